@@ -1,0 +1,250 @@
+/*
+ * ta.h — C ABI of the Transactional Attention (TA) KV-cache compaction library for NVIDIA B200 (sm_100a).
+ *
+ * The library implements one thing: the retention step of TA (Algorithm 1), run once over a prefilled KV cache,
+ * per layer and per KV head:
+ *
+ *   1. anchor detection + voucher allocation   (Section 3.2, Eq. 2, Algorithm 1 steps 1-6)   ta_sponsor_mask
+ *   2. attention part of the utility           (Eq. 1 terms alpha*A_i and delta*P_i)           ta_score
+ *   3. budget-K selection                      (Algorithm 1 step 8, Section 3.3)               ta_select_topk
+ *   4. eviction = gather of retained rows      (Algorithm 1 step 9, Section 3.2)               ta_compact_kv
+ *   all four in one enqueue                    (Algorithm 1)                                   ta_compress
+ *
+ * Conventions shared by every entry point
+ *   - Positions are 0-based; the paper's 1-based position i is i0 + 1.
+ *   - "DEVICE" pointers are CUDA device memory owned by the caller and must stay valid until the stream has
+ *     executed the call. "HOST" pointers are read before the call returns.
+ *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL = the legacy default stream),
+ *     allocate no memory, never throw and never abort. Host-detectable problems are returned as ta_status
+ *     and nothing is enqueued. Problems only the device can see (a token id outside the vocabulary, a sequence
+ *     longer than max_n, a pipeline wait that ran out) are recorded in the context and returned by ta_ctx_poll();
+ *     the kernels skip the offending access and still terminate.
+ *   - A batch holds B sequences. Uniform batches give every sequence n_uniform tokens; ragged batches pack
+ *     all tokens back to back and give cu_seqlens (B+1 ascending offsets, cu_seqlens[0] = 0). In both cases
+ *     token (b, i) has the packed index tok = cu_seqlens[b] + i (uniform: b*n_uniform + i). Per-token
+ *     arrays are indexed by tok; per-(layer, KV head, token) arrays are laid out [L][Hkv][total_tokens].
+ *   - A "unit" is one (layer l, sequence b, KV head g); units are independent.
+ *   - Supported shapes: head_dim d = 128; G = Hq/Hkv and observation window W with G*W <= 256 and W <= 64;
+ *     budget K <= 4096... see ta_limits below. Anything else returns TA_ERR_UNSUPPORTED: there is no fallback
+ *     path.
+ */
+#ifndef TA_H_
+#define TA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum ta_status {
+  TA_OK = 0,
+  TA_ERR_INVALID_ARG = 1,       /* NULL where data is required, negative size, inconsistent batch description   */
+  TA_ERR_UNSUPPORTED = 2,       /* shape or device outside the supported set                                     */
+  TA_ERR_ALIGNMENT = 3,         /* a bf16 view whose base or strides are not 16-byte multiples                   */
+  TA_ERR_SCRATCH_TOO_SMALL = 4, /* the context's scratch cannot hold this call (see ta_scratch_bytes)            */
+  TA_ERR_CUDA = 5,              /* a CUDA runtime / driver call failed; ta_ctx_last_cuda_error() has the code     */
+  TA_ERR_TIMEOUT = 6,           /* device: a bounded pipeline wait ran out                                       */
+  TA_ERR_DEVICE_BOUNDS = 7      /* device: token id >= vocab_size, or a sequence longer than max_n                */
+} ta_status;
+
+enum { TA_MODE_SCORED = 0, TA_MODE_FAST = 1 };
+
+/* bits of the per-token flag byte written by ta_sponsor_mask */
+enum {
+  TA_FLAG_ANCHOR_TOKEN = 1, /* S_i of Eq. 1: the token belongs to a matched anchor pattern            */
+  TA_FLAG_ANCHOR_END = 2,   /* the token is the last token of a match: "the anchor i" of Eq. 2        */
+  TA_FLAG_SPONSORED = 4     /* V_i > 0                                                                */
+};
+
+/* hard limits of this build (validated on every call) */
+enum {
+  TA_MAX_PATTERNS = 256,    /* patterns in one set                                                     */
+  TA_MAX_PATTERN_LEN = 8,   /* token ids per pattern                                                   */
+  TA_MAX_SPAN = 64,         /* sponsorship span L per pattern                                          */
+  TA_MAX_WINDOW = 64,       /* observation window W                                                    */
+  TA_MAX_SCORE_ROWS = 256,  /* G * W                                                                   */
+  TA_MAX_BUDGET = 4096,     /* K                                                                       */
+  TA_MAX_SEQ_LEN = 1 << 20, /* tokens per sequence                                                     */
+  TA_HEAD_DIM = 128         /* d                                                                       */
+};
+
+/*
+ * Hyper-parameters of Eq. 1 / Eq. 2 / Section 3.3. Paper defaults in brackets.
+ *   alpha, beta, gamma, delta, lambda  weights of Eq. 1                       [1.0 0.5 0.3 0.2 0.1]
+ *   voucher_decay                      base of the per-token voucher decay    [0.8]  (Eq. 2)
+ *   budget_decay, age_steps            B_i = B_p * budget_decay^age_steps     [0.9, 0] (Section 3.2, budgets decay per step)
+ *   n_sink, n_recent                   mandatory first / last tokens, taken from the main pool (Section 3.3)
+ *   k_protected                        slots reserved for sponsored tokens; < 0 means K_eff - n_sink - n_recent
+ *                                      (the K_p = K - 1 - W of Theorems 2-4)
+ *   obs_window                         W: number of trailing query positions whose attention is summed into A_i
+ *   pension_rho                        P_i is an exponential moving average over the W window rows with this
+ *                                      coefficient: P_i = sum_t (1-rho) rho^(W'-1-t) a_{t,i}
+ *   softmax_scale                      0 means 1/sqrt(d)
+ *   causal                             1: query row t (position n-W+t) sees keys i <= n-W+t
+ *   mode                               TA_MODE_SCORED (Eq. 1) or TA_MODE_FAST (Eq. 3: alpha = delta = 0, no Q/K read)
+ *   vocab_size                         token ids must lie in [0, vocab_size); sizes the frequency histogram of F_i
+ */
+typedef struct ta_policy {
+  float alpha, beta, gamma, delta, lambda;
+  float voucher_decay;
+  float budget_decay;
+  int32_t age_steps;
+  int32_t n_sink, n_recent, k_protected;
+  int32_t obs_window;
+  float pension_rho;
+  float softmax_scale;
+  int32_t causal;
+  int32_t mode;
+  int32_t vocab_size;
+} ta_policy;
+
+/* Named budget partitions. The paper states three that disagree; all are expressible in ta_policy:
+ *   TA_PRESET_THEOREM  1 sink, 4 recent, protected = the rest   (Theorems 2-4, Corollary on the minimum budget)
+ *   TA_PRESET_SEC33    1 sink, 2 recent, protected = K/4        (Section 3.3: K=16 -> 12 + 4)
+ *   TA_PRESET_AUDIT    4 sinks, 6 recent, 6 protected           (baseline-audit table, K=16)
+ * ta_policy_default fills every field with the paper's defaults for budget K and the given preset. */
+enum { TA_PRESET_THEOREM = 0, TA_PRESET_SEC33 = 1, TA_PRESET_AUDIT = 2 };
+ta_status ta_policy_default(int preset, int K, ta_policy* out /*HOST*/);
+
+typedef struct ta_batch {
+  int32_t n_layers;          /* L >= 1: layers handled by this call (independent; a launch-batching dimension) */
+  int32_t batch;             /* B >= 1                                                                       */
+  int32_t n_uniform;         /* tokens per sequence when cu_seqlens == NULL                                  */
+  int32_t max_n;             /* >= every sequence length (sizes the launch)                                  */
+  int64_t total_tokens;      /* sum of lengths (B * n_uniform when uniform)                                  */
+  const int32_t* cu_seqlens; /* DEVICE, B+1 entries, or NULL for a uniform batch                             */
+} ta_batch;
+
+/* A bf16 tensor with head_dim contiguous. Element (l, b, h, i, c) lives at
+ *   uniform batch: ptr + l*stride_l + b*stride_b + h*stride_h + i*stride_n + c
+ *   ragged batch : ptr + l*stride_l + h*stride_h + (cu_seqlens[b] + i)*stride_n + c        (stride_b unused)
+ * Strides are in elements and must be multiples of 8 (16 bytes); ptr must be 16-byte aligned.
+ * For q_obs the position axis is the window row t in [0, W) (row t is the query at position n - W + t; when
+ * n < W the first W - n rows are ignored) and the tensor is always dense per sequence (stride_b is used for
+ * ragged batches too). */
+typedef struct ta_bf16_view {
+  const void* ptr; /* DEVICE */
+  int64_t stride_l, stride_b, stride_h, stride_n;
+} ta_bf16_view;
+
+typedef struct ta_ctx ta_ctx;           /* opaque; one per device; owns scratch and the device status word      */
+typedef struct ta_patterns ta_patterns; /* opaque; device-resident matcher tables                               */
+
+/* ---- context ---------------------------------------------------------------------------------------------- */
+
+/* Creates a context on `device` (must be compute capability 10.x) with `scratch_bytes` of device scratch.
+ * The only entry points that allocate or free device memory are ta_ctx_create/destroy and
+ * ta_patterns_create/destroy. */
+ta_status ta_ctx_create(int device, size_t scratch_bytes, ta_ctx** out);
+void ta_ctx_destroy(ta_ctx* ctx);
+
+/* Scratch needed by the largest of the entry points for this problem size (ta_compress needs the most). */
+ta_status ta_scratch_bytes(const ta_batch* batch, int Hq, int Hkv, int d, int K, const ta_policy* policy,
+                           size_t* out_bytes);
+
+/* Synchronises the context's device, then returns and clears the first device-detected error (TA_OK if none). */
+ta_status ta_ctx_poll(ta_ctx* ctx);
+int ta_ctx_last_cuda_error(const ta_ctx* ctx);
+const char* ta_status_string(ta_status s);
+
+/* Optional per-kernel timing of ta_compress: when enabled, CUDA events are recorded on the call's stream around
+ * each kernel of the next ta_compress calls. ta_ctx_read_timing synchronises on those events and returns the
+ * milliseconds of the most recent call in out_ms[0..4] = {mask+static utility, score, select, compact, total}.
+ * Stages that did not run report 0. */
+ta_status ta_ctx_enable_timing(ta_ctx* ctx, int enable);
+ta_status ta_ctx_read_timing(ta_ctx* ctx, float out_ms[5] /*HOST*/);
+
+/* ---- anchor patterns (Section 3.2: the pattern set P; passing only allow-listed patterns is the allowlist
+ *      defence of Section 5.3) ------------------------------------------------------------------------------- */
+
+/* n_pat patterns; pattern p is ids_flat[offsets[p] .. offsets[p+1]) (1..TA_MAX_PATTERN_LEN token ids, all >= 0).
+ * budget[p] is the sponsor budget B (NULL: 15 for all), span[p] the span L in [1, TA_MAX_SPAN] (NULL: 6).
+ * All arrays HOST. n_pat may be 0 (no anchors: TA degenerates to plain score-based top-K). */
+ta_status ta_patterns_create(ta_ctx* ctx, int n_pat, const int32_t* ids_flat, const int32_t* offsets,
+                             const float* budget, const int32_t* span, ta_patterns** out);
+void ta_patterns_destroy(ta_patterns* pats);
+
+/* ---- step 1: sponsorship mask, vouchers and the attention-free utility ------------------------------------
+ * Algorithm 1 steps 1-6 and the attention-free part of step 7 (which is the whole TA-Fast score, Eq. 3).
+ * For every token: a pattern ends at position e when ids[e-len+1..e] equals it and the match does not cross
+ * the start of the sequence; if several patterns end at e the longest wins, then the lowest index. Every token of
+ * a match gets TA_FLAG_ANCHOR_TOKEN, its last token TA_FLAG_ANCHOR_END. Vouchers follow Eq. 2 with the winning
+ * pattern's budget (decayed age_steps times) and span, clipped at the end of the sequence; contributions of several
+ * anchors add, nearest anchor first. u_static = ((beta*R + gamma*S) - lambda*F) + V with R = (i0+1)/n and
+ * F = (occurrences of the token's id in its sequence)/n, every operation rounded to fp32.
+ *   token_ids  DEVICE int32 [total_tokens]
+ *   flags      DEVICE uint8 [total_tokens]   out
+ *   voucher    DEVICE float [total_tokens]   out
+ *   u_static   DEVICE float [total_tokens]   out
+ * Uses B*vocab_size*4 bytes of context scratch. batch->n_layers is ignored. */
+ta_status ta_sponsor_mask(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* policy, const ta_batch* batch,
+                          const int32_t* token_ids, uint8_t* flags, float* voucher, float* u_static, void* stream);
+
+/* ---- step 2: attention mass over the observation window ---------------------------------------------------
+ * Eq. 1's A_i and P_i, read as a one-shot compaction after prefill: for unit (l, b, g) the score rows are the
+ * last W' = min(W, n) query positions of the G = Hq/Hkv query heads of KV group g;
+ *   a_{h,t,i} = softmax_i( scale * <q_{h,t}, k_i> )   over the keys the row may see,
+ *   A_i = sum_{h,t} a_{h,t,i},      P_i = sum_{h,t} (1-rho) rho^(W'-1-t) a_{h,t,i}.
+ *   q_obs   bf16 view, positions = window rows, heads = Hq query heads
+ *   k       bf16 view, positions = context tokens, heads = Hkv
+ *   lse_obs DEVICE float [L][B][Hq][W] natural-log softmax normalisers of the same rows, or NULL. When given
+ *           (a prefill attention kernel has them), the keys are read once instead of twice.
+ *   A, P    DEVICE float [L][Hkv][total_tokens], out; P may be NULL.
+ * The contraction runs on the tensor cores (bf16 inputs, fp32 accumulation). */
+ta_status ta_score(ta_ctx* ctx, const ta_policy* policy, const ta_batch* batch, int Hq, int Hkv, int d,
+                   ta_bf16_view q_obs, ta_bf16_view k, const float* lse_obs, float* A, float* P, void* stream);
+
+/* ---- step 3: budget-K selection (Algorithm 1 step 8 with the partition of Section 3.3) --------------------
+ * Per unit: K_eff = min(K, n). If K_eff == n everything is kept. Otherwise p = k_protected (auto when < 0,
+ * clipped to [0, K_eff]) slots are protected and K_main = K_eff - p are main slots. Mandatory tokens (sinks
+ * 0.., then recents n-1, n-2, ..) are taken in that order while main slots last; the protected pool takes the
+ * sponsored tokens (voucher > 0) with the largest vouchers, lower position first among equals; what is left of
+ * the budget goes to the tokens with the largest u = (alpha*A + delta*P) + u_static (TA_MODE_SCORED) or
+ * u = u_static (TA_MODE_FAST), lower position first among equals (+0 and -0 compare equal; inputs must be finite).
+ *   flags, voucher, u_static  DEVICE, per token, as written by ta_sponsor_mask
+ *   A, P                      DEVICE float [L][Hkv][total_tokens] (scored mode; P may be NULL; both NULL in fast mode)
+ *   idx    DEVICE int32 [L][B][Hkv][K]  out: retained positions, ascending, padded with -1
+ *   count  DEVICE int32 [L][B][Hkv]     out: K_eff
+ * Uses total_tokens + 8*B bytes of context scratch. */
+ta_status ta_select_topk(ta_ctx* ctx, const ta_policy* policy, const ta_batch* batch, int Hkv, int K,
+                         const uint8_t* flags, const float* voucher, const float* u_static, const float* A,
+                         const float* P, int32_t* idx, int32_t* count, void* stream);
+
+/* ---- step 4: compaction (Algorithm 1 step 9: index_select along the sequence axis) ------------------------
+ *   k, v          bf16 views over the full cache
+ *   idx, count    as written by ta_select_topk
+ *   k_out, v_out  DEVICE bf16 [L][B][Hkv][K][d] out; rows at and beyond count are zero-filled. */
+ta_status ta_compact_kv(ta_ctx* ctx, const ta_batch* batch, int Hkv, int d, int K, ta_bf16_view k, ta_bf16_view v,
+                        const int32_t* idx, const int32_t* count, void* k_out, void* v_out, void* stream);
+
+/* ---- all steps in one enqueue (Algorithm 1) ---------------------------------------------------------------
+ * Steps 1-4 for batch->n_layers layers. The per-sequence results of step 1 (and, in fast mode, of step 3, which
+ * then does not depend on layer or head) are kept in the context and reused when seq_epoch is non-zero and equal
+ * to the previous call's: pass the same non-zero epoch for successive layers of one batch, a new one (or 0:
+ * never reuse) for a new batch. In scored mode the utilities stay in context scratch; A and P are not
+ * materialised. q_obs and k are not read in fast mode (their ptr may be NULL). */
+ta_status ta_compress(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* policy, const ta_batch* batch, int Hq,
+                      int Hkv, int d, int K, const int32_t* token_ids, ta_bf16_view q_obs, ta_bf16_view k,
+                      ta_bf16_view v, uint64_t seq_epoch, void* k_out, void* v_out, int32_t* idx, int32_t* count,
+                      void* stream);
+
+/* ---- host-buffer variant of ta_compress --------------------------------------------------------------------
+ * Same computation with every data pointer on the HOST (pinned memory makes the copies asynchronous):
+ * token_ids, cu_seqlens (inside batch: HOST here), the q_obs / k / v views, and the four outputs. The caller lends
+ * `workspace` (DEVICE, workspace_bytes >= ta_compress_host_workspace_bytes(...)) for the staged copies. Host to
+ * device copies, kernels and device to host copies are all enqueued on `stream`. Views must be dense in the
+ * order [L][B][Hkv or Hq][n or W][d] (ragged: [L][Hkv][total_tokens][d]); other strides return
+ * TA_ERR_UNSUPPORTED. */
+ta_status ta_compress_host_workspace_bytes(const ta_batch* batch, int Hq, int Hkv, int d, int K,
+                                           const ta_policy* policy, size_t* out_bytes);
+ta_status ta_compress_host(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* policy, const ta_batch* batch,
+                           int Hq, int Hkv, int d, int K, const int32_t* token_ids, const void* q_obs,
+                           const void* k, const void* v, void* k_out, void* v_out, int32_t* idx, int32_t* count,
+                           void* workspace, size_t workspace_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TA_H_ */
