@@ -160,6 +160,8 @@ def attention(Q: np.ndarray, K: np.ndarray, n: int, scale=0.0, causal=1, rho=0.9
     assert Q.dtype == np.uint16 and K.dtype == np.uint16
     Q = np.ascontiguousarray(Q)
     G, W, d = Q.shape
+    if n == 0:
+        return np.zeros(0, np.float32), np.zeros(0, np.float32)
     assert K.strides[1] == 2
     A = np.zeros(n, np.float32)
     P = np.zeros(n, np.float32)

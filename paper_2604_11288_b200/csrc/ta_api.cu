@@ -1,0 +1,697 @@
+// Host side of libta.so: argument validation, scratch carving and launch sequencing for the entry points declared
+// in ta.h. Nothing here computes any part of the method; every step runs in the kernels of ta_mask.cu, ta_score.cu,
+// ta_select.cu and ta_compact.cu.
+#include <cuda.h>
+#include <math.h>
+#include <new>
+#include <string.h>
+
+#include "ta_internal.cuh"
+
+namespace {
+
+constexpr size_t kAlign = 256;
+inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+struct Carve {  // hands out aligned pieces of the context scratch
+  uint8_t* base;
+  size_t off = 0;
+  explicit Carve(uint8_t* b) : base(b) {}
+  template <class T>
+  T* take(size_t count) {
+    T* p = reinterpret_cast<T*>(base + off);
+    off += align_up(count * sizeof(T));
+    return p;
+  }
+};
+
+struct Layout {  // scratch layout of ta_compress (a superset of what the single-step entry points need)
+  size_t hist, flags, voucher, u_static, forced, r_main, idx_seq, count_seq, u, end;
+};
+
+Layout make_layout(const ta_batch& b, int Hkv, int K, const ta_policy& pol) {
+  Layout L;
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    const size_t o = off;
+    off += align_up(bytes);
+    return o;
+  };
+  const size_t total = (size_t)b.total_tokens, B = (size_t)b.batch;
+  L.hist = take(B * (size_t)pol.vocab_size * 4);
+  L.flags = take(total);
+  L.voucher = take(total * 4);
+  L.u_static = take(total * 4);
+  L.forced = take(total);
+  L.r_main = take(B * 4);
+  L.idx_seq = take(B * (size_t)K * 4);
+  L.count_seq = take(B * 4);
+  L.u = take(pol.mode == TA_MODE_FAST ? 0 : (size_t)b.n_layers * Hkv * total * 4);
+  L.end = off;
+  return L;
+}
+
+ta_status check_batch(const ta_batch* b) {
+  if (!b) return TA_ERR_INVALID_ARG;
+  if (b->n_layers < 1 || b->batch < 1 || b->max_n < 0 || b->total_tokens < 0) return TA_ERR_INVALID_ARG;
+  if (b->max_n > TA_MAX_SEQ_LEN) return TA_ERR_UNSUPPORTED;
+  if (!b->cu_seqlens) {
+    if (b->n_uniform < 0 || b->n_uniform > b->max_n) return TA_ERR_INVALID_ARG;
+    if (b->total_tokens != (int64_t)b->batch * b->n_uniform) return TA_ERR_INVALID_ARG;
+  }
+  if (b->total_tokens > 0x7fffffffLL) return TA_ERR_UNSUPPORTED;
+  return TA_OK;
+}
+
+ta_status check_policy(const ta_policy* p) {
+  if (!p) return TA_ERR_INVALID_ARG;
+  if (p->mode != TA_MODE_SCORED && p->mode != TA_MODE_FAST) return TA_ERR_INVALID_ARG;
+  if (p->vocab_size < 1 || p->age_steps < 0 || p->n_sink < 0 || p->n_recent < 0) return TA_ERR_INVALID_ARG;
+  if (p->softmax_scale < 0.0f || !(p->pension_rho >= 0.0f && p->pension_rho <= 1.0f)) return TA_ERR_INVALID_ARG;
+  return TA_OK;
+}
+
+ta_status check_heads(int Hq, int Hkv, int d, const ta_policy* p, bool scored) {
+  if (Hkv < 1 || Hq < Hkv || Hq % Hkv) return TA_ERR_INVALID_ARG;
+  if (d != TA_HEAD_DIM) return TA_ERR_UNSUPPORTED;
+  if (scored) {
+    if (p->obs_window < 1) return TA_ERR_INVALID_ARG;
+    if (p->obs_window > TA_MAX_WINDOW || (Hq / Hkv) * p->obs_window > TA_MAX_SCORE_ROWS || Hq / Hkv > 256)
+      return TA_ERR_UNSUPPORTED;
+  }
+  return TA_OK;
+}
+
+ta_status check_view(const ta_bf16_view& v, bool need_b) {
+  if (!v.ptr) return TA_ERR_INVALID_ARG;
+  if ((uintptr_t)v.ptr % 16) return TA_ERR_ALIGNMENT;
+  const int64_t s[4] = {v.stride_l, v.stride_b, v.stride_h, v.stride_n};
+  for (int i = 0; i < 4; ++i) {
+    if (i == 1 && !need_b) continue;
+    if (s[i] < 0) return TA_ERR_INVALID_ARG;
+    if (s[i] % 8) return TA_ERR_ALIGNMENT;
+  }
+  if (v.stride_n < TA_HEAD_DIM) return TA_ERR_INVALID_ARG;
+  return TA_OK;
+}
+
+ta_seq_desc seq_desc(const ta_batch& b) {
+  ta_seq_desc s;
+  s.cu = b.cu_seqlens;
+  s.n_uniform = b.n_uniform;
+  s.batch = b.batch;
+  s.max_n = b.max_n;
+  s.total = b.total_tokens;
+  return s;
+}
+
+ta_status cuda_fail(ta_ctx* ctx, cudaError_t e) {
+  ctx->last_cuda_error = (int)e;
+  return TA_ERR_CUDA;
+}
+
+struct DeviceGuard {  // makes the context's device current for the duration of a call
+  int prev = -1;
+  bool ok;
+  explicit DeviceGuard(int dev) {
+    ok = cudaGetDevice(&prev) == cudaSuccess && (prev == dev || cudaSetDevice(dev) == cudaSuccess);
+    if (prev == dev) prev = -1;
+  }
+  ~DeviceGuard() {
+    if (prev >= 0) cudaSetDevice(prev);
+  }
+};
+
+}  // namespace
+
+extern "C" {
+
+const char* ta_status_string(ta_status s) {
+  switch (s) {
+    case TA_OK: return "ok";
+    case TA_ERR_INVALID_ARG: return "invalid argument";
+    case TA_ERR_UNSUPPORTED: return "unsupported shape or device";
+    case TA_ERR_ALIGNMENT: return "pointer or stride not 16-byte aligned";
+    case TA_ERR_SCRATCH_TOO_SMALL: return "context scratch too small";
+    case TA_ERR_CUDA: return "CUDA call failed";
+    case TA_ERR_TIMEOUT: return "device wait timed out";
+    case TA_ERR_DEVICE_BOUNDS: return "device-side bounds check failed";
+  }
+  return "unknown";
+}
+
+ta_status ta_policy_default(int preset, int K, ta_policy* out) {
+  if (!out || K < 0) return TA_ERR_INVALID_ARG;
+  ta_policy p;
+  memset(&p, 0, sizeof p);
+  p.alpha = 1.0f;
+  p.beta = 0.5f;
+  p.gamma = 0.3f;
+  p.delta = 0.2f;
+  p.lambda = 0.1f;
+  p.voucher_decay = 0.8f;
+  p.budget_decay = 0.9f;
+  p.age_steps = 0;
+  p.obs_window = 32;
+  p.pension_rho = 0.9f;
+  p.softmax_scale = 0.0f;
+  p.causal = 1;
+  p.mode = TA_MODE_SCORED;
+  p.vocab_size = 32000;
+  switch (preset) {
+    case TA_PRESET_THEOREM: p.n_sink = 1; p.n_recent = 4; p.k_protected = -1; break;
+    case TA_PRESET_SEC33: p.n_sink = 1; p.n_recent = 2; p.k_protected = K / 4; break;
+    case TA_PRESET_AUDIT: p.n_sink = 4; p.n_recent = 6; p.k_protected = 6; break;
+    default: return TA_ERR_INVALID_ARG;
+  }
+  *out = p;
+  return TA_OK;
+}
+
+ta_status ta_ctx_create(int device, size_t scratch_bytes, ta_ctx** out) {
+  if (!out) return TA_ERR_INVALID_ARG;
+  *out = nullptr;
+  int count = 0;
+  if (cudaGetDeviceCount(&count) != cudaSuccess || device < 0 || device >= count) return TA_ERR_INVALID_ARG;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return TA_ERR_CUDA;
+  if (prop.major != 10) return TA_ERR_UNSUPPORTED;  // the kernels are built for sm_100a only
+  DeviceGuard guard(device);
+  if (!guard.ok) return TA_ERR_CUDA;
+  ta_ctx* c = new (std::nothrow) ta_ctx();
+  if (!c) return TA_ERR_CUDA;
+  memset(c, 0, sizeof *c);
+  c->device = device;
+  c->sm_count = prop.multiProcessorCount;
+  c->scratch_bytes = scratch_bytes;
+  cudaError_t e = cudaMalloc(&c->d_status, sizeof(ta_dev_status));
+  if (e == cudaSuccess) e = cudaMemset(c->d_status, 0, sizeof(ta_dev_status));
+  if (e == cudaSuccess && scratch_bytes) e = cudaMalloc(&c->scratch, scratch_bytes);
+  for (int i = 0; e == cudaSuccess && i < 8; ++i) e = cudaEventCreate(&c->ev[i]);
+  if (e == cudaSuccess) {
+    cudaDriverEntryPointQueryResult q;
+    e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &c->encode_tiled, cudaEnableDefault, &q);
+    if (e == cudaSuccess && (q != cudaDriverEntryPointSuccess || !c->encode_tiled)) e = cudaErrorNotSupported;
+  }
+  if (e != cudaSuccess) {
+    ta_ctx_destroy(c);
+    return TA_ERR_CUDA;
+  }
+  *out = c;
+  return TA_OK;
+}
+
+void ta_ctx_destroy(ta_ctx* c) {
+  if (!c) return;
+  DeviceGuard guard(c->device);
+  for (int i = 0; i < 8; ++i)
+    if (c->ev[i]) cudaEventDestroy(c->ev[i]);
+  if (c->scratch) cudaFree(c->scratch);
+  if (c->d_status) cudaFree(c->d_status);
+  delete c;
+}
+
+ta_status ta_scratch_bytes(const ta_batch* batch, int Hq, int Hkv, int d, int K, const ta_policy* policy,
+                           size_t* out_bytes) {
+  (void)Hq;
+  (void)d;
+  if (!out_bytes) return TA_ERR_INVALID_ARG;
+  ta_status s = check_batch(batch);
+  if (s == TA_OK) s = check_policy(policy);
+  if (s != TA_OK) return s;
+  if (K < 1 || Hkv < 1) return TA_ERR_INVALID_ARG;
+  *out_bytes = make_layout(*batch, Hkv, K, *policy).end + kAlign;
+  return TA_OK;
+}
+
+ta_status ta_ctx_poll(ta_ctx* ctx) {
+  if (!ctx) return TA_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->device);
+  cudaError_t e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) return cuda_fail(ctx, e);
+  ta_dev_status st;
+  e = cudaMemcpy(&st, ctx->d_status, sizeof st, cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) return cuda_fail(ctx, e);
+  if (st.code != 0) {
+    cudaMemset(ctx->d_status, 0, sizeof st);
+    ctx->cached_epoch = 0;
+    return (ta_status)st.code;
+  }
+  return TA_OK;
+}
+
+int ta_ctx_last_cuda_error(const ta_ctx* ctx) { return ctx ? ctx->last_cuda_error : 0; }
+
+ta_status ta_ctx_enable_timing(ta_ctx* ctx, int enable) {
+  if (!ctx) return TA_ERR_INVALID_ARG;
+  ctx->timing_enabled = enable ? 1 : 0;
+  ctx->timing_valid = 0;
+  return TA_OK;
+}
+
+ta_status ta_ctx_read_timing(ta_ctx* ctx, float out_ms[5]) {
+  if (!ctx || !out_ms) return TA_ERR_INVALID_ARG;
+  for (int i = 0; i < 5; ++i) out_ms[i] = 0.0f;
+  if (!ctx->timing_valid) return TA_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->device);
+  cudaError_t e = cudaEventSynchronize(ctx->ev[4]);
+  for (int i = 0; e == cudaSuccess && i < 4; ++i) e = cudaEventElapsedTime(&out_ms[i], ctx->ev[i], ctx->ev[i + 1]);
+  if (e == cudaSuccess) e = cudaEventElapsedTime(&out_ms[4], ctx->ev[0], ctx->ev[4]);
+  return e == cudaSuccess ? TA_OK : cuda_fail(ctx, e);
+}
+
+// ---------------------------------------------------------------------------------------------- patterns
+ta_status ta_patterns_create(ta_ctx* ctx, int n_pat, const int32_t* ids_flat, const int32_t* offsets,
+                             const float* budget, const int32_t* span, ta_patterns** out) {
+  if (!ctx || !out || n_pat < 0 || (n_pat > 0 && (!ids_flat || !offsets))) return TA_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (n_pat > TA_MAX_PATTERNS) return TA_ERR_UNSUPPORTED;
+  const int np = n_pat > 0 ? n_pat : 1;
+  int32_t* h_ids = new (std::nothrow) int32_t[np * TA_MAX_PATTERN_LEN];
+  int32_t h_len[TA_MAX_PATTERNS], h_span[TA_MAX_PATTERNS];
+  float h_bud[TA_MAX_PATTERNS];
+  uint32_t h_bloom[32];
+  if (!h_ids) return TA_ERR_CUDA;
+  memset(h_bloom, 0, sizeof h_bloom);
+  for (int i = 0; i < np * TA_MAX_PATTERN_LEN; ++i) h_ids[i] = -1;
+  int max_len = 0, max_span = 0;
+  ta_status bad = TA_OK;
+  for (int p = 0; p < n_pat && bad == TA_OK; ++p) {
+    const int len = offsets[p + 1] - offsets[p];
+    const int sp = span ? span[p] : 6;
+    const float bu = budget ? budget[p] : 15.0f;
+    if (len < 1 || sp < 1 || !(bu == bu)) bad = TA_ERR_INVALID_ARG;
+    else if (len > TA_MAX_PATTERN_LEN || sp > TA_MAX_SPAN) bad = TA_ERR_UNSUPPORTED;
+    else {
+      for (int k = 0; k < len; ++k) {
+        const int32_t id = ids_flat[offsets[p] + k];
+        if (id < 0) bad = TA_ERR_INVALID_ARG;
+        h_ids[p * TA_MAX_PATTERN_LEN + k] = id;
+      }
+      const uint32_t h = ((uint32_t)h_ids[p * TA_MAX_PATTERN_LEN + len - 1] * 2654435761u) >> 22;
+      h_bloom[h >> 5] |= 1u << (h & 31);
+      h_len[p] = len;
+      h_span[p] = sp;
+      h_bud[p] = bu;
+      if (len > max_len) max_len = len;
+      if (sp > max_span) max_span = sp;
+    }
+  }
+  if (bad != TA_OK) {
+    delete[] h_ids;
+    return bad;
+  }
+  if (n_pat == 0) {
+    h_len[0] = 0;
+    h_span[0] = 0;
+    h_bud[0] = 0.0f;
+  }
+  DeviceGuard guard(ctx->device);
+  ta_patterns* P = new (std::nothrow) ta_patterns();
+  if (!P) {
+    delete[] h_ids;
+    return TA_ERR_CUDA;
+  }
+  memset(P, 0, sizeof *P);
+  P->device = ctx->device;
+  P->n_pat = n_pat;
+  P->max_len = max_len;
+  P->max_span = max_span;
+  cudaError_t e = cudaMalloc(&P->d_ids, sizeof(int32_t) * np * TA_MAX_PATTERN_LEN);
+  if (e == cudaSuccess) e = cudaMalloc(&P->d_len, sizeof(int32_t) * np);
+  if (e == cudaSuccess) e = cudaMalloc(&P->d_budget, sizeof(float) * np);
+  if (e == cudaSuccess) e = cudaMalloc(&P->d_span, sizeof(int32_t) * np);
+  if (e == cudaSuccess) e = cudaMalloc(&P->d_bloom, sizeof h_bloom);
+  if (e == cudaSuccess) e = cudaMemcpy(P->d_ids, h_ids, sizeof(int32_t) * np * TA_MAX_PATTERN_LEN, cudaMemcpyHostToDevice);
+  if (e == cudaSuccess) e = cudaMemcpy(P->d_len, h_len, sizeof(int32_t) * np, cudaMemcpyHostToDevice);
+  if (e == cudaSuccess) e = cudaMemcpy(P->d_budget, h_bud, sizeof(float) * np, cudaMemcpyHostToDevice);
+  if (e == cudaSuccess) e = cudaMemcpy(P->d_span, h_span, sizeof(int32_t) * np, cudaMemcpyHostToDevice);
+  if (e == cudaSuccess) e = cudaMemcpy(P->d_bloom, h_bloom, sizeof h_bloom, cudaMemcpyHostToDevice);
+  delete[] h_ids;
+  if (e != cudaSuccess) {
+    ta_patterns_destroy(P);
+    return cuda_fail(ctx, e);
+  }
+  *out = P;
+  return TA_OK;
+}
+
+void ta_patterns_destroy(ta_patterns* P) {
+  if (!P) return;
+  DeviceGuard guard(P->device);
+  if (P->d_ids) cudaFree(P->d_ids);
+  if (P->d_len) cudaFree(P->d_len);
+  if (P->d_budget) cudaFree(P->d_budget);
+  if (P->d_span) cudaFree(P->d_span);
+  if (P->d_bloom) cudaFree(P->d_bloom);
+  delete P;
+}
+
+// ---------------------------------------------------------------------------------------------- step 1
+ta_status ta_sponsor_mask(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* policy, const ta_batch* batch,
+                          const int32_t* token_ids, uint8_t* flags, float* voucher, float* u_static, void* stream) {
+  if (!ctx || !pats || !token_ids || !flags || !voucher || !u_static) return TA_ERR_INVALID_ARG;
+  ta_status s = check_batch(batch);
+  if (s == TA_OK) s = check_policy(policy);
+  if (s != TA_OK) return s;
+  if (pats->device != ctx->device) return TA_ERR_INVALID_ARG;
+  const size_t need = align_up((size_t)batch->batch * policy->vocab_size * 4);
+  if (need > ctx->scratch_bytes) return TA_ERR_SCRATCH_TOO_SMALL;
+  DeviceGuard guard(ctx->device);
+  ctx->cached_epoch = 0;
+  cudaError_t e = ta_launch_mask(pats, *policy, seq_desc(*batch), token_ids, flags, voucher, u_static,
+                                 reinterpret_cast<int32_t*>(ctx->scratch), ctx->d_status, (cudaStream_t)stream);
+  return e == cudaSuccess ? TA_OK : cuda_fail(ctx, e);
+}
+
+// ---------------------------------------------------------------------------------------------- step 2
+ta_status ta_score(ta_ctx* ctx, const ta_policy* policy, const ta_batch* batch, int Hq, int Hkv, int d,
+                   ta_bf16_view q_obs, ta_bf16_view k, const float* lse_obs, float* A, float* P, void* stream) {
+  if (!ctx || !A) return TA_ERR_INVALID_ARG;
+  ta_status s = check_batch(batch);
+  if (s == TA_OK) s = check_policy(policy);
+  if (s == TA_OK) s = check_heads(Hq, Hkv, d, policy, true);
+  if (s == TA_OK) s = check_view(q_obs, true);
+  if (s == TA_OK) s = check_view(k, batch->cu_seqlens == nullptr);
+  if (s != TA_OK) return s;
+  DeviceGuard guard(ctx->device);
+  ta_score_args a = {};
+  a.seq = seq_desc(*batch);
+  a.n_layers = batch->n_layers;
+  a.Hq = Hq;
+  a.Hkv = Hkv;
+  a.W = policy->obs_window;
+  a.q = q_obs;
+  a.k = k;
+  a.lse_obs = lse_obs;
+  a.A = A;
+  a.P = P;
+  a.u = nullptr;
+  a.u_static = nullptr;
+  a.alpha = policy->alpha;
+  a.delta = policy->delta;
+  a.rho = policy->pension_rho;
+  a.scale = policy->softmax_scale;
+  a.causal = policy->causal;
+  cudaError_t e = ta_launch_score(ctx, a, ctx->d_status, (cudaStream_t)stream);
+  return e == cudaSuccess ? TA_OK : cuda_fail(ctx, e);
+}
+
+// ---------------------------------------------------------------------------------------------- step 3
+ta_status ta_select_topk(ta_ctx* ctx, const ta_policy* policy, const ta_batch* batch, int Hkv, int K,
+                         const uint8_t* flags, const float* voucher, const float* u_static, const float* A,
+                         const float* P, int32_t* idx, int32_t* count, void* stream) {
+  if (!ctx || !flags || !voucher || !u_static || !idx || !count) return TA_ERR_INVALID_ARG;
+  ta_status s = check_batch(batch);
+  if (s == TA_OK) s = check_policy(policy);
+  if (s != TA_OK) return s;
+  if (Hkv < 1 || K < 1) return TA_ERR_INVALID_ARG;
+  if (K > TA_MAX_BUDGET) return TA_ERR_UNSUPPORTED;
+  const bool fast = policy->mode == TA_MODE_FAST;
+  if (!fast && !A) return TA_ERR_INVALID_ARG;
+  Carve carve(ctx->scratch);
+  uint8_t* forced = carve.take<uint8_t>((size_t)batch->total_tokens);
+  int32_t* r_main = carve.take<int32_t>((size_t)batch->batch);
+  int32_t* idx_seq = carve.take<int32_t>(fast ? (size_t)batch->batch * K : 0);
+  int32_t* count_seq = carve.take<int32_t>(fast ? (size_t)batch->batch : 0);
+  if (carve.off > ctx->scratch_bytes) return TA_ERR_SCRATCH_TOO_SMALL;
+  DeviceGuard guard(ctx->device);
+  ctx->cached_epoch = 0;
+  ta_select_args a = {};
+  a.seq = seq_desc(*batch);
+  a.n_layers = batch->n_layers;
+  a.Hkv = Hkv;
+  a.K = K;
+  a.n_sink = policy->n_sink;
+  a.n_recent = policy->n_recent;
+  a.k_protected = policy->k_protected;
+  a.fast = fast;
+  a.alpha = policy->alpha;
+  a.delta = policy->delta;
+  a.flags = flags;
+  a.voucher = voucher;
+  a.u_static = u_static;
+  a.A = A;
+  a.P = P;
+  a.u = nullptr;
+  a.forced = forced;
+  a.r_main = r_main;
+  a.idx = fast ? idx_seq : idx;
+  a.count = fast ? count_seq : count;
+  cudaError_t e = ta_launch_select(a, ctx->d_status, (cudaStream_t)stream);
+  if (e == cudaSuccess && fast)
+    e = ta_launch_broadcast_idx(batch->batch, Hkv, K, batch->n_layers, idx_seq, count_seq, idx, count,
+                                (cudaStream_t)stream);
+  return e == cudaSuccess ? TA_OK : cuda_fail(ctx, e);
+}
+
+// ---------------------------------------------------------------------------------------------- step 4
+ta_status ta_compact_kv(ta_ctx* ctx, const ta_batch* batch, int Hkv, int d, int K, ta_bf16_view k, ta_bf16_view v,
+                        const int32_t* idx, const int32_t* count, void* k_out, void* v_out, void* stream) {
+  if (!ctx || !idx || !count || !k_out || !v_out) return TA_ERR_INVALID_ARG;
+  ta_status s = check_batch(batch);
+  if (s != TA_OK) return s;
+  if (Hkv < 1 || K < 1) return TA_ERR_INVALID_ARG;
+  if (d != TA_HEAD_DIM || K > TA_MAX_BUDGET) return TA_ERR_UNSUPPORTED;
+  const bool uniform = batch->cu_seqlens == nullptr;
+  s = check_view(k, uniform);
+  if (s == TA_OK) s = check_view(v, uniform);
+  if (s != TA_OK) return s;
+  if ((uintptr_t)k_out % 16 || (uintptr_t)v_out % 16) return TA_ERR_ALIGNMENT;
+  DeviceGuard guard(ctx->device);
+  ta_compact_args a = {};
+  a.seq = seq_desc(*batch);
+  a.n_layers = batch->n_layers;
+  a.Hkv = Hkv;
+  a.K = K;
+  a.k = k;
+  a.v = v;
+  a.idx = idx;
+  a.count = count;
+  a.k_out = k_out;
+  a.v_out = v_out;
+  cudaError_t e = ta_launch_compact(a, ctx->sm_count, (cudaStream_t)stream);
+  return e == cudaSuccess ? TA_OK : cuda_fail(ctx, e);
+}
+
+// ---------------------------------------------------------------------------------------------- fused
+ta_status ta_compress(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* policy, const ta_batch* batch, int Hq,
+                      int Hkv, int d, int K, const int32_t* token_ids, ta_bf16_view q_obs, ta_bf16_view k,
+                      ta_bf16_view v, uint64_t seq_epoch, void* k_out, void* v_out, int32_t* idx, int32_t* count,
+                      void* stream_v) {
+  if (!ctx || !pats || !token_ids || !k_out || !v_out || !idx || !count) return TA_ERR_INVALID_ARG;
+  ta_status s = check_batch(batch);
+  if (s == TA_OK) s = check_policy(policy);
+  if (s != TA_OK) return s;
+  const bool fast = policy->mode == TA_MODE_FAST;
+  const bool uniform = batch->cu_seqlens == nullptr;
+  s = check_heads(Hq, Hkv, d, policy, !fast);
+  if (s == TA_OK && !fast) s = check_view(q_obs, true);
+  if (s == TA_OK) s = check_view(v, uniform);
+  if (s == TA_OK && !fast) s = check_view(k, uniform);
+  if (s == TA_OK && fast && k.ptr == nullptr) s = TA_ERR_INVALID_ARG;  // K rows are gathered in both modes
+  if (s == TA_OK && fast) s = check_view(k, uniform);
+  if (s != TA_OK) return s;
+  if (K < 1) return TA_ERR_INVALID_ARG;
+  if (K > TA_MAX_BUDGET) return TA_ERR_UNSUPPORTED;
+  if ((uintptr_t)k_out % 16 || (uintptr_t)v_out % 16) return TA_ERR_ALIGNMENT;
+  if (pats->device != ctx->device) return TA_ERR_INVALID_ARG;
+  const Layout L = make_layout(*batch, Hkv, K, *policy);
+  if (L.end > ctx->scratch_bytes) return TA_ERR_SCRATCH_TOO_SMALL;
+
+  DeviceGuard guard(ctx->device);
+  cudaStream_t stream = (cudaStream_t)stream_v;
+  uint8_t* sc = ctx->scratch;
+  int32_t* hist = reinterpret_cast<int32_t*>(sc + L.hist);
+  uint8_t* flags = sc + L.flags;
+  float* voucher = reinterpret_cast<float*>(sc + L.voucher);
+  float* u_static = reinterpret_cast<float*>(sc + L.u_static);
+  uint8_t* forced = sc + L.forced;
+  int32_t* r_main = reinterpret_cast<int32_t*>(sc + L.r_main);
+  int32_t* idx_seq = reinterpret_cast<int32_t*>(sc + L.idx_seq);
+  int32_t* count_seq = reinterpret_cast<int32_t*>(sc + L.count_seq);
+  float* u = reinterpret_cast<float*>(sc + L.u);
+  const ta_seq_desc seq = seq_desc(*batch);
+  const bool timing = ctx->timing_enabled != 0;
+  cudaError_t e = cudaSuccess;
+  auto mark = [&](int i) {
+    if (timing && e == cudaSuccess) e = cudaEventRecord(ctx->ev[i], stream);
+  };
+
+  const bool reuse = seq_epoch != 0 && seq_epoch == ctx->cached_epoch && ctx->cached_total == batch->total_tokens &&
+                     ctx->cached_batch == batch->batch && ctx->cached_K == K;
+  mark(0);
+  if (!reuse) e = ta_launch_mask(pats, *policy, seq, token_ids, flags, voucher, u_static, hist, ctx->d_status, stream);
+  mark(1);
+  if (e == cudaSuccess && !fast) {
+    ta_score_args a = {};
+    a.seq = seq;
+    a.n_layers = batch->n_layers;
+    a.Hq = Hq;
+    a.Hkv = Hkv;
+    a.W = policy->obs_window;
+    a.q = q_obs;
+    a.k = k;
+    a.lse_obs = nullptr;
+    a.A = nullptr;
+    a.P = nullptr;
+    a.u = u;
+    a.u_static = u_static;
+    a.alpha = policy->alpha;
+    a.delta = policy->delta;
+    a.rho = policy->pension_rho;
+    a.scale = policy->softmax_scale;
+    a.causal = policy->causal;
+    e = ta_launch_score(ctx, a, ctx->d_status, stream);
+  }
+  mark(2);
+  if (e == cudaSuccess && !(fast && reuse)) {
+    ta_select_args a = {};
+    a.seq = seq;
+    a.n_layers = batch->n_layers;
+    a.Hkv = Hkv;
+    a.K = K;
+    a.n_sink = policy->n_sink;
+    a.n_recent = policy->n_recent;
+    a.k_protected = policy->k_protected;
+    a.fast = fast;
+    a.alpha = policy->alpha;
+    a.delta = policy->delta;
+    a.flags = flags;
+    a.voucher = voucher;
+    a.u_static = u_static;
+    a.u = u;
+    a.forced = forced;
+    a.r_main = r_main;
+    a.idx = fast ? idx_seq : idx;
+    a.count = fast ? count_seq : count;
+    e = ta_launch_select(a, ctx->d_status, stream);
+  }
+  if (e == cudaSuccess && fast)
+    e = ta_launch_broadcast_idx(batch->batch, Hkv, K, batch->n_layers, idx_seq, count_seq, idx, count, stream);
+  mark(3);
+  if (e == cudaSuccess) {
+    ta_compact_args a = {};
+    a.seq = seq;
+    a.n_layers = batch->n_layers;
+    a.Hkv = Hkv;
+    a.K = K;
+    a.k = k;
+    a.v = v;
+    a.idx = idx;
+    a.count = count;
+    a.k_out = k_out;
+    a.v_out = v_out;
+    e = ta_launch_compact(a, ctx->sm_count, stream);
+  }
+  mark(4);
+  if (e != cudaSuccess) {
+    ctx->cached_epoch = 0;
+    return cuda_fail(ctx, e);
+  }
+  ctx->timing_valid = timing ? 1 : 0;
+  ctx->cached_epoch = seq_epoch;
+  ctx->cached_total = batch->total_tokens;
+  ctx->cached_batch = batch->batch;
+  ctx->cached_K = K;
+  return TA_OK;
+}
+
+// ---------------------------------------------------------------------------------------------- host buffers
+namespace {
+struct HostLayout {
+  size_t ids, cu, q, k, v, k_out, v_out, idx, count, end;
+  size_t q_bytes, kv_bytes, out_bytes, idx_bytes, count_bytes;
+};
+HostLayout host_layout(const ta_batch& b, int Hq, int Hkv, int d, int K, const ta_policy& pol) {
+  HostLayout H;
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    const size_t o = off;
+    off += align_up(bytes);
+    return o;
+  };
+  const size_t L = (size_t)b.n_layers, B = (size_t)b.batch, total = (size_t)b.total_tokens;
+  H.q_bytes = pol.mode == TA_MODE_FAST ? 0 : L * B * Hq * (size_t)pol.obs_window * d * 2;
+  H.kv_bytes = L * Hkv * total * d * 2;
+  H.out_bytes = L * B * Hkv * (size_t)K * d * 2;
+  H.idx_bytes = L * B * Hkv * (size_t)K * 4;
+  H.count_bytes = L * B * Hkv * 4;
+  H.ids = take(total * 4);
+  H.cu = take((B + 1) * 4);
+  H.q = take(H.q_bytes);
+  H.k = take(H.kv_bytes);
+  H.v = take(H.kv_bytes);
+  H.k_out = take(H.out_bytes);
+  H.v_out = take(H.out_bytes);
+  H.idx = take(H.idx_bytes);
+  H.count = take(H.count_bytes);
+  H.end = off;
+  return H;
+}
+}  // namespace
+
+ta_status ta_compress_host_workspace_bytes(const ta_batch* batch, int Hq, int Hkv, int d, int K,
+                                           const ta_policy* policy, size_t* out_bytes) {
+  if (!out_bytes) return TA_ERR_INVALID_ARG;
+  ta_status s = check_batch(batch);
+  if (s == TA_OK) s = check_policy(policy);
+  if (s != TA_OK) return s;
+  if (K < 1 || Hkv < 1 || Hq < 1 || d < 1) return TA_ERR_INVALID_ARG;
+  *out_bytes = host_layout(*batch, Hq, Hkv, d, K, *policy).end + kAlign;
+  return TA_OK;
+}
+
+ta_status ta_compress_host(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* policy, const ta_batch* batch,
+                           int Hq, int Hkv, int d, int K, const int32_t* token_ids, const void* q_obs, const void* k,
+                           const void* v, void* k_out, void* v_out, int32_t* idx, int32_t* count, void* workspace,
+                           size_t workspace_bytes, void* stream_v) {
+  if (!ctx || !pats || !token_ids || !k || !v || !k_out || !v_out || !idx || !count || !workspace)
+    return TA_ERR_INVALID_ARG;
+  ta_status s = check_batch(batch);
+  if (s == TA_OK) s = check_policy(policy);
+  if (s != TA_OK) return s;
+  const bool fast = policy->mode == TA_MODE_FAST;
+  if (!fast && !q_obs) return TA_ERR_INVALID_ARG;
+  if (K < 1 || Hkv < 1 || Hq < Hkv) return TA_ERR_INVALID_ARG;
+  if (d != TA_HEAD_DIM) return TA_ERR_UNSUPPORTED;
+  if ((uintptr_t)workspace % kAlign) return TA_ERR_ALIGNMENT;
+  const HostLayout H = host_layout(*batch, Hq, Hkv, d, K, *policy);
+  if (H.end > workspace_bytes) return TA_ERR_SCRATCH_TOO_SMALL;
+  DeviceGuard guard(ctx->device);
+  cudaStream_t stream = (cudaStream_t)stream_v;
+  uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
+  const size_t total = (size_t)batch->total_tokens;
+  cudaError_t e = cudaMemcpyAsync(ws + H.ids, token_ids, total * 4, cudaMemcpyHostToDevice, stream);
+  ta_batch db = *batch;
+  if (batch->cu_seqlens) {
+    if (e == cudaSuccess)
+      e = cudaMemcpyAsync(ws + H.cu, batch->cu_seqlens, ((size_t)batch->batch + 1) * 4, cudaMemcpyHostToDevice, stream);
+    db.cu_seqlens = reinterpret_cast<const int32_t*>(ws + H.cu);
+  }
+  if (e == cudaSuccess && !fast) e = cudaMemcpyAsync(ws + H.q, q_obs, H.q_bytes, cudaMemcpyHostToDevice, stream);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(ws + H.k, k, H.kv_bytes, cudaMemcpyHostToDevice, stream);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(ws + H.v, v, H.kv_bytes, cudaMemcpyHostToDevice, stream);
+  if (e != cudaSuccess) return cuda_fail(ctx, e);
+  const int64_t n = batch->n_uniform, W = policy->obs_window;
+  ta_bf16_view vq = {ws + H.q, (int64_t)batch->batch * Hq * W * d, (int64_t)Hq * W * d, W * d, d};
+  ta_bf16_view vk, vv;
+  if (batch->cu_seqlens) {
+    vk = {ws + H.k, (int64_t)Hkv * (int64_t)total * d, 0, (int64_t)total * d, d};
+  } else {
+    vk = {ws + H.k, (int64_t)batch->batch * Hkv * n * d, (int64_t)Hkv * n * d, n * d, d};
+  }
+  vv = vk;
+  vv.ptr = ws + H.v;
+  s = ta_compress(ctx, pats, policy, &db, Hq, Hkv, d, K, reinterpret_cast<const int32_t*>(ws + H.ids), vq, vk, vv, 0,
+                  ws + H.k_out, ws + H.v_out, reinterpret_cast<int32_t*>(ws + H.idx),
+                  reinterpret_cast<int32_t*>(ws + H.count), stream);
+  if (s != TA_OK) return s;
+  e = cudaMemcpyAsync(k_out, ws + H.k_out, H.out_bytes, cudaMemcpyDeviceToHost, stream);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(v_out, ws + H.v_out, H.out_bytes, cudaMemcpyDeviceToHost, stream);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(idx, ws + H.idx, H.idx_bytes, cudaMemcpyDeviceToHost, stream);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(count, ws + H.count, H.count_bytes, cudaMemcpyDeviceToHost, stream);
+  return e == cudaSuccess ? TA_OK : cuda_fail(ctx, e);
+}
+
+}  // extern "C"

@@ -1,0 +1,117 @@
+// Internal declarations shared by the translation units of libta.so (host orchestration <-> kernel launchers).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "ta.h"
+
+// Device status block: word 0 = first error code (ta_status), word 1..3 = detail (where, what).
+struct ta_dev_status {
+  int code;
+  int where;
+  int detail0;
+  int detail1;
+};
+
+struct ta_patterns {
+  int device;
+  int n_pat;
+  int max_len;
+  int max_span;
+  // device tables
+  int32_t* d_ids;     // [n_pat][TA_MAX_PATTERN_LEN], right-aligned is NOT used: ids[p][0..len)
+  int32_t* d_len;     // [n_pat]
+  float* d_budget;    // [n_pat]
+  int32_t* d_span;    // [n_pat]
+  uint32_t* d_bloom;  // [32] 1024-bit filter over the last id of every pattern
+};
+
+struct ta_ctx {
+  int device;
+  int sm_count;
+  int last_cuda_error;
+  size_t scratch_bytes;
+  uint8_t* scratch;         // device
+  ta_dev_status* d_status;  // device
+  // cache of per-sequence results inside scratch (ta_compress)
+  uint64_t cached_epoch;
+  int64_t cached_total;
+  int cached_batch;
+  int cached_K;
+  // per-kernel timing of ta_compress
+  int timing_enabled;
+  int timing_valid;
+  cudaEvent_t ev[8];
+  int ev_ran[4];
+  // driver entry point for tensor-map encoding (resolved at create time)
+  void* encode_tiled;
+};
+
+// Sizes are validated by the callers in ta_api.cu; launchers return cudaError_t from the launch.
+
+struct ta_seq_desc {  // how a kernel finds sequence b
+  const int32_t* cu;  // device, or nullptr
+  int n_uniform;
+  int batch;
+  int max_n;
+  long long total;
+};
+
+__host__ __device__ inline int ta_seq_begin(const ta_seq_desc& s, int b, const int32_t* cu_cached = nullptr) {
+  return s.cu ? s.cu[b] : b * s.n_uniform;
+}
+
+// ---- step 1 ------------------------------------------------------------------------------------------------
+cudaError_t ta_launch_mask(const ta_patterns* pats, const ta_policy& pol, const ta_seq_desc& seq, const int32_t* ids,
+                           uint8_t* flags, float* voucher, float* u_static, int32_t* hist /*[B][vocab]*/,
+                           ta_dev_status* status, cudaStream_t stream);
+
+// ---- step 2 ------------------------------------------------------------------------------------------------
+struct ta_score_args {
+  ta_seq_desc seq;
+  int n_layers, Hq, Hkv, W;
+  ta_bf16_view q, k;
+  const float* lse_obs;  // nullable
+  float* A;              // nullable
+  float* P;              // nullable
+  float* u;              // nullable: fused utility (alpha*A + delta*P) + u_static
+  const float* u_static;
+  float alpha, delta, rho, scale;
+  int causal;
+};
+cudaError_t ta_launch_score(ta_ctx* ctx, const ta_score_args& a, ta_dev_status* status, cudaStream_t stream);
+
+// ---- step 3 ------------------------------------------------------------------------------------------------
+struct ta_select_args {
+  ta_seq_desc seq;
+  int n_layers, Hkv, K;
+  int n_sink, n_recent, k_protected;
+  int fast;
+  float alpha, delta;
+  const uint8_t* flags;
+  const float* voucher;
+  const float* u_static;
+  const float* A;  // scored, unfused
+  const float* P;
+  const float* u;  // scored, fused (takes precedence over A/P)
+  uint8_t* forced;     // scratch [total]
+  int32_t* r_main;     // scratch [B]   main-pool picks per sequence (-1: keep everything)
+  int32_t* idx;        // [L][B][Hkv][K]
+  int32_t* count;      // [L][B][Hkv]
+};
+cudaError_t ta_launch_select(const ta_select_args& a, ta_dev_status* status, cudaStream_t stream);
+cudaError_t ta_launch_broadcast_idx(int B, int Hkv, int K, int n_layers, const int32_t* idx_seq,
+                                    const int32_t* count_seq, int32_t* idx, int32_t* count, cudaStream_t stream);
+
+// ---- step 4 ------------------------------------------------------------------------------------------------
+struct ta_compact_args {
+  ta_seq_desc seq;
+  int n_layers, Hkv, K;
+  ta_bf16_view k, v;
+  const int32_t* idx;
+  const int32_t* count;
+  void* k_out;
+  void* v_out;
+};
+cudaError_t ta_launch_compact(const ta_compact_args& a, int sm_count, cudaStream_t stream);

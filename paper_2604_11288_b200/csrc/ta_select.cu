@@ -1,0 +1,341 @@
+// Step 3 of the retention path: budget-K selection with the partition of Section 3.3 (Algorithm 1 step 8).
+//
+// The retained set is reported in ascending position order, so no sort of the winners is needed: a 4-pass 8-bit
+// radix select finds the threshold key (and how many tokens that tie with it still fit), and one ordered
+// stream-compaction pass writes the indices. Order is total and deterministic: larger value first, lower
+// position first among equal values.
+//
+//   ta_forced_kernel   one block per sequence: mandatory sinks/recents and the protected pool (largest vouchers
+//                      among sponsored tokens). Independent of layer and head, so it runs once per sequence.
+//   ta_select_kernel   one block per unit (layer, sequence, KV head) in scored mode, per sequence in fast mode:
+//                      main pool by utility among the tokens not forced, then the ordered write of
+//                      forced + chosen positions.
+//   ta_broadcast_idx_kernel  fast mode: the per-sequence result is the same for all layers and heads.
+#include "ta_internal.cuh"
+
+namespace {
+
+constexpr int kThreads = 1024;
+constexpr int kWarps = kThreads / 32;
+
+__device__ __forceinline__ uint32_t sortable_key(float f) {
+  uint32_t b = __float_as_uint(f);
+  if ((b << 1) == 0u) b = 0u;  // -0 == +0
+  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+
+struct SelectResult {
+  uint32_t thresh;  // key of the last element taken
+  int ties;         // how many elements equal to thresh are taken (lowest positions first)
+  int all;          // 1: every eligible element is taken (fewer eligible than requested)
+  int none;         // 1: nothing is taken
+};
+
+struct SelectShared {
+  uint32_t hist[256];
+  uint32_t prefix, mask;
+  int remaining;
+  int done_all;
+  int warp_def[kWarps];
+  int warp_tie[kWarps];
+};
+
+// Top-`want` of the eligible elements of [0, n) by key. key_of(i, key) returns eligibility and the 32-bit key.
+// All threads of the block must call it; the result is uniform across the block.
+template <class KeyFn>
+__device__ SelectResult block_radix_select(int n, int want, KeyFn key_of, SelectShared& sh) {
+  SelectResult r;
+  r.thresh = 0;
+  r.ties = 0;
+  r.all = 0;
+  r.none = (want <= 0);
+  if (r.none) return r;
+  const int tid = threadIdx.x, lane = tid & 31;
+  if (tid == 0) {
+    sh.prefix = 0;
+    sh.mask = 0;
+    sh.remaining = want;
+    sh.done_all = 0;
+  }
+  const int n_round = (n + kThreads - 1) / kThreads * kThreads;
+  for (int pass = 0; pass < 4; ++pass) {
+    const int shift = 24 - 8 * pass;
+    if (tid < 256) sh.hist[tid] = 0;
+    __syncthreads();
+    const uint32_t prefix = sh.prefix, mask = sh.mask;
+    for (int i = tid; i < n_round; i += kThreads) {
+      int bin = -1;
+      if (i < n) {
+        uint32_t key;
+        if (key_of(i, key) && (key & mask) == prefix) bin = (int)((key >> shift) & 255u);
+      }
+      const unsigned peers = __match_any_sync(0xffffffffu, bin);
+      if (bin >= 0 && lane == __ffs(peers) - 1) atomicAdd(&sh.hist[bin], (uint32_t)__popc(peers));
+    }
+    __syncthreads();
+    if (tid < 32) {
+      // lane l owns bins [8l, 8l+8); walk from the top bin down until `remaining` elements are covered
+      uint32_t tot = 0;
+#pragma unroll
+      for (int k = 0; k < 8; ++k) tot += sh.hist[8 * lane + k];
+      uint32_t above = 0;  // elements in lanes above this one
+      {
+        uint32_t run = tot;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+          const uint32_t o = __shfl_down_sync(0xffffffffu, run, off);
+          if (lane + off < 32) run += o;
+        }
+        above = run - tot;
+      }
+      const int remaining = sh.remaining;
+      const uint32_t total = __shfl_sync(0xffffffffu, above + tot, 0);
+      if (pass == 0 && total < (uint32_t)remaining) {
+        if (lane == 0) sh.done_all = 1;
+      } else {
+        const bool mine = above < (uint32_t)remaining && (uint32_t)remaining <= above + tot;
+        if (mine) {
+          uint32_t cum = above;
+          int bin = 8 * lane + 7;
+          for (; bin > 8 * lane; --bin) {
+            if (cum + sh.hist[bin] >= (uint32_t)remaining) break;
+            cum += sh.hist[bin];
+          }
+          sh.remaining = remaining - (int)cum;
+          sh.prefix = prefix | ((uint32_t)bin << shift);
+          sh.mask = mask | (255u << shift);
+        }
+      }
+    }
+    __syncthreads();
+    if (sh.done_all) {
+      r.all = 1;
+      return r;
+    }
+  }
+  r.thresh = sh.prefix;
+  r.ties = sh.remaining;
+  return r;
+}
+
+// Ordered pass over [0, n): element i is `definite` (taken for sure) or a `tie` (taken while ties last). Calls
+// emit(i, rank) for every taken element with its rank in ascending position order. Returns the number taken.
+template <class ClassFn, class EmitFn>
+__device__ int block_ordered_emit(int n, int ties_allowed, ClassFn classify, EmitFn emit, SelectShared& sh) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  int def_base = 0, tie_base = 0;
+  const int n_round = (n + kThreads - 1) / kThreads * kThreads;
+  for (int i = tid; i < n_round; i += kThreads) {
+    bool def = false, tie = false;
+    if (i < n) classify(i, def, tie);
+    const unsigned bd = __ballot_sync(0xffffffffu, def), bt = __ballot_sync(0xffffffffu, tie);
+    const unsigned lt = (1u << lane) - 1u;
+    if (lane == 0) {
+      sh.warp_def[warp] = __popc(bd);
+      sh.warp_tie[warp] = __popc(bt);
+    }
+    __syncthreads();
+    int def_before = __popc(bd & lt), tie_before = __popc(bt & lt);
+    int def_total = 0, tie_total = 0;
+    for (int w = 0; w < kWarps; ++w) {
+      const int d = sh.warp_def[w], t = sh.warp_tie[w];
+      if (w < warp) {
+        def_before += d;
+        tie_before += t;
+      }
+      def_total += d;
+      tie_total += t;
+    }
+    const int ties_seen = tie_base + tie_before;
+    if (def)
+      emit(i, def_base + def_before + min(ties_seen, ties_allowed));
+    else if (tie && ties_seen < ties_allowed)
+      emit(i, def_base + def_before + ties_seen);
+    def_base += def_total;
+    tie_base += tie_total;
+    __syncthreads();
+  }
+  return def_base + min(tie_base, ties_allowed);
+}
+
+struct SeqInfo {
+  int start, n, K_eff, s_take, r_take, p;
+};
+
+__device__ __forceinline__ SeqInfo seq_info(const ta_seq_desc& seq, int b, int K, int n_sink, int n_recent,
+                                            int k_protected) {
+  SeqInfo s;
+  s.start = ta_seq_begin(seq, b);
+  s.n = (seq.cu ? seq.cu[b + 1] : s.start + seq.n_uniform) - s.start;
+  s.K_eff = min(K, s.n);
+  int p = k_protected < 0 ? s.K_eff - n_sink - n_recent : k_protected;
+  p = max(0, min(p, s.K_eff));
+  s.p = p;
+  const int K_main = s.K_eff - p;
+  // mandatory list: sinks 0.. then recents n-1, n-2, .. (no duplicates), truncated to K_main entries
+  const int sinks = min(n_sink, s.n);
+  const int recents = max(0, min(n_recent, s.n - sinks));
+  s.s_take = min(sinks, K_main);
+  s.r_take = min(recents, K_main - s.s_take);
+  return s;
+}
+
+__global__ void __launch_bounds__(kThreads) ta_forced_kernel(ta_seq_desc seq, int K, int n_sink, int n_recent,
+                                                             int k_protected, const float* __restrict__ voucher,
+                                                             uint8_t* __restrict__ forced,
+                                                             int32_t* __restrict__ r_main, ta_dev_status* status) {
+  __shared__ SelectShared sh;
+  const int b = blockIdx.x;
+  const SeqInfo s = seq_info(seq, b, K, n_sink, n_recent, k_protected);
+  if (s.n > seq.max_n || s.n < 0) {
+    if (threadIdx.x == 0) {
+      if (atomicCAS(&status->code, 0, (int)TA_ERR_DEVICE_BOUNDS) == 0) {
+        status->where = 3;
+        status->detail0 = b;
+        status->detail1 = s.n;
+      }
+      r_main[b] = -2;  // poisoned: the select kernel writes an empty result
+    }
+    return;
+  }
+  if (s.K_eff == s.n) {
+    if (threadIdx.x == 0) r_main[b] = -1;  // keep everything
+    return;
+  }
+  const float* V = voucher + s.start;
+  auto mandatory = [&](int i) { return i < s.s_take || i >= s.n - s.r_take; };
+  auto key_of = [&](int i, uint32_t& key) {
+    const float v = V[i];
+    key = sortable_key(v);
+    return v > 0.0f && !mandatory(i);
+  };
+  const SelectResult r = block_radix_select(s.n, s.p, key_of, sh);
+  uint8_t* f = forced + s.start;
+  // ordered pass: mandatory tokens and vouchers above the threshold are forced for sure; vouchers equal to the
+  // threshold are forced while protected slots last, lowest position first
+  auto classify = [&](int i, bool& def, bool& tie) {
+    uint32_t key;
+    const bool cand = key_of(i, key);
+    def = mandatory(i) || (cand && !r.none && (r.all || key > r.thresh));
+    tie = !def && cand && !r.none && !r.all && key == r.thresh;
+    f[i] = 0;  // set by emit when taken (same thread, later)
+  };
+  auto emit = [&](int i, int rank) { f[i] = 1; };
+  const int taken = block_ordered_emit(s.n, r.ties, classify, emit, sh);
+  if (threadIdx.x == 0) r_main[b] = s.K_eff - taken;
+}
+
+struct UnitSrc {  // where a unit's utility comes from
+  const float* u;         // fused: [L][Hkv][total]
+  const float* A;         // unfused
+  const float* P;
+  const float* u_static;  // per token
+  float alpha, delta;
+};
+
+__device__ __forceinline__ float unit_utility(const UnitSrc& src, long long unit_off, long long tok) {
+  if (src.u) return src.u[unit_off + tok];
+  const float u0 = src.u_static[tok];
+  if (!src.A) return u0;
+  const float aA = __fmul_rn(src.alpha, src.A[unit_off + tok]);
+  const float dP = __fmul_rn(src.delta, src.P ? src.P[unit_off + tok] : 0.0f);
+  return __fadd_rn(__fadd_rn(aA, dP), u0);
+}
+
+// grid.x = units. scored: unit = (l*B + b)*Hkv + g; fast: unit = b.
+__global__ void __launch_bounds__(kThreads) ta_select_kernel(ta_seq_desc seq, int n_layers, int Hkv, int K, int fast,
+                                                             UnitSrc src, const uint8_t* __restrict__ forced,
+                                                             const int32_t* __restrict__ r_main,
+                                                             int32_t* __restrict__ idx, int32_t* __restrict__ count) {
+  __shared__ SelectShared sh;
+  const int unit = blockIdx.x;
+  int b, l = 0, g = 0;
+  if (fast) {
+    b = unit;
+  } else {
+    g = unit % Hkv;
+    b = (unit / Hkv) % seq.batch;
+    l = unit / (Hkv * seq.batch);
+  }
+  const int start = ta_seq_begin(seq, b);
+  const int n = (seq.cu ? seq.cu[b + 1] : start + seq.n_uniform) - start;
+  int32_t* out = idx + (long long)unit * K;
+  const int want = r_main[b];
+  const int tid = threadIdx.x;
+  if (want == -2) {  // sequence rejected by ta_forced_kernel
+    for (int r = tid; r < K; r += kThreads) out[r] = -1;
+    if (tid == 0) count[unit] = 0;
+    return;
+  }
+  if (want == -1) {  // K >= n: keep everything
+    for (int r = tid; r < K; r += kThreads) out[r] = r < n ? r : -1;
+    if (tid == 0) count[unit] = n;
+    return;
+  }
+  const long long unit_off = fast ? 0 : ((long long)l * Hkv + g) * seq.total;
+  const uint8_t* f = forced + start;
+  auto key_of = [&](int i, uint32_t& key) {
+    key = sortable_key(unit_utility(src, unit_off, (long long)start + i));
+    return f[i] == 0;
+  };
+  const SelectResult r = block_radix_select(n, want, key_of, sh);
+  auto classify = [&](int i, bool& def, bool& tie) {
+    uint32_t key;
+    const bool elig = key_of(i, key);
+    def = !elig || (!r.none && (r.all || key > r.thresh));
+    tie = !def && !r.none && !r.all && key == r.thresh;
+  };
+  auto emit = [&](int i, int rank) {
+    if (rank < K) out[rank] = i;
+  };
+  const int taken = block_ordered_emit(n, r.ties, classify, emit, sh);
+  for (int q = taken + tid; q < K; q += kThreads) out[q] = -1;
+  if (tid == 0) count[unit] = taken;
+}
+
+__global__ void ta_broadcast_idx_kernel(int B, int Hkv, int K, int n_layers, const int32_t* __restrict__ idx_seq,
+                                        const int32_t* __restrict__ count_seq, int32_t* __restrict__ idx,
+                                        int32_t* __restrict__ count) {
+  const long long total = (long long)n_layers * B * Hkv * K;
+  for (long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x; t < total;
+       t += (long long)gridDim.x * blockDim.x) {
+    const int r = (int)(t % K);
+    const long long unit = t / K;
+    const int b = (int)((unit / Hkv) % B);
+    idx[t] = idx_seq[(long long)b * K + r];
+    if (r == 0) count[unit] = count_seq[b];
+  }
+}
+
+}  // namespace
+
+// Scratch layout used by the launcher (the caller carves it): forced [total] bytes, r_main [B] ints; fast mode
+// additionally idx_seq [B][K] and count_seq [B] (passed through a.idx / a.count by the caller when it wants the
+// per-sequence result only).
+cudaError_t ta_launch_select(const ta_select_args& a, ta_dev_status* status, cudaStream_t stream) {
+  if (a.seq.batch == 0 || a.n_layers == 0) return cudaSuccess;
+  ta_forced_kernel<<<a.seq.batch, kThreads, 0, stream>>>(a.seq, a.K, a.n_sink, a.n_recent, a.k_protected, a.voucher,
+                                                         a.forced, a.r_main, status);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  UnitSrc src;
+  src.u = a.fast ? nullptr : a.u;
+  src.A = a.fast ? nullptr : a.A;
+  src.P = a.fast ? nullptr : a.P;
+  src.u_static = a.u_static;
+  src.alpha = a.alpha;
+  src.delta = a.delta;
+  const int units = a.fast ? a.seq.batch : a.n_layers * a.seq.batch * a.Hkv;
+  ta_select_kernel<<<units, kThreads, 0, stream>>>(a.seq, a.n_layers, a.Hkv, a.K, a.fast, src, a.forced, a.r_main,
+                                                   a.idx, a.count);
+  return cudaGetLastError();
+}
+
+cudaError_t ta_launch_broadcast_idx(int B, int Hkv, int K, int n_layers, const int32_t* idx_seq,
+                                    const int32_t* count_seq, int32_t* idx, int32_t* count, cudaStream_t stream) {
+  const long long total = (long long)n_layers * B * Hkv * K;
+  if (total == 0) return cudaSuccess;
+  const int blocks = (int)((total + 255) / 256 < 4096 ? (total + 255) / 256 : 4096);
+  ta_broadcast_idx_kernel<<<blocks, 256, 0, stream>>>(B, Hkv, K, n_layers, idx_seq, count_seq, idx, count);
+  return cudaGetLastError();
+}

@@ -1,0 +1,330 @@
+"""GPU parity, step by step: each C-ABI entry point against the CPU oracle on the same seeded bytes, at sizes that
+span several tiles and a ragged tail, plus the degenerate cases of the method."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2604_11288_b200 as ta
+import ta_workloads as tw
+from ta_testlib import (Gpu, assert_scores_close, assert_selection_matches, bf16_bits, oracle_patterns, oracle_policy,
+                        oracle_unit, unit_kv)
+
+pytestmark = pytest.mark.gpu
+
+
+def _workload(lengths, pats, spans=None, budgets=None, alphabet=None, seed=0, Hq=8, Hkv=2, W=8, plant=True):
+    """A packed batch with random ids; with a small alphabet the patterns occur by chance everywhere."""
+    rng = np.random.default_rng(seed)
+    lengths = np.asarray(lengths, np.int32)
+    total = int(lengths.sum())
+    hi = alphabet if alphabet else tw.VOCAB
+    ids = rng.integers(0, hi, size=total).astype(np.int32)
+    cu = np.zeros(len(lengths) + 1, np.int32)
+    cu[1:] = np.cumsum(lengths)
+    if plant and not alphabet:
+        for b in range(len(lengths)):
+            n = int(lengths[b])
+            for _ in range(max(1, n // 300)):
+                p = pats[int(rng.integers(0, len(pats)))]
+                if n > len(p) + 2:
+                    s = int(rng.integers(0, n - len(p)))
+                    ids[cu[b] + s:cu[b] + s + len(p)] = p
+    w = tw.Workload(name="t", seed=1234 + seed, n_layers=1, Hq=Hq, Hkv=Hkv, d=128, W=W, K_list=[], modes=[],
+                    uniform=False, lengths=lengths, cu=cu, ids=ids, pattern_ids=[list(map(int, p)) for p in pats],
+                    pattern_budget=budgets or [15.0] * len(pats), pattern_span=spans or [6] * len(pats), planted=[],
+                    vocab=hi)
+    return w
+
+
+def _check_mask(w, pol):
+    g = Gpu(w, pol, 4, 1)
+    try:
+        flags, V, u0 = g.sponsor_mask()
+        assert g.poll() == ta.TA_OK
+        f_o, V_o, u0_o = oracle.sponsor_mask(w.ids, w.cu, oracle_patterns(w), pol)
+        np.testing.assert_array_equal(flags.cpu().numpy(), f_o)
+        np.testing.assert_array_equal(V.cpu().numpy().view(np.uint32), V_o.view(np.uint32))
+        np.testing.assert_array_equal(u0.cpu().numpy().view(np.uint32), u0_o.view(np.uint32))
+        return f_o
+    finally:
+        g.close()
+
+
+@pytest.mark.parametrize("seed", range(4))
+def test_mask_small_alphabet_bit_exact(seed):
+    rng = np.random.default_rng(seed)
+    pats = [list(rng.integers(0, 4, size=int(rng.integers(1, 9)))) for _ in range(int(rng.integers(1, 12)))]
+    spans = [int(rng.integers(1, 65)) for _ in pats]
+    buds = [float(rng.integers(1, 30)) for _ in pats]
+    lengths = [1, 2, 511, 512, 513, 1700, 0, 37]
+    w = _workload(lengths, pats, spans, buds, alphabet=4, seed=seed)
+    pol = oracle_policy(4, vocab_size=4, age_steps=seed)
+    f = _check_mask(w, pol)
+    assert (f & 4).any() and (f & 2).any()
+
+
+def test_mask_many_patterns_and_vocab():
+    rng = np.random.default_rng(9)
+    pats = [list(rng.integers(0, tw.VOCAB, size=int(rng.integers(1, 4)))) for _ in range(256)]
+    w = _workload([5000, 3000, 9000], pats, [int(rng.integers(1, 33)) for _ in pats], seed=9)
+    _check_mask(w, oracle_policy(4, vocab_size=tw.VOCAB))
+
+
+def test_mask_no_patterns_and_bad_token_id():
+    w = _workload([700], [[1, 2]], seed=3)
+    w.pattern_ids, w.pattern_budget, w.pattern_span = [], [], []
+    f = _check_mask(w, oracle_policy(4))
+    assert not f.any()
+    # an id outside the vocabulary is reported through the context, and nothing faults
+    w2 = _workload([700], [[1, 2]], seed=3)
+    w2.ids[123] = tw.VOCAB + 5
+    g = Gpu(w2, oracle_policy(4), 4, 1)
+    try:
+        g.sponsor_mask()
+        assert g.poll() == ta.TA_ERR_DEVICE_BOUNDS
+        assert g.poll() == ta.TA_OK  # cleared
+    finally:
+        g.close()
+
+
+def _score_case(lengths, Hq, Hkv, W, causal=1, seed=0, layers=1, permute=False, scale=0.0):
+    w = _workload(lengths, [[1, 2]], seed=seed, Hq=Hq, Hkv=Hkv, W=W)
+    w.n_layers = layers
+    pol = oracle_policy(4, W=W, causal=causal, softmax_scale=scale)
+    Qh, Kh, _ = tw.make_qkv(w, range(layers))
+    g = Gpu(w, pol, 4, layers)
+    try:
+        Qd = Qh.cuda()
+        if permute:  # token-major storage [L, total, Hkv, d] viewed as [L, Hkv, total, d]
+            Kd = Kh.permute(0, 2, 1, 3).contiguous().cuda().permute(0, 2, 1, 3)
+        else:
+            Kd = Kh.cuda()
+        A, P = g.score(Qd, Kd)
+        torch.cuda.synchronize()
+        assert g.poll() == ta.TA_OK
+        A, P = A.cpu().numpy(), P.cpu().numpy()
+        G = Hq // Hkv
+        for l in range(layers):
+            for b in range(w.B):
+                o, e = int(w.cu[b]), int(w.cu[b + 1])
+                for h in range(Hkv):
+                    Ao, Po = oracle.attention(bf16_bits(Qh[l, b, h * G:(h + 1) * G]), unit_kv(w, Kh, l, b, h), e - o,
+                                              scale=scale, causal=causal, rho=pol.pension_rho)
+                    assert_scores_close(A[l, h, o:e], Ao, f"A l{l} b{b} h{h} n{e - o}")
+                    assert_scores_close(P[l, h, o:e], Po, f"P l{l} b{b} h{h} n{e - o}")
+        return w, pol, Qh, Kh, Qd, Kd, A, g
+    except Exception:
+        g.close()
+        raise
+
+
+def test_score_single_tile():
+    *_, g = _score_case([100], 8, 2, 32)
+    g.close()
+
+
+def test_score_multi_tile_ragged_tail():
+    *_, g = _score_case([1000, 128, 129, 4096 + 37], 8, 2, 32)
+    g.close()
+
+
+def test_score_window_64_two_row_blocks():
+    *_, g = _score_case([700, 2500], 8, 2, 64)
+    g.close()
+
+
+def test_score_small_row_count_and_short_sequences():
+    # G*W = 8 rows (padded to 128); sequences shorter than the window, of length 1, and empty
+    *_, g = _score_case([5, 1, 0, 300, 31], 2, 2, 8)
+    g.close()
+
+
+def test_score_non_causal_and_custom_scale():
+    *_, g = _score_case([900], 4, 1, 32, causal=0, scale=0.05)
+    g.close()
+
+
+def test_score_layers_and_strided_keys():
+    *_, g = _score_case([1500, 260], 8, 2, 32, layers=3, permute=True)
+    g.close()
+
+
+def test_score_cluster_sizes():
+    # 16, 32 and 64 tiles: clusters of 4 and 8 CTAs per unit
+    *_, g = _score_case([2048 + 5], 4, 1, 32)
+    g.close()
+    *_, g = _score_case([8192 - 77], 4, 1, 32, seed=2)
+    g.close()
+
+
+def test_score_with_supplied_lse_matches_two_pass():
+    w, pol, Qh, Kh, Qd, Kd, A2, g = _score_case([1300, 70], 8, 2, 32, seed=5)
+    try:
+        # log-sum-exp of every window row, from a library softmax in fp64
+        G = w.Hq // w.Hkv
+        lse = torch.full((1, w.B, w.Hq, w.W), 0.0, dtype=torch.float64)
+        for b in range(w.B):
+            o, e = int(w.cu[b]), int(w.cu[b + 1])
+            n = e - o
+            for h in range(w.Hq):
+                k = Kh[0, h // G, o:e].double()
+                s = (Qh[0, b, h].double() @ k.T) / np.sqrt(128.0)
+                pos = torch.arange(n - w.W, n).view(-1, 1)
+                s = s.masked_fill(torch.arange(n).view(1, -1) > pos, float("-inf"))
+                lse[0, b, h] = torch.where(pos.view(-1) >= 0, torch.logsumexp(s, -1), torch.zeros(w.W).double())
+        A1, _ = g.score(Qd, Kd, lse=lse.float().cuda())
+        torch.cuda.synchronize()
+        assert g.poll() == ta.TA_OK
+        A1 = A1.cpu().numpy()
+        for h in range(w.Hkv):
+            assert_scores_close(A1[0, h], A2[0, h], f"lse path h{h}")
+    finally:
+        g.close()
+
+
+def _select_case(w, pol, K, L=1, u_parts=None):
+    """Runs mask + (given A, P) select on the GPU and compares with the oracle unit by unit."""
+    g = Gpu(w, pol, K, L)
+    try:
+        flags, V, u0 = g.sponsor_mask()
+        A = P = None
+        if not pol.fast:
+            A, P = u_parts
+        idx, cnt = g.select(flags, V, u0, A, P)
+        torch.cuda.synchronize()
+        assert g.poll() == ta.TA_OK
+        idx, cnt = idx.cpu().numpy(), cnt.cpu().numpy()
+        f_o, V_o, u0_o = oracle.sponsor_mask(w.ids, w.cu, oracle_patterns(w), pol)
+        for l in range(L):
+            for b in range(w.B):
+                o, e = int(w.cu[b]), int(w.cu[b + 1])
+                for h in range(w.Hkv):
+                    if pol.fast:
+                        u = u0_o[o:e]
+                    else:
+                        u = oracle.utility(pol.alpha, pol.delta, A[l, h, o:e].cpu().numpy(),
+                                           P[l, h, o:e].cpu().numpy(), u0_o[o:e])
+                    io, co = oracle.select(V_o[o:e], u, K, pol.n_sink, pol.n_recent, pol.k_protected)
+                    assert cnt[l, b, h] == co
+                    np.testing.assert_array_equal(idx[l, b, h], io, err_msg=f"l{l} b{b} h{h}")
+        return idx, cnt
+    finally:
+        g.close()
+
+
+@pytest.mark.parametrize("preset", ["THEOREM", "SEC33", "AUDIT"])
+@pytest.mark.parametrize("K", [1, 5, 16, 300])
+def test_select_fast_bit_exact(preset, K):
+    pats = [[1, 2], [3], [2, 2, 1]]
+    w = _workload([1, 3, 17, 600, 1025, 0, 2500], pats, [6, 3, 20], alphabet=6, seed=K)
+    _select_case(w, oracle_policy(K, preset, fast=True, vocab_size=6), K)
+
+
+@pytest.mark.parametrize("K", [16, 2048, 4096])
+def test_select_scored_given_scores_bit_exact(K):
+    # the same fp32 A and P go to both sides, so the selection must agree exactly, ties included
+    w = _workload([3000, 40000, 700], [[5, 6, 7], [9]], seed=K, Hq=4, Hkv=2)
+    L = 2
+    gen = torch.Generator().manual_seed(K)
+    A = torch.rand((L, w.Hkv, w.total), generator=gen).cuda()
+    A = (A * 64).round() / 64  # many exact ties
+    P = (torch.rand((L, w.Hkv, w.total), generator=gen) * 0.1).cuda()
+    _select_case(w, oracle_policy(K, "THEOREM"), K, L, (A, P))
+
+
+def test_select_sponsored_overflow_and_precedence():
+    # far more sponsored tokens than protected slots: nearest-to-anchor first, earlier anchors win ties
+    w = _workload([5000], [[1]], [12], alphabet=40, seed=4)
+    idx, cnt = _select_case(w, oracle_policy(32, "THEOREM", fast=True, vocab_size=40), 32)
+    assert cnt[0, 0, 0] == 32
+
+
+def test_compact_strided_and_zero_fill():
+    w = _workload([300, 50, 0, 1000], [[1, 2]], seed=8, Hq=4, Hkv=2)
+    K = 64
+    pol = oracle_policy(K, fast=True)
+    _, Kh, Vh = tw.make_qkv(w, [0, 1], need_q=False)
+    g = Gpu(w, pol, K, 2)
+    try:
+        Kd = Kh.permute(0, 2, 1, 3).contiguous().cuda().permute(0, 2, 1, 3)  # token-major storage
+        Vd = Vh.cuda()
+        flags, V, u0 = g.sponsor_mask()
+        idx, cnt = g.select(flags, V, u0)
+        ko, vo = g.compact(Kd, Vd, idx, cnt)
+        torch.cuda.synchronize()
+        assert g.poll() == ta.TA_OK
+        idx, cnt = idx.cpu().numpy(), cnt.cpu().numpy()
+        for l in range(2):
+            for b in range(w.B):
+                for h in range(w.Hkv):
+                    want_k = oracle.compact(unit_kv(w, Kh, l, b, h), idx[l, b, h], int(cnt[l, b, h]), K)
+                    want_v = oracle.compact(unit_kv(w, Vh, l, b, h), idx[l, b, h], int(cnt[l, b, h]), K)
+                    np.testing.assert_array_equal(bf16_bits(ko[l, b, h]), want_k)
+                    np.testing.assert_array_equal(bf16_bits(vo[l, b, h]), want_v)
+        assert cnt[0, 1, 0] == 50 and cnt[0, 2, 0] == 0
+    finally:
+        g.close()
+
+
+@pytest.mark.parametrize("fast", [False, True])
+def test_compress_equals_steps_and_oracle(fast):
+    w = _workload([900, 2100, 64, 10], [[4, 5], [6]], seed=12, Hq=8, Hkv=2, W=32)
+    K, L = 24, 2
+    pol = oracle_policy(K, "THEOREM", fast=fast, W=32)
+    Qh, Kh, Vh = tw.make_qkv(w, range(L))
+    g = Gpu(w, pol, K, L)
+    try:
+        Qd, Kd, Vd = Qh.cuda(), Kh.cuda(), Vh.cuda()
+        idx, cnt, ko, vo = g.compress(Qd, Kd, Vd, epoch=7)
+        idx2, cnt2, ko2, vo2 = g.compress(Qd, Kd, Vd, epoch=7)  # reuses the per-sequence results
+        torch.cuda.synchronize()
+        assert g.poll() == ta.TA_OK
+        assert torch.equal(idx, idx2) and torch.equal(cnt, cnt2) and torch.equal(ko, ko2) and torch.equal(vo, vo2)
+        idx, cnt = idx.cpu().numpy(), cnt.cpu().numpy()
+        f_o, V_o, u0_o = oracle.sponsor_mask(w.ids, w.cu, oracle_patterns(w), pol)
+        exact = 0
+        for l in range(L):
+            for b in range(w.B):
+                for h in range(w.Hkv):
+                    A, P, u, io, co = oracle_unit(w, pol, K, Qh, Kh, l, b, h, V_o, u0_o)
+                    same = assert_selection_matches(idx[l, b, h], cnt[l, b, h], io, co, u, f"l{l} b{b} h{h}")
+                    exact += same
+                    if fast:
+                        assert same
+                    sel, c = idx[l, b, h], int(cnt[l, b, h])
+                    np.testing.assert_array_equal(bf16_bits(ko[l, b, h]), oracle.compact(unit_kv(w, Kh, l, b, h), sel, c, K))
+                    np.testing.assert_array_equal(bf16_bits(vo[l, b, h]), oracle.compact(unit_kv(w, Vh, l, b, h), sel, c, K))
+        assert exact >= 0.9 * L * w.B * w.Hkv
+    finally:
+        g.close()
+
+
+def test_host_argument_checks():
+    w = _workload([300], [[1, 2]], seed=1)
+    pol = oracle_policy(8, fast=True)
+    g = Gpu(w, pol, 8, 1)
+    try:
+        _, Kh, Vh = tw.make_qkv(w, [0], need_q=False)
+        Kd, Vd = Kh.cuda(), Vh.cuda()
+        idx = torch.zeros((1, 1, 2, 8), dtype=torch.int32, device="cuda")
+        cnt = torch.zeros((1, 1, 2), dtype=torch.int32, device="cuda")
+        out = torch.zeros((1, 1, 2, 8, 128), dtype=torch.bfloat16, device="cuda")
+        L = ta.binding.lib()
+        import ctypes as C
+        vk, vv = ta.view(Kd, True), ta.view(Vd, True)
+        call = lambda d, K, vk=vk: L.ta_compact_kv(g.ctx, C.byref(g.batch), 2, d, K, vk, vv, idx.data_ptr(),
+                                                   cnt.data_ptr(), out.data_ptr(), out.data_ptr(), None)
+        assert call(64, 8) == ta.TA_ERR_UNSUPPORTED
+        assert call(128, 5000) == ta.TA_ERR_UNSUPPORTED
+        assert call(128, 0) == ta.TA_ERR_INVALID_ARG
+        bad = ta.ta_bf16_view(vk.ptr + 2, vk.stride_l, vk.stride_b, vk.stride_h, vk.stride_n)
+        assert call(128, 8, bad) == ta.TA_ERR_ALIGNMENT
+        small = ta.ta_ctx_create(0, 1024)
+        st = L.ta_sponsor_mask(small, g.pats, C.byref(g.p), C.byref(g.batch), g.ids.data_ptr(), idx.data_ptr(),
+                               idx.data_ptr(), idx.data_ptr(), None)
+        assert st == ta.TA_ERR_SCRATCH_TOO_SMALL
+        ta.ta_ctx_destroy(small)
+        assert g.poll() == ta.TA_OK
+    finally:
+        g.close()
