@@ -1,0 +1,385 @@
+#!/usr/bin/env python
+"""Benchmark of the Transactional Attention KV-cache compaction path on B200.
+
+One step = one pass of the whole path (anchor mask, vouchers, attention-free utility, attention scores, budget-K
+selection, K/V gather) over one batch of seeded synthetic input, through the library's C ABI: a single ta_compress
+call covering all layers of the workload. The metric is context tokens compressed per second per layer, i.e.
+(tokens in the batch) / (step time / layers). Prints ONE JSON line on rank 0.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2] [--budget 16] [--mode scored|fast]
+  python bench.py --impl reference   # times the CPU oracle (the only baseline there is) on a bounded sample
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+import torch  # noqa: E402
+
+import ta_workloads as tw  # noqa: E402
+
+METRIC = "context tokens compressed/sec per layer (all heads)"
+UNIT = "tokens/s"
+
+
+# ------------------------------------------------------------------------------------------------ helpers
+def measured_peak_hbm():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            return float(json.load(open(p))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs (read-only queries)."""
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "50"], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            pass
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 6:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for nm, v in zip(names, f[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def build_workload(name, budget):
+    w = tw.CONFIGS[name]()
+    K = budget if budget else w.K_list[0]
+    return w, K
+
+
+def algorithmic_bytes(w, L, K, fast):
+    """Bytes the method itself must move for one step of L layers (what a perfect implementation reads + writes)."""
+    total, B = w.total, w.B
+    k_eff = int(sum(min(K, int(n)) for n in w.lengths))
+    score = 0 if fast else L * (total * w.Hkv * w.d * 2 + B * w.Hq * w.W * w.d * 2)
+    gather = L * 2 * 2 * w.Hkv * k_eff * w.d * 2          # K and V rows, read + write
+    idx = L * w.Hkv * k_eff * 4
+    per_seq = total * (4 + 1 + 4 + 4)                     # ids, flags, voucher, static utility: once per batch
+    return {"score": score, "gather": gather + idx, "per_sequence": per_seq, "total": score + gather + idx + per_seq}
+
+
+def score_kernel_bytes(w, L):
+    """Algorithmic bytes of one launch of the scoring kernel: every key row once, the query window once, one fused
+    fp32 utility written and one static utility read per (token, KV head)."""
+    return L * (w.total * w.Hkv * (w.d * 2 + 4 + 4) + w.B * w.Hq * w.W * w.d * 2)
+
+
+# ------------------------------------------------------------------------------------------------ CPU oracle legs
+def oracle_leg(w, K, fast, budget_s=12.0, max_layers=512):
+    """Times the CPU oracle (as it stands) on whole layers of the workload until about `budget_s` seconds are
+    spent. Inputs are drawn on the CPU from the same generator family."""
+    import oracle
+    pats = oracle.Patterns(w.pattern_ids, w.pattern_budget, w.pattern_span)
+    pol = oracle.preset("THEOREM", K, fast=1 if fast else 0, obs_window=w.W)
+    sub, note = w, "all sequences"
+    macs = float(w.total) * w.Hq * w.W * w.d  # multiply-adds of one layer's score matrix
+    if macs > 2e10 and not fast:
+        # a layer of this workload is minutes of CPU work: time a subset of sequences instead
+        keep = max(1, int(w.B * 2e10 / macs))
+        sub = subset_sequences(w, keep)
+        note = f"first {keep} of {w.B} sequences"
+    bits = lambda t: t.contiguous().view(torch.int16).numpy().view(np.uint16)
+    layers, spent, t_units = 0, 0.0, 0.0
+    while layers < max_layers and spent < budget_s:
+        Q, Kc, Vc = tw.make_qkv(sub, [layers % w.n_layers], need_q=not fast)
+        t0 = time.perf_counter()
+        oracle.compress_layer(sub.ids, sub.cu, sub.uniform, sub.Hq, sub.Hkv, sub.d, K, pats, pol,
+                              None if fast else bits(Q[0]), bits(Kc[0]), bits(Vc[0]))
+        dt = time.perf_counter() - t0
+        spent += dt
+        layers += 1
+    value = sub.total * layers / spent
+    return {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"{layers} layer(s) of {w.name}, {note}, {spent:.1f} s"}, spent / layers
+
+
+def subset_sequences(w, keep):
+    import copy
+    s = copy.copy(w)
+    s.lengths = w.lengths[:keep].copy()
+    s.cu = w.cu[:keep + 1].copy()
+    s.ids = w.ids[:int(s.cu[-1])].copy()
+    return s
+
+
+# ------------------------------------------------------------------------------------------------ GPU leg
+class Runner:
+    def __init__(self, w, K, L, fast, dev):
+        import paper_2604_11288_b200 as ta
+        self.ta, self.w, self.K, self.L, self.fast, self.dev = ta, w, K, L, fast, dev
+        p = ta.ta_policy_default(ta.TA_PRESET_THEOREM, K)
+        p.obs_window = w.W
+        p.mode = ta.TA_MODE_FAST if fast else ta.TA_MODE_SCORED
+        p.vocab_size = w.vocab
+        self.p = p
+        self.ids = torch.from_numpy(w.ids).to(dev)
+        self.cu = None if w.uniform else torch.from_numpy(w.cu).to(dev)
+        self.batch = ta.make_batch(L, w.B, int(w.lengths[0]) if w.uniform else 0, w.max_n, w.total, self.cu)
+        self.ctx = ta.ta_ctx_create(dev.index, ta.ta_scratch_bytes(self.batch, w.Hq, w.Hkv, w.d, K, p))
+        self.pats = ta.ta_patterns_create(self.ctx, w.pattern_ids, w.pattern_budget, w.pattern_span)
+        self.Q, self.Kc, self.Vc = tw.make_qkv(w, range(L), device=dev, need_q=not fast)
+        self.idx = torch.empty((L, w.B, w.Hkv, K), dtype=torch.int32, device=dev)
+        self.cnt = torch.empty((L, w.B, w.Hkv), dtype=torch.int32, device=dev)
+        self.ko = torch.empty((L, w.B, w.Hkv, K, w.d), dtype=torch.bfloat16, device=dev)
+        self.vo = torch.empty_like(self.ko)
+        self.rag = not w.uniform
+        self.stream = torch.cuda.current_stream(dev).cuda_stream
+        self.vq = ta.view(self.Q) if not fast else ta.view(None)
+        self.vk, self.vv = ta.view(self.Kc, self.rag), ta.view(self.Vc, self.rag)
+
+    def step(self):
+        w = self.w
+        self.ta.ta_compress(self.ctx, self.pats, self.p, self.batch, w.Hq, w.Hkv, w.d, self.K, self.ids, self.vq,
+                            self.vk, self.vv, 0, self.ko, self.vo, self.idx, self.cnt, self.stream)
+
+    def kernels_per_step(self):
+        # mask + static utility, [score], forced + select, [broadcast], gather
+        return 2 + (0 if self.fast else 1) + 2 + (1 if self.fast else 0) + 1
+
+    def close(self):
+        self.ta.ta_patterns_destroy(self.pats)
+        self.ta.ta_ctx_destroy(self.ctx)
+
+
+def time_steps(run, steps, warmup, barrier=None):
+    for _ in range(warmup):
+        run()
+    torch.cuda.synchronize()
+    if barrier:
+        barrier()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        run()
+    e1.record()
+    torch.cuda.synchronize()
+    if barrier:
+        barrier()
+    return e0.elapsed_time(e1) / steps
+
+
+def e2e_leg(r, steps, warmup):
+    """Same step through ta_compress_host: inputs start in pinned host memory, results end there."""
+    ta, w = r.ta, r.w
+    pin = lambda t: t.cpu().pin_memory()
+    ids_h = torch.from_numpy(w.ids).pin_memory()
+    q_h = pin(r.Q) if not r.fast else None
+    k_h, v_h = pin(r.Kc), pin(r.Vc)
+    ko_h, vo_h = torch.empty(r.ko.shape, dtype=torch.bfloat16).pin_memory(), torch.empty(r.vo.shape, dtype=torch.bfloat16).pin_memory()
+    idx_h, cnt_h = torch.empty(r.idx.shape, dtype=torch.int32).pin_memory(), torch.empty(r.cnt.shape, dtype=torch.int32).pin_memory()
+    hb = ta.make_batch(r.L, w.B, int(w.lengths[0]) if w.uniform else 0, w.max_n, w.total,
+                       None if w.uniform else w.cu.ctypes.data)
+    nbytes = ta.ta_compress_host_workspace_bytes(hb, w.Hq, w.Hkv, w.d, r.K, r.p)
+    ws = torch.empty(nbytes + 256, dtype=torch.uint8, device=r.dev)
+    ws_ptr = (ws.data_ptr() + 255) // 256 * 256
+
+    def run():
+        ta.ta_compress_host(r.ctx, r.pats, r.p, hb, w.Hq, w.Hkv, w.d, r.K, ids_h, q_h, k_h, v_h, ko_h, vo_h, idx_h,
+                            cnt_h, ws_ptr, nbytes, r.stream)
+
+    ms = time_steps(run, steps, warmup)
+    h2d = ids_h.numel() * 4 + (q_h.numel() * 2 if q_h is not None else 0) + k_h.numel() * 2 + v_h.numel() * 2
+    d2h = ko_h.numel() * 2 + vo_h.numel() * 2 + idx_h.numel() * 4 + cnt_h.numel() * 4
+    ok = bool((idx_h.to(r.dev) == r.idx).all()) and bool((ko_h.to(r.dev) == r.ko).all())
+    return ms, h2d, d2h, ok
+
+
+def kernel_breakdown(r, steps):
+    """Per-stage device times of ta_compress from CUDA events recorded on the call's stream inside the library."""
+    ta = r.ta
+    ta.ta_ctx_enable_timing(r.ctx, True)
+    acc = np.zeros(5)
+    for _ in range(steps):
+        r.step()
+        acc += np.array(ta.ta_ctx_read_timing(r.ctx))
+    ta.ta_ctx_enable_timing(r.ctx, False)
+    return acc / steps
+
+
+def measure_extra(name, L, dev, steps=5, warmup=3):
+    w, K = build_workload(name, 0)
+    fast = w.modes == ["fast"]
+    r = Runner(w, K, L, fast, dev)
+    try:
+        ms = time_steps(r.step, steps, warmup)
+        br = kernel_breakdown(r, steps)
+        ab = algorithmic_bytes(w, L, K, fast)
+        peak, how = measured_peak_hbm()
+        out = {"workload": name, "layers_per_call": L, "K": K, "mode": "fast" if fast else "scored",
+               "value": w.total * L / (ms * 1e-3), "unit": UNIT, "ms_per_step": ms,
+               "stage_ms": {"mask": br[0], "score": br[1], "select": br[2], "compact": br[3]},
+               "step_hbm_frac": ab["total"] / (ms * 1e-3) / 1e9 / peak}
+        if not fast and br[1] > 0:
+            out["score_hbm_frac"] = score_kernel_bytes(w, L) / (br[1] * 1e-3) / 1e9 / peak
+            out["score_tflops"] = 2.0 * (w.Hq // w.Hkv) * w.W * w.d * w.total * w.Hkv * L / (br[1] * 1e-3) / 1e12
+        if br[3] > 0:
+            out["compact_hbm_frac"] = ab["gather"] / (br[3] * 1e-3) / 1e9 / peak
+        return out
+    finally:
+        r.close()
+        torch.cuda.empty_cache()
+
+
+# ------------------------------------------------------------------------------------------------ main
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c2", choices=sorted(tw.CONFIGS))
+    ap.add_argument("--budget", type=int, default=0, help="K (default: the workload's first budget)")
+    ap.add_argument("--mode", default="", choices=["", "scored", "fast"])
+    ap.add_argument("--layers", type=int, default=0, help="layers per call (default: the workload's layer count)")
+    ap.add_argument("--no-extra", action="store_true", help="skip the supplementary workloads")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    a = ap.parse_args()
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    warmup = max(a.warmup, 3)
+    w, K = build_workload(a.workload, a.budget)
+    fast = (a.mode or w.modes[0]) == "fast"
+    L = a.layers or w.n_layers
+    config = {"workload": f"{w.name}: {L} layers x {w.B} seq, n={'ragged ' if not w.uniform else ''}{w.max_n}, "
+                          f"Hq={w.Hq} Hkv={w.Hkv} d={w.d}, W={w.W}, K={K}, {'TA-Fast' if fast else 'scored TA'}",
+              "layers_per_call": L, "budget_K": K, "mode": "fast" if fast else "scored", "preset": "THEOREM",
+              "l2": "inputs larger than L2 (every step streams all layers' keys)", "parallelism": f"replicas x{world}"}
+
+    if a.impl == "reference":
+        if rank != 0:
+            return
+        base, per_layer_s = oracle_leg(w, K, fast, budget_s=min(60.0, 4.0 * max(1, a.steps + warmup)))
+        line = {"impl": "reference", "metric": METRIC, "value": base["value"], "unit": UNIT, "n_gpus": a.gpus,
+                "steps": a.steps, "warmup": warmup, "ms_per_step": per_layer_s * 1e3 * L, "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": config,
+                "cpu_baseline": base,
+                "e2e": {"value": base["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+        print(json.dumps(line))
+        return
+
+    # the CPU leg runs before the first CUDA call of this process
+    cpu = None
+    if rank == 0 and world == 1 and not a.no_cpu:
+        cpu, _ = oracle_leg(w, K, fast)
+
+    dev = torch.device("cuda", local)
+    torch.cuda.set_device(dev)
+    barrier = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+        barrier = dist.barrier
+        w.seed += 7919 * rank  # every rank compacts its own batch (weak scaling, no exchange)
+
+    r = Runner(w, K, L, fast, dev)
+    sampler = ClockSampler(local)
+    sampler.start()
+    ms = time_steps(r.step, a.steps, warmup, barrier)
+    clocks = sampler.stop()
+    status = r.ta.ta_ctx_poll(r.ctx)
+    if status != 0:
+        raise SystemExit(f"device reported {r.ta.status_string(status)}")
+    if world > 1:
+        from paper_2604_11288_b200.sharding import max_over_ranks
+        ms = max_over_ranks(ms, dev)
+    value = world * w.total * L / (ms * 1e-3)
+
+    if rank != 0:
+        r.close()
+        return
+
+    br = kernel_breakdown(r, a.steps)
+    peak, how = measured_peak_hbm()
+    stage = {"mask": br[0], "score": br[1], "select": br[2], "compact": br[3]}
+    dom = "compact" if fast else "score"
+    ab = algorithmic_bytes(w, L, K, fast)
+    dom_bytes = ab["gather"] if fast else score_kernel_bytes(w, L)
+    achieved = dom_bytes / (stage[dom] * 1e-3) / 1e9 if stage[dom] > 0 else 0.0
+    roofline = {"kernel": "ta_compact_kernel" if fast else "ta_score_kernel", "bound": "hbm", "achieved": achieved,
+                "peak": peak, "peak_source": f"of {how}", "unit": "GB/s", "frac": achieved / peak, "traffic": None,
+                "ms_per_launch": stage[dom], "stage_ms": stage,
+                "step_algorithmic_bytes": ab["total"], "step_frac": ab["total"] / (ms * 1e-3) / 1e9 / peak}
+    if not fast:
+        roofline["tensor_tflops"] = 2.0 * (w.Hq // w.Hkv) * w.W * w.d * w.total * w.Hkv * L / (stage[dom] * 1e-3) / 1e12
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": a.steps, "warmup": warmup,
+            "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+            "data": "synthetic", "config": config, "clocks": clocks,
+            "gpu_launches": r.kernels_per_step() * a.steps, "roofline": roofline}
+    if not a.no_e2e and world == 1:
+        e_steps = max(3, min(a.steps, 10))
+        ems, h2d, d2h, same = e2e_leg(r, e_steps, 3)
+        line["e2e"] = {"value": w.total * L / (ems * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                       "d2h_bytes_per_step": d2h, "ms_per_step": ems, "matches_device_path": same}
+    if cpu:
+        line["cpu_baseline"] = cpu
+    r.close()
+    torch.cuda.empty_cache()
+    if not a.no_extra and world == 1:
+        extra = []
+        for name, layers in (("c3", 2), ("c4", 4), ("c5", 2)):
+            if name == a.workload:
+                continue
+            try:
+                extra.append(measure_extra(name, layers, dev))
+            except Exception as ex:  # supplementary only: never lose the main line
+                extra.append({"workload": name, "error": str(ex)[:200]})
+        line["other_workloads"] = extra
+    print(json.dumps(line))
+
+
+if __name__ == "__main__":
+    main()
