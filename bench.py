@@ -59,6 +59,9 @@ class ClockSampler:
             self.t.start()
         except Exception:
             self.proc = None
+        t0 = time.time()
+        while self.proc and not self.lines and time.time() - t0 < 3.0:  # first sample before the timed region
+            time.sleep(0.01)
 
     def _read(self):
         for line in self.proc.stdout:
@@ -67,6 +70,9 @@ class ClockSampler:
     def stop(self):
         if not self.proc:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
+        t0, have = time.time(), len(self.lines)
+        while len(self.lines) < have + 2 and time.time() - t0 < 0.5:  # the region may be shorter than one interval
+            time.sleep(0.01)
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
