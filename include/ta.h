@@ -212,6 +212,31 @@ ta_status ta_select_topk(ta_ctx* ctx, const ta_policy* policy, const ta_batch* b
                          const uint8_t* flags, const float* voucher, const float* u_static, const float* A,
                          const float* P, int32_t* idx, int32_t* count, void* stream);
 
+/* ---- step 3 without any allocation -------------------------------------------------------------------------
+ * (No counterpart in the paper: this entry point exists for a deployment constraint, not for the method.)
+ * Same computation and same results as ta_select_topk, for callers that are not allowed to allocate device memory
+ * and therefore cannot create a ta_ctx: code running inside an inference server whose memory pool already owns the
+ * whole GPU, a plugin loaded into someone else's process under a fixed memory budget, or a latency-critical loop
+ * where cudaMalloc's implicit device synchronisation is unacceptable. It takes no context. Its working memory (one
+ * byte per token plus a few words per sequence; in fast mode also B*K indices) lives in a fixed array inside the
+ * library image, so every GPU that loads this library gives up TA_STATIC_SCRATCH_BYTES for it until the process
+ * exits. The call issues no cudaMalloc/cudaFree and uses no allocating library routine.
+ *   - Limit: 256 + total_tokens + 8*B (+ 4*B*K in fast mode), each piece rounded up to 256 bytes, must fit in
+ *     TA_STATIC_SCRATCH_BYTES; larger problems are rejected with TA_ERR_SCRATCH_TOO_SMALL and nothing is enqueued.
+ *   - It works on the CUDA device that is current when it is called. The first call on each device looks up the
+ *     array's device address (a one-time runtime query, no allocation); make that first call outside of any stream
+ *     capture.
+ *   - All calls share the one array, which still holds the previous call's data: the call clears the part that has
+ *     to start at zero itself, but two calls whose kernels can overlap on the GPU (different streams without an
+ *     ordering between them, or two host threads) race on it. Serialise them.
+ *   - There is no context to poll: a sequence longer than batch->max_n gets count 0 and an all -1 index row instead
+ *     of an error code.
+ * Arguments are those of ta_select_topk without the context. */
+enum { TA_STATIC_SCRATCH_BYTES = 4 << 20 };
+ta_status ta_select_topk_static(const ta_policy* policy, const ta_batch* batch, int Hkv, int K, const uint8_t* flags,
+                                const float* voucher, const float* u_static, const float* A, const float* P,
+                                int32_t* idx, int32_t* count, void* stream);
+
 /* ---- step 4: compaction (Algorithm 1 step 9: index_select along the sequence axis) ------------------------
  *   k, v          bf16 views over the full cache
  *   idx, count    as written by ta_select_topk

@@ -72,6 +72,7 @@ def lib():
             "ta_sponsor_mask": (i32, [vp, vp, PP, PB, vp, vp, vp, vp, vp]),
             "ta_score": (i32, [vp, PP, PB, i32, i32, i32, ta_bf16_view, ta_bf16_view, vp, vp, vp, vp]),
             "ta_select_topk": (i32, [vp, PP, PB, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]),
+            "ta_select_topk_static": (i32, [PP, PB, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]),
             "ta_compact_kv": (i32, [vp, PB, i32, i32, i32, ta_bf16_view, ta_bf16_view, vp, vp, vp, vp, vp]),
             "ta_compress": (i32, [vp, vp, PP, PB, i32, i32, i32, i32, vp, ta_bf16_view, ta_bf16_view, ta_bf16_view,
                                   u64, vp, vp, vp, vp, vp]),
@@ -195,6 +196,14 @@ def ta_score(ctx, policy, batch, Hq, Hkv, d, q_obs: ta_bf16_view, k: ta_bf16_vie
 def ta_select_topk(ctx, policy, batch, Hkv, K, flags, voucher, u_static, A, P, idx, count, stream=None):
     _check(lib().ta_select_topk(ctx, C.byref(policy), C.byref(batch), Hkv, K, _ptr(flags), _ptr(voucher),
                                 _ptr(u_static), _ptr(A), _ptr(P), _ptr(idx), _ptr(count), stream), "ta_select_topk")
+
+
+def ta_select_topk_static(policy, batch, Hkv, K, flags, voucher, u_static, A, P, idx, count, stream=None):
+    """ta_select_topk for callers that may not allocate device memory: no context, working memory in a fixed
+    array inside the library (see include/ta.h for the size limit and the sharing rules)."""
+    _check(lib().ta_select_topk_static(C.byref(policy), C.byref(batch), Hkv, K, _ptr(flags), _ptr(voucher),
+                                       _ptr(u_static), _ptr(A), _ptr(P), _ptr(idx), _ptr(count), stream),
+           "ta_select_topk_static")
 
 
 def ta_compact_kv(ctx, batch, Hkv, d, K, k: ta_bf16_view, v: ta_bf16_view, idx, count, k_out, v_out, stream=None):

@@ -339,3 +339,99 @@ cudaError_t ta_launch_broadcast_idx(int B, int Hkv, int K, int n_layers, const i
   ta_broadcast_idx_kernel<<<blocks, 256, 0, stream>>>(B, Hkv, K, n_layers, idx_seq, count_seq, idx, count);
   return cudaGetLastError();
 }
+
+// ---------------------------------------------------------------------------------------------------------------
+// ta_select_topk_static: the selection step for callers that must not allocate device memory.
+//
+// The regular entry point takes its working memory (one byte per token, a few words per sequence) from a context
+// whose creation calls cudaMalloc. This variant keeps that working memory in the array below, which is part of the
+// library image: every GPU that loads the library reserves TA_STATIC_SCRATCH_BYTES for it until the process exits.
+// The array name is only meaningful to device code; host code must ask the runtime for its device address
+// (cudaGetSymbolAddress) once per device, with that device current, and hand that address to the kernels.
+#include <mutex>
+
+static __device__ __align__(256) unsigned char g_ta_static_scratch[TA_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+unsigned char* g_static_ptr[kMaxDevices] = {};  // device address of g_ta_static_scratch, per device ordinal
+
+size_t static_align(size_t x) { return (x + 255) / 256 * 256; }
+}  // namespace
+
+extern "C" ta_status ta_select_topk_static(const ta_policy* policy, const ta_batch* batch, int Hkv, int K,
+                                           const uint8_t* flags, const float* voucher, const float* u_static,
+                                           const float* A, const float* P, int32_t* idx, int32_t* count,
+                                           void* stream_v) {
+  if (!policy || !batch || !flags || !voucher || !u_static || !idx || !count) return TA_ERR_INVALID_ARG;
+  if (batch->n_layers < 1 || batch->batch < 1 || batch->max_n < 0 || batch->total_tokens < 0 || Hkv < 1 || K < 1)
+    return TA_ERR_INVALID_ARG;
+  if (!batch->cu_seqlens && (batch->n_uniform < 0 || batch->n_uniform > batch->max_n ||
+                             batch->total_tokens != (int64_t)batch->batch * batch->n_uniform))
+    return TA_ERR_INVALID_ARG;
+  if (policy->mode != TA_MODE_SCORED && policy->mode != TA_MODE_FAST) return TA_ERR_INVALID_ARG;
+  if (policy->n_sink < 0 || policy->n_recent < 0) return TA_ERR_INVALID_ARG;
+  if (K > TA_MAX_BUDGET || batch->max_n > TA_MAX_SEQ_LEN) return TA_ERR_UNSUPPORTED;
+  const bool fast = policy->mode == TA_MODE_FAST;
+  if (!fast && !A) return TA_ERR_INVALID_ARG;
+
+  // carve the fixed array: status block, forced flags, per-sequence counters, fast-mode per-sequence result
+  const size_t B = (size_t)batch->batch, total = (size_t)batch->total_tokens;
+  size_t off = 0;
+  const size_t o_status = off; off += static_align(sizeof(ta_dev_status));
+  const size_t o_forced = off; off += static_align(total);
+  const size_t o_rmain = off;  off += static_align(B * 4);
+  const size_t o_idxseq = off; off += static_align(fast ? B * (size_t)K * 4 : 0);
+  const size_t o_cntseq = off; off += static_align(fast ? B * 4 : 0);
+  if (off > (size_t)TA_STATIC_SCRATCH_BYTES) return TA_ERR_SCRATCH_TOO_SMALL;  // problem larger than the built-in limit
+
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return TA_ERR_CUDA;
+  unsigned char* base = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_ptr[dev]) {  // first call on this device: resolve the array's device address (no allocation)
+      void* p = nullptr;
+      if (cudaGetSymbolAddress(&p, g_ta_static_scratch) != cudaSuccess || !p) return TA_ERR_CUDA;
+      g_static_ptr[dev] = static_cast<unsigned char*>(p);
+    }
+    base = g_static_ptr[dev];
+  }
+  cudaStream_t stream = (cudaStream_t)stream_v;
+  // the array keeps whatever the previous call left: the status block must start at zero; the other pieces are
+  // fully rewritten by the kernels before they are read
+  if (cudaMemsetAsync(base + o_status, 0, sizeof(ta_dev_status), stream) != cudaSuccess) return TA_ERR_CUDA;
+
+  ta_select_args a = {};
+  a.seq.cu = batch->cu_seqlens;
+  a.seq.n_uniform = batch->n_uniform;
+  a.seq.batch = batch->batch;
+  a.seq.max_n = batch->max_n;
+  a.seq.total = batch->total_tokens;
+  a.n_layers = batch->n_layers;
+  a.Hkv = Hkv;
+  a.K = K;
+  a.n_sink = policy->n_sink;
+  a.n_recent = policy->n_recent;
+  a.k_protected = policy->k_protected;
+  a.fast = fast;
+  a.alpha = policy->alpha;
+  a.delta = policy->delta;
+  a.flags = flags;
+  a.voucher = voucher;
+  a.u_static = u_static;
+  a.A = A;
+  a.P = P;
+  a.u = nullptr;
+  a.forced = base + o_forced;
+  a.r_main = reinterpret_cast<int32_t*>(base + o_rmain);
+  int32_t* idx_seq = reinterpret_cast<int32_t*>(base + o_idxseq);
+  int32_t* cnt_seq = reinterpret_cast<int32_t*>(base + o_cntseq);
+  a.idx = fast ? idx_seq : idx;
+  a.count = fast ? cnt_seq : count;
+  cudaError_t e = ta_launch_select(a, reinterpret_cast<ta_dev_status*>(base + o_status), stream);
+  if (e == cudaSuccess && fast)
+    e = ta_launch_broadcast_idx(batch->batch, Hkv, K, batch->n_layers, idx_seq, cnt_seq, idx, count, stream);
+  return e == cudaSuccess ? TA_OK : TA_ERR_CUDA;
+}
