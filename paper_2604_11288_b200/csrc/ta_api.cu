@@ -188,6 +188,9 @@ ta_status ta_ctx_create(int device, size_t scratch_bytes, ta_ctx** out) {
   if (e == cudaSuccess) e = cudaMemset(c->d_status, 0, sizeof(ta_dev_status));
   if (e == cudaSuccess && scratch_bytes) e = cudaMalloc(&c->scratch, scratch_bytes);
   for (int i = 0; e == cudaSuccess && i < 8; ++i) e = cudaEventCreate(&c->ev[i]);
+  if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking);
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming);
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming);
   if (e == cudaSuccess) {
     cudaDriverEntryPointQueryResult q;
     e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &c->encode_tiled, cudaEnableDefault, &q);
@@ -206,6 +209,9 @@ void ta_ctx_destroy(ta_ctx* c) {
   DeviceGuard guard(c->device);
   for (int i = 0; i < 8; ++i)
     if (c->ev[i]) cudaEventDestroy(c->ev[i]);
+  if (c->ev_fork) cudaEventDestroy(c->ev_fork);
+  if (c->ev_join) cudaEventDestroy(c->ev_join);
+  if (c->side) cudaStreamDestroy(c->side);
   if (c->scratch) cudaFree(c->scratch);
   if (c->d_status) cudaFree(c->d_status);
   delete c;
@@ -255,7 +261,11 @@ ta_status ta_ctx_read_timing(ta_ctx* ctx, float out_ms[5]) {
   if (!ctx->timing_valid) return TA_ERR_INVALID_ARG;
   DeviceGuard guard(ctx->device);
   cudaError_t e = cudaEventSynchronize(ctx->ev[4]);
-  for (int i = 0; e == cudaSuccess && i < 4; ++i) e = cudaEventElapsedTime(&out_ms[i], ctx->ev[i], ctx->ev[i + 1]);
+  if (e == cudaSuccess && ctx->ev_ran[0]) {  // per-sequence work runs on the side stream, beside the score kernel
+    e = cudaEventSynchronize(ctx->ev[6]);
+    if (e == cudaSuccess) e = cudaEventElapsedTime(&out_ms[0], ctx->ev[5], ctx->ev[6]);
+  }
+  for (int i = 1; e == cudaSuccess && i < 4; ++i) e = cudaEventElapsedTime(&out_ms[i], ctx->ev[i], ctx->ev[i + 1]);
   if (e == cudaSuccess) e = cudaEventElapsedTime(&out_ms[4], ctx->ev[0], ctx->ev[4]);
   return e == cudaSuccess ? TA_OK : cuda_fail(ctx, e);
 }
@@ -520,8 +530,48 @@ ta_status ta_compress(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* pol
 
   const bool reuse = seq_epoch != 0 && seq_epoch == ctx->cached_epoch && ctx->cached_total == batch->total_tokens &&
                      ctx->cached_batch == batch->batch && ctx->cached_K == K;
+  ta_select_args sel = {};
+  sel.seq = seq;
+  sel.n_layers = batch->n_layers;
+  sel.Hkv = Hkv;
+  sel.K = K;
+  sel.n_sink = policy->n_sink;
+  sel.n_recent = policy->n_recent;
+  sel.k_protected = policy->k_protected;
+  sel.fast = fast;
+  sel.alpha = policy->alpha;
+  sel.delta = policy->delta;
+  sel.flags = flags;
+  sel.voucher = voucher;
+  sel.u_static = u_static;
+  sel.u = u;
+  sel.forced = forced;
+  sel.r_main = r_main;
+  sel.idx = fast ? idx_seq : idx;
+  sel.count = fast ? count_seq : count;
+
+  // Per-sequence work (anchor mask, vouchers, static utility, forced set) does not depend on Q/K: in scored mode it
+  // runs on the context's side stream beside the score kernel and joins before the per-unit selection.
   mark(0);
-  if (!reuse) e = ta_launch_mask(pats, *policy, seq, token_ids, flags, voucher, u_static, hist, ctx->d_status, stream);
+  ctx->ev_ran[0] = 0;
+  cudaStream_t seq_stream = stream;
+  const bool fork = !reuse && !fast;
+  if (fork) {
+    seq_stream = ctx->side;
+    e = cudaEventRecord(ctx->ev_fork, stream);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0);
+  }
+  if (!reuse) {
+    if (timing && e == cudaSuccess) e = cudaEventRecord(ctx->ev[5], seq_stream);
+    if (e == cudaSuccess)
+      e = ta_launch_mask(pats, *policy, seq, token_ids, flags, voucher, u_static, hist, ctx->d_status, seq_stream);
+    if (e == cudaSuccess) e = ta_launch_forced(sel, ctx->d_status, seq_stream);
+    if (timing && e == cudaSuccess) {
+      e = cudaEventRecord(ctx->ev[6], seq_stream);
+      ctx->ev_ran[0] = 1;
+    }
+  }
+  if (fork && e == cudaSuccess) e = cudaEventRecord(ctx->ev_join, ctx->side);
   mark(1);
   if (e == cudaSuccess && !fast) {
     ta_score_args a = {};
@@ -536,7 +586,7 @@ ta_status ta_compress(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* pol
     a.A = nullptr;
     a.P = nullptr;
     a.u = u;
-    a.u_static = u_static;
+    a.u_static = nullptr;
     a.alpha = policy->alpha;
     a.delta = policy->delta;
     a.rho = policy->pension_rho;
@@ -545,28 +595,8 @@ ta_status ta_compress(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* pol
     e = ta_launch_score(ctx, a, ctx->d_status, stream);
   }
   mark(2);
-  if (e == cudaSuccess && !(fast && reuse)) {
-    ta_select_args a = {};
-    a.seq = seq;
-    a.n_layers = batch->n_layers;
-    a.Hkv = Hkv;
-    a.K = K;
-    a.n_sink = policy->n_sink;
-    a.n_recent = policy->n_recent;
-    a.k_protected = policy->k_protected;
-    a.fast = fast;
-    a.alpha = policy->alpha;
-    a.delta = policy->delta;
-    a.flags = flags;
-    a.voucher = voucher;
-    a.u_static = u_static;
-    a.u = u;
-    a.forced = forced;
-    a.r_main = r_main;
-    a.idx = fast ? idx_seq : idx;
-    a.count = fast ? count_seq : count;
-    e = ta_launch_select(a, ctx->d_status, stream);
-  }
+  if (fork && e == cudaSuccess) e = cudaStreamWaitEvent(stream, ctx->ev_join, 0);
+  if (e == cudaSuccess && !(fast && reuse)) e = ta_launch_select_units(sel, stream);
   if (e == cudaSuccess && fast)
     e = ta_launch_broadcast_idx(batch->batch, Hkv, K, batch->n_layers, idx_seq, count_seq, idx, count, stream);
   mark(3);

@@ -44,6 +44,11 @@ struct ta_ctx {
   int timing_valid;
   cudaEvent_t ev[8];
   int ev_ran[4];
+  // fork/join of the per-sequence work (mask, vouchers, forced set) beside the score kernel
+  cudaStream_t side;
+  cudaEvent_t ev_fork, ev_join;
+  // launch shape of the most recent score kernel (diagnostics)
+  int score_cluster, score_clusters;
   // driver entry point for tensor-map encoding (resolved at create time)
   void* encode_tiled;
 };
@@ -75,8 +80,8 @@ struct ta_score_args {
   const float* lse_obs;  // nullable
   float* A;              // nullable
   float* P;              // nullable
-  float* u;              // nullable: fused utility (alpha*A + delta*P) + u_static
-  const float* u_static;
+  float* u;              // nullable: fused attention part alpha*A + delta*P (u_static is added by the selection)
+  const float* u_static; // unused
   float alpha, delta, rho, scale;
   int causal;
 };
@@ -94,13 +99,15 @@ struct ta_select_args {
   const float* u_static;
   const float* A;  // scored, unfused
   const float* P;
-  const float* u;  // scored, fused (takes precedence over A/P)
+  const float* u;  // scored, fused: alpha*A + delta*P as written by the score kernel (takes precedence over A/P)
   uint8_t* forced;     // scratch [total]
   int32_t* r_main;     // scratch [B]   main-pool picks per sequence (-1: keep everything)
   int32_t* idx;        // [L][B][Hkv][K]
   int32_t* count;      // [L][B][Hkv]
 };
-cudaError_t ta_launch_select(const ta_select_args& a, ta_dev_status* status, cudaStream_t stream);
+cudaError_t ta_launch_select(const ta_select_args& a, ta_dev_status* status, cudaStream_t stream);  // both below
+cudaError_t ta_launch_forced(const ta_select_args& a, ta_dev_status* status, cudaStream_t stream);
+cudaError_t ta_launch_select_units(const ta_select_args& a, cudaStream_t stream);
 cudaError_t ta_launch_broadcast_idx(int B, int Hkv, int K, int n_layers, const int32_t* idx_seq,
                                     const int32_t* count_seq, int32_t* idx, int32_t* count, cudaStream_t stream);
 

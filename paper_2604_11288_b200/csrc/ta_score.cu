@@ -10,13 +10,19 @@
 // Both passes use the same shared-memory operand tiles (both K-major, 128-byte swizzle); only the roles in the
 // instruction descriptor swap, which puts the reduction axis of each pass along a thread's own registers.
 // The keys of a unit are split over the CTAs of a cluster (each CTA owns a contiguous range of 128-key tiles);
-// between the passes the CTAs exchange their per-row statistics through distributed shared memory. Pass 2
-// re-reads the CTA's own tiles, which are still in L2, so HBM sees every key once.
-// When the caller supplies the rows' log-sum-exp (lse_obs), pass 1 is skipped.
+// between the passes the CTAs exchange their per-row statistics through distributed shared memory (remote stores
+// followed by a remote mbarrier arrive). Pass 2 re-reads the CTA's own tiles, which are still in L2, so HBM sees
+// every key once. When the caller supplies the rows' log-sum-exp (lse_obs), pass 1 is skipped.
+//
+// The grid is persistent: as many clusters as the device can hold at once, each walking over units
+// cluster, cluster + n_clusters, ...; the TMA and MMA warps run ahead across unit boundaries (double-buffered query
+// tile, ring of key tiles, two accumulator stages), so barrier set-up, TMEM allocation and pipeline fill are paid
+// once per CTA and not once per unit.
 //
 // Warp roles (320 threads): warp 0 TMA producer, warp 1 MMA issuer + TMEM owner, warps 2-9 two softmax groups that
 // alternate over the two accumulator stages. Every wait on an mbarrier is bounded by wall time; when one runs out
 // the CTA records TA_ERR_TIMEOUT, stops waiting anywhere, drains its copies, frees its tensor memory and returns.
+// The only unbounded waits are two hardware cluster barriers (start, end) that every thread reaches on every path.
 #include <cuda.h>
 
 #include "ta_internal.cuh"
@@ -27,10 +33,8 @@ constexpr int kTileN = 128;                       // keys per tile
 constexpr int kD = TA_HEAD_DIM;                   // 128
 constexpr int kHalfBytes = kTileN * 128;          // one 64-column half of a 128-row operand tile: 16 KB
 constexpr int kKTileBytes = 2 * kHalfBytes;       // 32 KB
-constexpr int kStages = 4;                        // shared-memory ring of key tiles
 constexpr int kMaxCluster = 8;
 constexpr int kThreads = 320;
-constexpr int kSoftmaxThreads = 256;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s
 
 struct ScoreParams {
@@ -38,6 +42,7 @@ struct ScoreParams {
   int n_layers, Hq, Hkv, G, W;
   int rows;           // G*W
   int cluster;        // CTAs per unit
+  int units;          // L * B * Hkv
   int two_pass;       // 0 when lse_obs is given
   int causal;
   float c;            // softmax scale * log2(e)
@@ -144,9 +149,10 @@ __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 
-// 32 lanes x 32 consecutive fp32 columns: thread i of the warp receives lane (quadrant base + i).
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
-  uint32_t r[32];
+// 32 lanes x 32 consecutive 32-bit columns: thread i of the warp receives lane (quadrant base + i). The load is
+// asynchronous; tmem_ld_wait() must be called on the same registers before they are read. Passing the registers
+// through the wait as read-write operands keeps the compiler from moving their uses above it.
+__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t (&r)[32]) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
       "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
@@ -157,9 +163,16 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
         "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
       : "r"(taddr)
       : "memory");
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-  for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
+}
+__device__ __forceinline__ void tmem_ld_wait(uint32_t (&r)[32]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+                 "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
+                 "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]),
+                 "+r"(r[23]), "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]),
+                 "+r"(r[30]), "+r"(r[31])
+               :
+               : "memory");
 }
 
 __device__ __forceinline__ float ex2(float x) {
@@ -180,6 +193,25 @@ __device__ __forceinline__ void st_cluster_f32(uint32_t local_addr, uint32_t ran
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
   asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote), "f"(v) : "memory");
 }
+// arrive (release at cluster scope) on the mbarrier at the same shared-memory offset in CTA `rank` of the cluster
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t local_bar, uint32_t rank) {
+  uint32_t remote;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_bar), "r"(rank));
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n"
+      "selp.u32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
 __device__ __forceinline__ void softmax_bar() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 
 // Shared-memory matrix descriptor for a K-major operand tile stored as rows of 128 bytes with the 128-byte swizzle
@@ -199,21 +231,57 @@ __device__ __forceinline__ uint32_t idesc_bf16(int M, int N) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 
+// Bounded wait with cluster-scope acquire (for barriers that peers of the cluster arrive on).
+__device__ __noinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                               ta_dev_status* status, int where) {
+  if (*abort_flag) return false;
+  if (mbar_try_wait_cluster(bar, parity)) return true;
+  const unsigned long long t0 = globaltimer_ns();
+  for (;;) {
+#pragma unroll 1
+    for (int it = 0; it < 64; ++it)
+      if (mbar_try_wait_cluster(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (globaltimer_ns() - t0 > kWaitLimitNs) {
+      *abort_flag = 1;
+      if (atomicCAS(&status->code, 0, (int)TA_ERR_TIMEOUT) == 0) {
+        status->where = where;
+        status->detail0 = (int)blockIdx.x;
+        status->detail1 = (int)parity;
+      }
+      return false;
+    }
+  }
+}
+
 // ---------------------------------------------------------------------------------------------- shared memory
 template <int MB>
+struct ScoreCfg {
+  static constexpr int kQBufs = MB == 1 ? 2 : 1;   // query tiles in flight (next unit's tile loads early)
+  static constexpr int kStages = MB == 1 ? 4 : 3;  // ring of key tiles
+  static constexpr int kRowsPad = MB * 128;
+};
+
+template <int MB>
 struct alignas(1024) ScoreSmem {
-  uint8_t q[MB * 2 * kHalfBytes];         // [half][MB*128 rows][128 B]
-  uint8_t k[kStages][kKTileBytes];        // [stage][half][128 rows][128 B]
-  float xchg_m[kMaxCluster][MB * 128];    // per-CTA row statistics of every CTA of the cluster
-  float xchg_z[kMaxCluster][MB * 128];
-  float part_m[2][MB * 128];              // per softmax group
+  using Cfg = ScoreCfg<MB>;
+  uint8_t q[Cfg::kQBufs][MB * 2 * kHalfBytes];    // [buffer][half][MB*128 rows][128 B]
+  uint8_t k[Cfg::kStages][kKTileBytes];           // [stage][half][128 rows][128 B]
+  float xchg_m[2][kMaxCluster][MB * 128];         // [unit parity][cluster rank][row]: per-CTA row statistics
+  float xchg_z[2][kMaxCluster][MB * 128];
+  float part_m[2][MB * 128];                      // per softmax group
   float part_z[2][MB * 128];
-  float lse2[MB * 128];                   // log2-domain log-sum-exp per row (+inf: row contributes nothing)
-  float wrow[MB * 128];                   // pension weight per row
-  int lim[MB * 128];                      // last key a row may see (-1: none)
-  unsigned long long full[kStages], empty[kStages], acc_full[2], acc_empty[2], q_full, drain;
+  float lse2[2][MB * 128];                        // [unit parity][row] log2-domain log-sum-exp (+inf: row is mute)
+  float wrow[MB * 128];                           // pension weight per row
+  int row_t[MB * 128];                            // window index t of the row, -1 for padding rows
+  unsigned long long full[Cfg::kStages], empty[Cfg::kStages], acc_full[2], acc_empty[2];
+  unsigned long long q_full[Cfg::kQBufs], q_empty[Cfg::kQBufs], xchg_full[2], drain;
   uint32_t tmem_base;
   int abort_flag;
+};
+
+struct UnitInfo {
+  int l, b, g, tok0, n, t_begin, T;
 };
 
 // ---------------------------------------------------------------------------------------------- the kernel
@@ -221,36 +289,42 @@ template <int MB, bool kNeedP>
 __global__ void __launch_bounds__(kThreads, 1)
 ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                 const __grid_constant__ ScoreParams p) {
+  using Cfg = ScoreCfg<MB>;
+  constexpr int kStages = Cfg::kStages, kQBufs = Cfg::kQBufs, kRowsPad = Cfg::kRowsPad;
+  constexpr uint32_t kTmemCols = MB * 256;
+  constexpr int kQBytes = MB * 2 * kHalfBytes;
   extern __shared__ uint8_t smem_raw[];
   ScoreSmem<MB>& sm = *reinterpret_cast<ScoreSmem<MB>*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const uint32_t rank = cluster_ctarank();
-  const int unit = blockIdx.x / p.cluster;
-  const int g = unit % p.Hkv;
-  const int b = (unit / p.Hkv) % p.seq.batch;
-  const int l = unit / (p.Hkv * p.seq.batch);
-  const int tok0 = ta_seq_begin(p.seq, b);
-  int n = (p.seq.cu ? p.seq.cu[b + 1] : tok0 + p.seq.n_uniform) - tok0;
-  if (n > p.seq.max_n || n < 0) {  // reported by the selection step as well; here: just do nothing harmful
-    if (tid == 0 && atomicCAS(&p.status->code, 0, (int)TA_ERR_DEVICE_BOUNDS) == 0) {
-      p.status->where = 2;
-      p.status->detail0 = b;
-      p.status->detail1 = n;
-    }
-    n = 0;
-  }
-  const int Wp = min(p.W, n);
-  const int tiles_total = (n + kTileN - 1) / kTileN;
-  const int t_begin = (int)((long long)tiles_total * rank / p.cluster);
-  const int t_end = (int)((long long)tiles_total * (rank + 1) / p.cluster);
-  const int T = t_end - t_begin;
-  const int n_jobs = p.two_pass ? 2 * T : T;
+  const int cluster_id = blockIdx.x / p.cluster;
+  const int n_clusters = gridDim.x / p.cluster;
   volatile int* abort_flag = &sm.abort_flag;
-  constexpr uint32_t kTmemCols = MB * 256;
-  constexpr int kRowsPad = MB * 128;
 
-  // ---- set-up
+  auto get_unit = [&](int u) {
+    UnitInfo ui;
+    ui.g = u % p.Hkv;
+    ui.b = (u / p.Hkv) % p.seq.batch;
+    ui.l = u / (p.Hkv * p.seq.batch);
+    ui.tok0 = ta_seq_begin(p.seq, ui.b);
+    int n = (p.seq.cu ? p.seq.cu[ui.b + 1] : ui.tok0 + p.seq.n_uniform) - ui.tok0;
+    if (n > p.seq.max_n || n < 0) {  // the selection step rejects this sequence; here it is simply skipped
+      if (tid == 0 && atomicCAS(&p.status->code, 0, (int)TA_ERR_DEVICE_BOUNDS) == 0) {
+        p.status->where = 2;
+        p.status->detail0 = ui.b;
+        p.status->detail1 = n;
+      }
+      n = 0;
+    }
+    ui.n = n;
+    const int tiles_total = (n + kTileN - 1) / kTileN;
+    ui.t_begin = (int)((long long)tiles_total * rank / p.cluster);
+    ui.T = (int)((long long)tiles_total * (rank + 1) / p.cluster) - ui.t_begin;
+    return ui;
+  };
+
+  // ---- set-up (once per CTA)
   if (tid == 0) {
     for (int s = 0; s < kStages; ++s) {
       mbar_init(smem_u32(&sm.full[s]), 1);
@@ -259,8 +333,12 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     for (int a = 0; a < 2; ++a) {
       mbar_init(smem_u32(&sm.acc_full[a]), 1);
       mbar_init(smem_u32(&sm.acc_empty[a]), 4);
+      mbar_init(smem_u32(&sm.xchg_full[a]), (uint32_t)(p.cluster * kRowsPad));
     }
-    mbar_init(smem_u32(&sm.q_full), 1);
+    for (int qb = 0; qb < kQBufs; ++qb) {
+      mbar_init(smem_u32(&sm.q_full[qb]), 1);
+      mbar_init(smem_u32(&sm.q_empty[qb]), 1);
+    }
     mbar_init(smem_u32(&sm.drain), 1);
     // a wait that ran out in an earlier CTA or call (not yet polled) makes the remaining CTAs skip their waits
     sm.abort_flag = (*reinterpret_cast<volatile int*>(&p.status->code) == (int)TA_ERR_TIMEOUT) ? 1 : 0;
@@ -270,39 +348,21 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     tmem_alloc(smem_u32(&sm.tmem_base), kTmemCols);
     tmem_relinquish();
   }
-  // per-row tables: last visible key and pension weight. Row r = h*W + t; its query sits at position n - W + t.
+  // per-row tables: row r = h*W + t
   for (int r = tid; r < kRowsPad; r += kThreads) {
-    int lim = -1;
-    float w = 0.0f;
-    if (r < p.rows) {
-      const int t = r % p.W;
-      const int pos = n - p.W + t;
-      if (pos >= 0) {
-        lim = p.causal ? pos : n - 1;
-        // weight (1-rho) rho^(W'-1-t') with t' = t - (W - W'): the exponent is W-1-t for every valid row
-        w = p.wrow[t];
-      }
-    }
-    sm.lim[r] = lim;
-    sm.wrow[r] = w;
-    if (!p.two_pass) {
-      float lse2 = INFINITY;
-      if (lim >= 0) {
-        const int h = r / p.W, t = r % p.W;
-        const float lse = p.lse_obs[(((long long)l * p.seq.batch + b) * p.Hq + (g * p.G + h)) * p.W + t];
-        lse2 = lse * 1.4426950408889634f;
-      }
-      sm.lse2[r] = lse2;
-    }
+    const int t = r < p.rows ? r % p.W : -1;
+    sm.row_t[r] = t;
+    sm.wrow[r] = t >= 0 ? p.wrow[t] : 0.0f;  // (1-rho) rho^(W-1-t); also right for W' < W (same exponent)
   }
   // Rows of the query tile that the TMA box does not cover are multiplied like any other row: make them zeros so
   // that the padded score columns are finite.
   if (p.rows < kRowsPad) {
     const int pad_rows = kRowsPad - p.rows;
-    for (int i = tid; i < 2 * pad_rows * 8; i += kThreads) {
-      const int half = i / (pad_rows * 8), rem = i % (pad_rows * 8);
+    for (int i = tid; i < kQBufs * 2 * pad_rows * 8; i += kThreads) {
+      const int qb = i / (2 * pad_rows * 8), i2 = i % (2 * pad_rows * 8);
+      const int half = i2 / (pad_rows * 8), rem = i2 % (pad_rows * 8);
       const int row = p.rows + rem / 8, chunk = rem % 8;
-      *reinterpret_cast<uint4*>(&sm.q[half * (MB * kHalfBytes) + row * 128 + chunk * 16]) = make_uint4(0, 0, 0, 0);
+      *reinterpret_cast<uint4*>(&sm.q[qb][half * (MB * kHalfBytes) + row * 128 + chunk * 16]) = make_uint4(0, 0, 0, 0);
     }
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -310,44 +370,47 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = sm.tmem_base;
-  // every CTA of the cluster must be running before any of them writes into a peer's shared memory
+  // every CTA of the cluster must be running (barriers initialised) before any peer writes into its shared memory
   cluster_arrive();
   cluster_wait();
 
-  const uint32_t q_smem = smem_u32(sm.q);
   const uint32_t k_smem = smem_u32(sm.k);
-  const int row_coord_base = p.seq.cu ? tok0 : 0;  // ragged: tokens are packed along the row axis
-  const int b_coord = p.seq.cu ? 0 : b;
 
   if (warp == 0) {
     // =========================================================================== TMA producer
-    int issued[kStages];
+    if (lane == 0) {
+      int issued[kStages];
 #pragma unroll
-    for (int s = 0; s < kStages; ++s) issued[s] = 0;
-    auto issue = [&](int j) {
-      const int s = j % kStages;
-      const uint32_t ph = (uint32_t)(j / kStages) & 1u;
-      mbar_wait(smem_u32(&sm.empty[s]), ph ^ 1u, abort_flag, p.status, 10);
-      const int tile = t_begin + (p.two_pass ? j % T : j);
-      const uint32_t bar = smem_u32(&sm.full[s]);
-      mbar_expect_tx(bar, kKTileBytes);
-      const uint32_t dst = k_smem + s * kKTileBytes;
-      tma_load_5d(dst, &map_k, bar, 0, row_coord_base + tile * kTileN, g, b_coord, l);
-      tma_load_5d(dst + kHalfBytes, &map_k, bar, 64, row_coord_base + tile * kTileN, g, b_coord, l);
-      issued[s] = j + 1;
-    };
-    if (lane == 0 && T > 0) {
-      const uint32_t bar = smem_u32(&sm.q_full);
-      mbar_expect_tx(bar, (uint32_t)(2 * p.rows * 128));
-      tma_load_5d(q_smem, &map_q, bar, 0, 0, g * p.G, b, l);
-      tma_load_5d(q_smem + MB * kHalfBytes, &map_q, bar, 64, 0, g * p.G, b, l);
-      if (p.two_pass)
-        for (int j = 0; j < T; ++j) issue(j);
-    }
-    __syncwarp();
-    cluster_arrive();
-    if (lane == 0 && T > 0) {
-      for (int j = p.two_pass ? T : 0; j < n_jobs; ++j) issue(j);
+      for (int s = 0; s < kStages; ++s) issued[s] = 0;
+      int jg = 0, qn = 0;
+      for (int u = cluster_id; u < p.units; u += n_clusters) {
+        const UnitInfo ui = get_unit(u);
+        if (ui.T == 0) continue;
+        const int qb = qn % kQBufs;
+        mbar_wait(smem_u32(&sm.q_empty[qb]), ((uint32_t)(qn / kQBufs) & 1u) ^ 1u, abort_flag, p.status, 11);
+        {
+          const uint32_t bar = smem_u32(&sm.q_full[qb]);
+          const uint32_t dst = smem_u32(sm.q[qb]);
+          mbar_expect_tx(bar, (uint32_t)(2 * p.rows * 128));
+          tma_load_5d(dst, &map_q, bar, 0, 0, ui.g * p.G, ui.b, ui.l);
+          tma_load_5d(dst + MB * kHalfBytes, &map_q, bar, 64, 0, ui.g * p.G, ui.b, ui.l);
+        }
+        ++qn;
+        const int row0 = p.seq.cu ? ui.tok0 : 0;  // ragged: tokens are packed along the row axis
+        const int bc = p.seq.cu ? 0 : ui.b;
+        const int n_jobs = p.two_pass ? 2 * ui.T : ui.T;
+        for (int j = 0; j < n_jobs; ++j, ++jg) {
+          const int s = jg % kStages;
+          mbar_wait(smem_u32(&sm.empty[s]), ((uint32_t)(jg / kStages) & 1u) ^ 1u, abort_flag, p.status, 10);
+          const int tile = ui.t_begin + (j >= ui.T ? j - ui.T : j);
+          const uint32_t bar = smem_u32(&sm.full[s]);
+          mbar_expect_tx(bar, kKTileBytes);
+          const uint32_t dst = k_smem + s * kKTileBytes;
+          tma_load_5d(dst, &map_k, bar, 0, row0 + tile * kTileN, ui.g, bc, ui.l);
+          tma_load_5d(dst + kHalfBytes, &map_k, bar, 64, row0 + tile * kTileN, ui.g, bc, ui.l);
+          issued[s] = jg + 1;
+        }
+      }
       if (*abort_flag) {  // drain: every armed stage must have landed before the CTA may leave
         for (int s = 0; s < kStages; ++s) {
           if (!issued[s]) continue;
@@ -358,55 +421,54 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         }
       }
     }
-    __syncwarp();
-    cluster_wait();
   } else if (warp == 1) {
     // =========================================================================== MMA issuer
-    auto issue = [&](int j) {
-      const int s = j % kStages;
-      const uint32_t ph = (uint32_t)(j / kStages) & 1u;
-      const int a = j & 1;
-      const uint32_t aph = (uint32_t)(j >> 1) & 1u;
-      const bool stats = p.two_pass && j < T;
-      mbar_wait(smem_u32(&sm.full[s]), ph, abort_flag, p.status, 20);
-      mbar_wait(smem_u32(&sm.acc_empty[a]), aph ^ 1u, abort_flag, p.status, 21);
-      tc_fence_after();
-      const uint32_t kt = k_smem + s * kKTileBytes;
-      const uint32_t acc = tmem_base + (uint32_t)(a * kRowsPad);
-      if (stats) {
-        const uint32_t idesc = idesc_bf16(128, kTileN);
+    if (lane == 0) {
+      int jg = 0, qn = 0;
+      for (int u = cluster_id; u < p.units; u += n_clusters) {
+        const UnitInfo ui = get_unit(u);
+        if (ui.T == 0) continue;
+        const int qb = qn % kQBufs;
+        mbar_wait(smem_u32(&sm.q_full[qb]), (uint32_t)(qn / kQBufs) & 1u, abort_flag, p.status, 22);
+        const uint32_t q_smem = smem_u32(sm.q[qb]);
+        const int n_jobs = p.two_pass ? 2 * ui.T : ui.T;
+        for (int j = 0; j < n_jobs; ++j, ++jg) {
+          const int s = jg % kStages;
+          const int a = jg & 1;
+          const bool stats = p.two_pass && j < ui.T;
+          mbar_wait(smem_u32(&sm.full[s]), (uint32_t)(jg / kStages) & 1u, abort_flag, p.status, 20);
+          mbar_wait(smem_u32(&sm.acc_empty[a]), ((uint32_t)(jg >> 1) & 1u) ^ 1u, abort_flag, p.status, 21);
+          tc_fence_after();
+          const uint32_t kt = k_smem + s * kKTileBytes;
+          const uint32_t acc = tmem_base + (uint32_t)(a * kRowsPad);
+          if (stats) {
+            const uint32_t idesc = idesc_bf16(128, kTileN);
 #pragma unroll
-        for (int mb = 0; mb < MB; ++mb) {
+            for (int mb = 0; mb < MB; ++mb) {
 #pragma unroll
-          for (int k = 0; k < 8; ++k) {
-            const uint32_t off = (uint32_t)(k & 3) * 32u;
-            const uint64_t da = smem_desc_sw128(q_smem + (k >> 2) * (MB * kHalfBytes) + mb * kHalfBytes + off);
-            const uint64_t db = smem_desc_sw128(kt + (k >> 2) * kHalfBytes + off);
-            umma_bf16(acc + mb * 128, da, db, idesc, k > 0);
+              for (int k = 0; k < 8; ++k) {
+                const uint32_t off = (uint32_t)(k & 3) * 32u;
+                const uint64_t da = smem_desc_sw128(q_smem + (k >> 2) * (MB * kHalfBytes) + mb * kHalfBytes + off);
+                const uint64_t db = smem_desc_sw128(kt + (k >> 2) * kHalfBytes + off);
+                umma_bf16(acc + mb * 128, da, db, idesc, k > 0);
+              }
+            }
+          } else {
+            const uint32_t idesc = idesc_bf16(128, kRowsPad);
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+              const uint32_t off = (uint32_t)(k & 3) * 32u;
+              const uint64_t da = smem_desc_sw128(kt + (k >> 2) * kHalfBytes + off);
+              const uint64_t db = smem_desc_sw128(q_smem + (k >> 2) * (MB * kHalfBytes) + off);
+              umma_bf16(acc, da, db, idesc, k > 0);
+            }
           }
+          umma_commit(smem_u32(&sm.empty[s]));
+          umma_commit(smem_u32(&sm.acc_full[a]));
         }
-      } else {
-        const uint32_t idesc = idesc_bf16(128, kRowsPad);
-#pragma unroll
-        for (int k = 0; k < 8; ++k) {
-          const uint32_t off = (uint32_t)(k & 3) * 32u;
-          const uint64_t da = smem_desc_sw128(kt + (k >> 2) * kHalfBytes + off);
-          const uint64_t db = smem_desc_sw128(q_smem + (k >> 2) * (MB * kHalfBytes) + off);
-          umma_bf16(acc, da, db, idesc, k > 0);
-        }
+        umma_commit(smem_u32(&sm.q_empty[qb]));  // the query tile may be overwritten once these MMAs are done
+        ++qn;
       }
-      umma_commit(smem_u32(&sm.empty[s]));
-      umma_commit(smem_u32(&sm.acc_full[a]));
-    };
-    if (lane == 0 && T > 0) {
-      mbar_wait(smem_u32(&sm.q_full), 0, abort_flag, p.status, 22);
-      if (p.two_pass)
-        for (int j = 0; j < T; ++j) issue(j);
-    }
-    __syncwarp();
-    cluster_arrive();
-    if (lane == 0 && T > 0) {
-      for (int j = p.two_pass ? T : 0; j < n_jobs; ++j) issue(j);
       if (*abort_flag) {  // make sure no MMA is still writing tensor memory before it is freed
         umma_commit(smem_u32(&sm.drain));
         const unsigned long long t0 = globaltimer_ns();
@@ -414,52 +476,72 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         }
       }
     }
-    __syncwarp();
-    cluster_wait();
   } else {
     // =========================================================================== softmax warps
     const int st = tid - 64;              // 0..255
     const int grp = st >> 7;              // accumulator stage this group serves
     const int quad = warp & 3;            // TMEM lane quadrant this warp may read
     const int row_in_tile = quad * 32 + lane;
-    const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
+    const uint32_t tbase = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(grp * kRowsPad);
     const float c = p.c;
-
-    // ---- pass 1: running max / sum of exponentials for rows row_in_tile (+128 when MB == 2)
-    float m_run[MB], z_run[MB];
-    int lim_row[MB];
+    const int n_chunks2 = (p.rows + 31) >> 5;
+    int my_t[MB];
 #pragma unroll
-    for (int mb = 0; mb < MB; ++mb) {
-      m_run[mb] = -INFINITY;
-      z_run[mb] = 0.0f;
-      lim_row[mb] = sm.lim[mb * 128 + row_in_tile];
-    }
-    if (p.two_pass) {
-      for (int j = grp; j < T; j += 2) {
-        const uint32_t aph = (uint32_t)(j >> 1) & 1u;
-        mbar_wait(smem_u32(&sm.acc_full[grp]), aph, abort_flag, p.status, 30);
-        tc_fence_after();
-        const int key0 = (t_begin + j) * kTileN;
+    for (int mb = 0; mb < MB; ++mb) my_t[mb] = sm.row_t[mb * 128 + row_in_tile];
+
+    int jg = 0, it = 0;
+    for (int u = cluster_id; u < p.units; u += n_clusters, ++it) {
+      const UnitInfo ui = get_unit(u);
+      const int n = ui.n, T = ui.T;
+      const int up = it & 1;
+      const int Wp = min(p.W, n);
+
+      if (p.two_pass) {
+        // ---- pass 1: running max / sum of exponentials for rows row_in_tile (+128 when MB == 2)
+        float m_run[MB], z_run[MB];
+        int lim_row[MB];
 #pragma unroll
         for (int mb = 0; mb < MB; ++mb) {
-          const int lim = lim_row[mb];
-          const bool skip = __all_sync(0xffffffffu, lim < 0);
-          const bool full = __all_sync(0xffffffffu, key0 + kTileN - 1 <= lim);
-#pragma unroll 1
-          for (int ch = 0; ch < 4; ++ch) {
-            float v[32];
-            tmem_ld32(tmem_base + lane_addr + (uint32_t)(grp * kRowsPad + mb * 128 + ch * 32), v);
-            if (mb == MB - 1 && ch == 3) {  // all of this job's accumulator is in registers: hand the stage back
+          m_run[mb] = -INFINITY;
+          z_run[mb] = 0.0f;
+          const int pos = n - p.W + my_t[mb];
+          lim_row[mb] = (my_t[mb] >= 0 && pos >= 0) ? (p.causal ? pos : n - 1) : -1;
+        }
+        for (int j = ((jg & 1) == grp) ? 0 : 1; j < T; j += 2) {
+          const int jj = jg + j;
+          mbar_wait(smem_u32(&sm.acc_full[grp]), (uint32_t)(jj >> 1) & 1u, abort_flag, p.status, 30);
+          tc_fence_after();
+          const int key0 = (ui.t_begin + j) * kTileN;
+          bool skip[MB], full[MB];
+#pragma unroll
+          for (int mb = 0; mb < MB; ++mb) {
+            skip[mb] = __all_sync(0xffffffffu, lim_row[mb] < 0);
+            full[mb] = __all_sync(0xffffffffu, key0 + kTileN - 1 <= lim_row[mb]);
+          }
+          uint32_t ra[32], rb[32];
+          tmem_ld32_issue(tbase, ra);
+#pragma unroll
+          for (int cc = 0; cc < 4 * MB; ++cc) {
+            uint32_t(&cur)[32] = (cc & 1) ? rb : ra;
+            uint32_t(&nxt)[32] = (cc & 1) ? ra : rb;
+            tmem_ld_wait(cur);
+            if (cc + 1 < 4 * MB) {
+              tmem_ld32_issue(tbase + (uint32_t)((cc + 1) * 32), nxt);
+            } else {  // the whole accumulator of this job is in registers: hand the stage back to the MMA warp
               tc_fence_before();
               __syncwarp();
               if (lane == 0) mbar_arrive(smem_u32(&sm.acc_empty[grp]));
             }
-            if (skip) continue;
-            if (!full) {
+            const int mb = cc >> 2, ch = cc & 3;
+            if (skip[mb]) continue;
+            float v[32];
+#pragma unroll
+            for (int q = 0; q < 32; ++q) v[q] = __uint_as_float(cur[q]);
+            if (!full[mb]) {
               const int kbase = key0 + ch * 32;
 #pragma unroll
               for (int q = 0; q < 32; ++q)
-                if (kbase + q > lim) v[q] = -INFINITY;
+                if (kbase + q > lim_row[mb]) v[q] = -INFINITY;
             }
             float cmax = v[0];
 #pragma unroll
@@ -467,108 +549,131 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             const float m_new = fmaxf(m_run[mb], cmax);
             if (m_new > -INFINITY) {
               const float mc = m_new * c;
-              float acc = z_run[mb] * ex2(m_run[mb] * c - mc);
+              float acc0 = z_run[mb] * ex2(m_run[mb] * c - mc), acc1 = 0.0f, acc2 = 0.0f, acc3 = 0.0f;
 #pragma unroll
-              for (int q = 0; q < 32; ++q) acc += ex2(fmaf(v[q], c, -mc));
-              z_run[mb] = acc;
+              for (int q = 0; q < 32; q += 4) {
+                acc0 += ex2(fmaf(v[q + 0], c, -mc));
+                acc1 += ex2(fmaf(v[q + 1], c, -mc));
+                acc2 += ex2(fmaf(v[q + 2], c, -mc));
+                acc3 += ex2(fmaf(v[q + 3], c, -mc));
+              }
+              z_run[mb] = (acc0 + acc1) + (acc2 + acc3);
               m_run[mb] = m_new;
             }
           }
         }
-      }
-      // ---- exchange: group partials -> CTA partial -> every CTA of the cluster
+        // ---- exchange: group partials -> CTA partial -> every CTA of the cluster
 #pragma unroll
-      for (int mb = 0; mb < MB; ++mb) {
-        sm.part_m[grp][mb * 128 + row_in_tile] = m_run[mb];
-        sm.part_z[grp][mb * 128 + row_in_tile] = z_run[mb];
-      }
-      softmax_bar();
-      if (st < kRowsPad) {
-        const float m0 = sm.part_m[0][st], m1 = sm.part_m[1][st];
-        const float m = fmaxf(m0, m1);
-        float z = 0.0f;
-        if (m > -INFINITY) z = sm.part_z[0][st] * ex2((m0 - m) * c) + sm.part_z[1][st] * ex2((m1 - m) * c);
-        for (int r = 0; r < p.cluster; ++r) {
-          st_cluster_f32(smem_u32(&sm.xchg_m[rank][st]), (uint32_t)r, m);
-          st_cluster_f32(smem_u32(&sm.xchg_z[rank][st]), (uint32_t)r, z);
+        for (int mb = 0; mb < MB; ++mb) {
+          sm.part_m[grp][mb * 128 + row_in_tile] = m_run[mb];
+          sm.part_z[grp][mb * 128 + row_in_tile] = z_run[mb];
         }
+        softmax_bar();
+        if (st < kRowsPad) {
+          const float m0 = sm.part_m[0][st], m1 = sm.part_m[1][st];
+          float m = fmaxf(m0, m1);
+          float z = 0.0f;
+          if (m > -INFINITY) z = sm.part_z[0][st] * ex2((m0 - m) * c) + sm.part_z[1][st] * ex2((m1 - m) * c);
+          const uint32_t bar = smem_u32(&sm.xchg_full[up]);
+          for (int r = 0; r < p.cluster; ++r) {
+            st_cluster_f32(smem_u32(&sm.xchg_m[up][rank][st]), (uint32_t)r, m);
+            st_cluster_f32(smem_u32(&sm.xchg_z[up][rank][st]), (uint32_t)r, z);
+            mbar_arrive_remote(bar, (uint32_t)r);  // release: the two stores above are visible to who acquires
+          }
+          mbar_wait_cluster(bar, (uint32_t)(it >> 1) & 1u, abort_flag, p.status, 32);
+          m = -INFINITY;
+          for (int r = 0; r < p.cluster; ++r) m = fmaxf(m, sm.xchg_m[up][r][st]);
+          z = 0.0f;
+          if (m > -INFINITY)
+            for (int r = 0; r < p.cluster; ++r) z += sm.xchg_z[up][r][st] * ex2((sm.xchg_m[up][r][st] - m) * c);
+          sm.lse2[up][st] = (z > 0.0f) ? m * c + log2f(z) : INFINITY;
+        }
+        softmax_bar();
+      } else {
+        if (st < kRowsPad) {
+          float lse2 = INFINITY;
+          const int t = sm.row_t[st];
+          if (t >= 0 && n - p.W + t >= 0) {
+            const int h = st / p.W;
+            const float lse = p.lse_obs[(((long long)ui.l * p.seq.batch + ui.b) * p.Hq + (ui.g * p.G + h)) * p.W + t];
+            lse2 = lse * 1.4426950408889634f;
+          }
+          sm.lse2[up][st] = lse2;
+        }
+        softmax_bar();
       }
-    }
-    cluster_arrive();
-    cluster_wait();
-    if (p.two_pass) {
-      if (st < kRowsPad) {
-        float m = -INFINITY;
-        for (int r = 0; r < p.cluster; ++r) m = fmaxf(m, sm.xchg_m[r][st]);
-        float z = 0.0f;
-        if (m > -INFINITY)
-          for (int r = 0; r < p.cluster; ++r) z += sm.xchg_z[r][st] * ex2((sm.xchg_m[r][st] - m) * c);
-        sm.lse2[st] = (z > 0.0f) ? m * c + log2f(z) : INFINITY;
-      }
-      softmax_bar();
-    }
 
-    // ---- pass 2: column sums for key row_in_tile of each tile
-    const int min_lim = p.causal ? n - Wp : n - 1;  // every valid row sees keys up to here
-    const int j0 = p.two_pass ? T : 0;
-    const int first = j0 + (((j0 & 1) == grp) ? 0 : 1);
-    const long long unit_off = ((long long)l * p.Hkv + g) * p.seq.total;
-    for (int j = first; j < n_jobs; j += 2) {
-      const uint32_t aph = (uint32_t)(j >> 1) & 1u;
-      mbar_wait(smem_u32(&sm.acc_full[grp]), aph, abort_flag, p.status, 31);
-      tc_fence_after();
-      const int key = (t_begin + (j - j0)) * kTileN + row_in_tile;
-      const bool fast_path = __all_sync(0xffffffffu, key <= min_lim || key >= n);
-      float sumA = 0.0f, sumP = 0.0f;
-      const int n_chunks = (p.rows + 31) >> 5;
-#pragma unroll 1
-      for (int ch = 0; ch < n_chunks; ++ch) {
-        float v[32];
-        tmem_ld32(tmem_base + lane_addr + (uint32_t)(grp * kRowsPad + ch * 32), v);
-        if (ch == n_chunks - 1) {
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(smem_u32(&sm.acc_empty[grp]));
-        }
-        const float4* l4 = reinterpret_cast<const float4*>(&sm.lse2[ch * 32]);
-        const float4* w4 = reinterpret_cast<const float4*>(&sm.wrow[ch * 32]);
-        if (fast_path) {
+      // ---- pass 2: column sums for key row_in_tile of each tile
+      const int min_lim = p.causal ? n - Wp : n - 1;  // every valid row sees keys up to here
+      const int j0 = p.two_pass ? T : 0;
+      const int n_jobs = j0 + T;
+      const long long unit_off = ((long long)ui.l * p.Hkv + ui.g) * p.seq.total;
+      const float4* l4 = reinterpret_cast<const float4*>(sm.lse2[up]);
+      const float4* w4 = reinterpret_cast<const float4*>(sm.wrow);
+      for (int j = j0 + ((((jg + j0) & 1) == grp) ? 0 : 1); j < n_jobs; j += 2) {
+        const int jj = jg + j;
+        mbar_wait(smem_u32(&sm.acc_full[grp]), (uint32_t)(jj >> 1) & 1u, abort_flag, p.status, 31);
+        tc_fence_after();
+        const int key = (ui.t_begin + (j - j0)) * kTileN + row_in_tile;
+        const bool fast_path = __all_sync(0xffffffffu, key <= min_lim || key >= n);
+        float sA0 = 0.0f, sA1 = 0.0f, sP0 = 0.0f, sP1 = 0.0f;
+        uint32_t ra[32], rb[32];
+        tmem_ld32_issue(tbase, ra);
 #pragma unroll
-          for (int q = 0; q < 8; ++q) {
-            const float4 ls = l4[q];
-            const float a0 = ex2(fmaf(v[4 * q + 0], c, -ls.x));
-            const float a1 = ex2(fmaf(v[4 * q + 1], c, -ls.y));
-            const float a2 = ex2(fmaf(v[4 * q + 2], c, -ls.z));
-            const float a3 = ex2(fmaf(v[4 * q + 3], c, -ls.w));
-            sumA += (a0 + a1) + (a2 + a3);
-            if (kNeedP) {
-              const float4 ws = w4[q];
-              sumP = fmaf(ws.x, a0, sumP);
-              sumP = fmaf(ws.y, a1, sumP);
-              sumP = fmaf(ws.z, a2, sumP);
-              sumP = fmaf(ws.w, a3, sumP);
+        for (int cc = 0; cc < 4 * MB; ++cc) {
+          if (cc < n_chunks2) {
+            uint32_t(&cur)[32] = (cc & 1) ? rb : ra;
+            uint32_t(&nxt)[32] = (cc & 1) ? ra : rb;
+            tmem_ld_wait(cur);
+            if (cc + 1 < n_chunks2) {
+              tmem_ld32_issue(tbase + (uint32_t)((cc + 1) * 32), nxt);
+            } else {
+              tc_fence_before();
+              __syncwarp();
+              if (lane == 0) mbar_arrive(smem_u32(&sm.acc_empty[grp]));
+            }
+            if (fast_path) {
+#pragma unroll
+              for (int q = 0; q < 8; ++q) {
+                const float4 ls = l4[cc * 8 + q];
+                const float a0 = ex2(fmaf(__uint_as_float(cur[4 * q + 0]), c, -ls.x));
+                const float a1 = ex2(fmaf(__uint_as_float(cur[4 * q + 1]), c, -ls.y));
+                const float a2 = ex2(fmaf(__uint_as_float(cur[4 * q + 2]), c, -ls.z));
+                const float a3 = ex2(fmaf(__uint_as_float(cur[4 * q + 3]), c, -ls.w));
+                sA0 += a0 + a1;
+                sA1 += a2 + a3;
+                if (kNeedP) {
+                  const float4 ws = w4[cc * 8 + q];
+                  sP0 = fmaf(ws.x, a0, sP0);
+                  sP1 = fmaf(ws.y, a1, sP1);
+                  sP0 = fmaf(ws.z, a2, sP0);
+                  sP1 = fmaf(ws.w, a3, sP1);
+                }
+              }
+            } else {
+#pragma unroll
+              for (int q = 0; q < 32; ++q) {
+                const int r = cc * 32 + q;
+                const int t = sm.row_t[r];
+                const int pos = n - p.W + t;
+                const int lim = (t >= 0 && pos >= 0) ? (p.causal ? pos : n - 1) : -1;
+                float a = 0.0f;
+                if (key <= lim) a = ex2(fmaf(__uint_as_float(cur[q]), c, -sm.lse2[up][r]));
+                sA0 += a;
+                if (kNeedP) sP0 = fmaf(sm.wrow[r], a, sP0);
+              }
             }
           }
-        } else {
-#pragma unroll
-          for (int q = 0; q < 32; ++q) {
-            const int r = ch * 32 + q;
-            float a = 0.0f;
-            if (key <= sm.lim[r]) a = ex2(fmaf(v[q], c, -sm.lse2[r]));
-            sumA += a;
-            if (kNeedP) sumP = fmaf(sm.wrow[r], a, sumP);
-          }
+        }
+        if (key < n) {
+          const float sumA = sA0 + sA1, sumP = sP0 + sP1;
+          const long long o = unit_off + ui.tok0 + key;
+          if (p.A) p.A[o] = sumA;
+          if (p.P) p.P[o] = sumP;
+          if (p.u) p.u[o] = __fadd_rn(__fmul_rn(p.alpha, sumA), __fmul_rn(p.delta, sumP));
         }
       }
-      if (key < n) {
-        const long long o = unit_off + tok0 + key;
-        if (p.A) p.A[o] = sumA;
-        if (p.P) p.P[o] = sumP;
-        if (p.u) {
-          const float t = __fadd_rn(__fmul_rn(p.alpha, sumA), __fmul_rn(p.delta, sumP));
-          p.u[o] = __fadd_rn(t, p.u_static[tok0 + key]);
-        }
-      }
+      if (T > 0) jg += n_jobs;
     }
   }
 
@@ -579,6 +684,9 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     tc_fence_after();
     tmem_dealloc(tmem_base, kTmemCols);
   }
+  // no CTA may leave while a peer can still store into its shared memory or arrive on its barriers
+  cluster_arrive();
+  cluster_wait();
 }
 
 template <int MB>
@@ -606,14 +714,18 @@ CUresult encode_5d(void* fn, CUtensorMap* map, const void* base, const uint64_t 
 }
 
 template <int MB, bool NP>
-cudaError_t launch_variant(const CUtensorMap& mq, const CUtensorMap& mk, const ScoreParams& sp, int units,
+cudaError_t launch_variant(ta_ctx* ctx, const CUtensorMap& mq, const CUtensorMap& mk, ScoreParams& sp,
                            cudaStream_t stream) {
   auto kern = ta_score_kernel<MB, NP>;
   const size_t smem = score_smem_bytes<MB>();
-  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  if (e != cudaSuccess) return e;
+  static bool attr_set_dev[64] = {};  // per device and instantiation; the attribute is sticky
+  bool& attr_set = attr_set_dev[ctx->device & 63];
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)(units * sp.cluster), 1, 1);
   cfg.blockDim = dim3(kThreads, 1, 1);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = stream;
@@ -624,6 +736,21 @@ cudaError_t launch_variant(const CUtensorMap& mq, const CUtensorMap& mk, const S
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
+  // persistent grid: as many clusters as can be resident at once (queried once per cluster size)
+  static int max_clusters_dev[64][kMaxCluster + 1] = {};
+  int* max_clusters = max_clusters_dev[ctx->device & 63];
+  if (max_clusters[sp.cluster] == 0) {
+    cfg.gridDim = dim3((unsigned)(ctx->sm_count / sp.cluster * sp.cluster), 1, 1);
+    int n = 0;
+    cudaError_t e = cudaOccupancyMaxActiveClusters(&n, kern, &cfg);
+    if (e != cudaSuccess) return e;
+    if (n < 1) return cudaErrorLaunchOutOfResources;
+    max_clusters[sp.cluster] = n;
+  }
+  const int n_clusters = sp.units < max_clusters[sp.cluster] ? sp.units : max_clusters[sp.cluster];
+  ctx->score_cluster = sp.cluster;
+  ctx->score_clusters = n_clusters;
+  cfg.gridDim = dim3((unsigned)(n_clusters * sp.cluster), 1, 1);
   return cudaLaunchKernelEx(&cfg, kern, mq, mk, sp);
 }
 
@@ -662,8 +789,13 @@ cudaError_t ta_launch_score(ta_ctx* ctx, const ta_score_args& a, ta_dev_status* 
   sp.status = status;
   sp.rho = a.rho;
   for (int t = 0; t < a.W; ++t) sp.wrow[t] = (float)((1.0 - (double)a.rho) * pow((double)a.rho, (double)(a.W - 1 - t)));
+  sp.units = units;
+  // CTAs per unit: at least four 128-key tiles per CTA, and more CTAs per unit when there are few units
   const int tiles_max = (a.seq.max_n + kTileN - 1) / kTileN;
-  sp.cluster = tiles_max >= 32 ? 8 : tiles_max >= 16 ? 4 : tiles_max >= 8 ? 2 : 1;
+  int cl = 4;
+  while (cl > 1 && tiles_max < 4 * cl) cl >>= 1;
+  if (cl == 4 && units * 8 <= ctx->sm_count && tiles_max >= 32) cl = 8;
+  sp.cluster = cl;
 
   // tensor maps: dims (d, position, head, batch, layer)
   CUtensorMap mq, mk;
@@ -684,8 +816,7 @@ cudaError_t ta_launch_score(ta_ctx* ctx, const ta_score_args& a, ta_dev_status* 
     if (encode_5d(ctx->encode_tiled, &mk, a.k.ptr, dims, str, box) != CUDA_SUCCESS) return cudaErrorInvalidValue;
   }
   const bool need_p = a.P != nullptr || (a.u != nullptr && a.delta != 0.0f);
-  if (MB == 1) return need_p ? launch_variant<1, true>(mq, mk, sp, units, stream)
-                             : launch_variant<1, false>(mq, mk, sp, units, stream);
-  return need_p ? launch_variant<2, true>(mq, mk, sp, units, stream)
-                : launch_variant<2, false>(mq, mk, sp, units, stream);
+  if (MB == 1) return need_p ? launch_variant<1, true>(ctx, mq, mk, sp, stream)
+                             : launch_variant<1, false>(ctx, mq, mk, sp, stream);
+  return need_p ? launch_variant<2, true>(ctx, mq, mk, sp, stream) : launch_variant<2, false>(ctx, mq, mk, sp, stream);
 }

@@ -234,8 +234,8 @@ struct UnitSrc {  // where a unit's utility comes from
 };
 
 __device__ __forceinline__ float unit_utility(const UnitSrc& src, long long unit_off, long long tok) {
-  if (src.u) return src.u[unit_off + tok];
   const float u0 = src.u_static[tok];
+  if (src.u) return __fadd_rn(src.u[unit_off + tok], u0);
   if (!src.A) return u0;
   const float aA = __fmul_rn(src.alpha, src.A[unit_off + tok]);
   const float dP = __fmul_rn(src.delta, src.P ? src.P[unit_off + tok] : 0.0f);
@@ -312,12 +312,15 @@ __global__ void ta_broadcast_idx_kernel(int B, int Hkv, int K, int n_layers, con
 // Scratch layout used by the launcher (the caller carves it): forced [total] bytes, r_main [B] ints; fast mode
 // additionally idx_seq [B][K] and count_seq [B] (passed through a.idx / a.count by the caller when it wants the
 // per-sequence result only).
-cudaError_t ta_launch_select(const ta_select_args& a, ta_dev_status* status, cudaStream_t stream) {
+cudaError_t ta_launch_forced(const ta_select_args& a, ta_dev_status* status, cudaStream_t stream) {
   if (a.seq.batch == 0 || a.n_layers == 0) return cudaSuccess;
   ta_forced_kernel<<<a.seq.batch, kThreads, 0, stream>>>(a.seq, a.K, a.n_sink, a.n_recent, a.k_protected, a.voucher,
                                                          a.forced, a.r_main, status);
-  cudaError_t e = cudaGetLastError();
-  if (e != cudaSuccess) return e;
+  return cudaGetLastError();
+}
+
+cudaError_t ta_launch_select_units(const ta_select_args& a, cudaStream_t stream) {
+  if (a.seq.batch == 0 || a.n_layers == 0) return cudaSuccess;
   UnitSrc src;
   src.u = a.fast ? nullptr : a.u;
   src.A = a.fast ? nullptr : a.A;
@@ -329,6 +332,12 @@ cudaError_t ta_launch_select(const ta_select_args& a, ta_dev_status* status, cud
   ta_select_kernel<<<units, kThreads, 0, stream>>>(a.seq, a.n_layers, a.Hkv, a.K, a.fast, src, a.forced, a.r_main,
                                                    a.idx, a.count);
   return cudaGetLastError();
+}
+
+cudaError_t ta_launch_select(const ta_select_args& a, ta_dev_status* status, cudaStream_t stream) {
+  cudaError_t e = ta_launch_forced(a, status, stream);
+  if (e != cudaSuccess) return e;
+  return ta_launch_select_units(a, stream);
 }
 
 cudaError_t ta_launch_broadcast_idx(int B, int Hkv, int K, int n_layers, const int32_t* idx_seq,
