@@ -19,11 +19,14 @@
 // tile, ring of key tiles, two accumulator stages), so barrier set-up, TMEM allocation and pipeline fill are paid
 // once per CTA and not once per unit.
 //
-// Warp roles (320 threads): warp 0 TMA producer, warp 1 MMA issuer + TMEM owner, warps 2-9 two softmax groups that
-// alternate over the two accumulator stages. Every wait on an mbarrier is bounded by wall time; when one runs out
+// Warp roles (384 threads, three warpgroups): warps 0-7 are two softmax groups that alternate over the accumulator
+// stages, warp 8 is the TMA producer, warp 9 the MMA issuer and TMEM owner, warps 10-11 idle. After set-up the third
+// warpgroup gives registers back (setmaxnreg) and the softmax warpgroups take them. Every wait on an mbarrier is bounded by wall time; when one runs out
 // the CTA records TA_ERR_TIMEOUT, stops waiting anywhere, drains its copies, frees its tensor memory and returns.
 // The only unbounded waits are two hardware cluster barriers (start, end) that every thread reaches on every path.
 #include <cuda.h>
+
+#include <type_traits>
 
 #include "ta_internal.cuh"
 
@@ -34,7 +37,10 @@ constexpr int kD = TA_HEAD_DIM;                   // 128
 constexpr int kHalfBytes = kTileN * 128;          // one 64-column half of a 128-row operand tile: 16 KB
 constexpr int kKTileBytes = 2 * kHalfBytes;       // 32 KB
 constexpr int kMaxCluster = 8;
-constexpr int kThreads = 320;
+constexpr int kThreads = 384;                     // warps 0-7 softmax, 8 TMA producer, 9 MMA issuer, 10-11 idle
+constexpr int kRegsSoftmax = 216;                 // register split after set-up (setmaxnreg): 8 softmax warps
+constexpr int kRegsOther = 72;                    // ... and the 4 warps of the third warpgroup
+constexpr int kRegsNeeded = (8 * kRegsSoftmax + 4 * kRegsOther) * 32;  // must fit in threads x registers at launch
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s
 
 struct ScoreParams {
@@ -89,11 +95,10 @@ __device__ __forceinline__ unsigned long long globaltimer_ns() {
 }
 
 // Bounded wait. Returns false (and raises the CTA's abort flag) when the limit is reached or another thread of the
-// CTA already gave up.
-__device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                       ta_dev_status* status, int where) {
+// CTA already gave up. The common case (the phase has completed) is one inlined try_wait.
+__device__ __forceinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                            ta_dev_status* status, int where) {
   if (*abort_flag) return false;
-  if (mbar_try_wait(bar, parity)) return true;
   const unsigned long long t0 = globaltimer_ns();
   for (;;) {
 #pragma unroll 1
@@ -110,6 +115,11 @@ __device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile i
       return false;
     }
   }
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          ta_dev_status* status, int where) {
+  if (mbar_try_wait(bar, parity)) return true;
+  return mbar_wait_slow(bar, parity, abort_flag, status, where);
 }
 
 __device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1,
@@ -188,6 +198,14 @@ __device__ __forceinline__ uint32_t cluster_ctarank() {
   asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
   return r;
 }
+__device__ __forceinline__ float ld_cluster_f32(uint32_t local_addr, uint32_t rank) {
+  uint32_t remote;
+  float v;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
+  asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(remote) : "memory");
+  return v;
+}
+__device__ __forceinline__ void fence_cluster() { asm volatile("fence.acq_rel.cluster;" ::: "memory"); }
 __device__ __forceinline__ void st_cluster_f32(uint32_t local_addr, uint32_t rank, float v) {
   uint32_t remote;
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
@@ -232,10 +250,10 @@ __device__ __forceinline__ uint32_t idesc_bf16(int M, int N) {
 }
 
 // Bounded wait with cluster-scope acquire (for barriers that peers of the cluster arrive on).
-__device__ __noinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag,
                                                ta_dev_status* status, int where) {
-  if (*abort_flag) return false;
   if (mbar_try_wait_cluster(bar, parity)) return true;
+  if (*abort_flag) return false;
   const unsigned long long t0 = globaltimer_ns();
   for (;;) {
 #pragma unroll 1
@@ -260,6 +278,7 @@ struct ScoreCfg {
   static constexpr int kQBufs = MB == 1 ? 2 : 1;   // query tiles in flight (next unit's tile loads early)
   static constexpr int kStages = MB == 1 ? 4 : 3;  // ring of key tiles
   static constexpr int kRowsPad = MB * 128;
+  static constexpr int kAcc = MB == 1 ? 4 : 2;     // accumulator stages in tensor memory (kAcc * kRowsPad = 512 columns)
 };
 
 template <int MB>
@@ -267,31 +286,40 @@ struct alignas(1024) ScoreSmem {
   using Cfg = ScoreCfg<MB>;
   uint8_t q[Cfg::kQBufs][MB * 2 * kHalfBytes];    // [buffer][half][MB*128 rows][128 B]
   uint8_t k[Cfg::kStages][kKTileBytes];           // [stage][half][128 rows][128 B]
-  float xchg_m[2][kMaxCluster][MB * 128];         // [unit parity][cluster rank][row]: per-CTA row statistics
-  float xchg_z[2][kMaxCluster][MB * 128];
+  float mine_m[2][MB * 128];                      // [unit parity][row]: this CTA's row statistics, read by its peers
+  float mine_z[2][MB * 128];
   float part_m[2][MB * 128];                      // per softmax group
   float part_z[2][MB * 128];
   float lse2[2][MB * 128];                        // [unit parity][row] log2-domain log-sum-exp (+inf: row is mute)
   float wrow[MB * 128];                           // pension weight per row
   int row_t[MB * 128];                            // window index t of the row, -1 for padding rows
-  unsigned long long full[Cfg::kStages], empty[Cfg::kStages], acc_full[2], acc_empty[2];
+  unsigned long long full[Cfg::kStages], empty[Cfg::kStages], acc_full[Cfg::kAcc], acc_empty[Cfg::kAcc];
   unsigned long long q_full[Cfg::kQBufs], q_empty[Cfg::kQBufs], xchg_full[2], drain;
   uint32_t tmem_base;
   int abort_flag;
 };
+
+// Pass-2 order of the 32-row chunks of an accumulator (as a TMEM column offset). With W = 64 and the pension term
+// (PM 2) the chunks holding window positions 0..31 of every head come first, then those holding 32..63.
+template <int MB, int PM>
+__device__ __forceinline__ uint32_t chunk_col(int ci) {
+  if (PM == 2) return (uint32_t)((ci < 2 * MB ? 2 * ci : 2 * (ci - 2 * MB) + 1) * 32);
+  return (uint32_t)(ci * 32);
+}
 
 struct UnitInfo {
   int l, b, g, tok0, n, t_begin, T;
 };
 
 // ---------------------------------------------------------------------------------------------- the kernel
-template <int MB, bool kNeedP>
+template <int MB, int PM>
 __global__ void __launch_bounds__(kThreads, 1)
 ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                 const __grid_constant__ ScoreParams p) {
   using Cfg = ScoreCfg<MB>;
   constexpr int kStages = Cfg::kStages, kQBufs = Cfg::kQBufs, kRowsPad = Cfg::kRowsPad;
-  constexpr uint32_t kTmemCols = MB * 256;
+  constexpr int kAcc = Cfg::kAcc;
+  constexpr uint32_t kTmemCols = 512;  // kAcc accumulator stages of kRowsPad columns
   constexpr int kQBytes = MB * 2 * kHalfBytes;
   extern __shared__ uint8_t smem_raw[];
   ScoreSmem<MB>& sm = *reinterpret_cast<ScoreSmem<MB>*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -330,11 +358,11 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
       mbar_init(smem_u32(&sm.full[s]), 1);
       mbar_init(smem_u32(&sm.empty[s]), 1);
     }
-    for (int a = 0; a < 2; ++a) {
+    for (int a = 0; a < kAcc; ++a) {
       mbar_init(smem_u32(&sm.acc_full[a]), 1);
       mbar_init(smem_u32(&sm.acc_empty[a]), 4);
-      mbar_init(smem_u32(&sm.xchg_full[a]), (uint32_t)(p.cluster * kRowsPad));
     }
+    for (int a = 0; a < 2; ++a) mbar_init(smem_u32(&sm.xchg_full[a]), (uint32_t)p.cluster);
     for (int qb = 0; qb < kQBufs; ++qb) {
       mbar_init(smem_u32(&sm.q_full[qb]), 1);
       mbar_init(smem_u32(&sm.q_empty[qb]), 1);
@@ -344,7 +372,7 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     sm.abort_flag = (*reinterpret_cast<volatile int*>(&p.status->code) == (int)TA_ERR_TIMEOUT) ? 1 : 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 1) {
+  if (warp == 9) {
     tmem_alloc(smem_u32(&sm.tmem_base), kTmemCols);
     tmem_relinquish();
   }
@@ -376,7 +404,9 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 
   const uint32_t k_smem = smem_u32(sm.k);
 
-  if (warp == 0) {
+  if (warp >= 8) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsOther));
+  if (warp == 8) {
     // =========================================================================== TMA producer
     if (lane == 0) {
       int issued[kStages];
@@ -421,46 +451,44 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         }
       }
     }
-  } else if (warp == 1) {
+  } else if (warp == 9) {
     // =========================================================================== MMA issuer
     if (lane == 0) {
       int jg = 0, qn = 0;
+      const uint64_t dk_base = smem_desc_sw128(k_smem);
+      const uint32_t idesc1 = idesc_bf16(128, kTileN), idesc2 = idesc_bf16(128, kRowsPad);
       for (int u = cluster_id; u < p.units; u += n_clusters) {
         const UnitInfo ui = get_unit(u);
         if (ui.T == 0) continue;
         const int qb = qn % kQBufs;
         mbar_wait(smem_u32(&sm.q_full[qb]), (uint32_t)(qn / kQBufs) & 1u, abort_flag, p.status, 22);
-        const uint32_t q_smem = smem_u32(sm.q[qb]);
+        const uint64_t dq = smem_desc_sw128(smem_u32(sm.q[qb]));
         const int n_jobs = p.two_pass ? 2 * ui.T : ui.T;
         for (int j = 0; j < n_jobs; ++j, ++jg) {
           const int s = jg % kStages;
-          const int a = jg & 1;
+          const int a = jg % kAcc;
           const bool stats = p.two_pass && j < ui.T;
           mbar_wait(smem_u32(&sm.full[s]), (uint32_t)(jg / kStages) & 1u, abort_flag, p.status, 20);
-          mbar_wait(smem_u32(&sm.acc_empty[a]), ((uint32_t)(jg >> 1) & 1u) ^ 1u, abort_flag, p.status, 21);
+          mbar_wait(smem_u32(&sm.acc_empty[a]), ((uint32_t)(jg / kAcc) & 1u) ^ 1u, abort_flag, p.status, 21);
           tc_fence_after();
-          const uint32_t kt = k_smem + s * kKTileBytes;
+          const uint64_t dk = dk_base + (uint64_t)((uint32_t)(s * kKTileBytes) >> 4);
           const uint32_t acc = tmem_base + (uint32_t)(a * kRowsPad);
           if (stats) {
-            const uint32_t idesc = idesc_bf16(128, kTileN);
 #pragma unroll
             for (int mb = 0; mb < MB; ++mb) {
 #pragma unroll
               for (int k = 0; k < 8; ++k) {
-                const uint32_t off = (uint32_t)(k & 3) * 32u;
-                const uint64_t da = smem_desc_sw128(q_smem + (k >> 2) * (MB * kHalfBytes) + mb * kHalfBytes + off);
-                const uint64_t db = smem_desc_sw128(kt + (k >> 2) * kHalfBytes + off);
-                umma_bf16(acc + mb * 128, da, db, idesc, k > 0);
+                const uint64_t da = dq + (uint64_t)(((k >> 2) * (MB * kHalfBytes) + mb * kHalfBytes + (k & 3) * 32) >> 4);
+                const uint64_t db = dk + (uint64_t)(((k >> 2) * kHalfBytes + (k & 3) * 32) >> 4);
+                umma_bf16(acc + mb * 128, da, db, idesc1, k > 0);
               }
             }
           } else {
-            const uint32_t idesc = idesc_bf16(128, kRowsPad);
 #pragma unroll
             for (int k = 0; k < 8; ++k) {
-              const uint32_t off = (uint32_t)(k & 3) * 32u;
-              const uint64_t da = smem_desc_sw128(kt + (k >> 2) * kHalfBytes + off);
-              const uint64_t db = smem_desc_sw128(q_smem + (k >> 2) * (MB * kHalfBytes) + off);
-              umma_bf16(acc, da, db, idesc, k > 0);
+              const uint64_t da = dk + (uint64_t)(((k >> 2) * kHalfBytes + (k & 3) * 32) >> 4);
+              const uint64_t db = dq + (uint64_t)(((k >> 2) * (MB * kHalfBytes) + (k & 3) * 32) >> 4);
+              umma_bf16(acc, da, db, idesc2, k > 0);
             }
           }
           umma_commit(smem_u32(&sm.empty[s]));
@@ -476,18 +504,31 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         }
       }
     }
+  }
   } else {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmax));
     // =========================================================================== softmax warps
-    const int st = tid - 64;              // 0..255
-    const int grp = st >> 7;              // accumulator stage this group serves
+    const int st = tid;                   // 0..255
+    const int grp = st >> 7;              // this group serves jobs with (global job index & 1) == grp
     const int quad = warp & 3;            // TMEM lane quadrant this warp may read
     const int row_in_tile = quad * 32 + lane;
-    const uint32_t tbase = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(grp * kRowsPad);
+    const uint32_t tlane = tmem_base + ((uint32_t)(quad * 32) << 16);
     const float c = p.c;
     const int n_chunks2 = (p.rows + 31) >> 5;
     int my_t[MB];
 #pragma unroll
     for (int mb = 0; mb < MB; ++mb) my_t[mb] = sm.row_t[mb * 128 + row_in_tile];
+
+    auto acc_addr = [&](int jj) { return tlane + (uint32_t)((jj % kAcc) * kRowsPad); };
+    auto wait_full = [&](int jj, int where) {
+      mbar_wait(smem_u32(&sm.acc_full[jj % kAcc]), (uint32_t)(jj / kAcc) & 1u, abort_flag, p.status, where);
+      tc_fence_after();
+    };
+    auto release = [&](int jj) {  // the whole accumulator of the job is in registers: hand the stage back
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&sm.acc_empty[jj % kAcc]));
+    };
 
     int jg = 0, it = 0;
     for (int u = cluster_id; u < p.units; u += n_clusters, ++it) {
@@ -497,96 +538,145 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
       const int Wp = min(p.W, n);
 
       if (p.two_pass) {
-        // ---- pass 1: running max / sum of exponentials for rows row_in_tile (+128 when MB == 2)
-        float m_run[MB], z_run[MB];
+        // ---- pass 1: per row, sum of exp2(s*c - ref) against a reference `ref` that trails the running maximum:
+        // the exponentials of a chunk use the reference left by the previous chunks, so they do not wait for the
+        // chunk's own maximum; only when the maximum jumps by more than 2^8 is the chunk redone with a new reference.
+        float ref_c[MB], z_run[MB];
         int lim_row[MB];
 #pragma unroll
         for (int mb = 0; mb < MB; ++mb) {
-          m_run[mb] = -INFINITY;
+          ref_c[mb] = -1e30f;
           z_run[mb] = 0.0f;
           const int pos = n - p.W + my_t[mb];
           lim_row[mb] = (my_t[mb] >= 0 && pos >= 0) ? (p.causal ? pos : n - 1) : -1;
         }
-        for (int j = ((jg & 1) == grp) ? 0 : 1; j < T; j += 2) {
+        // one 32-key chunk of one row; `lim` < INT_MAX masks keys beyond it (cold tiles only)
+        auto chunk1 = [&](auto masked_tag, const uint32_t(&cur)[32], float& rc_io, float& z_io, int kbase, int lim) {
+          constexpr bool masked = decltype(masked_tag)::value;
+          float v[32];
+#pragma unroll
+          for (int q = 0; q < 32; ++q) v[q] = __uint_as_float(cur[q]);
+          if (masked) {
+#pragma unroll
+            for (int q = 0; q < 32; ++q)
+              if (kbase + q > lim) v[q] = -INFINITY;
+          }
+          const float rc = rc_io;
+          float a0 = 0.0f, a1 = 0.0f, a2 = 0.0f, a3 = 0.0f;
+#pragma unroll
+          for (int q = 0; q < 32; q += 4) {
+            a0 += ex2(fmaf(v[q + 0], c, -rc));
+            a1 += ex2(fmaf(v[q + 1], c, -rc));
+            a2 += ex2(fmaf(v[q + 2], c, -rc));
+            a3 += ex2(fmaf(v[q + 3], c, -rc));
+          }
+          float t8[8];
+#pragma unroll
+          for (int q = 0; q < 8; ++q) t8[q] = fmaxf(fmaxf(v[4 * q], v[4 * q + 1]), fmaxf(v[4 * q + 2], v[4 * q + 3]));
+          const float cmax = fmaxf(fmaxf(fmaxf(t8[0], t8[1]), fmaxf(t8[2], t8[3])),
+                                   fmaxf(fmaxf(t8[4], t8[5]), fmaxf(t8[6], t8[7])));
+          const float cm_c = cmax * c;
+          const bool jump = cm_c > rc + 8.0f;
+          float add = (a0 + a1) + (a2 + a3);
+          if (__any_sync(0xffffffffu, jump)) {
+            if (jump) {  // new reference = this chunk's maximum; earlier sums are rescaled, the chunk is redone
+              z_io *= ex2(rc - cm_c);
+              rc_io = cm_c;
+              float b0 = 0.0f, b1 = 0.0f;
+#pragma unroll
+              for (int q = 0; q < 32; q += 2) {
+                b0 += ex2(fmaf(v[q + 0], c, -cm_c));
+                b1 += ex2(fmaf(v[q + 1], c, -cm_c));
+              }
+              add = b0 + b1;
+            }
+          }
+          z_io += add;
+        };
+        uint32_t ra[32], rb[32];
+        int j = ((jg & 1) == grp) ? 0 : 1;
+        if (j < T) {
+          wait_full(jg + j, 30);
+          tmem_ld32_issue(acc_addr(jg + j), ra);
+        }
+        // one job: all chunks of the accumulator, two register sets in flight, the next job's first load issued
+        // before the last chunk is computed
+        auto job1 = [&](auto masked_tag, int j) {
           const int jj = jg + j;
-          mbar_wait(smem_u32(&sm.acc_full[grp]), (uint32_t)(jj >> 1) & 1u, abort_flag, p.status, 30);
-          tc_fence_after();
           const int key0 = (ui.t_begin + j) * kTileN;
-          bool skip[MB], full[MB];
+          const uint32_t abase = acc_addr(jj);
 #pragma unroll
           for (int mb = 0; mb < MB; ++mb) {
-            skip[mb] = __all_sync(0xffffffffu, lim_row[mb] < 0);
-            full[mb] = __all_sync(0xffffffffu, key0 + kTileN - 1 <= lim_row[mb]);
-          }
-          uint32_t ra[32], rb[32];
-          tmem_ld32_issue(tbase, ra);
-#pragma unroll
-          for (int cc = 0; cc < 4 * MB; ++cc) {
-            uint32_t(&cur)[32] = (cc & 1) ? rb : ra;
-            uint32_t(&nxt)[32] = (cc & 1) ? ra : rb;
-            tmem_ld_wait(cur);
-            if (cc + 1 < 4 * MB) {
-              tmem_ld32_issue(tbase + (uint32_t)((cc + 1) * 32), nxt);
-            } else {  // the whole accumulator of this job is in registers: hand the stage back to the MMA warp
-              tc_fence_before();
-              __syncwarp();
-              if (lane == 0) mbar_arrive(smem_u32(&sm.acc_empty[grp]));
-            }
-            const int mb = cc >> 2, ch = cc & 3;
-            if (skip[mb]) continue;
-            float v[32];
-#pragma unroll
-            for (int q = 0; q < 32; ++q) v[q] = __uint_as_float(cur[q]);
-            if (!full[mb]) {
-              const int kbase = key0 + ch * 32;
-#pragma unroll
-              for (int q = 0; q < 32; ++q)
-                if (kbase + q > lim_row[mb]) v[q] = -INFINITY;
-            }
-            float cmax = v[0];
-#pragma unroll
-            for (int q = 1; q < 32; ++q) cmax = fmaxf(cmax, v[q]);
-            const float m_new = fmaxf(m_run[mb], cmax);
-            if (m_new > -INFINITY) {
-              const float mc = m_new * c;
-              float acc0 = z_run[mb] * ex2(m_run[mb] * c - mc), acc1 = 0.0f, acc2 = 0.0f, acc3 = 0.0f;
-#pragma unroll
-              for (int q = 0; q < 32; q += 4) {
-                acc0 += ex2(fmaf(v[q + 0], c, -mc));
-                acc1 += ex2(fmaf(v[q + 1], c, -mc));
-                acc2 += ex2(fmaf(v[q + 2], c, -mc));
-                acc3 += ex2(fmaf(v[q + 3], c, -mc));
+            const int lim = lim_row[mb];
+#pragma unroll 1
+            for (int half = 0; half < 2; ++half) {
+              const int cc = mb * 4 + half * 2;  // chunks cc (in ra) and cc + 1 (in rb)
+              tmem_ld_wait(ra);
+              tmem_ld32_issue(abase + (uint32_t)((cc + 1) * 32), rb);
+              chunk1(masked_tag, ra, ref_c[mb], z_run[mb], key0 + (half * 2) * 32, lim);
+              tmem_ld_wait(rb);
+              if (mb == MB - 1 && half == 1) {
+                release(jj);
+                if (j + 2 < T) {
+                  wait_full(jj + 2, 30);
+                  tmem_ld32_issue(acc_addr(jj + 2), ra);
+                }
+              } else {
+                tmem_ld32_issue(abase + (uint32_t)((cc + 2) * 32), ra);
               }
-              z_run[mb] = (acc0 + acc1) + (acc2 + acc3);
-              m_run[mb] = m_new;
+              chunk1(masked_tag, rb, ref_c[mb], z_run[mb], key0 + (half * 2 + 1) * 32, lim);
             }
           }
+        };
+        for (; j < T; j += 2) {
+          // tiles that every row of the warp sees completely take the unmasked path (rows that see nothing at all,
+          // i.e. padding, still run: their sums are never used)
+          bool masked = false;
+#pragma unroll
+          for (int mb = 0; mb < MB; ++mb)
+            masked = masked || (lim_row[mb] >= 0 && (ui.t_begin + j) * kTileN + kTileN - 1 > lim_row[mb]);
+          if (__any_sync(0xffffffffu, masked)) job1(std::true_type{}, j);
+          else job1(std::false_type{}, j);
         }
-        // ---- exchange: group partials -> CTA partial -> every CTA of the cluster
+        // ---- exchange: group partials -> CTA partial -> every CTA of the cluster reads every other's
 #pragma unroll
         for (int mb = 0; mb < MB; ++mb) {
-          sm.part_m[grp][mb * 128 + row_in_tile] = m_run[mb];
-          sm.part_z[grp][mb * 128 + row_in_tile] = z_run[mb];
+          // rows that see no key at all (padding, window positions before the sequence start) stay mute
+          sm.part_m[grp][mb * 128 + row_in_tile] = lim_row[mb] >= 0 ? ref_c[mb] : -1e30f;
+          sm.part_z[grp][mb * 128 + row_in_tile] = lim_row[mb] >= 0 ? z_run[mb] : 0.0f;
         }
         softmax_bar();
         if (st < kRowsPad) {
           const float m0 = sm.part_m[0][st], m1 = sm.part_m[1][st];
-          float m = fmaxf(m0, m1);
-          float z = 0.0f;
-          if (m > -INFINITY) z = sm.part_z[0][st] * ex2((m0 - m) * c) + sm.part_z[1][st] * ex2((m1 - m) * c);
-          const uint32_t bar = smem_u32(&sm.xchg_full[up]);
-          for (int r = 0; r < p.cluster; ++r) {
-            st_cluster_f32(smem_u32(&sm.xchg_m[up][rank][st]), (uint32_t)r, m);
-            st_cluster_f32(smem_u32(&sm.xchg_z[up][rank][st]), (uint32_t)r, z);
-            mbar_arrive_remote(bar, (uint32_t)r);  // release: the two stores above are visible to who acquires
+          const float m = fmaxf(m0, m1);
+          sm.mine_m[up][st] = m;
+          sm.mine_z[up][st] = sm.part_z[0][st] * ex2(m0 - m) + sm.part_z[1][st] * ex2(m1 - m);
+        }
+        softmax_bar();
+        // one thread per peer tells that peer that this CTA's statistics of the unit are in place
+        if (st < p.cluster) {
+          fence_cluster();
+          mbar_arrive_remote(smem_u32(&sm.xchg_full[up]), (uint32_t)st);
+        }
+        if (st < kRowsPad) {
+          mbar_wait_cluster(smem_u32(&sm.xchg_full[up]), (uint32_t)(it >> 1) & 1u, abort_flag, p.status, 32);
+          float pm[kMaxCluster], pz[kMaxCluster];
+#pragma unroll
+          for (int r = 0; r < kMaxCluster; ++r) {
+            pm[r] = -1e30f;
+            pz[r] = 0.0f;
+            if (r < p.cluster) {
+              pm[r] = ld_cluster_f32(smem_u32(&sm.mine_m[up][st]), (uint32_t)r);
+              pz[r] = ld_cluster_f32(smem_u32(&sm.mine_z[up][st]), (uint32_t)r);
+            }
           }
-          mbar_wait_cluster(bar, (uint32_t)(it >> 1) & 1u, abort_flag, p.status, 32);
-          m = -INFINITY;
-          for (int r = 0; r < p.cluster; ++r) m = fmaxf(m, sm.xchg_m[up][r][st]);
-          z = 0.0f;
-          if (m > -INFINITY)
-            for (int r = 0; r < p.cluster; ++r) z += sm.xchg_z[up][r][st] * ex2((sm.xchg_m[up][r][st] - m) * c);
-          sm.lse2[up][st] = (z > 0.0f) ? m * c + log2f(z) : INFINITY;
+          float m = pm[0];
+#pragma unroll
+          for (int r = 1; r < kMaxCluster; ++r) m = fmaxf(m, pm[r]);
+          float z = 0.0f;
+#pragma unroll
+          for (int r = 0; r < kMaxCluster; ++r) z += pz[r] * ex2(pm[r] - m);
+          sm.lse2[up][st] = (z > 0.0f) ? m + log2f(z) : INFINITY;
         }
         softmax_bar();
       } else {
@@ -610,67 +700,117 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
       const long long unit_off = ((long long)ui.l * p.Hkv + ui.g) * p.seq.total;
       const float4* l4 = reinterpret_cast<const float4*>(sm.lse2[up]);
       const float4* w4 = reinterpret_cast<const float4*>(sm.wrow);
-      for (int j = j0 + ((((jg + j0) & 1) == grp) ? 0 : 1); j < n_jobs; j += 2) {
-        const int jj = jg + j;
-        mbar_wait(smem_u32(&sm.acc_full[grp]), (uint32_t)(jj >> 1) & 1u, abort_flag, p.status, 31);
-        tc_fence_after();
-        const int key = (ui.t_begin + (j - j0)) * kTileN + row_in_tile;
-        const bool fast_path = __all_sync(0xffffffffu, key <= min_lim || key >= n);
-        float sA0 = 0.0f, sA1 = 0.0f, sP0 = 0.0f, sP1 = 0.0f;
-        uint32_t ra[32], rb[32];
-        tmem_ld32_issue(tbase, ra);
+      const bool pipelined = (n_chunks2 == 4 * MB);  // an even chunk count keeps the two register sets in step
+      {
+        float sT[32];  // PM 0..2: partial column sums per register position (window position q % W); PM 3: unused
+        float sA = 0.0f, sP = 0.0f;
+        // 32 rows (chunk cc) of this thread's key; masked: keys inside the observation window (cold tiles only)
+        auto chunk2 = [&](auto masked_tag, const uint32_t(&cur)[32], int cc, int key) {
+          constexpr bool masked = decltype(masked_tag)::value;
 #pragma unroll
-        for (int cc = 0; cc < 4 * MB; ++cc) {
-          if (cc < n_chunks2) {
-            uint32_t(&cur)[32] = (cc & 1) ? rb : ra;
-            uint32_t(&nxt)[32] = (cc & 1) ? ra : rb;
-            tmem_ld_wait(cur);
-            if (cc + 1 < n_chunks2) {
-              tmem_ld32_issue(tbase + (uint32_t)((cc + 1) * 32), nxt);
-            } else {
-              tc_fence_before();
-              __syncwarp();
-              if (lane == 0) mbar_arrive(smem_u32(&sm.acc_empty[grp]));
-            }
-            if (fast_path) {
+          for (int q4 = 0; q4 < 8; ++q4) {
+            const float4 ls = l4[cc * 8 + q4];
+            float a[4];
+            a[0] = ex2(fmaf(__uint_as_float(cur[4 * q4 + 0]), c, -ls.x));
+            a[1] = ex2(fmaf(__uint_as_float(cur[4 * q4 + 1]), c, -ls.y));
+            a[2] = ex2(fmaf(__uint_as_float(cur[4 * q4 + 2]), c, -ls.z));
+            a[3] = ex2(fmaf(__uint_as_float(cur[4 * q4 + 3]), c, -ls.w));
+            if (masked) {  // row r sees key i only if i <= the row's own position
 #pragma unroll
-              for (int q = 0; q < 8; ++q) {
-                const float4 ls = l4[cc * 8 + q];
-                const float a0 = ex2(fmaf(__uint_as_float(cur[4 * q + 0]), c, -ls.x));
-                const float a1 = ex2(fmaf(__uint_as_float(cur[4 * q + 1]), c, -ls.y));
-                const float a2 = ex2(fmaf(__uint_as_float(cur[4 * q + 2]), c, -ls.z));
-                const float a3 = ex2(fmaf(__uint_as_float(cur[4 * q + 3]), c, -ls.w));
-                sA0 += a0 + a1;
-                sA1 += a2 + a3;
-                if (kNeedP) {
-                  const float4 ws = w4[cc * 8 + q];
-                  sP0 = fmaf(ws.x, a0, sP0);
-                  sP1 = fmaf(ws.y, a1, sP1);
-                  sP0 = fmaf(ws.z, a2, sP0);
-                  sP1 = fmaf(ws.w, a3, sP1);
-                }
-              }
-            } else {
-#pragma unroll
-              for (int q = 0; q < 32; ++q) {
-                const int r = cc * 32 + q;
-                const int t = sm.row_t[r];
+              for (int e = 0; e < 4; ++e) {
+                const int t = sm.row_t[cc * 32 + 4 * q4 + e];
                 const int pos = n - p.W + t;
                 const int lim = (t >= 0 && pos >= 0) ? (p.causal ? pos : n - 1) : -1;
-                float a = 0.0f;
-                if (key <= lim) a = ex2(fmaf(__uint_as_float(cur[q]), c, -sm.lse2[up][r]));
-                sA0 += a;
-                if (kNeedP) sP0 = fmaf(sm.wrow[r], a, sP0);
+                if (key > lim) a[e] = 0.0f;
               }
             }
+            if (PM == 3) {
+              const float4 ws = w4[cc * 8 + q4];
+              sA += (a[0] + a[1]) + (a[2] + a[3]);
+              sP = fmaf(ws.x, a[0], sP);
+              sP = fmaf(ws.y, a[1], sP);
+              sP = fmaf(ws.z, a[2], sP);
+              sP = fmaf(ws.w, a[3], sP);
+            } else {
+#pragma unroll
+              for (int e = 0; e < 4; ++e) sT[4 * q4 + e] += a[e];
+            }
           }
+        };
+        // fold the per-position sums into A (and P with the weights starting at w4[wbase])
+        auto fold = [&](int wbase) {
+#pragma unroll
+          for (int q4 = 0; q4 < 8; ++q4) {
+            sA += (sT[4 * q4] + sT[4 * q4 + 1]) + (sT[4 * q4 + 2] + sT[4 * q4 + 3]);
+            if (PM == 1 || PM == 2) {
+              const float4 ws = w4[wbase + q4];
+              sP = fmaf(ws.x, sT[4 * q4 + 0], sP);
+              sP = fmaf(ws.y, sT[4 * q4 + 1], sP);
+              sP = fmaf(ws.z, sT[4 * q4 + 2], sP);
+              sP = fmaf(ws.w, sT[4 * q4 + 3], sP);
+            }
+            sT[4 * q4] = sT[4 * q4 + 1] = sT[4 * q4 + 2] = sT[4 * q4 + 3] = 0.0f;
+          }
+        };
+        uint32_t ra[32], rb[32];
+        int j = j0 + ((((jg + j0) & 1) == grp) ? 0 : 1);
+        if (pipelined && j < n_jobs) {
+          wait_full(jg + j, 31);
+          tmem_ld32_issue(acc_addr(jg + j) + chunk_col<MB, PM>(0), ra);
         }
-        if (key < n) {
-          const float sumA = sA0 + sA1, sumP = sP0 + sP1;
-          const long long o = unit_off + ui.tok0 + key;
-          if (p.A) p.A[o] = sumA;
-          if (p.P) p.P[o] = sumP;
-          if (p.u) p.u[o] = __fadd_rn(__fmul_rn(p.alpha, sumA), __fmul_rn(p.delta, sumP));
+        auto job2 = [&](auto masked_tag, int j, int key) {
+          const int jj = jg + j;
+          const uint32_t abase = acc_addr(jj);
+          if (pipelined) {
+#pragma unroll 1
+            for (int cp = 0; cp < 2 * MB; ++cp) {  // chunk pair: sequence positions 2cp (in ra), 2cp + 1 (in rb)
+              const int ci = 2 * cp;
+              tmem_ld_wait(ra);
+              tmem_ld32_issue(abase + chunk_col<MB, PM>(ci + 1), rb);
+              chunk2(masked_tag, ra, (int)(chunk_col<MB, PM>(ci) >> 5), key);
+              tmem_ld_wait(rb);
+              if (cp == 2 * MB - 1) {
+                release(jj);
+                if (j + 2 < n_jobs) {
+                  wait_full(jj + 2, 31);
+                  tmem_ld32_issue(acc_addr(jj + 2) + chunk_col<MB, PM>(0), ra);
+                }
+              } else {
+                tmem_ld32_issue(abase + chunk_col<MB, PM>(ci + 2), ra);
+              }
+              chunk2(masked_tag, rb, (int)(chunk_col<MB, PM>(ci + 1) >> 5), key);
+              // W = 64 with pension: window positions 0..31 end with the first half of the sequence
+              if (PM == 2 && cp == MB - 1) fold(0);
+            }
+            if (PM == 2) fold(8);
+            if (PM == 0 || PM == 1) fold(0);
+          } else {  // few rows (G*W < 128*MB - 31): one chunk at a time, no prefetch across jobs
+            wait_full(jj, 31);
+#pragma unroll 1
+            for (int ci = 0; ci < n_chunks2; ++ci) {
+              tmem_ld32_issue(abase + (uint32_t)(ci * 32), ra);
+              tmem_ld_wait(ra);
+              if (ci == n_chunks2 - 1) release(jj);
+              chunk2(masked_tag, ra, ci, key);
+            }
+            if (PM != 3) fold(0);  // PM 2 needs rows == 256, so it never gets here
+          }
+        };
+        for (; j < n_jobs; j += 2) {
+          const int key = (ui.t_begin + (j - j0)) * kTileN + row_in_tile;
+#pragma unroll
+          for (int q = 0; q < 32; ++q) sT[q] = 0.0f;
+          sA = 0.0f;
+          sP = 0.0f;
+          // only the last W-1 keys of a sequence are hidden from some rows: those tiles take the masked path
+          if (__all_sync(0xffffffffu, key <= min_lim || key >= n)) job2(std::false_type{}, j, key);
+          else job2(std::true_type{}, j, key);
+          if (key < n) {
+            const long long o = unit_off + ui.tok0 + key;
+            if (p.A) p.A[o] = sA;
+            if (p.P) p.P[o] = sP;
+            if (p.u) p.u[o] = __fadd_rn(__fmul_rn(p.alpha, sA), __fmul_rn(p.delta, sP));
+          }
         }
       }
       if (T > 0) jg += n_jobs;
@@ -680,7 +820,7 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
   // ---- teardown
   tc_fence_before();
   __syncthreads();
-  if (warp == 1) {
+  if (warp == 9) {
     tc_fence_after();
     tmem_dealloc(tmem_base, kTmemCols);
   }
@@ -713,16 +853,21 @@ CUresult encode_5d(void* fn, CUtensorMap* map, const void* base, const uint64_t 
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
 }
 
-template <int MB, bool NP>
+template <int MB, int PM>
 cudaError_t launch_variant(ta_ctx* ctx, const CUtensorMap& mq, const CUtensorMap& mk, ScoreParams& sp,
                            cudaStream_t stream) {
-  auto kern = ta_score_kernel<MB, NP>;
+  auto kern = ta_score_kernel<MB, PM>;
   const size_t smem = score_smem_bytes<MB>();
   static bool attr_set_dev[64] = {};  // per device and instantiation; the attribute is sticky
   bool& attr_set = attr_set_dev[ctx->device & 63];
   if (!attr_set) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
+    // the in-kernel register split must fit in what the launch provides, or the warps asking for more wait forever
+    cudaFuncAttributes fa;
+    e = cudaFuncGetAttributes(&fa, kern);
+    if (e != cudaSuccess) return e;
+    if (fa.numRegs * kThreads < kRegsNeeded) return cudaErrorLaunchOutOfResources;
     attr_set = true;
   }
   cudaLaunchConfig_t cfg = {};
@@ -815,8 +960,20 @@ cudaError_t ta_launch_score(ta_ctx* ctx, const ta_score_args& a, ta_dev_status* 
     const uint32_t box[5] = {64, (uint32_t)kTileN, 1, 1, 1};
     if (encode_5d(ctx->encode_tiled, &mk, a.k.ptr, dims, str, box) != CUDA_SUCCESS) return cudaErrorInvalidValue;
   }
+  // how the pension term is accumulated: 0 none, 1 W divides 32, 2 W == 64, 3 any W (per-element weights)
   const bool need_p = a.P != nullptr || (a.u != nullptr && a.delta != 0.0f);
-  if (MB == 1) return need_p ? launch_variant<1, true>(ctx, mq, mk, sp, stream)
-                             : launch_variant<1, false>(ctx, mq, mk, sp, stream);
-  return need_p ? launch_variant<2, true>(ctx, mq, mk, sp, stream) : launch_variant<2, false>(ctx, mq, mk, sp, stream);
+  const int pm = !need_p ? 0 : (32 % a.W == 0) ? 1 : (a.W == 64 && rows == 256) ? 2 : 3;
+  if (MB == 1) {
+    switch (pm) {
+      case 0: return launch_variant<1, 0>(ctx, mq, mk, sp, stream);
+      case 1: return launch_variant<1, 1>(ctx, mq, mk, sp, stream);
+      default: return launch_variant<1, 3>(ctx, mq, mk, sp, stream);
+    }
+  }
+  switch (pm) {
+    case 0: return launch_variant<2, 0>(ctx, mq, mk, sp, stream);
+    case 1: return launch_variant<2, 1>(ctx, mq, mk, sp, stream);
+    case 2: return launch_variant<2, 2>(ctx, mq, mk, sp, stream);
+    default: return launch_variant<2, 3>(ctx, mq, mk, sp, stream);
+  }
 }
