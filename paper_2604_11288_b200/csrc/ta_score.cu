@@ -102,8 +102,10 @@ __device__ __forceinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, vo
   const unsigned long long t0 = globaltimer_ns();
   for (;;) {
 #pragma unroll 1
-    for (int it = 0; it < 64; ++it)
+    for (int it = 0; it < 64; ++it) {
       if (mbar_try_wait(bar, parity)) return true;
+      __nanosleep(100);  // a polling warp must not eat the issue slots of the softmax warps on its sub-partition
+    }
     if (*abort_flag) return false;
     if (globaltimer_ns() - t0 > kWaitLimitNs) {
       *abort_flag = 1;
@@ -181,6 +183,24 @@ __device__ __forceinline__ void tmem_ld_wait(uint32_t (&r)[32]) {
                  "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]),
                  "+r"(r[23]), "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]),
                  "+r"(r[30]), "+r"(r[31])
+               :
+               : "memory");
+}
+
+// 16-column variants: half the registers per load in flight
+__device__ __forceinline__ void tmem_ld16_issue(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];\n"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait(uint32_t (&r)[16]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+                 "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15])
                :
                : "memory");
 }
@@ -550,32 +570,30 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           const int pos = n - p.W + my_t[mb];
           lim_row[mb] = (my_t[mb] >= 0 && pos >= 0) ? (p.causal ? pos : n - 1) : -1;
         }
-        // one 32-key chunk of one row; `lim` < INT_MAX masks keys beyond it (cold tiles only)
-        auto chunk1 = [&](auto masked_tag, const uint32_t(&cur)[32], float& rc_io, float& z_io, int kbase, int lim) {
+        // 16 keys of one row (half of a 32-key chunk); masked tiles (cold) drop keys beyond `lim`
+        auto chunk1 = [&](auto masked_tag, const uint32_t(&cur)[16], float& rc_io, float& z_io, int kbase, int lim) {
           constexpr bool masked = decltype(masked_tag)::value;
-          float v[32];
+          float v[16];
 #pragma unroll
-          for (int q = 0; q < 32; ++q) v[q] = __uint_as_float(cur[q]);
+          for (int q = 0; q < 16; ++q) v[q] = __uint_as_float(cur[q]);
           if (masked) {
 #pragma unroll
-            for (int q = 0; q < 32; ++q)
+            for (int q = 0; q < 16; ++q)
               if (kbase + q > lim) v[q] = -INFINITY;
           }
           const float rc = rc_io;
           float a0 = 0.0f, a1 = 0.0f, a2 = 0.0f, a3 = 0.0f;
 #pragma unroll
-          for (int q = 0; q < 32; q += 4) {
+          for (int q = 0; q < 16; q += 4) {
             a0 += ex2(fmaf(v[q + 0], c, -rc));
             a1 += ex2(fmaf(v[q + 1], c, -rc));
             a2 += ex2(fmaf(v[q + 2], c, -rc));
             a3 += ex2(fmaf(v[q + 3], c, -rc));
           }
-          float t8[8];
+          float t4[4];
 #pragma unroll
-          for (int q = 0; q < 8; ++q) t8[q] = fmaxf(fmaxf(v[4 * q], v[4 * q + 1]), fmaxf(v[4 * q + 2], v[4 * q + 3]));
-          const float cmax = fmaxf(fmaxf(fmaxf(t8[0], t8[1]), fmaxf(t8[2], t8[3])),
-                                   fmaxf(fmaxf(t8[4], t8[5]), fmaxf(t8[6], t8[7])));
-          const float cm_c = cmax * c;
+          for (int q = 0; q < 4; ++q) t4[q] = fmaxf(fmaxf(v[4 * q], v[4 * q + 1]), fmaxf(v[4 * q + 2], v[4 * q + 3]));
+          const float cm_c = fmaxf(fmaxf(t4[0], t4[1]), fmaxf(t4[2], t4[3])) * c;
           const bool jump = cm_c > rc + 8.0f;
           float add = (a0 + a1) + (a2 + a3);
           if (__any_sync(0xffffffffu, jump)) {
@@ -584,7 +602,7 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
               rc_io = cm_c;
               float b0 = 0.0f, b1 = 0.0f;
 #pragma unroll
-              for (int q = 0; q < 32; q += 2) {
+              for (int q = 0; q < 16; q += 2) {
                 b0 += ex2(fmaf(v[q + 0], c, -cm_c));
                 b1 += ex2(fmaf(v[q + 1], c, -cm_c));
               }
@@ -593,14 +611,14 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           }
           z_io += add;
         };
-        uint32_t ra[32], rb[32];
+        uint32_t ra[16], rb[16];
         int j = ((jg & 1) == grp) ? 0 : 1;
         if (j < T) {
           wait_full(jg + j, 30);
-          tmem_ld32_issue(acc_addr(jg + j), ra);
+          tmem_ld16_issue(acc_addr(jg + j), ra);
         }
-        // one job: all chunks of the accumulator, two register sets in flight, the next job's first load issued
-        // before the last chunk is computed
+        // one job: the accumulator in 32-column chunks, each fetched as two 16-column loads (ra, rb) so that one
+        // load is always in flight; the next job's first load is issued before the last half-chunk is computed
         auto job1 = [&](auto masked_tag, int j) {
           const int jj = jg + j;
           const int key0 = (ui.t_begin + j) * kTileN;
@@ -609,22 +627,22 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           for (int mb = 0; mb < MB; ++mb) {
             const int lim = lim_row[mb];
 #pragma unroll 1
-            for (int half = 0; half < 2; ++half) {
-              const int cc = mb * 4 + half * 2;  // chunks cc (in ra) and cc + 1 (in rb)
+            for (int c4 = 0; c4 < 4; ++c4) {
+              const uint32_t col = (uint32_t)(mb * 128 + c4 * 32);
               tmem_ld_wait(ra);
-              tmem_ld32_issue(abase + (uint32_t)((cc + 1) * 32), rb);
-              chunk1(masked_tag, ra, ref_c[mb], z_run[mb], key0 + (half * 2) * 32, lim);
+              tmem_ld16_issue(abase + col + 16, rb);
+              chunk1(masked_tag, ra, ref_c[mb], z_run[mb], key0 + c4 * 32, lim);
               tmem_ld_wait(rb);
-              if (mb == MB - 1 && half == 1) {
+              if (mb == MB - 1 && c4 == 3) {
                 release(jj);
                 if (j + 2 < T) {
                   wait_full(jj + 2, 30);
-                  tmem_ld32_issue(acc_addr(jj + 2), ra);
+                  tmem_ld16_issue(acc_addr(jj + 2), ra);
                 }
               } else {
-                tmem_ld32_issue(abase + (uint32_t)((cc + 2) * 32), ra);
+                tmem_ld16_issue(abase + col + 32, ra);
               }
-              chunk1(masked_tag, rb, ref_c[mb], z_run[mb], key0 + (half * 2 + 1) * 32, lim);
+              chunk1(masked_tag, rb, ref_c[mb], z_run[mb], key0 + c4 * 32 + 16, lim);
             }
           }
         };
@@ -700,16 +718,17 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
       const long long unit_off = ((long long)ui.l * p.Hkv + ui.g) * p.seq.total;
       const float4* l4 = reinterpret_cast<const float4*>(sm.lse2[up]);
       const float4* w4 = reinterpret_cast<const float4*>(sm.wrow);
-      const bool pipelined = (n_chunks2 == 4 * MB);  // an even chunk count keeps the two register sets in step
       {
         float sT[32];  // PM 0..2: partial column sums per register position (window position q % W); PM 3: unused
         float sA = 0.0f, sP = 0.0f;
-        // 32 rows (chunk cc) of this thread's key; masked: keys inside the observation window (cold tiles only)
-        auto chunk2 = [&](auto masked_tag, const uint32_t(&cur)[32], int cc, int key) {
+        // 16 rows (half `hi` of the 32-row chunk cc) of this thread's key; masked: keys inside the observation
+        // window (cold tiles only)
+        auto chunk2 = [&](auto masked_tag, auto hi_tag, const uint32_t(&cur)[16], int cc, int key) {
           constexpr bool masked = decltype(masked_tag)::value;
+          constexpr int hi = decltype(hi_tag)::value;  // 0: rows 32cc..32cc+15, 1: rows 32cc+16..32cc+31
 #pragma unroll
-          for (int q4 = 0; q4 < 8; ++q4) {
-            const float4 ls = l4[cc * 8 + q4];
+          for (int q4 = 0; q4 < 4; ++q4) {
+            const float4 ls = l4[cc * 8 + hi * 4 + q4];
             float a[4];
             a[0] = ex2(fmaf(__uint_as_float(cur[4 * q4 + 0]), c, -ls.x));
             a[1] = ex2(fmaf(__uint_as_float(cur[4 * q4 + 1]), c, -ls.y));
@@ -718,14 +737,14 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             if (masked) {  // row r sees key i only if i <= the row's own position
 #pragma unroll
               for (int e = 0; e < 4; ++e) {
-                const int t = sm.row_t[cc * 32 + 4 * q4 + e];
+                const int t = sm.row_t[cc * 32 + hi * 16 + 4 * q4 + e];
                 const int pos = n - p.W + t;
                 const int lim = (t >= 0 && pos >= 0) ? (p.causal ? pos : n - 1) : -1;
                 if (key > lim) a[e] = 0.0f;
               }
             }
             if (PM == 3) {
-              const float4 ws = w4[cc * 8 + q4];
+              const float4 ws = w4[cc * 8 + hi * 4 + q4];
               sA += (a[0] + a[1]) + (a[2] + a[3]);
               sP = fmaf(ws.x, a[0], sP);
               sP = fmaf(ws.y, a[1], sP);
@@ -733,7 +752,7 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
               sP = fmaf(ws.w, a[3], sP);
             } else {
 #pragma unroll
-              for (int e = 0; e < 4; ++e) sT[4 * q4 + e] += a[e];
+              for (int e = 0; e < 4; ++e) sT[hi * 16 + 4 * q4 + e] += a[e];
             }
           }
         };
@@ -752,49 +771,39 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             sT[4 * q4] = sT[4 * q4 + 1] = sT[4 * q4 + 2] = sT[4 * q4 + 3] = 0.0f;
           }
         };
-        uint32_t ra[32], rb[32];
+        uint32_t ra[16], rb[16];
         int j = j0 + ((((jg + j0) & 1) == grp) ? 0 : 1);
-        if (pipelined && j < n_jobs) {
+        if (j < n_jobs) {
           wait_full(jg + j, 31);
-          tmem_ld32_issue(acc_addr(jg + j) + chunk_col<MB, PM>(0), ra);
+          tmem_ld16_issue(acc_addr(jg + j) + chunk_col<MB, PM>(0), ra);
         }
+        // one job: 32-row chunks in the order chunk_col gives, each as two 16-column loads (ra low half, rb high half)
         auto job2 = [&](auto masked_tag, int j, int key) {
           const int jj = jg + j;
           const uint32_t abase = acc_addr(jj);
-          if (pipelined) {
 #pragma unroll 1
-            for (int cp = 0; cp < 2 * MB; ++cp) {  // chunk pair: sequence positions 2cp (in ra), 2cp + 1 (in rb)
-              const int ci = 2 * cp;
-              tmem_ld_wait(ra);
-              tmem_ld32_issue(abase + chunk_col<MB, PM>(ci + 1), rb);
-              chunk2(masked_tag, ra, (int)(chunk_col<MB, PM>(ci) >> 5), key);
-              tmem_ld_wait(rb);
-              if (cp == 2 * MB - 1) {
-                release(jj);
-                if (j + 2 < n_jobs) {
-                  wait_full(jj + 2, 31);
-                  tmem_ld32_issue(acc_addr(jj + 2) + chunk_col<MB, PM>(0), ra);
-                }
-              } else {
-                tmem_ld32_issue(abase + chunk_col<MB, PM>(ci + 2), ra);
+          for (int ci = 0; ci < n_chunks2; ++ci) {
+            const uint32_t col = chunk_col<MB, PM>(ci);
+            const int cc = (int)(col >> 5);
+            tmem_ld_wait(ra);
+            tmem_ld16_issue(abase + col + 16, rb);
+            chunk2(masked_tag, std::integral_constant<int, 0>{}, ra, cc, key);
+            tmem_ld_wait(rb);
+            if (ci == n_chunks2 - 1) {
+              release(jj);
+              if (j + 2 < n_jobs) {
+                wait_full(jj + 2, 31);
+                tmem_ld16_issue(acc_addr(jj + 2) + chunk_col<MB, PM>(0), ra);
               }
-              chunk2(masked_tag, rb, (int)(chunk_col<MB, PM>(ci + 1) >> 5), key);
-              // W = 64 with pension: window positions 0..31 end with the first half of the sequence
-              if (PM == 2 && cp == MB - 1) fold(0);
+            } else {
+              tmem_ld16_issue(abase + chunk_col<MB, PM>(ci + 1), ra);
             }
-            if (PM == 2) fold(8);
-            if (PM == 0 || PM == 1) fold(0);
-          } else {  // few rows (G*W < 128*MB - 31): one chunk at a time, no prefetch across jobs
-            wait_full(jj, 31);
-#pragma unroll 1
-            for (int ci = 0; ci < n_chunks2; ++ci) {
-              tmem_ld32_issue(abase + (uint32_t)(ci * 32), ra);
-              tmem_ld_wait(ra);
-              if (ci == n_chunks2 - 1) release(jj);
-              chunk2(masked_tag, ra, ci, key);
-            }
-            if (PM != 3) fold(0);  // PM 2 needs rows == 256, so it never gets here
+            chunk2(masked_tag, std::integral_constant<int, 1>{}, rb, cc, key);
+            // W = 64 with pension: window positions 0..31 end with the first half of the sequence
+            if (PM == 2 && ci == 2 * MB - 1) fold(0);
           }
+          if (PM == 2) fold(8);
+          if (PM == 0 || PM == 1) fold(0);
         };
         for (; j < n_jobs; j += 2) {
           const int key = (ui.t_begin + (j - j0)) * kTileN + row_in_tile;
