@@ -161,33 +161,9 @@ __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 
-// 32 lanes x 32 consecutive 32-bit columns: thread i of the warp receives lane (quadrant base + i). The load is
-// asynchronous; tmem_ld_wait() must be called on the same registers before they are read. Passing the registers
-// through the wait as read-write operands keeps the compiler from moving their uses above it.
-__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t (&r)[32]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];\n"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
-        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
-        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr)
-      : "memory");
-}
-__device__ __forceinline__ void tmem_ld_wait(uint32_t (&r)[32]) {
-  asm volatile("tcgen05.wait::ld.sync.aligned;"
-               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
-                 "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
-                 "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]),
-                 "+r"(r[23]), "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]),
-                 "+r"(r[30]), "+r"(r[31])
-               :
-               : "memory");
-}
-
-// 16-column variants: half the registers per load in flight
+// Tensor-memory loads, shape 32x32b: thread i of the warp receives lane (quadrant base + i) and 16 consecutive 32-bit
+// columns. The load is asynchronous; tmem_ld_wait() must be called on the same registers before they are read.
+// Passing the registers through the wait as read-write operands keeps the compiler from moving their uses above it.
 __device__ __forceinline__ void tmem_ld16_issue(uint32_t taddr, uint32_t (&r)[16]) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
@@ -226,11 +202,6 @@ __device__ __forceinline__ float ld_cluster_f32(uint32_t local_addr, uint32_t ra
   return v;
 }
 __device__ __forceinline__ void fence_cluster() { asm volatile("fence.acq_rel.cluster;" ::: "memory"); }
-__device__ __forceinline__ void st_cluster_f32(uint32_t local_addr, uint32_t rank, float v) {
-  uint32_t remote;
-  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
-  asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote), "f"(v) : "memory");
-}
 // arrive (release at cluster scope) on the mbarrier at the same shared-memory offset in CTA `rank` of the cluster
 __device__ __forceinline__ void mbar_arrive_remote(uint32_t local_bar, uint32_t rank) {
   uint32_t remote;
@@ -340,7 +311,6 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
   constexpr int kStages = Cfg::kStages, kQBufs = Cfg::kQBufs, kRowsPad = Cfg::kRowsPad;
   constexpr int kAcc = Cfg::kAcc;
   constexpr uint32_t kTmemCols = 512;  // kAcc accumulator stages of kRowsPad columns
-  constexpr int kQBytes = MB * 2 * kHalfBytes;
   extern __shared__ uint8_t smem_raw[];
   ScoreSmem<MB>& sm = *reinterpret_cast<ScoreSmem<MB>*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
 
@@ -864,7 +834,7 @@ CUresult encode_5d(void* fn, CUtensorMap* map, const void* base, const uint64_t 
 
 template <int MB, int PM>
 cudaError_t launch_variant(ta_ctx* ctx, const CUtensorMap& mq, const CUtensorMap& mk, ScoreParams& sp,
-                           cudaStream_t stream) {
+                           int tiles_max, cudaStream_t stream) {
   auto kern = ta_score_kernel<MB, PM>;
   const size_t smem = score_smem_bytes<MB>();
   static bool attr_set_dev[64] = {};  // per device and instantiation; the attribute is sticky
@@ -890,18 +860,35 @@ cudaError_t launch_variant(ta_ctx* ctx, const CUtensorMap& mq, const CUtensorMap
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  // persistent grid: as many clusters as can be resident at once (queried once per cluster size)
+  // Persistent grid: as many clusters as can be resident at once (queried once per cluster size). CTAs per unit:
+  // the size with the fewest tile-times on the busiest CTA, counting ~1 tile-time of overhead per unit and ~2 more
+  // for the statistics exchange when a unit spans several CTAs.
   static int max_clusters_dev[64][kMaxCluster + 1] = {};
   int* max_clusters = max_clusters_dev[ctx->device & 63];
-  if (max_clusters[sp.cluster] == 0) {
-    cfg.gridDim = dim3((unsigned)(ctx->sm_count / sp.cluster * sp.cluster), 1, 1);
-    int n = 0;
-    cudaError_t e = cudaOccupancyMaxActiveClusters(&n, kern, &cfg);
-    if (e != cudaSuccess) return e;
-    if (n < 1) return cudaErrorLaunchOutOfResources;
-    max_clusters[sp.cluster] = n;
+  int best_cl = 1;
+  long long best_cost = -1;
+  for (int cl = 1; cl <= kMaxCluster; cl *= 2) {
+    if (cl > 1 && tiles_max < 2 * cl) break;
+    if (max_clusters[cl] == 0) {
+      attr[0].val.clusterDim.x = (unsigned)cl;
+      cfg.gridDim = dim3((unsigned)(ctx->sm_count / cl * cl), 1, 1);
+      int n = 0;
+      cudaError_t e = cudaOccupancyMaxActiveClusters(&n, kern, &cfg);
+      if (e != cudaSuccess) return e;
+      max_clusters[cl] = n < 1 ? -1 : n;
+    }
+    if (max_clusters[cl] < 1) continue;
+    const long long rounds = (sp.units + max_clusters[cl] - 1) / max_clusters[cl];
+    const long long cost = rounds * ((tiles_max + cl - 1) / cl + (cl > 1 ? 3 : 1));
+    if (best_cost < 0 || cost < best_cost) {
+      best_cost = cost;
+      best_cl = cl;
+    }
   }
-  const int n_clusters = sp.units < max_clusters[sp.cluster] ? sp.units : max_clusters[sp.cluster];
+  if (best_cost < 0) return cudaErrorLaunchOutOfResources;
+  sp.cluster = best_cl;
+  attr[0].val.clusterDim.x = (unsigned)best_cl;
+  const int n_clusters = sp.units < max_clusters[best_cl] ? sp.units : max_clusters[best_cl];
   ctx->score_cluster = sp.cluster;
   ctx->score_clusters = n_clusters;
   cfg.gridDim = dim3((unsigned)(n_clusters * sp.cluster), 1, 1);
@@ -944,12 +931,8 @@ cudaError_t ta_launch_score(ta_ctx* ctx, const ta_score_args& a, ta_dev_status* 
   sp.rho = a.rho;
   for (int t = 0; t < a.W; ++t) sp.wrow[t] = (float)((1.0 - (double)a.rho) * pow((double)a.rho, (double)(a.W - 1 - t)));
   sp.units = units;
-  // CTAs per unit: at least four 128-key tiles per CTA, and more CTAs per unit when there are few units
   const int tiles_max = (a.seq.max_n + kTileN - 1) / kTileN;
-  int cl = 4;
-  while (cl > 1 && tiles_max < 4 * cl) cl >>= 1;
-  if (cl == 4 && units * 8 <= ctx->sm_count && tiles_max >= 32) cl = 8;
-  sp.cluster = cl;
+  sp.cluster = 1;  // chosen at launch
 
   // tensor maps: dims (d, position, head, batch, layer)
   CUtensorMap mq, mk;
@@ -974,15 +957,15 @@ cudaError_t ta_launch_score(ta_ctx* ctx, const ta_score_args& a, ta_dev_status* 
   const int pm = !need_p ? 0 : (32 % a.W == 0) ? 1 : (a.W == 64 && rows == 256) ? 2 : 3;
   if (MB == 1) {
     switch (pm) {
-      case 0: return launch_variant<1, 0>(ctx, mq, mk, sp, stream);
-      case 1: return launch_variant<1, 1>(ctx, mq, mk, sp, stream);
-      default: return launch_variant<1, 3>(ctx, mq, mk, sp, stream);
+      case 0: return launch_variant<1, 0>(ctx, mq, mk, sp, tiles_max, stream);
+      case 1: return launch_variant<1, 1>(ctx, mq, mk, sp, tiles_max, stream);
+      default: return launch_variant<1, 3>(ctx, mq, mk, sp, tiles_max, stream);
     }
   }
   switch (pm) {
-    case 0: return launch_variant<2, 0>(ctx, mq, mk, sp, stream);
-    case 1: return launch_variant<2, 1>(ctx, mq, mk, sp, stream);
-    case 2: return launch_variant<2, 2>(ctx, mq, mk, sp, stream);
-    default: return launch_variant<2, 3>(ctx, mq, mk, sp, stream);
+    case 0: return launch_variant<2, 0>(ctx, mq, mk, sp, tiles_max, stream);
+    case 1: return launch_variant<2, 1>(ctx, mq, mk, sp, tiles_max, stream);
+    case 2: return launch_variant<2, 2>(ctx, mq, mk, sp, tiles_max, stream);
+    default: return launch_variant<2, 3>(ctx, mq, mk, sp, tiles_max, stream);
   }
 }
