@@ -592,6 +592,7 @@ ta_status ta_compress(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* pol
     a.rho = policy->pension_rho;
     a.scale = policy->softmax_scale;
     a.causal = policy->causal;
+    a.reserve_sms = fork ? 4 : 0;
     e = ta_launch_score(ctx, a, ctx->d_status, stream);
   }
   mark(2);

@@ -84,6 +84,7 @@ struct ta_score_args {
   const float* u_static; // unused
   float alpha, delta, rho, scale;
   int causal;
+  int reserve_sms;       // SMs left free for kernels running beside the (persistent) score kernel
 };
 cudaError_t ta_launch_score(ta_ctx* ctx, const ta_score_args& a, ta_dev_status* status, cudaStream_t stream);
 

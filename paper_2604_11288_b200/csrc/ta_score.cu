@@ -834,7 +834,7 @@ CUresult encode_5d(void* fn, CUtensorMap* map, const void* base, const uint64_t 
 
 template <int MB, int PM>
 cudaError_t launch_variant(ta_ctx* ctx, const CUtensorMap& mq, const CUtensorMap& mk, ScoreParams& sp,
-                           int tiles_max, cudaStream_t stream) {
+                           int tiles_max, int reserve_sms, cudaStream_t stream) {
   auto kern = ta_score_kernel<MB, PM>;
   const size_t smem = score_smem_bytes<MB>();
   static bool attr_set_dev[64] = {};  // per device and instantiation; the attribute is sticky
@@ -878,7 +878,8 @@ cudaError_t launch_variant(ta_ctx* ctx, const CUtensorMap& mq, const CUtensorMap
       max_clusters[cl] = n < 1 ? -1 : n;
     }
     if (max_clusters[cl] < 1) continue;
-    const long long rounds = (sp.units + max_clusters[cl] - 1) / max_clusters[cl];
+    const int avail = max_clusters[cl] - (reserve_sms + cl - 1) / cl > 0 ? max_clusters[cl] - (reserve_sms + cl - 1) / cl : 1;
+    const long long rounds = (sp.units + avail - 1) / avail;
     const long long cost = rounds * ((tiles_max + cl - 1) / cl + (cl > 1 ? 3 : 1));
     if (best_cost < 0 || cost < best_cost) {
       best_cost = cost;
@@ -888,7 +889,9 @@ cudaError_t launch_variant(ta_ctx* ctx, const CUtensorMap& mq, const CUtensorMap
   if (best_cost < 0) return cudaErrorLaunchOutOfResources;
   sp.cluster = best_cl;
   attr[0].val.clusterDim.x = (unsigned)best_cl;
-  const int n_clusters = sp.units < max_clusters[best_cl] ? sp.units : max_clusters[best_cl];
+  int n_clusters = max_clusters[best_cl] - (reserve_sms + best_cl - 1) / best_cl;
+  if (n_clusters < 1) n_clusters = 1;
+  if (n_clusters > sp.units) n_clusters = sp.units;
   ctx->score_cluster = sp.cluster;
   ctx->score_clusters = n_clusters;
   cfg.gridDim = dim3((unsigned)(n_clusters * sp.cluster), 1, 1);
@@ -957,15 +960,15 @@ cudaError_t ta_launch_score(ta_ctx* ctx, const ta_score_args& a, ta_dev_status* 
   const int pm = !need_p ? 0 : (32 % a.W == 0) ? 1 : (a.W == 64 && rows == 256) ? 2 : 3;
   if (MB == 1) {
     switch (pm) {
-      case 0: return launch_variant<1, 0>(ctx, mq, mk, sp, tiles_max, stream);
-      case 1: return launch_variant<1, 1>(ctx, mq, mk, sp, tiles_max, stream);
-      default: return launch_variant<1, 3>(ctx, mq, mk, sp, tiles_max, stream);
+      case 0: return launch_variant<1, 0>(ctx, mq, mk, sp, tiles_max, a.reserve_sms, stream);
+      case 1: return launch_variant<1, 1>(ctx, mq, mk, sp, tiles_max, a.reserve_sms, stream);
+      default: return launch_variant<1, 3>(ctx, mq, mk, sp, tiles_max, a.reserve_sms, stream);
     }
   }
   switch (pm) {
-    case 0: return launch_variant<2, 0>(ctx, mq, mk, sp, tiles_max, stream);
-    case 1: return launch_variant<2, 1>(ctx, mq, mk, sp, tiles_max, stream);
-    case 2: return launch_variant<2, 2>(ctx, mq, mk, sp, tiles_max, stream);
-    default: return launch_variant<2, 3>(ctx, mq, mk, sp, tiles_max, stream);
+    case 0: return launch_variant<2, 0>(ctx, mq, mk, sp, tiles_max, a.reserve_sms, stream);
+    case 1: return launch_variant<2, 1>(ctx, mq, mk, sp, tiles_max, a.reserve_sms, stream);
+    case 2: return launch_variant<2, 2>(ctx, mq, mk, sp, tiles_max, a.reserve_sms, stream);
+    default: return launch_variant<2, 3>(ctx, mq, mk, sp, tiles_max, a.reserve_sms, stream);
   }
 }

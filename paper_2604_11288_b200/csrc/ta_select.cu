@@ -36,14 +36,67 @@ struct SelectShared {
   uint32_t prefix, mask;
   int remaining;
   int done_all;
-  int warp_def[kWarps];
-  int warp_tie[kWarps];
+  __align__(16) uint32_t warp_cnt[kWarps];  // per warp: definite count (low 16 bits) | tie count (high 16 bits)
 };
 
-// Top-`want` of the eligible elements of [0, n) by key. key_of(i, key) returns eligibility and the 32-bit key.
-// All threads of the block must call it; the result is uniform across the block.
+// Keys of a unit are read once into registers when the unit is short enough (kItems per thread), else they are
+// re-read from L2 on every sweep in batches whose loads are all issued before the first use.
+constexpr int kItems = 8;
+constexpr int kBatch = 8;
+struct KeyCache {
+  uint32_t key[kItems];
+  uint32_t elig;  // bit `it`: element tid + it*kThreads exists and is eligible
+};
+
 template <class KeyFn>
-__device__ SelectResult block_radix_select(int n, int want, KeyFn key_of, SelectShared& sh) {
+__device__ __forceinline__ void fill_cache(int n, KeyFn key_of, KeyCache& kc) {
+  kc.elig = 0;
+#pragma unroll
+  for (int it = 0; it < kItems; ++it) {
+    const int i = (int)threadIdx.x + it * kThreads;
+    kc.key[it] = 0;
+    if (i < n && key_of(i, kc.key[it])) kc.elig |= 1u << it;
+  }
+}
+
+// Calls body(i, exists, eligible, key) for every element slot in ascending chunks of kThreads; every thread of the
+// block makes the same number of calls (the body may hold block-wide barriers).
+template <bool CACHED, class KeyFn, class Body>
+__device__ __forceinline__ void sweep(int n, KeyFn key_of, const KeyCache& kc, Body body) {
+  const int tid = threadIdx.x;
+  if (CACHED) {
+#pragma unroll
+    for (int it = 0; it < kItems; ++it) {
+      if (it * kThreads < n) {
+        const int i = tid + it * kThreads;
+        body(i, i < n, ((kc.elig >> it) & 1u) != 0, kc.key[it]);
+      }
+    }
+  } else {
+    for (int base = 0; base < n; base += kBatch * kThreads) {
+      uint32_t k[kBatch];
+      uint32_t e = 0;
+#pragma unroll
+      for (int b = 0; b < kBatch; ++b) {
+        const int i = base + b * kThreads + tid;
+        k[b] = 0;
+        if (i < n && key_of(i, k[b])) e |= 1u << b;
+      }
+#pragma unroll
+      for (int b = 0; b < kBatch; ++b) {
+        if (base + b * kThreads < n) {
+          const int i = base + b * kThreads + tid;
+          body(i, i < n, ((e >> b) & 1u) != 0, k[b]);
+        }
+      }
+    }
+  }
+}
+
+// Top-`want` of the eligible elements of [0, n) by key. All threads of the block must call it; the result is uniform
+// across the block.
+template <bool CACHED, class KeyFn>
+__device__ SelectResult block_radix_select(int n, int want, KeyFn key_of, const KeyCache& kc, SelectShared& sh) {
   SelectResult r;
   r.thresh = 0;
   r.ties = 0;
@@ -57,21 +110,16 @@ __device__ SelectResult block_radix_select(int n, int want, KeyFn key_of, Select
     sh.remaining = want;
     sh.done_all = 0;
   }
-  const int n_round = (n + kThreads - 1) / kThreads * kThreads;
   for (int pass = 0; pass < 4; ++pass) {
     const int shift = 24 - 8 * pass;
     if (tid < 256) sh.hist[tid] = 0;
     __syncthreads();
     const uint32_t prefix = sh.prefix, mask = sh.mask;
-    for (int i = tid; i < n_round; i += kThreads) {
-      int bin = -1;
-      if (i < n) {
-        uint32_t key;
-        if (key_of(i, key) && (key & mask) == prefix) bin = (int)((key >> shift) & 255u);
-      }
+    sweep<CACHED>(n, key_of, kc, [&](int, bool, bool elig, uint32_t key) {
+      const int bin = (elig && (key & mask) == prefix) ? (int)((key >> shift) & 255u) : -1;
       const unsigned peers = __match_any_sync(0xffffffffu, bin);
       if (bin >= 0 && lane == __ffs(peers) - 1) atomicAdd(&sh.hist[bin], (uint32_t)__popc(peers));
-    }
+    });
     __syncthreads();
     if (tid < 32) {
       // lane l owns bins [8l, 8l+8); walk from the top bin down until `remaining` elements are covered
@@ -118,43 +166,43 @@ __device__ SelectResult block_radix_select(int n, int want, KeyFn key_of, Select
   return r;
 }
 
-// Ordered pass over [0, n): element i is `definite` (taken for sure) or a `tie` (taken while ties last). Calls
-// emit(i, rank) for every taken element with its rank in ascending position order. Returns the number taken.
-template <class ClassFn, class EmitFn>
-__device__ int block_ordered_emit(int n, int ties_allowed, ClassFn classify, EmitFn emit, SelectShared& sh) {
+// Ordered pass over [0, n): classify(i, eligible, key, def, tie) marks element i `definite` (taken for sure) or a
+// `tie` (taken while ties last). Calls emit(i, rank) for every taken element with its rank in ascending position
+// order. Returns the number taken.
+template <bool CACHED, class KeyFn, class ClassFn, class EmitFn>
+__device__ int block_ordered_emit(int n, int ties_allowed, KeyFn key_of, const KeyCache& kc, ClassFn classify,
+                                  EmitFn emit, SelectShared& sh) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   int def_base = 0, tie_base = 0;
-  const int n_round = (n + kThreads - 1) / kThreads * kThreads;
-  for (int i = tid; i < n_round; i += kThreads) {
+  sweep<CACHED>(n, key_of, kc, [&](int i, bool exists, bool elig, uint32_t key) {
     bool def = false, tie = false;
-    if (i < n) classify(i, def, tie);
+    if (exists) classify(i, elig, key, def, tie);
     const unsigned bd = __ballot_sync(0xffffffffu, def), bt = __ballot_sync(0xffffffffu, tie);
     const unsigned lt = (1u << lane) - 1u;
-    if (lane == 0) {
-      sh.warp_def[warp] = __popc(bd);
-      sh.warp_tie[warp] = __popc(bt);
-    }
+    if (lane == 0) sh.warp_cnt[warp] = (uint32_t)__popc(bd) | ((uint32_t)__popc(bt) << 16);
     __syncthreads();
-    int def_before = __popc(bd & lt), tie_before = __popc(bt & lt);
-    int def_total = 0, tie_total = 0;
-    for (int w = 0; w < kWarps; ++w) {
-      const int d = sh.warp_def[w], t = sh.warp_tie[w];
-      if (w < warp) {
-        def_before += d;
-        tie_before += t;
+    uint32_t before = 0, total = 0;
+    const uint4* wc = reinterpret_cast<const uint4*>(sh.warp_cnt);
+#pragma unroll
+    for (int q = 0; q < kWarps / 4; ++q) {
+      const uint4 c4 = wc[q];
+      const uint32_t cs[4] = {c4.x, c4.y, c4.z, c4.w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        total += cs[e];
+        if (4 * q + e < warp) before += cs[e];
       }
-      def_total += d;
-      tie_total += t;
     }
-    const int ties_seen = tie_base + tie_before;
+    const int def_before = (int)(before & 0xffffu) + __popc(bd & lt);
+    const int ties_seen = tie_base + (int)(before >> 16) + __popc(bt & lt);
     if (def)
       emit(i, def_base + def_before + min(ties_seen, ties_allowed));
     else if (tie && ties_seen < ties_allowed)
       emit(i, def_base + def_before + ties_seen);
-    def_base += def_total;
-    tie_base += tie_total;
+    def_base += (int)(total & 0xffffu);
+    tie_base += (int)(total >> 16);
     __syncthreads();
-  }
+  });
   return def_base + min(tie_base, ties_allowed);
 }
 
@@ -180,6 +228,7 @@ __device__ __forceinline__ SeqInfo seq_info(const ta_seq_desc& seq, int b, int K
   return s;
 }
 
+template <bool CACHED>
 __global__ void __launch_bounds__(kThreads) ta_forced_kernel(ta_seq_desc seq, int K, int n_sink, int n_recent,
                                                              int k_protected, const float* __restrict__ voucher,
                                                              uint8_t* __restrict__ forced,
@@ -209,19 +258,19 @@ __global__ void __launch_bounds__(kThreads) ta_forced_kernel(ta_seq_desc seq, in
     key = sortable_key(v);
     return v > 0.0f && !mandatory(i);
   };
-  const SelectResult r = block_radix_select(s.n, s.p, key_of, sh);
+  KeyCache kc;
+  if (CACHED) fill_cache(s.n, key_of, kc);
+  const SelectResult r = block_radix_select<CACHED>(s.n, s.p, key_of, kc, sh);
   uint8_t* f = forced + s.start;
   // ordered pass: mandatory tokens and vouchers above the threshold are forced for sure; vouchers equal to the
   // threshold are forced while protected slots last, lowest position first
-  auto classify = [&](int i, bool& def, bool& tie) {
-    uint32_t key;
-    const bool cand = key_of(i, key);
+  auto classify = [&](int i, bool cand, uint32_t key, bool& def, bool& tie) {
     def = mandatory(i) || (cand && !r.none && (r.all || key > r.thresh));
     tie = !def && cand && !r.none && !r.all && key == r.thresh;
     f[i] = 0;  // set by emit when taken (same thread, later)
   };
   auto emit = [&](int i, int rank) { f[i] = 1; };
-  const int taken = block_ordered_emit(s.n, r.ties, classify, emit, sh);
+  const int taken = block_ordered_emit<CACHED>(s.n, r.ties, key_of, kc, classify, emit, sh);
   if (threadIdx.x == 0) r_main[b] = s.K_eff - taken;
 }
 
@@ -243,6 +292,7 @@ __device__ __forceinline__ float unit_utility(const UnitSrc& src, long long unit
 }
 
 // grid.x = units. scored: unit = (l*B + b)*Hkv + g; fast: unit = b.
+template <bool CACHED>
 __global__ void __launch_bounds__(kThreads) ta_select_kernel(ta_seq_desc seq, int n_layers, int Hkv, int K, int fast,
                                                              UnitSrc src, const uint8_t* __restrict__ forced,
                                                              const int32_t* __restrict__ r_main,
@@ -278,17 +328,17 @@ __global__ void __launch_bounds__(kThreads) ta_select_kernel(ta_seq_desc seq, in
     key = sortable_key(unit_utility(src, unit_off, (long long)start + i));
     return f[i] == 0;
   };
-  const SelectResult r = block_radix_select(n, want, key_of, sh);
-  auto classify = [&](int i, bool& def, bool& tie) {
-    uint32_t key;
-    const bool elig = key_of(i, key);
+  KeyCache kc;
+  if (CACHED) fill_cache(n, key_of, kc);
+  const SelectResult r = block_radix_select<CACHED>(n, want, key_of, kc, sh);
+  auto classify = [&](int, bool elig, uint32_t key, bool& def, bool& tie) {
     def = !elig || (!r.none && (r.all || key > r.thresh));
     tie = !def && !r.none && !r.all && key == r.thresh;
   };
   auto emit = [&](int i, int rank) {
     if (rank < K) out[rank] = i;
   };
-  const int taken = block_ordered_emit(n, r.ties, classify, emit, sh);
+  const int taken = block_ordered_emit<CACHED>(n, r.ties, key_of, kc, classify, emit, sh);
   for (int q = taken + tid; q < K; q += kThreads) out[q] = -1;
   if (tid == 0) count[unit] = taken;
 }
@@ -314,8 +364,12 @@ __global__ void ta_broadcast_idx_kernel(int B, int Hkv, int K, int n_layers, con
 // per-sequence result only).
 cudaError_t ta_launch_forced(const ta_select_args& a, ta_dev_status* status, cudaStream_t stream) {
   if (a.seq.batch == 0 || a.n_layers == 0) return cudaSuccess;
-  ta_forced_kernel<<<a.seq.batch, kThreads, 0, stream>>>(a.seq, a.K, a.n_sink, a.n_recent, a.k_protected, a.voucher,
-                                                         a.forced, a.r_main, status);
+  if (a.seq.max_n <= kItems * kThreads)
+    ta_forced_kernel<true><<<a.seq.batch, kThreads, 0, stream>>>(a.seq, a.K, a.n_sink, a.n_recent, a.k_protected,
+                                                               a.voucher, a.forced, a.r_main, status);
+  else
+    ta_forced_kernel<false><<<a.seq.batch, kThreads, 0, stream>>>(a.seq, a.K, a.n_sink, a.n_recent, a.k_protected,
+                                                                a.voucher, a.forced, a.r_main, status);
   return cudaGetLastError();
 }
 
@@ -329,8 +383,12 @@ cudaError_t ta_launch_select_units(const ta_select_args& a, cudaStream_t stream)
   src.alpha = a.alpha;
   src.delta = a.delta;
   const int units = a.fast ? a.seq.batch : a.n_layers * a.seq.batch * a.Hkv;
-  ta_select_kernel<<<units, kThreads, 0, stream>>>(a.seq, a.n_layers, a.Hkv, a.K, a.fast, src, a.forced, a.r_main,
-                                                   a.idx, a.count);
+  if (a.seq.max_n <= kItems * kThreads)
+    ta_select_kernel<true><<<units, kThreads, 0, stream>>>(a.seq, a.n_layers, a.Hkv, a.K, a.fast, src, a.forced,
+                                                         a.r_main, a.idx, a.count);
+  else
+    ta_select_kernel<false><<<units, kThreads, 0, stream>>>(a.seq, a.n_layers, a.Hkv, a.K, a.fast, src, a.forced,
+                                                          a.r_main, a.idx, a.count);
   return cudaGetLastError();
 }
 
