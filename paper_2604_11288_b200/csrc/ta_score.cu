@@ -540,8 +540,10 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           const int pos = n - p.W + my_t[mb];
           lim_row[mb] = (my_t[mb] >= 0 && pos >= 0) ? (p.causal ? pos : n - 1) : -1;
         }
-        // 16 keys of one row (half of a 32-key chunk); masked tiles (cold) drop keys beyond `lim`
-        auto chunk1 = [&](auto masked_tag, const uint32_t(&cur)[16], float& rc_io, float& z_io, int kbase, int lim) {
+        // 16 keys of one row (half of a 32-key chunk): adds exp2(s*c - rc) to `sum`, tracks the largest s*c.
+        // Masked tiles (cold) drop keys beyond `lim`.
+        auto half1 = [&](auto masked_tag, const uint32_t(&cur)[16], float rc, float& sum, float& mx, int kbase,
+                         int lim) {
           constexpr bool masked = decltype(masked_tag)::value;
           float v[16];
 #pragma unroll
@@ -551,7 +553,6 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             for (int q = 0; q < 16; ++q)
               if (kbase + q > lim) v[q] = -INFINITY;
           }
-          const float rc = rc_io;
           float a0 = 0.0f, a1 = 0.0f, a2 = 0.0f, a3 = 0.0f;
 #pragma unroll
           for (int q = 0; q < 16; q += 4) {
@@ -563,23 +564,8 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           float t4[4];
 #pragma unroll
           for (int q = 0; q < 4; ++q) t4[q] = fmaxf(fmaxf(v[4 * q], v[4 * q + 1]), fmaxf(v[4 * q + 2], v[4 * q + 3]));
-          const float cm_c = fmaxf(fmaxf(t4[0], t4[1]), fmaxf(t4[2], t4[3])) * c;
-          const bool jump = cm_c > rc + 8.0f;
-          float add = (a0 + a1) + (a2 + a3);
-          if (__any_sync(0xffffffffu, jump)) {
-            if (jump) {  // new reference = this chunk's maximum; earlier sums are rescaled, the chunk is redone
-              z_io *= ex2(rc - cm_c);
-              rc_io = cm_c;
-              float b0 = 0.0f, b1 = 0.0f;
-#pragma unroll
-              for (int q = 0; q < 16; q += 2) {
-                b0 += ex2(fmaf(v[q + 0], c, -cm_c));
-                b1 += ex2(fmaf(v[q + 1], c, -cm_c));
-              }
-              add = b0 + b1;
-            }
-          }
-          z_io += add;
+          mx = fmaxf(mx, fmaxf(fmaxf(t4[0], t4[1]), fmaxf(t4[2], t4[3])));
+          sum += (a0 + a1) + (a2 + a3);
         };
         uint32_t ra[16], rb[16];
         int j = ((jg & 1) == grp) ? 0 : 1;
@@ -587,8 +573,11 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           wait_full(jg + j, 30);
           tmem_ld16_issue(acc_addr(jg + j), ra);
         }
-        // one job: the accumulator in 32-column chunks, each fetched as two 16-column loads (ra, rb) so that one
-        // load is always in flight; the next job's first load is issued before the last half-chunk is computed
+        // One job: the accumulator in 32-column chunks, each fetched as two 16-column loads (ra, rb) so that one
+        // load is always in flight; the next job's first load is issued before the last half-chunk is computed.
+        // The exponentials of the whole tile use the reference left by the previous tiles; only after the tile is
+        // it checked whether its maximum ran more than 2^8 ahead of that reference, in which case the tile is
+        // read again (the accumulator stage is released after the check) with its own maximum as the new reference.
         auto job1 = [&](auto masked_tag, int j) {
           const int jj = jg + j;
           const int key0 = (ui.t_begin + j) * kTileN;
@@ -596,24 +585,48 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 #pragma unroll
           for (int mb = 0; mb < MB; ++mb) {
             const int lim = lim_row[mb];
+            const float rc = ref_c[mb];
+            float sum = 0.0f, mx = -INFINITY;
 #pragma unroll 1
             for (int c4 = 0; c4 < 4; ++c4) {
               const uint32_t col = (uint32_t)(mb * 128 + c4 * 32);
               tmem_ld_wait(ra);
               tmem_ld16_issue(abase + col + 16, rb);
-              chunk1(masked_tag, ra, ref_c[mb], z_run[mb], key0 + c4 * 32, lim);
+              half1(masked_tag, ra, rc, sum, mx, key0 + c4 * 32, lim);
               tmem_ld_wait(rb);
               if (mb == MB - 1 && c4 == 3) {
-                release(jj);
-                if (j + 2 < T) {
+                // with more than one stage per group the next job's accumulator is a different stage: fetch ahead
+                if (kAcc > 2 && j + 2 < T) {
                   wait_full(jj + 2, 30);
                   tmem_ld16_issue(acc_addr(jj + 2), ra);
                 }
               } else {
                 tmem_ld16_issue(abase + col + 32, ra);
               }
-              chunk1(masked_tag, rb, ref_c[mb], z_run[mb], key0 + c4 * 32 + 16, lim);
+              half1(masked_tag, rb, rc, sum, mx, key0 + c4 * 32 + 16, lim);
             }
+            const float mx_c = mx * c;
+            const bool jump = mx_c > rc + 8.0f;
+            if (__any_sync(0xffffffffu, jump)) {  // rare: first tiles of a unit, or a score far above all before
+              float sum2 = 0.0f, mx2 = -INFINITY;
+#pragma unroll 1
+              for (int h = 0; h < 8; ++h) {
+                tmem_ld16_issue(abase + (uint32_t)(mb * 128 + h * 16), rb);
+                tmem_ld_wait(rb);
+                half1(masked_tag, rb, jump ? mx_c : rc, sum2, mx2, key0 + h * 16, lim);
+              }
+              if (jump) {
+                z_run[mb] *= ex2(rc - mx_c);
+                ref_c[mb] = mx_c;
+                sum = sum2;
+              }
+            }
+            z_run[mb] += sum;
+          }
+          release(jj);
+          if (kAcc == 2 && j + 2 < T) {  // one stage per group: the next job can only be fetched once this one is released
+            wait_full(jj + 2, 30);
+            tmem_ld16_issue(acc_addr(jj + 2), ra);
           }
         };
         for (; j < T; j += 2) {
