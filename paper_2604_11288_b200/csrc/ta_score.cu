@@ -422,7 +422,8 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         for (int j = 0; j < n_jobs; ++j, ++jg) {
           const int s = jg % kStages;
           mbar_wait(smem_u32(&sm.empty[s]), ((uint32_t)(jg / kStages) & 1u) ^ 1u, abort_flag, p.status, 10);
-          const int tile = ui.t_begin + (j >= ui.T ? j - ui.T : j);
+          // the second sweep walks the CTA's tiles backwards: the tiles read last are the ones still in L2
+          const int tile = ui.t_begin + (j >= ui.T ? 2 * ui.T - 1 - j : j);
           const uint32_t bar = smem_u32(&sm.full[s]);
           mbar_expect_tx(bar, kKTileBytes);
           const uint32_t dst = k_smem + s * kKTileBytes;
@@ -789,7 +790,7 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           if (PM == 0 || PM == 1) fold(0);
         };
         for (; j < n_jobs; j += 2) {
-          const int key = (ui.t_begin + (j - j0)) * kTileN + row_in_tile;
+          const int key = (ui.t_begin + (p.two_pass ? n_jobs - 1 - j : j)) * kTileN + row_in_tile;
 #pragma unroll
           for (int q = 0; q < 32; ++q) sT[q] = 0.0f;
           sA = 0.0f;
