@@ -252,7 +252,11 @@ def e2e_leg(r, steps, warmup):
                             cnt_h, ws_ptr, nbytes, r.stream)
 
     ms = time_steps(run, steps, warmup)
-    h2d = ids_h.numel() * 4 + (q_h.numel() * 2 if q_h is not None else 0) + k_h.numel() * 2 + v_h.numel() * 2
+    # V is pinned: only its retained rows cross the bus (read in place by the gather kernel); same for K in fast mode
+    k_eff = int(sum(min(r.K, int(x)) for x in w.lengths)) * r.L * w.Hkv
+    row = w.d * 2
+    h2d = ids_h.numel() * 4 + (q_h.numel() * 2 if q_h is not None else 0)
+    h2d += (k_eff * row if r.fast else k_h.numel() * 2) + k_eff * row
     d2h = ko_h.numel() * 2 + vo_h.numel() * 2 + idx_h.numel() * 4 + cnt_h.numel() * 4
     ok = bool((idx_h.to(r.dev) == r.idx).all()) and bool((ko_h.to(r.dev) == r.ko).all())
     return ms, h2d, d2h, ok
@@ -408,7 +412,7 @@ def main():
     torch.cuda.empty_cache()
     if not a.no_extra and world == 1:
         extra = []
-        for name, layers in (("c3", 2), ("c4", 4), ("c5", 2)):
+        for name, layers in (("c3", 2), ("c4", 16), ("c5", 2)):
             if name == a.workload:
                 continue
             try:

@@ -259,7 +259,9 @@ ta_status ta_compress(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* pol
  * Same computation with every data pointer on the HOST (pinned memory makes the copies asynchronous):
  * token_ids, cu_seqlens (inside batch: HOST here), the q_obs / k / v views, and the four outputs. The caller lends
  * `workspace` (DEVICE, workspace_bytes >= ta_compress_host_workspace_bytes(...)) for the staged copies. Host to
- * device copies, kernels and device to host copies are all enqueued on `stream`. Views must be dense in the
+ * device copies, kernels and device to host copies are all enqueued on `stream`. A V cache (and, in fast mode, a K
+ * cache) that lies in pinned or registered host memory is not copied at all: only its retained rows are read, directly
+ * over the bus, by the gather kernel. Views must be dense in the
  * order [L][B][Hkv or Hq][n or W][d] (ragged: [L][Hkv][total_tokens][d]); other strides return
  * TA_ERR_UNSUPPORTED. */
 ta_status ta_compress_host_workspace_bytes(const ta_batch* batch, int Hq, int Hkv, int d, int K,

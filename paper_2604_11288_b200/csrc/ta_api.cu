@@ -701,19 +701,36 @@ ta_status ta_compress_host(ta_ctx* ctx, const ta_patterns* pats, const ta_policy
     db.cu_seqlens = reinterpret_cast<const int32_t*>(ws + H.cu);
   }
   if (e == cudaSuccess && !fast) e = cudaMemcpyAsync(ws + H.q, q_obs, H.q_bytes, cudaMemcpyHostToDevice, stream);
-  if (e == cudaSuccess) e = cudaMemcpyAsync(ws + H.k, k, H.kv_bytes, cudaMemcpyHostToDevice, stream);
-  if (e == cudaSuccess) e = cudaMemcpyAsync(ws + H.v, v, H.kv_bytes, cudaMemcpyHostToDevice, stream);
+  // Only the retained rows of V are ever read (and, in fast mode, of K): when such a cache sits in pinned or
+  // registered host memory the gather kernel reads those rows straight over the bus and the full copy is skipped.
+  auto device_visible_host = [&](const void* ptr, const void** dev_alias) {
+    cudaPointerAttributes at;
+    if (cudaPointerGetAttributes(&at, ptr) != cudaSuccess) {
+      cudaGetLastError();
+      return false;
+    }
+    if (at.type != cudaMemoryTypeHost || !at.devicePointer) return false;
+    *dev_alias = at.devicePointer;
+    return true;
+  };
+  const void* k_src = ws + H.k;
+  const void* v_src = ws + H.v;
+  const void* alias = nullptr;
+  if (fast && device_visible_host(k, &alias)) k_src = alias;
+  else if (e == cudaSuccess) e = cudaMemcpyAsync(ws + H.k, k, H.kv_bytes, cudaMemcpyHostToDevice, stream);
+  if (device_visible_host(v, &alias)) v_src = alias;
+  else if (e == cudaSuccess) e = cudaMemcpyAsync(ws + H.v, v, H.kv_bytes, cudaMemcpyHostToDevice, stream);
   if (e != cudaSuccess) return cuda_fail(ctx, e);
   const int64_t n = batch->n_uniform, W = policy->obs_window;
   ta_bf16_view vq = {ws + H.q, (int64_t)batch->batch * Hq * W * d, (int64_t)Hq * W * d, W * d, d};
   ta_bf16_view vk, vv;
   if (batch->cu_seqlens) {
-    vk = {ws + H.k, (int64_t)Hkv * (int64_t)total * d, 0, (int64_t)total * d, d};
+    vk = {k_src, (int64_t)Hkv * (int64_t)total * d, 0, (int64_t)total * d, d};
   } else {
-    vk = {ws + H.k, (int64_t)batch->batch * Hkv * n * d, (int64_t)Hkv * n * d, n * d, d};
+    vk = {k_src, (int64_t)batch->batch * Hkv * n * d, (int64_t)Hkv * n * d, n * d, d};
   }
   vv = vk;
-  vv.ptr = ws + H.v;
+  vv.ptr = v_src;
   s = ta_compress(ctx, pats, policy, &db, Hq, Hkv, d, K, reinterpret_cast<const int32_t*>(ws + H.ids), vq, vk, vv, 0,
                   ws + H.k_out, ws + H.v_out, reinterpret_cast<int32_t*>(ws + H.idx),
                   reinterpret_cast<int32_t*>(ws + H.count), stream);

@@ -328,3 +328,35 @@ def test_host_argument_checks():
         assert g.poll() == ta.TA_OK
     finally:
         g.close()
+
+
+@pytest.mark.parametrize("fast", [False, True])
+@pytest.mark.parametrize("pinned", [True, False])
+def test_compress_host_matches_device_path(fast, pinned):
+    """The host-buffer entry point (staged copies; pinned caches gathered in place) gives the device path's result."""
+    w = tw.config1(n=1500, Hq=8, Hkv=2)  # uniform batch of one sequence
+    K, L = 16, 2
+    pol = oracle_policy(K, "THEOREM", fast=fast, W=w.W)
+    Qh, Kh, Vh = tw.make_qkv(w, range(L))
+    g = Gpu(w, pol, K, L)
+    try:
+        idx, cnt, ko, vo = g.compress(Qh.cuda(), Kh.cuda(), Vh.cuda())
+        torch.cuda.synchronize()
+        pin = (lambda t: t.pin_memory()) if pinned else (lambda t: t)
+        ids_h = pin(torch.from_numpy(w.ids))
+        q_h, k_h, v_h = pin(Qh.contiguous()), pin(Kh.contiguous()), pin(Vh.contiguous())
+        ko_h, vo_h = pin(torch.zeros(ko.shape, dtype=torch.bfloat16)), pin(torch.zeros(vo.shape, dtype=torch.bfloat16))
+        idx_h, cnt_h = pin(torch.zeros(idx.shape, dtype=torch.int32)), pin(torch.zeros(cnt.shape, dtype=torch.int32))
+        hb = ta.make_batch(L, w.B, int(w.lengths[0]), w.max_n, w.total, None)
+        nbytes = ta.ta_compress_host_workspace_bytes(hb, w.Hq, w.Hkv, w.d, K, g.p)
+        ws = torch.empty(nbytes + 256, dtype=torch.uint8, device="cuda")
+        ws_ptr = (ws.data_ptr() + 255) // 256 * 256
+        ta.ta_compress_host(g.ctx, g.pats, g.p, hb, w.Hq, w.Hkv, w.d, K, ids_h, None if fast else q_h, k_h, v_h, ko_h,
+                            vo_h, idx_h, cnt_h, ws_ptr, nbytes, g.stream)
+        torch.cuda.synchronize()
+        assert g.poll() == ta.TA_OK
+        assert torch.equal(idx_h, idx.cpu()) and torch.equal(cnt_h, cnt.cpu())
+        assert torch.equal(ko_h.view(torch.int16), ko.cpu().view(torch.int16))
+        assert torch.equal(vo_h.view(torch.int16), vo.cpu().view(torch.int16))
+    finally:
+        g.close()
