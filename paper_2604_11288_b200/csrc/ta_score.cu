@@ -37,10 +37,16 @@ constexpr int kD = TA_HEAD_DIM;                   // 128
 constexpr int kHalfBytes = kTileN * 128;          // one 64-column half of a 128-row operand tile: 16 KB
 constexpr int kKTileBytes = 2 * kHalfBytes;       // 32 KB
 constexpr int kMaxCluster = 8;
-constexpr int kThreads = 384;                     // warps 0-7 softmax, 8 TMA producer, 9 MMA issuer, 10-11 idle
-constexpr int kRegsSoftmax = 216;                 // register split after set-up (setmaxnreg): 8 softmax warps
-constexpr int kRegsOther = 72;                    // ... and the 4 warps of the third warpgroup
-constexpr int kRegsNeeded = (8 * kRegsSoftmax + 4 * kRegsOther) * 32;  // must fit in threads x registers at launch
+// NG softmax warpgroups (4 warps each) plus one warpgroup holding the TMA producer warp, the MMA issuer warp and
+// two idle warps. Register split after set-up (setmaxnreg); the shares must fit in threads x registers at launch:
+//   NG = 2: 384 threads x 168 = 64512 = 8*32*216 + 4*32*72        NG = 3: 512 threads x 128 = 65536 = 12*32*152 + 4*32*56
+template <int NG>
+struct GroupCfg {
+  static constexpr int kThreads = (NG + 1) * 128;
+  static constexpr int kRegsSoftmax = NG == 2 ? 216 : 152;
+  static constexpr int kRegsOther = NG == 2 ? 72 : 56;
+  static constexpr int kRegsNeeded = (NG * 4 * kRegsSoftmax + 4 * kRegsOther) * 32;
+};
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s
 
 struct ScoreParams {
@@ -221,7 +227,10 @@ __device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t par
       : "memory");
   return ok != 0;
 }
-__device__ __forceinline__ void softmax_bar() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+template <int NG>
+__device__ __forceinline__ void softmax_bar() {
+  asm volatile("bar.sync 1, %0;" ::"n"(NG * 128) : "memory");
+}
 
 // Shared-memory matrix descriptor for a K-major operand tile stored as rows of 128 bytes with the 128-byte swizzle
 // (what a TMA box of 64 bf16 x rows with CU_TENSOR_MAP_SWIZZLE_128B writes): 8-row groups are 1024 bytes apart.
@@ -264,23 +273,25 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity,
 }
 
 // ---------------------------------------------------------------------------------------------- shared memory
-template <int MB>
+template <int MB, int NG>
 struct ScoreCfg {
   static constexpr int kQBufs = MB == 1 ? 2 : 1;   // query tiles in flight (next unit's tile loads early)
   static constexpr int kStages = MB == 1 ? 4 : 3;  // ring of key tiles
   static constexpr int kRowsPad = MB * 128;
-  static constexpr int kAcc = MB == 1 ? 4 : 2;     // accumulator stages in tensor memory (kAcc * kRowsPad = 512 columns)
+  // accumulator stages in tensor memory (at most 512 columns): two per softmax group when they fit (the group can
+  // then fetch its next job before releasing the current one), else one per group
+  static constexpr int kAcc = MB == 1 ? (NG == 2 ? 4 : 3) : 2;
 };
 
-template <int MB>
+template <int MB, int NG>
 struct alignas(1024) ScoreSmem {
-  using Cfg = ScoreCfg<MB>;
+  using Cfg = ScoreCfg<MB, NG>;
   uint8_t q[Cfg::kQBufs][MB * 2 * kHalfBytes];    // [buffer][half][MB*128 rows][128 B]
   uint8_t k[Cfg::kStages][kKTileBytes];           // [stage][half][128 rows][128 B]
   float mine_m[2][MB * 128];                      // [unit parity][row]: this CTA's row statistics, read by its peers
   float mine_z[2][MB * 128];
-  float part_m[2][MB * 128];                      // per softmax group
-  float part_z[2][MB * 128];
+  float part_m[NG][MB * 128];                     // per softmax group
+  float part_z[NG][MB * 128];
   float lse2[2][MB * 128];                        // [unit parity][row] log2-domain log-sum-exp (+inf: row is mute)
   float wrow[MB * 128];                           // pension weight per row
   int row_t[MB * 128];                            // window index t of the row, -1 for padding rows
@@ -303,16 +314,18 @@ struct UnitInfo {
 };
 
 // ---------------------------------------------------------------------------------------------- the kernel
-template <int MB, int PM>
-__global__ void __launch_bounds__(kThreads, 1)
+template <int MB, int PM, int NG>
+__global__ void __launch_bounds__(GroupCfg<NG>::kThreads, 1)
 ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                 const __grid_constant__ ScoreParams p) {
-  using Cfg = ScoreCfg<MB>;
+  using Cfg = ScoreCfg<MB, NG>;
+  constexpr int kThreads = GroupCfg<NG>::kThreads;
+  constexpr int kWarpTma = NG * 4, kWarpMma = NG * 4 + 1;
   constexpr int kStages = Cfg::kStages, kQBufs = Cfg::kQBufs, kRowsPad = Cfg::kRowsPad;
   constexpr int kAcc = Cfg::kAcc;
   constexpr uint32_t kTmemCols = 512;  // kAcc accumulator stages of kRowsPad columns
   extern __shared__ uint8_t smem_raw[];
-  ScoreSmem<MB>& sm = *reinterpret_cast<ScoreSmem<MB>*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  ScoreSmem<MB, NG>& sm = *reinterpret_cast<ScoreSmem<MB, NG>*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const uint32_t rank = cluster_ctarank();
@@ -362,7 +375,7 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     sm.abort_flag = (*reinterpret_cast<volatile int*>(&p.status->code) == (int)TA_ERR_TIMEOUT) ? 1 : 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 9) {
+  if (warp == kWarpMma) {
     tmem_alloc(smem_u32(&sm.tmem_base), kTmemCols);
     tmem_relinquish();
   }
@@ -394,9 +407,9 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 
   const uint32_t k_smem = smem_u32(sm.k);
 
-  if (warp >= 8) {
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsOther));
-  if (warp == 8) {
+  if (warp >= kWarpTma) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(GroupCfg<NG>::kRegsOther));
+  if (warp == kWarpTma) {
     // =========================================================================== TMA producer
     if (lane == 0) {
       int issued[kStages];
@@ -442,7 +455,7 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         }
       }
     }
-  } else if (warp == 9) {
+  } else if (warp == kWarpMma) {
     // =========================================================================== MMA issuer
     if (lane == 0) {
       int jg = 0, qn = 0;
@@ -497,10 +510,11 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     }
   }
   } else {
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmax));
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(GroupCfg<NG>::kRegsSoftmax));
     // =========================================================================== softmax warps
     const int st = tid;                   // 0..255
-    const int grp = st >> 7;              // this group serves jobs with (global job index & 1) == grp
+    const int grp = st >> 7;              // this group serves jobs with (global job index % NG) == grp
+    constexpr bool kAhead = (kAcc >= 2 * NG);  // two stages per group: fetch the next job before releasing this one
     const int quad = warp & 3;            // TMEM lane quadrant this warp may read
     const int row_in_tile = quad * 32 + lane;
     const uint32_t tlane = tmem_base + ((uint32_t)(quad * 32) << 16);
@@ -569,7 +583,7 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           sum += (a0 + a1) + (a2 + a3);
         };
         uint32_t ra[16], rb[16];
-        int j = ((jg & 1) == grp) ? 0 : 1;
+        int j = (grp - jg % NG + NG) % NG;  // first job of this pass that belongs to the group
         if (j < T) {
           wait_full(jg + j, 30);
           tmem_ld16_issue(acc_addr(jg + j), ra);
@@ -597,9 +611,9 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
               tmem_ld_wait(rb);
               if (mb == MB - 1 && c4 == 3) {
                 // with more than one stage per group the next job's accumulator is a different stage: fetch ahead
-                if (kAcc > 2 && j + 2 < T) {
-                  wait_full(jj + 2, 30);
-                  tmem_ld16_issue(acc_addr(jj + 2), ra);
+                if (kAhead && j + NG < T) {
+                  wait_full(jj + NG, 30);
+                  tmem_ld16_issue(acc_addr(jj + NG), ra);
                 }
               } else {
                 tmem_ld16_issue(abase + col + 32, ra);
@@ -625,12 +639,12 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             z_run[mb] += sum;
           }
           release(jj);
-          if (kAcc == 2 && j + 2 < T) {  // one stage per group: the next job can only be fetched once this one is released
-            wait_full(jj + 2, 30);
-            tmem_ld16_issue(acc_addr(jj + 2), ra);
+          if (!kAhead && j + NG < T) {  // one stage per group: the next job can only be fetched once this one is released
+            wait_full(jj + NG, 30);
+            tmem_ld16_issue(acc_addr(jj + NG), ra);
           }
         };
-        for (; j < T; j += 2) {
+        for (; j < T; j += NG) {
           // tiles that every row of the warp sees completely take the unmasked path (rows that see nothing at all,
           // i.e. padding, still run: their sums are never used)
           bool masked = false;
@@ -647,14 +661,18 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           sm.part_m[grp][mb * 128 + row_in_tile] = lim_row[mb] >= 0 ? ref_c[mb] : -1e30f;
           sm.part_z[grp][mb * 128 + row_in_tile] = lim_row[mb] >= 0 ? z_run[mb] : 0.0f;
         }
-        softmax_bar();
+        softmax_bar<NG>();
         if (st < kRowsPad) {
-          const float m0 = sm.part_m[0][st], m1 = sm.part_m[1][st];
-          const float m = fmaxf(m0, m1);
+          float m = sm.part_m[0][st];
+#pragma unroll
+          for (int gq = 1; gq < NG; ++gq) m = fmaxf(m, sm.part_m[gq][st]);
+          float z = 0.0f;
+#pragma unroll
+          for (int gq = 0; gq < NG; ++gq) z += sm.part_z[gq][st] * ex2(sm.part_m[gq][st] - m);
           sm.mine_m[up][st] = m;
-          sm.mine_z[up][st] = sm.part_z[0][st] * ex2(m0 - m) + sm.part_z[1][st] * ex2(m1 - m);
+          sm.mine_z[up][st] = z;
         }
-        softmax_bar();
+        softmax_bar<NG>();
         // one thread per peer tells that peer that this CTA's statistics of the unit are in place
         if (st < p.cluster) {
           fence_cluster();
@@ -680,7 +698,7 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           for (int r = 0; r < kMaxCluster; ++r) z += pz[r] * ex2(pm[r] - m);
           sm.lse2[up][st] = (z > 0.0f) ? m + log2f(z) : INFINITY;
         }
-        softmax_bar();
+        softmax_bar<NG>();
       } else {
         if (st < kRowsPad) {
           float lse2 = INFINITY;
@@ -692,7 +710,7 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           }
           sm.lse2[up][st] = lse2;
         }
-        softmax_bar();
+        softmax_bar<NG>();
       }
 
       // ---- pass 2: column sums for key row_in_tile of each tile
@@ -756,7 +774,7 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           }
         };
         uint32_t ra[16], rb[16];
-        int j = j0 + ((((jg + j0) & 1) == grp) ? 0 : 1);
+        int j = j0 + (grp - (jg + j0) % NG + NG) % NG;
         if (j < n_jobs) {
           wait_full(jg + j, 31);
           tmem_ld16_issue(acc_addr(jg + j) + chunk_col<MB, PM>(0), ra);
@@ -775,9 +793,9 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             tmem_ld_wait(rb);
             if (ci == n_chunks2 - 1) {
               release(jj);
-              if (j + 2 < n_jobs) {
-                wait_full(jj + 2, 31);
-                tmem_ld16_issue(acc_addr(jj + 2) + chunk_col<MB, PM>(0), ra);
+              if (j + NG < n_jobs) {
+                wait_full(jj + NG, 31);
+                tmem_ld16_issue(acc_addr(jj + NG) + chunk_col<MB, PM>(0), ra);
               }
             } else {
               tmem_ld16_issue(abase + chunk_col<MB, PM>(ci + 1), ra);
@@ -789,7 +807,7 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           if (PM == 2) fold(8);
           if (PM == 0 || PM == 1) fold(0);
         };
-        for (; j < n_jobs; j += 2) {
+        for (; j < n_jobs; j += NG) {
           const int key = (ui.t_begin + (p.two_pass ? n_jobs - 1 - j : j)) * kTileN + row_in_tile;
 #pragma unroll
           for (int q = 0; q < 32; ++q) sT[q] = 0.0f;
@@ -813,7 +831,7 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
   // ---- teardown
   tc_fence_before();
   __syncthreads();
-  if (warp == 9) {
+  if (warp == kWarpMma) {
     tc_fence_after();
     tmem_dealloc(tmem_base, kTmemCols);
   }
@@ -822,9 +840,9 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
   cluster_wait();
 }
 
-template <int MB>
+template <int MB, int NG>
 size_t score_smem_bytes() {
-  return sizeof(ScoreSmem<MB>) + 1024;
+  return sizeof(ScoreSmem<MB, NG>) + 1024;
 }
 
 CUresult encode_5d(void* fn, CUtensorMap* map, const void* base, const uint64_t dims[5], const uint64_t strides_el[4],
@@ -846,11 +864,12 @@ CUresult encode_5d(void* fn, CUtensorMap* map, const void* base, const uint64_t 
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
 }
 
-template <int MB, int PM>
+template <int MB, int PM, int NG>
 cudaError_t launch_variant(ta_ctx* ctx, const CUtensorMap& mq, const CUtensorMap& mk, ScoreParams& sp,
                            int tiles_max, int reserve_sms, cudaStream_t stream) {
-  auto kern = ta_score_kernel<MB, PM>;
-  const size_t smem = score_smem_bytes<MB>();
+  auto kern = ta_score_kernel<MB, PM, NG>;
+  const size_t smem = score_smem_bytes<MB, NG>();
+  constexpr int kThreads = GroupCfg<NG>::kThreads;
   static bool attr_set_dev[64] = {};  // per device and instantiation; the attribute is sticky
   bool& attr_set = attr_set_dev[ctx->device & 63];
   if (!attr_set) {
@@ -860,7 +879,7 @@ cudaError_t launch_variant(ta_ctx* ctx, const CUtensorMap& mq, const CUtensorMap
     cudaFuncAttributes fa;
     e = cudaFuncGetAttributes(&fa, kern);
     if (e != cudaSuccess) return e;
-    if (fa.numRegs * kThreads < kRegsNeeded) return cudaErrorLaunchOutOfResources;
+    if (fa.numRegs * kThreads < GroupCfg<NG>::kRegsNeeded) return cudaErrorLaunchOutOfResources;
     attr_set = true;
   }
   cudaLaunchConfig_t cfg = {};
@@ -974,15 +993,15 @@ cudaError_t ta_launch_score(ta_ctx* ctx, const ta_score_args& a, ta_dev_status* 
   const int pm = !need_p ? 0 : (32 % a.W == 0) ? 1 : (a.W == 64 && rows == 256) ? 2 : 3;
   if (MB == 1) {
     switch (pm) {
-      case 0: return launch_variant<1, 0>(ctx, mq, mk, sp, tiles_max, a.reserve_sms, stream);
-      case 1: return launch_variant<1, 1>(ctx, mq, mk, sp, tiles_max, a.reserve_sms, stream);
-      default: return launch_variant<1, 3>(ctx, mq, mk, sp, tiles_max, a.reserve_sms, stream);
+      case 0: return launch_variant<1, 0, 3>(ctx, mq, mk, sp, tiles_max, a.reserve_sms, stream);
+      case 1: return launch_variant<1, 1, 3>(ctx, mq, mk, sp, tiles_max, a.reserve_sms, stream);
+      default: return launch_variant<1, 3, 3>(ctx, mq, mk, sp, tiles_max, a.reserve_sms, stream);
     }
   }
   switch (pm) {
-    case 0: return launch_variant<2, 0>(ctx, mq, mk, sp, tiles_max, a.reserve_sms, stream);
-    case 1: return launch_variant<2, 1>(ctx, mq, mk, sp, tiles_max, a.reserve_sms, stream);
-    case 2: return launch_variant<2, 2>(ctx, mq, mk, sp, tiles_max, a.reserve_sms, stream);
-    default: return launch_variant<2, 3>(ctx, mq, mk, sp, tiles_max, a.reserve_sms, stream);
+    case 0: return launch_variant<2, 0, 2>(ctx, mq, mk, sp, tiles_max, a.reserve_sms, stream);
+    case 1: return launch_variant<2, 1, 2>(ctx, mq, mk, sp, tiles_max, a.reserve_sms, stream);
+    case 2: return launch_variant<2, 2, 2>(ctx, mq, mk, sp, tiles_max, a.reserve_sms, stream);
+    default: return launch_variant<2, 3, 2>(ctx, mq, mk, sp, tiles_max, a.reserve_sms, stream);
   }
 }
