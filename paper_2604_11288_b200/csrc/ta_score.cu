@@ -170,19 +170,19 @@ __device__ __forceinline__ void umma_commit(uint32_t bar) {
 // Tensor-memory loads, shape 32x32b: thread i of the warp receives lane (quadrant base + i) and 16 consecutive 32-bit
 // columns. The load is asynchronous; tmem_ld_wait() must be called on the same registers before they are read.
 // Passing the registers through the wait as read-write operands keeps the compiler from moving their uses above it.
-__device__ __forceinline__ void tmem_ld16_issue(uint32_t taddr, uint32_t (&r)[16]) {
+__device__ __forceinline__ void tmem_ld16_issue(uint32_t taddr, float (&r)[16]) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
       "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];\n"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "=f"(r[0]), "=f"(r[1]), "=f"(r[2]), "=f"(r[3]), "=f"(r[4]), "=f"(r[5]), "=f"(r[6]), "=f"(r[7]), "=f"(r[8]),
+        "=f"(r[9]), "=f"(r[10]), "=f"(r[11]), "=f"(r[12]), "=f"(r[13]), "=f"(r[14]), "=f"(r[15])
       : "r"(taddr)
       : "memory");
 }
-__device__ __forceinline__ void tmem_ld_wait(uint32_t (&r)[16]) {
+__device__ __forceinline__ void tmem_ld_wait(float (&r)[16]) {
   asm volatile("tcgen05.wait::ld.sync.aligned;"
-               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
-                 "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15])
+               : "+f"(r[0]), "+f"(r[1]), "+f"(r[2]), "+f"(r[3]), "+f"(r[4]), "+f"(r[5]), "+f"(r[6]), "+f"(r[7]),
+                 "+f"(r[8]), "+f"(r[9]), "+f"(r[10]), "+f"(r[11]), "+f"(r[12]), "+f"(r[13]), "+f"(r[14]), "+f"(r[15])
                :
                : "memory");
 }
@@ -557,12 +557,12 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         }
         // 16 keys of one row (half of a 32-key chunk): adds exp2(s*c - rc) to `sum`, tracks the largest s*c.
         // Masked tiles (cold) drop keys beyond `lim`.
-        auto half1 = [&](auto masked_tag, const uint32_t(&cur)[16], float rc, float& sum, float& mx, int kbase,
+        auto half1 = [&](auto masked_tag, const float(&cur)[16], float rc, float& sum, float& mx, int kbase,
                          int lim) {
           constexpr bool masked = decltype(masked_tag)::value;
           float v[16];
 #pragma unroll
-          for (int q = 0; q < 16; ++q) v[q] = __uint_as_float(cur[q]);
+          for (int q = 0; q < 16; ++q) v[q] = cur[q];
           if (masked) {
 #pragma unroll
             for (int q = 0; q < 16; ++q)
@@ -582,7 +582,7 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           mx = fmaxf(mx, fmaxf(fmaxf(t4[0], t4[1]), fmaxf(t4[2], t4[3])));
           sum += (a0 + a1) + (a2 + a3);
         };
-        uint32_t ra[16], rb[16];
+        float ra[16], rb[16];
         int j = (grp - jg % NG + NG) % NG;  // first job of this pass that belongs to the group
         if (j < T) {
           wait_full(jg + j, 30);
@@ -725,17 +725,17 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         float sA = 0.0f, sP = 0.0f;
         // 16 rows (half `hi` of the 32-row chunk cc) of this thread's key; masked: keys inside the observation
         // window (cold tiles only)
-        auto chunk2 = [&](auto masked_tag, auto hi_tag, const uint32_t(&cur)[16], int cc, int key) {
+        auto chunk2 = [&](auto masked_tag, auto hi_tag, const float(&cur)[16], int cc, int key) {
           constexpr bool masked = decltype(masked_tag)::value;
           constexpr int hi = decltype(hi_tag)::value;  // 0: rows 32cc..32cc+15, 1: rows 32cc+16..32cc+31
 #pragma unroll
           for (int q4 = 0; q4 < 4; ++q4) {
             const float4 ls = l4[cc * 8 + hi * 4 + q4];
             float a[4];
-            a[0] = ex2(fmaf(__uint_as_float(cur[4 * q4 + 0]), c, -ls.x));
-            a[1] = ex2(fmaf(__uint_as_float(cur[4 * q4 + 1]), c, -ls.y));
-            a[2] = ex2(fmaf(__uint_as_float(cur[4 * q4 + 2]), c, -ls.z));
-            a[3] = ex2(fmaf(__uint_as_float(cur[4 * q4 + 3]), c, -ls.w));
+            a[0] = ex2(fmaf(cur[4 * q4 + 0], c, -ls.x));
+            a[1] = ex2(fmaf(cur[4 * q4 + 1], c, -ls.y));
+            a[2] = ex2(fmaf(cur[4 * q4 + 2], c, -ls.z));
+            a[3] = ex2(fmaf(cur[4 * q4 + 3], c, -ls.w));
             if (masked) {  // row r sees key i only if i <= the row's own position
 #pragma unroll
               for (int e = 0; e < 4; ++e) {
@@ -773,7 +773,7 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             sT[4 * q4] = sT[4 * q4 + 1] = sT[4 * q4 + 2] = sT[4 * q4 + 3] = 0.0f;
           }
         };
-        uint32_t ra[16], rb[16];
+        float ra[16], rb[16];
         int j = j0 + (grp - (jg + j0) % NG + NG) % NG;
         if (j < n_jobs) {
           wait_full(jg + j, 31);
