@@ -11,7 +11,11 @@
 //                      main pool by utility among the tokens not forced, then the ordered write of
 //                      forced + chosen positions.
 //   ta_broadcast_idx_kernel  fast mode: the per-sequence result is the same for all layers and heads.
+#include <cooperative_groups.h>
+
 #include "ta_internal.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace {
 
@@ -37,7 +41,12 @@ struct SelectShared {
   int remaining;
   int done_all;
   __align__(16) uint32_t warp_cnt[kWarps];  // per warp: definite count (low 16 bits) | tie count (high 16 bits)
+  // long sequences are split over the CTAs of a cluster: histogram of the whole unit (on rank 0, two buffers
+  // alternating by pass) and every CTA's (definite, tie) totals
+  uint32_t ghist[2][256];
+  int totals[8][2];
 };
+constexpr int kSelectCluster = 8;  // CTAs per unit when a sequence is longer than kItems * kThreads
 
 // Keys of a unit are read once into registers when the unit is short enough (kItems per thread), else they are
 // re-read from L2 on every sweep in batches whose loads are all issued before the first use.
@@ -95,7 +104,7 @@ __device__ __forceinline__ void sweep(int n, KeyFn key_of, const KeyCache& kc, B
 
 // Top-`want` of the eligible elements of [0, n) by key. All threads of the block must call it; the result is uniform
 // across the block.
-template <bool CACHED, class KeyFn>
+template <bool CACHED, int CL, class KeyFn>
 __device__ SelectResult block_radix_select(int n, int want, KeyFn key_of, const KeyCache& kc, SelectShared& sh) {
   SelectResult r;
   r.thresh = 0;
@@ -110,10 +119,16 @@ __device__ SelectResult block_radix_select(int n, int want, KeyFn key_of, const 
     sh.remaining = want;
     sh.done_all = 0;
   }
+  uint32_t* ghist0 = nullptr;
+  if (CL > 1) ghist0 = cg::this_cluster().map_shared_rank(&sh.ghist[0][0], 0);
   for (int pass = 0; pass < 4; ++pass) {
     const int shift = 24 - 8 * pass;
-    if (tid < 256) sh.hist[tid] = 0;
-    __syncthreads();
+    if (tid < 256) {
+      sh.hist[tid] = 0;
+      if (CL > 1) sh.ghist[pass & 1][tid] = 0;  // only rank 0's copy is used; its readers of two passes ago are done
+    }
+    if (CL > 1) cg::this_cluster().sync();
+    else __syncthreads();
     const uint32_t prefix = sh.prefix, mask = sh.mask;
     sweep<CACHED>(n, key_of, kc, [&](int, bool, bool elig, uint32_t key) {
       const int bin = (elig && (key & mask) == prefix) ? (int)((key >> shift) & 255u) : -1;
@@ -121,11 +136,21 @@ __device__ SelectResult block_radix_select(int n, int want, KeyFn key_of, const 
       if (bin >= 0 && lane == __ffs(peers) - 1) atomicAdd(&sh.hist[bin], (uint32_t)__popc(peers));
     });
     __syncthreads();
+    const uint32_t* hist = sh.hist;
+    if (CL > 1) {  // merge the slices' histograms on rank 0, then every CTA takes the same decision from the sum
+      uint32_t* gh = ghist0 + (pass & 1) * 256;
+      if (tid < 256 && sh.hist[tid]) atomicAdd(&gh[tid], sh.hist[tid]);
+      cg::this_cluster().sync();
+      hist = gh;
+    }
     if (tid < 32) {
       // lane l owns bins [8l, 8l+8); walk from the top bin down until `remaining` elements are covered
+      uint32_t hl[8];
+#pragma unroll
+      for (int k = 0; k < 8; ++k) hl[k] = hist[8 * lane + k];
       uint32_t tot = 0;
 #pragma unroll
-      for (int k = 0; k < 8; ++k) tot += sh.hist[8 * lane + k];
+      for (int k = 0; k < 8; ++k) tot += hl[k];
       uint32_t above = 0;  // elements in lanes above this one
       {
         uint32_t run = tot;
@@ -144,11 +169,15 @@ __device__ SelectResult block_radix_select(int n, int want, KeyFn key_of, const 
         const bool mine = above < (uint32_t)remaining && (uint32_t)remaining <= above + tot;
         if (mine) {
           uint32_t cum = above;
-          int bin = 8 * lane + 7;
-          for (; bin > 8 * lane; --bin) {
-            if (cum + sh.hist[bin] >= (uint32_t)remaining) break;
-            cum += sh.hist[bin];
+          int k = 7;
+#pragma unroll
+          for (int kk = 7; kk > 0; --kk) {
+            if (k == kk && cum + hl[kk] < (uint32_t)remaining) {
+              cum += hl[kk];
+              k = kk - 1;
+            }
           }
+          const int bin = 8 * lane + k;
           sh.remaining = remaining - (int)cum;
           sh.prefix = prefix | ((uint32_t)bin << shift);
           sh.mask = mask | (255u << shift);
@@ -171,9 +200,10 @@ __device__ SelectResult block_radix_select(int n, int want, KeyFn key_of, const 
 // order. Returns the number taken.
 template <bool CACHED, class KeyFn, class ClassFn, class EmitFn>
 __device__ int block_ordered_emit(int n, int ties_allowed, KeyFn key_of, const KeyCache& kc, ClassFn classify,
-                                  EmitFn emit, SelectShared& sh) {
+                                  EmitFn emit, SelectShared& sh, int def_base = 0, int tie_base = 0,
+                                  int* def_total_out = nullptr, int* tie_total_out = nullptr) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  int def_base = 0, tie_base = 0;
+  const int def0 = def_base, tie0 = tie_base;
   sweep<CACHED>(n, key_of, kc, [&](int i, bool exists, bool elig, uint32_t key) {
     bool def = false, tie = false;
     if (exists) classify(i, elig, key, def, tie);
@@ -203,7 +233,55 @@ __device__ int block_ordered_emit(int n, int ties_allowed, KeyFn key_of, const K
     tie_base += (int)(total >> 16);
     __syncthreads();
   });
+  if (def_total_out) *def_total_out = def_base - def0;
+  if (tie_total_out) *tie_total_out = tie_base - tie0;
   return def_base + min(tie_base, ties_allowed);
+}
+
+// The ordered pass for a unit split over CL CTAs (rank r owns a contiguous, ascending slice): a counting sweep
+// gives every CTA its (definite, tie) totals, the totals are exchanged through distributed shared memory, and the
+// emitting sweep starts from the sums of the lower ranks. Returns the number taken over the whole unit.
+template <bool CACHED, int CL, class KeyFn, class ClassFn, class EmitFn>
+__device__ int cluster_ordered_emit(int n, int ties_allowed, KeyFn key_of, const KeyCache& kc, ClassFn classify,
+                                    EmitFn emit, SelectShared& sh) {
+  if (CL == 1) return block_ordered_emit<CACHED>(n, ties_allowed, key_of, kc, classify, emit, sh);
+  cg::cluster_group cluster = cg::this_cluster();
+  const int rank = (int)cluster.block_rank();
+  int dt = 0, tt = 0;
+  block_ordered_emit<CACHED>(n, 0, key_of, kc, classify, [](int, int) {}, sh, 0, 0, &dt, &tt);
+  if (threadIdx.x < CL) {
+    int* peer = cluster.map_shared_rank(&sh.totals[0][0], threadIdx.x);
+    peer[rank * 2 + 0] = dt;
+    peer[rank * 2 + 1] = tt;
+  }
+  cluster.sync();
+  int def_base = 0, tie_base = 0, def_all = 0, tie_all = 0;
+#pragma unroll
+  for (int r = 0; r < CL; ++r) {
+    if (r < rank) {
+      def_base += sh.totals[r][0];
+      tie_base += sh.totals[r][1];
+    }
+    def_all += sh.totals[r][0];
+    tie_all += sh.totals[r][1];
+  }
+  block_ordered_emit<CACHED>(n, ties_allowed, key_of, kc, classify, emit, sh, def_base, tie_base);
+  return def_all + min(tie_all, ties_allowed);
+}
+
+// Slice [lo, hi) of a unit of n elements owned by this CTA when the unit is split over CL CTAs (whole chunks of
+// kThreads elements per CTA so that the slices stay aligned).
+template <int CL>
+__device__ __forceinline__ void unit_slice(int n, int& lo, int& hi) {
+  if (CL == 1) {
+    lo = 0;
+    hi = n;
+    return;
+  }
+  const int rank = (int)cg::this_cluster().block_rank();
+  const int per = ((n + CL - 1) / CL + kThreads - 1) / kThreads * kThreads;
+  lo = min(n, rank * per);
+  hi = min(n, lo + per);
 }
 
 struct SeqInfo {
@@ -228,13 +306,13 @@ __device__ __forceinline__ SeqInfo seq_info(const ta_seq_desc& seq, int b, int K
   return s;
 }
 
-template <bool CACHED>
+template <bool CACHED, int CL>
 __global__ void __launch_bounds__(kThreads) ta_forced_kernel(ta_seq_desc seq, int K, int n_sink, int n_recent,
                                                              int k_protected, const float* __restrict__ voucher,
                                                              uint8_t* __restrict__ forced,
                                                              int32_t* __restrict__ r_main, ta_dev_status* status) {
   __shared__ SelectShared sh;
-  const int b = blockIdx.x;
+  const int b = blockIdx.x / CL;
   const SeqInfo s = seq_info(seq, b, K, n_sink, n_recent, k_protected);
   if (s.n > seq.max_n || s.n < 0) {
     if (threadIdx.x == 0) {
@@ -251,27 +329,29 @@ __global__ void __launch_bounds__(kThreads) ta_forced_kernel(ta_seq_desc seq, in
     if (threadIdx.x == 0) r_main[b] = -1;  // keep everything
     return;
   }
-  const float* V = voucher + s.start;
+  int lo, hi;
+  unit_slice<CL>(s.n, lo, hi);
+  const float* V = voucher + s.start + lo;  // this CTA's slice; local index il <-> position lo + il
   auto mandatory = [&](int i) { return i < s.s_take || i >= s.n - s.r_take; };
-  auto key_of = [&](int i, uint32_t& key) {
-    const float v = V[i];
+  auto key_of = [&](int il, uint32_t& key) {
+    const float v = V[il];
     key = sortable_key(v);
-    return v > 0.0f && !mandatory(i);
+    return v > 0.0f && !mandatory(lo + il);
   };
   KeyCache kc;
-  if (CACHED) fill_cache(s.n, key_of, kc);
-  const SelectResult r = block_radix_select<CACHED>(s.n, s.p, key_of, kc, sh);
-  uint8_t* f = forced + s.start;
+  if (CACHED) fill_cache(hi - lo, key_of, kc);
+  const SelectResult r = block_radix_select<CACHED, CL>(hi - lo, s.p, key_of, kc, sh);
+  uint8_t* f = forced + s.start + lo;
   // ordered pass: mandatory tokens and vouchers above the threshold are forced for sure; vouchers equal to the
   // threshold are forced while protected slots last, lowest position first
-  auto classify = [&](int i, bool cand, uint32_t key, bool& def, bool& tie) {
-    def = mandatory(i) || (cand && !r.none && (r.all || key > r.thresh));
+  auto classify = [&](int il, bool cand, uint32_t key, bool& def, bool& tie) {
+    def = mandatory(lo + il) || (cand && !r.none && (r.all || key > r.thresh));
     tie = !def && cand && !r.none && !r.all && key == r.thresh;
-    f[i] = 0;  // set by emit when taken (same thread, later)
+    f[il] = 0;  // set by emit when taken (same thread, later)
   };
-  auto emit = [&](int i, int rank) { f[i] = 1; };
-  const int taken = block_ordered_emit<CACHED>(s.n, r.ties, key_of, kc, classify, emit, sh);
-  if (threadIdx.x == 0) r_main[b] = s.K_eff - taken;
+  auto emit = [&](int il, int rank) { f[il] = 1; };
+  const int taken = cluster_ordered_emit<CACHED, CL>(hi - lo, r.ties, key_of, kc, classify, emit, sh);
+  if (threadIdx.x == 0 && blockIdx.x % CL == 0) r_main[b] = s.K_eff - taken;
 }
 
 struct UnitSrc {  // where a unit's utility comes from
@@ -292,13 +372,14 @@ __device__ __forceinline__ float unit_utility(const UnitSrc& src, long long unit
 }
 
 // grid.x = units. scored: unit = (l*B + b)*Hkv + g; fast: unit = b.
-template <bool CACHED>
+template <bool CACHED, int CL>
 __global__ void __launch_bounds__(kThreads) ta_select_kernel(ta_seq_desc seq, int n_layers, int Hkv, int K, int fast,
                                                              UnitSrc src, const uint8_t* __restrict__ forced,
                                                              const int32_t* __restrict__ r_main,
                                                              int32_t* __restrict__ idx, int32_t* __restrict__ count) {
   __shared__ SelectShared sh;
-  const int unit = blockIdx.x;
+  const int unit = blockIdx.x / CL;
+  const bool lead = blockIdx.x % CL == 0;
   int b, l = 0, g = 0;
   if (fast) {
     b = unit;
@@ -313,32 +394,39 @@ __global__ void __launch_bounds__(kThreads) ta_select_kernel(ta_seq_desc seq, in
   const int want = r_main[b];
   const int tid = threadIdx.x;
   if (want == -2) {  // sequence rejected by ta_forced_kernel
-    for (int r = tid; r < K; r += kThreads) out[r] = -1;
-    if (tid == 0) count[unit] = 0;
+    if (lead) {
+      for (int r = tid; r < K; r += kThreads) out[r] = -1;
+      if (tid == 0) count[unit] = 0;
+    }
     return;
   }
   if (want == -1) {  // K >= n: keep everything
-    for (int r = tid; r < K; r += kThreads) out[r] = r < n ? r : -1;
-    if (tid == 0) count[unit] = n;
+    if (lead) {
+      for (int r = tid; r < K; r += kThreads) out[r] = r < n ? r : -1;
+      if (tid == 0) count[unit] = n;
+    }
     return;
   }
   const long long unit_off = fast ? 0 : ((long long)l * Hkv + g) * seq.total;
-  const uint8_t* f = forced + start;
-  auto key_of = [&](int i, uint32_t& key) {
-    key = sortable_key(unit_utility(src, unit_off, (long long)start + i));
-    return f[i] == 0;
+  int lo, hi;
+  unit_slice<CL>(n, lo, hi);
+  const uint8_t* f = forced + start + lo;
+  auto key_of = [&](int il, uint32_t& key) {
+    key = sortable_key(unit_utility(src, unit_off, (long long)start + lo + il));
+    return f[il] == 0;
   };
   KeyCache kc;
-  if (CACHED) fill_cache(n, key_of, kc);
-  const SelectResult r = block_radix_select<CACHED>(n, want, key_of, kc, sh);
+  if (CACHED) fill_cache(hi - lo, key_of, kc);
+  const SelectResult r = block_radix_select<CACHED, CL>(hi - lo, want, key_of, kc, sh);
   auto classify = [&](int, bool elig, uint32_t key, bool& def, bool& tie) {
     def = !elig || (!r.none && (r.all || key > r.thresh));
     tie = !def && !r.none && !r.all && key == r.thresh;
   };
-  auto emit = [&](int i, int rank) {
-    if (rank < K) out[rank] = i;
+  auto emit = [&](int il, int rank) {
+    if (rank < K) out[rank] = lo + il;
   };
-  const int taken = block_ordered_emit<CACHED>(n, r.ties, key_of, kc, classify, emit, sh);
+  const int taken = cluster_ordered_emit<CACHED, CL>(hi - lo, r.ties, key_of, kc, classify, emit, sh);
+  if (!lead) return;
   for (int q = taken + tid; q < K; q += kThreads) out[q] = -1;
   if (tid == 0) count[unit] = taken;
 }
@@ -362,15 +450,53 @@ __global__ void ta_broadcast_idx_kernel(int B, int Hkv, int K, int n_layers, con
 // Scratch layout used by the launcher (the caller carves it): forced [total] bytes, r_main [B] ints; fast mode
 // additionally idx_seq [B][K] and count_seq [B] (passed through a.idx / a.count by the caller when it wants the
 // per-sequence result only).
+// Sequences that fit kItems keys per thread run one CTA per unit with the keys in registers; longer ones are split
+// over a cluster of kSelectCluster CTAs (keys in registers up to kSelectCluster * kItems * kThreads elements).
+// Splitting pays only while the clusters of all units fit on the device about at once; with many units one CTA per
+// unit (keys re-read in batches when they do not fit in registers) keeps every SM busy without cluster barriers.
+bool split_units(int units, int max_n) {
+  if (max_n <= kItems * kThreads) return false;
+  static int sms = 0;
+  if (sms == 0) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1)
+      sms = 148;
+  }
+  return units * kSelectCluster <= 2 * sms;
+}
+
+template <class Kern, class... Args>
+cudaError_t launch_clustered(Kern kern, int units, int cl, cudaStream_t stream, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(units * cl), 1, 1);
+  cfg.blockDim = dim3(kThreads, 1, 1);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = (unsigned)cl;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, args...);
+}
+
 cudaError_t ta_launch_forced(const ta_select_args& a, ta_dev_status* status, cudaStream_t stream) {
   if (a.seq.batch == 0 || a.n_layers == 0) return cudaSuccess;
+  const int B = a.seq.batch;
   if (a.seq.max_n <= kItems * kThreads)
-    ta_forced_kernel<true><<<a.seq.batch, kThreads, 0, stream>>>(a.seq, a.K, a.n_sink, a.n_recent, a.k_protected,
-                                                               a.voucher, a.forced, a.r_main, status);
-  else
-    ta_forced_kernel<false><<<a.seq.batch, kThreads, 0, stream>>>(a.seq, a.K, a.n_sink, a.n_recent, a.k_protected,
-                                                                a.voucher, a.forced, a.r_main, status);
-  return cudaGetLastError();
+    return launch_clustered(ta_forced_kernel<true, 1>, B, 1, stream, a.seq, a.K, a.n_sink, a.n_recent, a.k_protected,
+                            a.voucher, a.forced, a.r_main, status);
+  if (!split_units(B, a.seq.max_n))
+    return launch_clustered(ta_forced_kernel<false, 1>, B, 1, stream, a.seq, a.K, a.n_sink, a.n_recent, a.k_protected,
+                            a.voucher, a.forced, a.r_main, status);
+  if (a.seq.max_n <= kSelectCluster * kItems * kThreads)
+    return launch_clustered(ta_forced_kernel<true, kSelectCluster>, B, kSelectCluster, stream, a.seq, a.K, a.n_sink,
+                            a.n_recent, a.k_protected, a.voucher, a.forced, a.r_main, status);
+  return launch_clustered(ta_forced_kernel<false, kSelectCluster>, B, kSelectCluster, stream, a.seq, a.K, a.n_sink,
+                          a.n_recent, a.k_protected, a.voucher, a.forced, a.r_main, status);
 }
 
 cudaError_t ta_launch_select_units(const ta_select_args& a, cudaStream_t stream) {
@@ -384,12 +510,16 @@ cudaError_t ta_launch_select_units(const ta_select_args& a, cudaStream_t stream)
   src.delta = a.delta;
   const int units = a.fast ? a.seq.batch : a.n_layers * a.seq.batch * a.Hkv;
   if (a.seq.max_n <= kItems * kThreads)
-    ta_select_kernel<true><<<units, kThreads, 0, stream>>>(a.seq, a.n_layers, a.Hkv, a.K, a.fast, src, a.forced,
-                                                         a.r_main, a.idx, a.count);
-  else
-    ta_select_kernel<false><<<units, kThreads, 0, stream>>>(a.seq, a.n_layers, a.Hkv, a.K, a.fast, src, a.forced,
-                                                          a.r_main, a.idx, a.count);
-  return cudaGetLastError();
+    return launch_clustered(ta_select_kernel<true, 1>, units, 1, stream, a.seq, a.n_layers, a.Hkv, a.K, a.fast, src,
+                            a.forced, a.r_main, a.idx, a.count);
+  if (!split_units(units, a.seq.max_n))
+    return launch_clustered(ta_select_kernel<false, 1>, units, 1, stream, a.seq, a.n_layers, a.Hkv, a.K, a.fast, src,
+                            a.forced, a.r_main, a.idx, a.count);
+  if (a.seq.max_n <= kSelectCluster * kItems * kThreads)
+    return launch_clustered(ta_select_kernel<true, kSelectCluster>, units, kSelectCluster, stream, a.seq, a.n_layers,
+                            a.Hkv, a.K, a.fast, src, a.forced, a.r_main, a.idx, a.count);
+  return launch_clustered(ta_select_kernel<false, kSelectCluster>, units, kSelectCluster, stream, a.seq, a.n_layers,
+                          a.Hkv, a.K, a.fast, src, a.forced, a.r_main, a.idx, a.count);
 }
 
 cudaError_t ta_launch_select(const ta_select_args& a, ta_dev_status* status, cudaStream_t stream) {
