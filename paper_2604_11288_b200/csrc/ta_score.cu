@@ -5,25 +5,27 @@
 // For unit (l, b, g) the score matrix is S = Q_obs[heads of g] * K^T, M = G*W rows (<= 256) by n keys. Each row is
 // softmax-normalised over the keys it may see and the result is summed over rows per key. The normaliser of a row
 // needs every key before any column sum can be finished, so the keys are swept twice:
-//   pass 1  S = Q * Ktile^T   (TMEM lane = query row)  -> running max and sum of exponentials per row
+//   pass 1  S = Q * Ktile^T   (TMEM lane = query row)  -> reference and sum of exponentials per row
 //   pass 2  S^T = Ktile * Q^T (TMEM lane = key)        -> A_i = sum_rows exp2(s*c - lse_row), P_i likewise
 // Both passes use the same shared-memory operand tiles (both K-major, 128-byte swizzle); only the roles in the
 // instruction descriptor swap, which puts the reduction axis of each pass along a thread's own registers.
-// The keys of a unit are split over the CTAs of a cluster (each CTA owns a contiguous range of 128-key tiles);
-// between the passes the CTAs exchange their per-row statistics through distributed shared memory (remote stores
-// followed by a remote mbarrier arrive). Pass 2 re-reads the CTA's own tiles, which are still in L2, so HBM sees
-// every key once. When the caller supplies the rows' log-sum-exp (lse_obs), pass 1 is skipped.
+// A unit is handled by a cluster of 1, 2, 4 or 8 CTAs (chosen per launch: one CTA when there are many units, more when
+// there are few); each CTA owns a contiguous range of 128-key tiles. Between the passes every CTA publishes its
+// per-row (reference, sum) pairs in its own shared memory, signals its peers with a remote mbarrier arrive, and reads
+// the peers' pairs with distributed-shared-memory loads. Pass 2 walks the CTA's tiles backwards so that the tiles read
+// last are re-read first from L2. When the caller supplies the rows' log-sum-exp (lse_obs), pass 1 is skipped.
 //
 // The grid is persistent: as many clusters as the device can hold at once, each walking over units
-// cluster, cluster + n_clusters, ...; the TMA and MMA warps run ahead across unit boundaries (double-buffered query
-// tile, ring of key tiles, two accumulator stages), so barrier set-up, TMEM allocation and pipeline fill are paid
-// once per CTA and not once per unit.
+// cluster, cluster + n_clusters, ...; the TMA and MMA warps run ahead across pass and unit boundaries (double-buffered
+// query tile, ring of key tiles, one accumulator stage per softmax group or two where tensor memory allows), so
+// barrier set-up, TMEM allocation and pipeline fill are paid once per CTA and not once per unit.
 //
-// Warp roles (384 threads, three warpgroups): warps 0-7 are two softmax groups that alternate over the accumulator
-// stages, warp 8 is the TMA producer, warp 9 the MMA issuer and TMEM owner, warps 10-11 idle. After set-up the third
-// warpgroup gives registers back (setmaxnreg) and the softmax warpgroups take them. Every wait on an mbarrier is bounded by wall time; when one runs out
-// the CTA records TA_ERR_TIMEOUT, stops waiting anywhere, drains its copies, frees its tensor memory and returns.
-// The only unbounded waits are two hardware cluster barriers (start, end) that every thread reaches on every path.
+// Warp roles: NG softmax warpgroups (3 for M = 128, 2 for M = 256) that take the jobs round-robin, plus one warpgroup
+// with the TMA producer warp, the MMA issuer warp (TMEM owner) and two idle warps. After set-up that last warpgroup
+// gives registers back (setmaxnreg) and the softmax warpgroups take them. Every wait on an mbarrier is bounded by
+// wall time; when one runs out the CTA records TA_ERR_TIMEOUT, stops waiting anywhere, drains its copies, frees its
+// tensor memory and returns. The only unbounded waits are two hardware cluster barriers (start, end) that every
+// thread reaches on every path.
 #include <cuda.h>
 
 #include <type_traits>

@@ -360,3 +360,28 @@ def test_compress_host_matches_device_path(fast, pinned):
         assert torch.equal(vo_h.view(torch.int16), vo.cpu().view(torch.int16))
     finally:
         g.close()
+
+
+def test_fused_path_is_deterministic():
+    """Three runs on the same inputs give bit-identical indices and caches (no atomics on the data path decide
+    anything: histograms are integer, ties break by position)."""
+    w = _workload([2500, 700, 4100], [[4, 5], [6]], seed=31, Hq=8, Hkv=2, W=32)
+    K, L = 40, 2
+    pol = oracle_policy(K, "THEOREM", W=32)
+    Qh, Kh, Vh = tw.make_qkv(w, range(L))
+    g = Gpu(w, pol, K, L)
+    try:
+        Qd, Kd, Vd = Qh.cuda(), Kh.cuda(), Vh.cuda()
+        ref = None
+        for _ in range(3):
+            out = g.compress(Qd, Kd, Vd)
+            torch.cuda.synchronize()
+            if ref is None:
+                ref = out
+            else:
+                for a, b in zip(ref, out):
+                    assert torch.equal(a.view(torch.int16) if a.dtype == torch.bfloat16 else a,
+                                       b.view(torch.int16) if b.dtype == torch.bfloat16 else b)
+        assert g.poll() == ta.TA_OK
+    finally:
+        g.close()
