@@ -385,3 +385,43 @@ def test_fused_path_is_deterministic():
         assert g.poll() == ta.TA_OK
     finally:
         g.close()
+
+
+def test_score_general_window_sizes():
+    # windows that do not divide 32 use per-element pension weights: 96 rows (one row block) and 192 rows (two)
+    *_, g = _score_case([777, 130], 4, 1, 24, seed=7)
+    g.close()
+    *_, g = _score_case([1500], 4, 1, 48, seed=8)
+    g.close()
+
+
+def test_score_without_pension_output():
+    w, pol, Qh, Kh, Qd, Kd, A_ref, g = _score_case([900, 260], 8, 2, 32, seed=9)
+    try:
+        A, P = g.score(Qd, Kd, want_P=False)
+        torch.cuda.synchronize()
+        assert P is None and g.poll() == ta.TA_OK
+        np.testing.assert_allclose(A.cpu().numpy(), A_ref, rtol=1e-5, atol=1e-7)
+    finally:
+        g.close()
+
+
+def test_compress_with_zero_pension_weight():
+    # delta = 0: the fused kernel skips the pension sums altogether
+    w = _workload([1200, 300], [[4, 5]], seed=14, Hq=8, Hkv=2, W=32)
+    K = 20
+    pol = oracle_policy(K, "SEC33", W=32, delta=0.0)
+    Qh, Kh, Vh = tw.make_qkv(w, [0])
+    g = Gpu(w, pol, K, 1)
+    try:
+        idx, cnt, ko, vo = g.compress(Qh.cuda(), Kh.cuda(), Vh.cuda())
+        torch.cuda.synchronize()
+        assert g.poll() == ta.TA_OK
+        idx, cnt = idx.cpu().numpy(), cnt.cpu().numpy()
+        f_o, V_o, u0_o = oracle.sponsor_mask(w.ids, w.cu, oracle_patterns(w), pol)
+        for b in range(w.B):
+            for h in range(w.Hkv):
+                A, P, u, io, co = oracle_unit(w, pol, K, Qh, Kh, 0, b, h, V_o, u0_o)
+                assert_selection_matches(idx[0, b, h], cnt[0, b, h], io, co, u, f"b{b} h{h}")
+    finally:
+        g.close()
