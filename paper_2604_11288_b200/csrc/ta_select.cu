@@ -19,7 +19,7 @@ namespace cg = cooperative_groups;
 
 namespace {
 
-constexpr int kThreads = 1024;
+constexpr int kThreads = 512;
 constexpr int kWarps = kThreads / 32;
 
 __device__ __forceinline__ uint32_t sortable_key(float f) {
@@ -50,7 +50,7 @@ constexpr int kSelectCluster = 8;  // CTAs per unit when a sequence is longer th
 
 // Keys of a unit are read once into registers when the unit is short enough (kItems per thread), else they are
 // re-read from L2 on every sweep in batches whose loads are all issued before the first use.
-constexpr int kItems = 8;
+constexpr int kItems = 16;
 constexpr int kBatch = 8;
 struct KeyCache {
   uint32_t key[kItems];
@@ -479,7 +479,7 @@ cudaError_t launch_clustered(Kern kern, int units, int cl, cudaStream_t stream, 
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = cl > 1 ? 1 : 0;  // a plain launch when no cluster is needed
   return cudaLaunchKernelEx(&cfg, kern, args...);
 }
 
