@@ -93,6 +93,35 @@ void ora_anchors(int n, const int32_t* ids, int n_pat, const int32_t* pat_ids, c
 }
 
 // ---------------------------------------------------------------------------------------------------------
+// Anchor detection by a learned detector (Section 5.1 "Learned Anchor Detection"), for ONE sequence. The detector
+// itself (an MLP on hidden states) is outside this path: its per-token confidence f(h_i) in [0, 1] is an input.
+// Token i is an anchor iff f(h_i) > threshold (strictly, as the paper writes it); anchors are single tokens, so
+// S_i = 1 exactly on them. Two variants, both feeding the voucher sum of Eq. 2 unchanged:
+//   TA-Learned   (rank = 0): threshold 0.5, every anchor sponsors with the fixed budget B.
+//   TA-LearnRank (rank = 1): threshold 0.3, the confidence takes the place of the budget: B_i = budget * f(h_i)
+//                (budget = 1 gives the paper's equation V_j = sum_i f(h_i) 0.8^(j-i) 1[f(h_i) > 0.3, i < j <= i+L]).
+// The budget is aged like a pattern's (age_steps products with budget_decay, fp32). A NaN confidence is no anchor.
+// Pinned by: closed forms f*0.8^k; threshold edge (equal is not above); rank = 0 on the indicator of a token id
+// equals the pattern detector with that one-token pattern.
+void ora_anchors_conf(int n, const float* conf, float threshold, float budget, int span, int rank,
+                      float budget_decay, int age_steps, uint8_t* anchor_tok, uint8_t* anchor_end, float* B_e,
+                      int32_t* L_e) {
+  for (int i = 0; i < n; ++i) {
+    const bool is_anchor = conf[i] > threshold;
+    anchor_tok[i] = is_anchor ? 1 : 0;
+    anchor_end[i] = is_anchor ? 1 : 0;
+    B_e[i] = 0.0f;
+    L_e[i] = 0;
+    if (is_anchor) {
+      float B = rank ? budget * conf[i] : budget;
+      for (int t = 0; t < age_steps; ++t) B = B * budget_decay;
+      B_e[i] = B;
+      L_e[i] = span;
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------------------
 // Voucher allocation (Eq. 2; Algorithm 1 steps 2-6) for one sequence:
 //   V_j = sum over anchors i with i < j <= i + L_i of B_i * decay^(j-i).
 // decay^k is built by repeated fp32 multiplication (w[1] = decay, w[k] = w[k-1]*decay); the sum over anchors is

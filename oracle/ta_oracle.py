@@ -113,6 +113,21 @@ def anchors(ids: np.ndarray, pats: Patterns, budget_decay=0.9, age_steps=0):
     return atok, aend, Be, Le
 
 
+def anchors_conf(conf: np.ndarray, threshold, budget, span, rank, budget_decay=0.9, age_steps=0):
+    """Anchors from a detector's per-token confidence (Section 5.1): same outputs as anchors()."""
+    lib = _load()
+    conf = np.ascontiguousarray(conf, np.float32)
+    n = conf.shape[0]
+    atok = np.zeros(n, np.uint8)
+    aend = np.zeros(n, np.uint8)
+    Be = np.zeros(n, np.float32)
+    Le = np.zeros(n, np.int32)
+    lib.ora_anchors_conf(C.c_int(n), _p(conf, C.c_float), C.c_float(threshold), C.c_float(budget), C.c_int(span),
+                         C.c_int(1 if rank else 0), C.c_float(budget_decay), C.c_int(age_steps), _p(atok, C.c_uint8),
+                         _p(aend, C.c_uint8), _p(Be, C.c_float), _p(Le, C.c_int32))
+    return atok, aend, Be, Le
+
+
 def vouchers(aend, Be, Le, voucher_decay=0.8):
     lib = _load()
     n = aend.shape[0]
@@ -147,6 +162,22 @@ def sponsor_mask(ids, cu, pats: Patterns, pol: Policy):
     for b in range(len(cu) - 1):
         o, e = int(cu[b]), int(cu[b + 1])
         atok, aend, Be, Le = anchors(ids[o:e], pats, pol.budget_decay, pol.age_steps)
+        v = vouchers(aend, Be, Le, pol.voucher_decay)
+        V[o:e] = v
+        u0[o:e] = static_utility(ids[o:e], atok, v, pol.beta, pol.gamma, pol.lam, vocab=pol.vocab_size)
+        flags[o:e] = atok | (aend << 1) | ((v > 0).astype(np.uint8) << 2)
+    return flags, V, u0
+
+
+def sponsor_mask_conf(ids, cu, conf, threshold, budget, span, rank, pol: Policy):
+    """sponsor_mask() with the anchors taken from a detector's confidences instead of token-id patterns."""
+    total = int(cu[-1])
+    flags = np.zeros(total, np.uint8)
+    V = np.zeros(total, np.float32)
+    u0 = np.zeros(total, np.float32)
+    for b in range(len(cu) - 1):
+        o, e = int(cu[b]), int(cu[b + 1])
+        atok, aend, Be, Le = anchors_conf(conf[o:e], threshold, budget, span, rank, pol.budget_decay, pol.age_steps)
         v = vouchers(aend, Be, Le, pol.voucher_decay)
         V[o:e] = v
         u0[o:e] = static_utility(ids[o:e], atok, v, pol.beta, pol.gamma, pol.lam, vocab=pol.vocab_size)

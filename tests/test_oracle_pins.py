@@ -393,3 +393,46 @@ def test_compress_layer_matches_step_by_step():
             assert cnt[b, g] == c2
             np.testing.assert_array_equal(ko[b, g], oracle.compact(Kb[g, o:e], i2, c2, 12))
             np.testing.assert_array_equal(vo[b, g], oracle.compact(Vb[g, o:e], i2, c2, 12))
+
+
+# ------------------------------------------------------------------------- learned-detector anchors (Section 5.1)
+def test_conf_anchors_rank_mode_closed_form():
+    # TA-LearnRank: V_j = sum_i f_i 0.8^(j-i) 1[f_i > 0.3, i < j <= i+L]; two anchors, one below the threshold
+    conf = np.array([0.0, 0.9, 0.2, 0.0, 0.6, 0.3, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0], np.float32)
+    L = 6
+    atok, aend, Be, Le = oracle.anchors_conf(conf, 0.3, 1.0, L, True)
+    assert aend.tolist() == [0, 1, 0, 0, 1, 0, 0, 0, 0, 0, 0, 0]  # 0.2 and exactly 0.3 are not above 0.3
+    assert (atok == aend).all()
+    V = oracle.vouchers(aend, Be, Le)
+    f1, f4 = float(np.float32(0.9)), float(np.float32(0.6))
+    for j in range(12):
+        want = 0.0
+        if 1 < j <= 1 + L:
+            want += f1 * 0.8 ** (j - 1)
+        if 4 < j <= 4 + L:
+            want += f4 * 0.8 ** (j - 4)
+        assert V[j] == pytest.approx(want, rel=1e-6, abs=1e-12)
+    # "higher-confidence anchors receive more protection": right after each anchor the ratio is the confidence ratio
+    assert V[2] / 0.8 == pytest.approx(f1, rel=1e-6)
+
+
+def test_conf_anchors_fixed_budget_equals_one_token_pattern():
+    # TA-Learned with the indicator of a token id as "confidence" is the pattern detector with that one-token pattern
+    rng = np.random.default_rng(5)
+    ids = rng.integers(0, 4, 200).astype(np.int32)
+    conf = (ids == 2).astype(np.float32)
+    for age in (0, 3):
+        a1 = oracle.anchors_conf(conf, 0.5, 15.0, 6, False, age_steps=age)
+        a2 = oracle.anchors(ids, oracle.Patterns([[2]]), age_steps=age)
+        for x, y in zip(a1, a2):
+            np.testing.assert_array_equal(x, y)
+    # rank mode with confidence 1 everywhere an anchor is: budget * 1 = budget
+    a3 = oracle.anchors_conf(conf, 0.3, 15.0, 6, True)
+    np.testing.assert_array_equal(a3[2], oracle.anchors(ids, oracle.Patterns([[2]]))[2])
+
+
+def test_conf_anchors_nan_and_budget_age():
+    conf = np.array([np.nan, 0.8, 1.0], np.float32)
+    atok, aend, Be, Le = oracle.anchors_conf(conf, 0.5, 2.0, 4, True, budget_decay=0.9, age_steps=2)
+    assert aend.tolist() == [0, 1, 1] and Le.tolist() == [0, 4, 4]
+    assert Be[1] == pytest.approx(2.0 * 0.8 * 0.81, rel=1e-6) and Be[2] == pytest.approx(2.0 * 0.81, rel=1e-6)
