@@ -182,6 +182,23 @@ void ta_patterns_destroy(ta_patterns* pats);
 ta_status ta_sponsor_mask(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* policy, const ta_batch* batch,
                           const int32_t* token_ids, uint8_t* flags, float* voucher, float* u_static, void* stream);
 
+/* ---- step 1 with a learned anchor detector (Section 5.1, "Learned Anchor Detection") ----------------------
+ * The detector itself (an MLP on hidden states, or an embedding similarity) runs in the caller's model; its
+ * per-token confidence f(h_i) is the input here. Token i is an anchor iff conf[i] > threshold (NaN: no anchor).
+ * Anchors are single tokens: TA_FLAG_ANCHOR_TOKEN and TA_FLAG_ANCHOR_END are set together, all anchors share the
+ * span L = span, and vouchers, flags and u_static follow exactly as in ta_sponsor_mask (Eq. 2, Eq. 3) with the
+ * per-anchor budget
+ *   rank_by_confidence == 0 : B_i = budget                  TA-Learned   (paper: threshold 0.5, B = 15)
+ *   rank_by_confidence != 0 : B_i = budget * conf[i]        TA-LearnRank (paper: threshold 0.3, budget = 1, i.e.
+ *                             V_j = sum_i f(h_i) 0.8^(j-i) 1[f(h_i) > 0.3, i < j <= i+L])
+ * decayed age_steps times like a pattern's budget; every product rounded to fp32.
+ *   conf  DEVICE float [total_tokens]
+ * span in [1, TA_MAX_SPAN]. Other arguments, outputs and scratch use as ta_sponsor_mask. The outputs feed
+ * ta_select_topk / ta_compact_kv unchanged. */
+ta_status ta_sponsor_mask_conf(ta_ctx* ctx, const ta_policy* policy, const ta_batch* batch, const int32_t* token_ids,
+                               const float* conf, float threshold, float budget, int span, int rank_by_confidence,
+                               uint8_t* flags, float* voucher, float* u_static, void* stream);
+
 /* ---- step 2: attention mass over the observation window ---------------------------------------------------
  * Eq. 1's A_i and P_i, read as a one-shot compaction after prefill: for unit (l, b, g) the score rows are the
  * last W' = min(W, n) query positions of the G = Hq/Hkv query heads of KV group g;

@@ -70,6 +70,7 @@ def lib():
             "ta_patterns_create": (i32, [vp, i32, vp, vp, vp, vp, C.POINTER(vp)]),
             "ta_patterns_destroy": (None, [vp]),
             "ta_sponsor_mask": (i32, [vp, vp, PP, PB, vp, vp, vp, vp, vp]),
+            "ta_sponsor_mask_conf": (i32, [vp, PP, PB, vp, vp, C.c_float, C.c_float, i32, i32, vp, vp, vp, vp]),
             "ta_score": (i32, [vp, PP, PB, i32, i32, i32, ta_bf16_view, ta_bf16_view, vp, vp, vp, vp]),
             "ta_select_topk": (i32, [vp, PP, PB, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]),
             "ta_select_topk_static": (i32, [PP, PB, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]),
@@ -181,6 +182,13 @@ def ta_patterns_create(ctx, pattern_ids, budget=None, span=None):
 
 def ta_patterns_destroy(pats):
     lib().ta_patterns_destroy(pats)
+
+
+def ta_sponsor_mask_conf(ctx, policy, batch, token_ids, conf, threshold, budget, span, rank_by_confidence, flags,
+                         voucher, u_static, stream=None):
+    _check(lib().ta_sponsor_mask_conf(ctx, C.byref(policy), C.byref(batch), _ptr(token_ids), _ptr(conf),
+                                      C.c_float(threshold), C.c_float(budget), int(span), int(rank_by_confidence),
+                                      _ptr(flags), _ptr(voucher), _ptr(u_static), stream), "ta_sponsor_mask_conf")
 
 
 def ta_sponsor_mask(ctx, pats, policy, batch, token_ids, flags, voucher, u_static, stream=None):

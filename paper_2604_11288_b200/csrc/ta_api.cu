@@ -374,6 +374,25 @@ ta_status ta_sponsor_mask(ta_ctx* ctx, const ta_patterns* pats, const ta_policy*
   return e == cudaSuccess ? TA_OK : cuda_fail(ctx, e);
 }
 
+ta_status ta_sponsor_mask_conf(ta_ctx* ctx, const ta_policy* policy, const ta_batch* batch, const int32_t* token_ids,
+                               const float* conf, float threshold, float budget, int span, int rank_by_confidence,
+                               uint8_t* flags, float* voucher, float* u_static, void* stream) {
+  if (!ctx || !token_ids || !conf || !flags || !voucher || !u_static) return TA_ERR_INVALID_ARG;
+  ta_status s = check_batch(batch);
+  if (s == TA_OK) s = check_policy(policy);
+  if (s != TA_OK) return s;
+  if (!(threshold == threshold) || !(budget == budget) || span < 1) return TA_ERR_INVALID_ARG;
+  if (span > TA_MAX_SPAN) return TA_ERR_UNSUPPORTED;
+  const size_t need = align_up((size_t)batch->batch * policy->vocab_size * 4);
+  if (need > ctx->scratch_bytes) return TA_ERR_SCRATCH_TOO_SMALL;
+  DeviceGuard guard(ctx->device);
+  ctx->cached_epoch = 0;
+  cudaError_t e = ta_launch_mask_conf(*policy, seq_desc(*batch), token_ids, conf, threshold, budget, span,
+                                      rank_by_confidence ? 1 : 0, flags, voucher, u_static,
+                                      reinterpret_cast<int32_t*>(ctx->scratch), ctx->d_status, (cudaStream_t)stream);
+  return e == cudaSuccess ? TA_OK : cuda_fail(ctx, e);
+}
+
 // ---------------------------------------------------------------------------------------------- step 2
 ta_status ta_score(ta_ctx* ctx, const ta_policy* policy, const ta_batch* batch, int Hq, int Hkv, int d,
                    ta_bf16_view q_obs, ta_bf16_view k, const float* lse_obs, float* A, float* P, void* stream) {

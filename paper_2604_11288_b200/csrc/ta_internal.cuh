@@ -72,6 +72,11 @@ cudaError_t ta_launch_mask(const ta_patterns* pats, const ta_policy& pol, const 
                            uint8_t* flags, float* voucher, float* u_static, int32_t* hist /*[B][vocab]*/,
                            ta_dev_status* status, cudaStream_t stream);
 
+// the same with anchors from a detector's per-token confidences (single-token anchors, one span for all)
+cudaError_t ta_launch_mask_conf(const ta_policy& pol, const ta_seq_desc& seq, const int32_t* ids, const float* conf,
+                                float threshold, float budget, int span, int rank, uint8_t* flags, float* voucher,
+                                float* u_static, int32_t* hist, ta_dev_status* status, cudaStream_t stream);
+
 // ---- step 2 ------------------------------------------------------------------------------------------------
 struct ta_score_args {
   ta_seq_desc seq;

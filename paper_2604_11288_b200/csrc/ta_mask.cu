@@ -11,6 +11,8 @@
 //            token whether any earlier anchor of its own sequence reaches it; only those tokens add up their
 //            vouchers, nearest anchor first, in fp32 with one rounding per operation (bit-exact by construction)
 // Kernel ta_ustatic_kernel then combines recency, anchor flag, frequency and voucher into u_static.
+// With a detector's per-token confidences instead of a pattern set (Section 5.1) phase b is a threshold test: the
+// anchors are single tokens, all with the same span, and their budget is fixed or proportional to the confidence.
 #include "ta_internal.cuh"
 
 namespace {
@@ -42,6 +44,14 @@ __device__ __forceinline__ void report(ta_dev_status* st, int code, int where, i
   }
 }
 
+struct ConfAnchors {   // anchors from a detector's confidences; conf == nullptr: token-id patterns are matched
+  const float* conf;   // [total]
+  float threshold;     // anchor iff conf > threshold
+  float budget;        // sponsor budget B (rank: B_i = budget * conf_i)
+  int span;            // L
+  int rank;
+};
+
 struct SegMax {  // element of the segmented max-scan: flag = a segment starts at or before this element
   int flag;
   int val;
@@ -62,7 +72,8 @@ __global__ void __launch_bounds__(kTile) ta_mask_kernel(ta_seq_desc seq, const i
                                                         int max_len, int max_span, float voucher_decay,
                                                         float budget_decay, int age_steps, int vocab,
                                                         uint8_t* __restrict__ flags, float* __restrict__ voucher,
-                                                        int32_t* __restrict__ hist, ta_dev_status* status) {
+                                                        int32_t* __restrict__ hist, ta_dev_status* status,
+                                                        ConfAnchors ca) {
   __shared__ int32_t s_id[kExt];
   __shared__ int32_t s_start[kExt];     // packed index of the first token of the position's sequence
   __shared__ int16_t s_apat[kExt];      // winning pattern ending here, -1 none
@@ -79,13 +90,21 @@ __global__ void __launch_bounds__(kTile) ta_mask_kernel(ta_seq_desc seq, const i
   const long long T0 = (long long)blockIdx.x * kTile;  // first packed token of the tile
   const long long ext0 = T0 - kHaloL;                  // packed token of s_id[0]
 
-  for (int i = tid; i < n_pat * TA_MAX_PATTERN_LEN; i += kTile) s_pid[i] = p_ids[i];
-  for (int i = tid; i < n_pat; i += kTile) {
-    s_plen[i] = p_len[i];
-    s_pspan[i] = p_span[i];
-    s_pbud[i] = p_budget[i];
+  if (ca.conf) {  // one pseudo-pattern of length 1 stands for "the detector fired here"
+    if (tid == 0) {
+      s_plen[0] = 1;
+      s_pspan[0] = ca.span;
+      s_pbud[0] = ca.budget;
+    }
+  } else {
+    for (int i = tid; i < n_pat * TA_MAX_PATTERN_LEN; i += kTile) s_pid[i] = p_ids[i];
+    for (int i = tid; i < n_pat; i += kTile) {
+      s_plen[i] = p_len[i];
+      s_pspan[i] = p_span[i];
+      s_pbud[i] = p_budget[i];
+    }
+    if (tid < 32) s_bloom[tid] = n_pat ? p_bloom[tid] : 0u;
   }
-  if (tid < 32) s_bloom[tid] = n_pat ? p_bloom[tid] : 0u;
   if (tid == 0) {
     float w = voucher_decay;
     s_w[0] = 1.0f;
@@ -119,7 +138,14 @@ __global__ void __launch_bounds__(kTile) ta_mask_kernel(ta_seq_desc seq, const i
   for (int i = tid; i < kExt; i += kTile) {
     int best = -1, best_len = 0;
     const int32_t x = s_id[i];
-    if (x >= 0 && i >= TA_MAX_PATTERN_LEN) {
+    float cf = 0.0f;
+    if (ca.conf) {
+      const long long tok = ext0 + i;
+      if (tok >= 0 && tok < seq.total) {
+        cf = ca.conf[tok];
+        if (cf > ca.threshold) best = 0;  // false for NaN
+      }
+    } else if (x >= 0 && i >= TA_MAX_PATTERN_LEN) {
       const uint32_t h = bloom_hash(x);
       if (s_bloom[h >> 5] & (1u << (h & 31))) {
         const long long tok = ext0 + i;
@@ -142,6 +168,7 @@ __global__ void __launch_bounds__(kTile) ta_mask_kernel(ta_seq_desc seq, const i
     float B = 0.0f;
     if (best >= 0) {
       B = s_pbud[best];
+      if (ca.conf && ca.rank) B = __fmul_rn(B, cf);
       for (int t = 0; t < age_steps; ++t) B = __fmul_rn(B, budget_decay);
     }
     s_abud[i] = B;
@@ -288,6 +315,32 @@ __global__ void __launch_bounds__(256) ta_ustatic_kernel(ta_seq_desc seq, const 
 
 }  // namespace
 
+namespace {
+cudaError_t finish_static_utility(const ta_policy& pol, const ta_seq_desc& seq, const int32_t* ids, const uint8_t* flags,
+                                  const float* voucher, const int32_t* hist, float* u_static, cudaStream_t stream) {
+  const int blocks = (int)((seq.total + 255) / 256);
+  ta_ustatic_kernel<<<blocks, 256, 0, stream>>>(seq, ids, flags, voucher, hist, pol.vocab_size, pol.beta, pol.gamma,
+                                                pol.lambda, u_static);
+  return cudaGetLastError();
+}
+}  // namespace
+
+cudaError_t ta_launch_mask_conf(const ta_policy& pol, const ta_seq_desc& seq, const int32_t* ids, const float* conf,
+                                float threshold, float budget, int span, int rank, uint8_t* flags, float* voucher,
+                                float* u_static, int32_t* hist, ta_dev_status* status, cudaStream_t stream) {
+  if (seq.total == 0) return cudaSuccess;
+  cudaError_t e = cudaMemsetAsync(hist, 0, (size_t)seq.batch * pol.vocab_size * sizeof(int32_t), stream);
+  if (e != cudaSuccess) return e;
+  const int tiles = (int)((seq.total + kTile - 1) / kTile);
+  ConfAnchors ca = {conf, threshold, budget, span, rank};
+  ta_mask_kernel<<<tiles, kTile, 0, stream>>>(seq, ids, nullptr, nullptr, nullptr, nullptr, nullptr, 1, 1, span,
+                                              pol.voucher_decay, pol.budget_decay, pol.age_steps, pol.vocab_size, flags,
+                                              voucher, hist, status, ca);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  return finish_static_utility(pol, seq, ids, flags, voucher, hist, u_static, stream);
+}
+
 cudaError_t ta_launch_mask(const ta_patterns* pats, const ta_policy& pol, const ta_seq_desc& seq, const int32_t* ids,
                            uint8_t* flags, float* voucher, float* u_static, int32_t* hist, ta_dev_status* status,
                            cudaStream_t stream) {
@@ -298,11 +351,8 @@ cudaError_t ta_launch_mask(const ta_patterns* pats, const ta_policy& pol, const 
   ta_mask_kernel<<<tiles, kTile, 0, stream>>>(seq, ids, pats->d_ids, pats->d_len, pats->d_budget, pats->d_span,
                                               pats->d_bloom, pats->n_pat, pats->max_len, pats->max_span,
                                               pol.voucher_decay, pol.budget_decay, pol.age_steps, pol.vocab_size, flags,
-                                              voucher, hist, status);
+                                              voucher, hist, status, ConfAnchors{nullptr, 0.0f, 0.0f, 0, 0});
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  const int blocks = (int)((seq.total + 255) / 256);
-  ta_ustatic_kernel<<<blocks, 256, 0, stream>>>(seq, ids, flags, voucher, hist, pol.vocab_size, pol.beta, pol.gamma,
-                                                pol.lambda, u_static);
-  return cudaGetLastError();
+  return finish_static_utility(pol, seq, ids, flags, voucher, hist, u_static, stream);
 }

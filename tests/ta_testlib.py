@@ -60,6 +60,15 @@ class Gpu:
         ta.ta_sponsor_mask(self.ctx, self.pats, self.p, self.batch, self.ids, flags, V, u0, self.stream)
         return flags, V, u0
 
+    def sponsor_mask_conf(self, conf, threshold, budget, span, rank):
+        t = self.w.total
+        flags = torch.empty(t, dtype=torch.uint8, device=self.dev)
+        V = torch.empty(t, dtype=torch.float32, device=self.dev)
+        u0 = torch.empty(t, dtype=torch.float32, device=self.dev)
+        ta.ta_sponsor_mask_conf(self.ctx, self.p, self.batch, self.ids, conf, threshold, budget, span, rank, flags, V,
+                                u0, self.stream)
+        return flags, V, u0
+
     def score(self, Q, K, lse=None, want_P=True):
         w = self.w
         A = torch.full((self.L, w.Hkv, w.total), float("nan"), dtype=torch.float32, device=self.dev)

@@ -88,6 +88,48 @@ def test_mask_no_patterns_and_bad_token_id():
         g.close()
 
 
+@pytest.mark.parametrize("rank,threshold,budget,span", [(False, 0.5, 15.0, 6), (True, 0.3, 1.0, 6), (True, 0.3, 15.0, 64)])
+def test_mask_from_detector_confidences_bit_exact(rank, threshold, budget, span):
+    # Section 5.1: anchors from a learned detector's confidences (TA-Learned, TA-LearnRank), ragged batch with
+    # sequences shorter than a span, spans that run into each other and across tile borders, NaN and exact-threshold
+    # confidences; aged budgets
+    lengths = [700, 3, 1, 0, 1500, 513, 64]
+    w = _workload(lengths, [[1, 2]], seed=21)
+    rng = np.random.default_rng(77)
+    conf = rng.random(w.total).astype(np.float32)
+    conf[rng.random(w.total) < 0.9] *= 0.25          # most tokens well below either threshold
+    conf[rng.integers(0, w.total, 20)] = threshold   # equal is not above
+    conf[rng.integers(0, w.total, 5)] = np.nan
+    conf[508:516] = 0.97                             # a run of anchors across the first tile border
+    pol = oracle_policy(8, age_steps=2)
+    g = Gpu(w, pol, 8, 1)
+    try:
+        flags, V, u0 = g.sponsor_mask_conf(torch.from_numpy(conf).cuda(), threshold, budget, span, rank)
+        torch.cuda.synchronize()
+        assert g.poll() == ta.TA_OK
+        f_o, V_o, u0_o = oracle.sponsor_mask_conf(w.ids, w.cu, conf, threshold, budget, span, rank, pol)
+        np.testing.assert_array_equal(flags.cpu().numpy(), f_o)
+        np.testing.assert_array_equal(V.cpu().numpy().view(np.uint32), V_o.view(np.uint32))
+        np.testing.assert_array_equal(u0.cpu().numpy().view(np.uint32), u0_o.view(np.uint32))
+        assert (f_o & ta.TA_FLAG_SPONSORED).any() and (f_o & ta.TA_FLAG_ANCHOR_END).sum() > 50
+        # the outputs feed the unchanged selection step: fast-mode selection equals the oracle's
+        polf = oracle_policy(8, fast=True, age_steps=2)
+        g2 = Gpu(w, polf, 8, 1)
+        try:
+            idx, cnt = g2.select(flags, V, u0)
+            torch.cuda.synchronize()
+            idx, cnt = idx.cpu().numpy(), cnt.cpu().numpy()
+            for b in range(w.B):
+                o, e = int(w.cu[b]), int(w.cu[b + 1])
+                io, co = oracle.select(V_o[o:e], u0_o[o:e], 8, polf.n_sink, polf.n_recent, polf.k_protected)
+                assert cnt[0, b, 0] == co
+                np.testing.assert_array_equal(idx[0, b, 0], io)
+        finally:
+            g2.close()
+    finally:
+        g.close()
+
+
 def _score_case(lengths, Hq, Hkv, W, causal=1, seed=0, layers=1, permute=False, scale=0.0):
     w = _workload(lengths, [[1, 2]], seed=seed, Hq=Hq, Hkv=Hkv, W=W)
     w.n_layers = layers
