@@ -272,6 +272,21 @@ ta_status ta_compress(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* pol
                       ta_bf16_view v, uint64_t seq_epoch, void* k_out, void* v_out, int32_t* idx, int32_t* count,
                       void* stream);
 
+/* ---- composition with another eviction score (Section 4.5 "Composability") ---------------------------------
+ * TA changes the scoring function, not the eviction policy: sponsorship is added on top of whatever importance
+ * score a pipeline already has (accumulated attention of H2O, the pooled prefill-window attention of SnapKV, a
+ * per-layer or per-head budgeted score, ...). This entry point is ta_compress with the attention terms of Eq. 1
+ * supplied by the caller instead of computed from Q and K:
+ *   u = (alpha*score + delta*score2) + u_static,  then selection (Section 3.3) and the gather, as in ta_compress.
+ *   score   DEVICE float [L][Hkv][total_tokens]   the caller's per-token importance (takes the place of A_i)
+ *   score2  DEVICE float, same shape, or NULL     a second term weighted by delta (takes the place of P_i)
+ * policy->mode must be TA_MODE_SCORED; obs_window and the softmax fields are ignored. Values must be finite.
+ * Everything else (patterns, seq_epoch reuse of the per-sequence step, outputs, scratch) as ta_compress. */
+ta_status ta_compress_scores(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* policy, const ta_batch* batch,
+                             int Hkv, int d, int K, const int32_t* token_ids, const float* score,
+                             const float* score2, ta_bf16_view k, ta_bf16_view v, uint64_t seq_epoch, void* k_out,
+                             void* v_out, int32_t* idx, int32_t* count, void* stream);
+
 /* ---- host-buffer variant of ta_compress --------------------------------------------------------------------
  * Same computation with every data pointer on the HOST (pinned memory makes the copies asynchronous):
  * token_ids, cu_seqlens (inside batch: HOST here), the q_obs / k / v views, and the four outputs. The caller lends

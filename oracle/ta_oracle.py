@@ -207,9 +207,10 @@ def utility(alpha, delta, A, P, u0):
     n = u0.shape[0]
     u = np.zeros(n, np.float32)
     A = np.ascontiguousarray(A, np.float32)
-    P = np.ascontiguousarray(P, np.float32)
+    P = None if P is None else np.ascontiguousarray(P, np.float32)
     u0 = np.ascontiguousarray(u0, np.float32)
-    lib.ora_utility(C.c_int(n), C.c_float(alpha), C.c_float(delta), _p(A, C.c_float), _p(P, C.c_float),
+    lib.ora_utility(C.c_int(n), C.c_float(alpha), C.c_float(delta), _p(A, C.c_float),
+                    C.POINTER(C.c_float)() if P is None else _p(P, C.c_float),
                     _p(u0, C.c_float), _p(u, C.c_float))
     return u
 

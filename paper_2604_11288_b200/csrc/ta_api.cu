@@ -504,22 +504,26 @@ ta_status ta_compact_kv(ta_ctx* ctx, const ta_batch* batch, int Hkv, int d, int 
 }
 
 // ---------------------------------------------------------------------------------------------- fused
-ta_status ta_compress(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* policy, const ta_batch* batch, int Hq,
-                      int Hkv, int d, int K, const int32_t* token_ids, ta_bf16_view q_obs, ta_bf16_view k,
-                      ta_bf16_view v, uint64_t seq_epoch, void* k_out, void* v_out, int32_t* idx, int32_t* count,
-                      void* stream_v) {
+namespace {
+// ext_A != nullptr: the attention terms come from the caller (ext_A, ext_P per layer, KV head and token) and the
+// score kernel is not run; q_obs is then unused.
+ta_status compress_impl(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* policy, const ta_batch* batch, int Hq,
+                        int Hkv, int d, int K, const int32_t* token_ids, ta_bf16_view q_obs, ta_bf16_view k,
+                        ta_bf16_view v, uint64_t seq_epoch, void* k_out, void* v_out, int32_t* idx, int32_t* count,
+                        void* stream_v, const float* ext_A, const float* ext_P) {
   if (!ctx || !pats || !token_ids || !k_out || !v_out || !idx || !count) return TA_ERR_INVALID_ARG;
   ta_status s = check_batch(batch);
   if (s == TA_OK) s = check_policy(policy);
   if (s != TA_OK) return s;
   const bool fast = policy->mode == TA_MODE_FAST;
+  const bool external = ext_A != nullptr;
+  if (external && fast) return TA_ERR_INVALID_ARG;
   const bool uniform = batch->cu_seqlens == nullptr;
-  s = check_heads(Hq, Hkv, d, policy, !fast);
-  if (s == TA_OK && !fast) s = check_view(q_obs, true);
+  s = check_heads(Hq, Hkv, d, policy, !fast && !external);
+  if (s == TA_OK && !fast && !external) s = check_view(q_obs, true);
   if (s == TA_OK) s = check_view(v, uniform);
-  if (s == TA_OK && !fast) s = check_view(k, uniform);
-  if (s == TA_OK && fast && k.ptr == nullptr) s = TA_ERR_INVALID_ARG;  // K rows are gathered in both modes
-  if (s == TA_OK && fast) s = check_view(k, uniform);
+  if (s == TA_OK && k.ptr == nullptr) s = TA_ERR_INVALID_ARG;  // K rows are gathered in every mode
+  if (s == TA_OK) s = check_view(k, uniform);
   if (s != TA_OK) return s;
   if (K < 1) return TA_ERR_INVALID_ARG;
   if (K > TA_MAX_BUDGET) return TA_ERR_UNSUPPORTED;
@@ -563,7 +567,9 @@ ta_status ta_compress(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* pol
   sel.flags = flags;
   sel.voucher = voucher;
   sel.u_static = u_static;
-  sel.u = u;
+  sel.u = external ? nullptr : u;
+  sel.A = ext_A;
+  sel.P = ext_P;
   sel.forced = forced;
   sel.r_main = r_main;
   sel.idx = fast ? idx_seq : idx;
@@ -574,7 +580,7 @@ ta_status ta_compress(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* pol
   mark(0);
   ctx->ev_ran[0] = 0;
   cudaStream_t seq_stream = stream;
-  const bool fork = !reuse && !fast;
+  const bool fork = !reuse && !fast && !external;
   if (fork) {
     seq_stream = ctx->side;
     e = cudaEventRecord(ctx->ev_fork, stream);
@@ -592,7 +598,7 @@ ta_status ta_compress(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* pol
   }
   if (fork && e == cudaSuccess) e = cudaEventRecord(ctx->ev_join, ctx->side);
   mark(1);
-  if (e == cudaSuccess && !fast) {
+  if (e == cudaSuccess && !fast && !external) {
     ta_score_args a = {};
     a.seq = seq;
     a.n_layers = batch->n_layers;
@@ -645,6 +651,26 @@ ta_status ta_compress(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* pol
   ctx->cached_batch = batch->batch;
   ctx->cached_K = K;
   return TA_OK;
+}
+}  // namespace
+
+ta_status ta_compress(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* policy, const ta_batch* batch, int Hq,
+                      int Hkv, int d, int K, const int32_t* token_ids, ta_bf16_view q_obs, ta_bf16_view k,
+                      ta_bf16_view v, uint64_t seq_epoch, void* k_out, void* v_out, int32_t* idx, int32_t* count,
+                      void* stream) {
+  return compress_impl(ctx, pats, policy, batch, Hq, Hkv, d, K, token_ids, q_obs, k, v, seq_epoch, k_out, v_out, idx,
+                       count, stream, nullptr, nullptr);
+}
+
+ta_status ta_compress_scores(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* policy, const ta_batch* batch,
+                             int Hkv, int d, int K, const int32_t* token_ids, const float* score,
+                             const float* score2, ta_bf16_view k, ta_bf16_view v, uint64_t seq_epoch, void* k_out,
+                             void* v_out, int32_t* idx, int32_t* count, void* stream) {
+  if (!score || !policy) return TA_ERR_INVALID_ARG;
+  if (policy->mode != TA_MODE_SCORED) return TA_ERR_INVALID_ARG;
+  ta_bf16_view none = {};
+  return compress_impl(ctx, pats, policy, batch, Hkv, Hkv, d, K, token_ids, none, k, v, seq_epoch, k_out, v_out, idx,
+                       count, stream, score, score2);
 }
 
 // ---------------------------------------------------------------------------------------------- host buffers

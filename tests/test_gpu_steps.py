@@ -342,6 +342,48 @@ def test_compress_equals_steps_and_oracle(fast):
         g.close()
 
 
+@pytest.mark.parametrize("with_second", [False, True])
+def test_compress_with_external_scores_bit_exact(with_second):
+    # Section 4.5: sponsorship on top of another method's importance score. Here the provider is a SnapKV-style
+    # max-pooled attention mass (computed on the host) and, optionally, a second arbitrary term weighted by delta.
+    w = _workload([1200, 300, 40, 2600], [[4, 5], [9]], seed=31, Hq=8, Hkv=2, W=32)
+    K, L = 24, 2
+    pol = oracle_policy(K, "SEC33", W=32)
+    Qh, Kh, Vh = tw.make_qkv(w, range(L))
+    rng = np.random.default_rng(3)
+    G = w.Hq // w.Hkv
+    score = np.zeros((L, w.Hkv, w.total), np.float32)
+    for l in range(L):
+        for b in range(w.B):
+            o, e = int(w.cu[b]), int(w.cu[b + 1])
+            for h in range(w.Hkv):
+                A, _ = oracle.attention(bf16_bits(Qh[l, b, h * G:(h + 1) * G]), unit_kv(w, Kh, l, b, h), e - o)
+                pad = np.pad(A, 3, constant_values=-np.inf)
+                score[l, h, o:e] = np.max(np.stack([pad[k:k + e - o] for k in range(7)]), axis=0)
+    score2 = rng.standard_normal(score.shape).astype(np.float32) if with_second else None
+    g = Gpu(w, pol, K, L)
+    try:
+        s2 = None if score2 is None else torch.from_numpy(score2).cuda()
+        idx, cnt, ko, vo = g.compress_scores(torch.from_numpy(score).cuda(), s2, Kh.cuda(), Vh.cuda())
+        torch.cuda.synchronize()
+        assert g.poll() == ta.TA_OK
+        idx, cnt = idx.cpu().numpy(), cnt.cpu().numpy()
+        f_o, V_o, u0_o = oracle.sponsor_mask(w.ids, w.cu, oracle_patterns(w), pol)
+        for l in range(L):
+            for b in range(w.B):
+                o, e = int(w.cu[b]), int(w.cu[b + 1])
+                for h in range(w.Hkv):
+                    u = oracle.utility(pol.alpha, pol.delta, score[l, h, o:e],
+                                       None if score2 is None else score2[l, h, o:e], u0_o[o:e])
+                    io, co = oracle.select(V_o[o:e], u, K, pol.n_sink, pol.n_recent, pol.k_protected)
+                    assert cnt[l, b, h] == co
+                    np.testing.assert_array_equal(idx[l, b, h], io, err_msg=f"l{l} b{b} h{h}")
+                    np.testing.assert_array_equal(bf16_bits(ko[l, b, h]), oracle.compact(unit_kv(w, Kh, l, b, h), io, co, K))
+                    np.testing.assert_array_equal(bf16_bits(vo[l, b, h]), oracle.compact(unit_kv(w, Vh, l, b, h), io, co, K))
+    finally:
+        g.close()
+
+
 def test_host_argument_checks():
     w = _workload([300], [[1, 2]], seed=1)
     pol = oracle_policy(8, fast=True)
