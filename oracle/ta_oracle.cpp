@@ -246,6 +246,54 @@ void ora_attention(int n, int G, int W, int d, const uint16_t* Q, int64_t q_stri
 }
 
 // ---------------------------------------------------------------------------------------------------------
+// The same sums taken over ALL query heads of a layer (the literal "cumulative attention across heads" of Eq. 1 and
+// Appendix A Definition 1): query head h attends to the keys of its KV head h / G. One A and one P per token, shared
+// by every KV head of the layer.
+//   Q: [Hq][W][d] as above; K: Hkv blocks of n rows, block g at K + g*k_stride_h.
+// Pinned by: sum_i A_i = Hq*W'; equals the sum over KV heads of ora_attention (a different summation order in
+// double, so equal to rounding); with Hkv = 1 it is ora_attention.
+void ora_attention_allheads(int n, int Hq, int Hkv, int W, int d, const uint16_t* Q, int64_t q_stride_h,
+                            int64_t q_stride_t, const uint16_t* K, int64_t k_stride_h, int64_t k_stride_n,
+                            double scale, int causal, double rho, float* A_out, float* P_out) {
+  if (scale <= 0.0) scale = 1.0 / std::sqrt((double)d);
+  const int G = Hq / Hkv;
+  const int Wp = W < n ? W : n;
+  std::vector<double> A(n, 0.0), P(n, 0.0), s(n), q(d);
+  for (int h = 0; h < Hq; ++h) {
+    const uint16_t* Kg = K + (int64_t)(h / G) * k_stride_h;
+    for (int tp = 0; tp < Wp; ++tp) {
+      const int t = W - Wp + tp;
+      const int pos = n - Wp + tp;
+      const int last = causal ? pos : n - 1;
+      for (int c = 0; c < d; ++c) q[c] = bf16_to_double(Q[h * q_stride_h + t * q_stride_t + c]);
+      double mx = -INFINITY;
+      for (int i = 0; i <= last; ++i) {
+        const uint16_t* kr = Kg + (int64_t)i * k_stride_n;
+        double acc = 0.0;
+        for (int c = 0; c < d; ++c) acc += q[c] * bf16_to_double(kr[c]);
+        s[i] = scale * acc;
+        if (s[i] > mx) mx = s[i];
+      }
+      double Z = 0.0;
+      for (int i = 0; i <= last; ++i) {
+        s[i] = std::exp(s[i] - mx);
+        Z += s[i];
+      }
+      const double wt = (1.0 - rho) * std::pow(rho, (double)(Wp - 1 - tp));
+      for (int i = 0; i <= last; ++i) {
+        const double a = s[i] / Z;
+        A[i] += a;
+        P[i] += wt * a;
+      }
+    }
+  }
+  for (int i = 0; i < n; ++i) {
+    A_out[i] = (float)A[i];
+    if (P_out) P_out[i] = (float)P[i];
+  }
+}
+
+// ---------------------------------------------------------------------------------------------------------
 // Full utility of Eq. 1 from its parts: u = (alpha*A + delta*P) + u0, fp32, one rounding per operation.
 void ora_utility(int n, float alpha, float delta, const float* A, const float* P, const float* u0, float* u) {
   for (int i = 0; i < n; ++i) {

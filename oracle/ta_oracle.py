@@ -202,6 +202,25 @@ def attention(Q: np.ndarray, K: np.ndarray, n: int, scale=0.0, causal=1, rho=0.9
     return A, P
 
 
+def attention_allheads(Q: np.ndarray, K: np.ndarray, n: int, scale=0.0, causal=1, rho=0.9):
+    """Q: uint16 [Hq, W, d]; K: uint16 [Hkv, n, d] (contiguous). A, P float32 [n] summed over all query heads."""
+    lib = _load()
+    assert Q.dtype == np.uint16 and K.dtype == np.uint16
+    Q = np.ascontiguousarray(Q)
+    K = np.ascontiguousarray(K)
+    Hq, W, d = Q.shape
+    Hkv = K.shape[0]
+    if n == 0:
+        return np.zeros(0, np.float32), np.zeros(0, np.float32)
+    A = np.zeros(n, np.float32)
+    P = np.zeros(n, np.float32)
+    lib.ora_attention_allheads(C.c_int(n), C.c_int(Hq), C.c_int(Hkv), C.c_int(W), C.c_int(d), _p(Q, C.c_uint16),
+                               C.c_int64(W * d), C.c_int64(d), _p(K, C.c_uint16), C.c_int64(K.shape[1] * d),
+                               C.c_int64(d), C.c_double(scale), C.c_int(causal), C.c_double(rho), _p(A, C.c_float),
+                               _p(P, C.c_float))
+    return A, P
+
+
 def utility(alpha, delta, A, P, u0):
     lib = _load()
     n = u0.shape[0]

@@ -436,3 +436,28 @@ def test_conf_anchors_nan_and_budget_age():
     atok, aend, Be, Le = oracle.anchors_conf(conf, 0.5, 2.0, 4, True, budget_decay=0.9, age_steps=2)
     assert aend.tolist() == [0, 1, 1] and Le.tolist() == [0, 4, 4]
     assert Be[1] == pytest.approx(2.0 * 0.8 * 0.81, rel=1e-6) and Be[2] == pytest.approx(2.0 * 0.81, rel=1e-6)
+
+
+# ------------------------------------------------------------------------------- attention summed over all heads
+def test_attention_allheads_is_sum_over_kv_heads_and_normalised():
+    g = torch.Generator().manual_seed(11)
+    Hq, Hkv, W, d, n = 8, 2, 5, 16, 37
+    Q = bf16_bits(torch.randn(Hq, W, d, generator=g))
+    K = bf16_bits(torch.randn(Hkv, n, d, generator=g))
+    A, P = oracle.attention_allheads(Q, K, n, rho=0.7)
+    G = Hq // Hkv
+    As = np.zeros(n)
+    Ps = np.zeros(n)
+    for h in range(Hkv):
+        a, p = oracle.attention(Q[h * G:(h + 1) * G], K[h], n, rho=0.7)
+        As += a
+        Ps += p
+    np.testing.assert_allclose(A, As, rtol=1e-6, atol=1e-9)
+    np.testing.assert_allclose(P, Ps, rtol=1e-6, atol=1e-9)
+    assert A.sum() == pytest.approx(Hq * W, rel=1e-6)          # every softmax row sums to one
+    assert P.sum() == pytest.approx(Hq * (1 - 0.7 ** W), rel=1e-6)
+    # one KV head: the per-group routine
+    A1, P1 = oracle.attention_allheads(Q[:G], K[:1], n, rho=0.7)
+    a, p = oracle.attention(Q[:G], K[0], n, rho=0.7)
+    np.testing.assert_array_equal(A1, a)
+    np.testing.assert_array_equal(P1, p)
