@@ -272,6 +272,19 @@ ta_status ta_compress(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* pol
                       ta_bf16_view v, uint64_t seq_epoch, void* k_out, void* v_out, int32_t* idx, int32_t* count,
                       void* stream);
 
+/* ---- one selection per layer, shared by its KV heads (Eq. 1: A_i "across heads") -----------------------------
+ * Eq. 1 and Appendix A Definition 1 define A_i as attention accumulated over ALL heads, which gives one retained
+ * set per layer. ta_compress reads them per KV head (every head keeps its own K tokens); this entry point takes
+ * the literal reading: A_i and P_i are summed over the Hq query heads of the layer (each attending to the keys of
+ * its own KV head), u = (alpha*A + delta*P) + u_static is formed once per (layer, sequence), one selection is
+ * made from it, and every KV head of the layer gathers the same positions: idx[l][b][g][:] is the same for all g.
+ * The head sum is taken in fp32 over the per-head fused terms, KV head 0 first.
+ * Arguments, outputs and scratch as ta_compress; policy->mode must be TA_MODE_SCORED. */
+ta_status ta_compress_allheads(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* policy, const ta_batch* batch,
+                               int Hq, int Hkv, int d, int K, const int32_t* token_ids, ta_bf16_view q_obs,
+                               ta_bf16_view k, ta_bf16_view v, uint64_t seq_epoch, void* k_out, void* v_out,
+                               int32_t* idx, int32_t* count, void* stream);
+
 /* ---- composition with another eviction score (Section 4.5 "Composability") ---------------------------------
  * TA changes the scoring function, not the eviction policy: sponsorship is added on top of whatever importance
  * score a pipeline already has (accumulated attention of H2O, the pooled prefill-window attention of SnapKV, a

@@ -77,6 +77,8 @@ def lib():
             "ta_compact_kv": (i32, [vp, PB, i32, i32, i32, ta_bf16_view, ta_bf16_view, vp, vp, vp, vp, vp]),
             "ta_compress": (i32, [vp, vp, PP, PB, i32, i32, i32, i32, vp, ta_bf16_view, ta_bf16_view, ta_bf16_view,
                                   u64, vp, vp, vp, vp, vp]),
+            "ta_compress_allheads": (i32, [vp, vp, PP, PB, i32, i32, i32, i32, vp, ta_bf16_view, ta_bf16_view,
+                                           ta_bf16_view, u64, vp, vp, vp, vp, vp]),
             "ta_compress_scores": (i32, [vp, vp, PP, PB, i32, i32, i32, vp, vp, vp, ta_bf16_view, ta_bf16_view, u64, vp,
                                          vp, vp, vp, vp]),
             "ta_compress_host_workspace_bytes": (i32, [PB, i32, i32, i32, i32, PP, C.POINTER(sz)]),
@@ -225,6 +227,13 @@ def ta_compress(ctx, pats, policy, batch, Hq, Hkv, d, K, token_ids, q_obs: ta_bf
                 v: ta_bf16_view, seq_epoch, k_out, v_out, idx, count, stream=None):
     _check(lib().ta_compress(ctx, pats, C.byref(policy), C.byref(batch), Hq, Hkv, d, K, _ptr(token_ids), q_obs, k, v,
                              int(seq_epoch), _ptr(k_out), _ptr(v_out), _ptr(idx), _ptr(count), stream), "ta_compress")
+
+
+def ta_compress_allheads(ctx, pats, policy, batch, Hq, Hkv, d, K, token_ids, q_obs: ta_bf16_view, k: ta_bf16_view,
+                         v: ta_bf16_view, seq_epoch, k_out, v_out, idx, count, stream=None):
+    _check(lib().ta_compress_allheads(ctx, pats, C.byref(policy), C.byref(batch), Hq, Hkv, d, K, _ptr(token_ids), q_obs,
+                                      k, v, int(seq_epoch), _ptr(k_out), _ptr(v_out), _ptr(idx), _ptr(count), stream),
+           "ta_compress_allheads")
 
 
 def ta_compress_scores(ctx, pats, policy, batch, Hkv, d, K, token_ids, score, score2, k: ta_bf16_view,

@@ -26,7 +26,7 @@ struct Carve {  // hands out aligned pieces of the context scratch
 };
 
 struct Layout {  // scratch layout of ta_compress (a superset of what the single-step entry points need)
-  size_t hist, flags, voucher, u_static, forced, r_main, idx_seq, count_seq, u, end;
+  size_t hist, flags, voucher, u_static, forced, r_main, idx_seq, count_seq, u, u_all, idx_lb, count_lb, end;
 };
 
 Layout make_layout(const ta_batch& b, int Hkv, int K, const ta_policy& pol) {
@@ -47,6 +47,11 @@ Layout make_layout(const ta_batch& b, int Hkv, int K, const ta_policy& pol) {
   L.idx_seq = take(B * (size_t)K * 4);
   L.count_seq = take(B * 4);
   L.u = take(pol.mode == TA_MODE_FAST ? 0 : (size_t)b.n_layers * Hkv * total * 4);
+  // selection shared by the heads of a layer (ta_compress_allheads): head sums and the per-(layer, sequence) result
+  const bool scored = pol.mode != TA_MODE_FAST;
+  L.u_all = take(scored ? (size_t)b.n_layers * total * 4 : 0);
+  L.idx_lb = take(scored ? (size_t)b.n_layers * B * K * 4 : 0);
+  L.count_lb = take(scored ? (size_t)b.n_layers * B * 4 : 0);
   L.end = off;
   return L;
 }
@@ -510,14 +515,15 @@ namespace {
 ta_status compress_impl(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* policy, const ta_batch* batch, int Hq,
                         int Hkv, int d, int K, const int32_t* token_ids, ta_bf16_view q_obs, ta_bf16_view k,
                         ta_bf16_view v, uint64_t seq_epoch, void* k_out, void* v_out, int32_t* idx, int32_t* count,
-                        void* stream_v, const float* ext_A, const float* ext_P) {
+                        void* stream_v, const float* ext_A, const float* ext_P, bool share_heads) {
   if (!ctx || !pats || !token_ids || !k_out || !v_out || !idx || !count) return TA_ERR_INVALID_ARG;
   ta_status s = check_batch(batch);
   if (s == TA_OK) s = check_policy(policy);
   if (s != TA_OK) return s;
   const bool fast = policy->mode == TA_MODE_FAST;
   const bool external = ext_A != nullptr;
-  if (external && fast) return TA_ERR_INVALID_ARG;
+  if ((external || share_heads) && fast) return TA_ERR_INVALID_ARG;
+  if (external && share_heads) return TA_ERR_INVALID_ARG;
   const bool uniform = batch->cu_seqlens == nullptr;
   s = check_heads(Hq, Hkv, d, policy, !fast && !external);
   if (s == TA_OK && !fast && !external) s = check_view(q_obs, true);
@@ -544,6 +550,9 @@ ta_status compress_impl(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* p
   int32_t* idx_seq = reinterpret_cast<int32_t*>(sc + L.idx_seq);
   int32_t* count_seq = reinterpret_cast<int32_t*>(sc + L.count_seq);
   float* u = reinterpret_cast<float*>(sc + L.u);
+  float* u_all = reinterpret_cast<float*>(sc + L.u_all);
+  int32_t* idx_lb = reinterpret_cast<int32_t*>(sc + L.idx_lb);
+  int32_t* count_lb = reinterpret_cast<int32_t*>(sc + L.count_lb);
   const ta_seq_desc seq = seq_desc(*batch);
   const bool timing = ctx->timing_enabled != 0;
   cudaError_t e = cudaSuccess;
@@ -574,6 +583,12 @@ ta_status compress_impl(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* p
   sel.r_main = r_main;
   sel.idx = fast ? idx_seq : idx;
   sel.count = fast ? count_seq : count;
+  if (share_heads) {  // one selection per (layer, sequence) on the head sums
+    sel.Hkv = 1;
+    sel.u = u_all;
+    sel.idx = idx_lb;
+    sel.count = count_lb;
+  }
 
   // Per-sequence work (anchor mask, vouchers, static utility, forced set) does not depend on Q/K: in scored mode it
   // runs on the context's side stream beside the score kernel and joins before the per-unit selection.
@@ -622,7 +637,10 @@ ta_status compress_impl(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* p
   }
   mark(2);
   if (fork && e == cudaSuccess) e = cudaStreamWaitEvent(stream, ctx->ev_join, 0);
+  if (e == cudaSuccess && share_heads) e = ta_launch_headsum(batch->n_layers, Hkv, batch->total_tokens, u, u_all, stream);
   if (e == cudaSuccess && !(fast && reuse)) e = ta_launch_select_units(sel, stream);
+  if (e == cudaSuccess && share_heads)
+    e = ta_launch_broadcast_heads(batch->n_layers, batch->batch, Hkv, K, idx_lb, count_lb, idx, count, stream);
   if (e == cudaSuccess && fast)
     e = ta_launch_broadcast_idx(batch->batch, Hkv, K, batch->n_layers, idx_seq, count_seq, idx, count, stream);
   mark(3);
@@ -659,7 +677,16 @@ ta_status ta_compress(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* pol
                       ta_bf16_view v, uint64_t seq_epoch, void* k_out, void* v_out, int32_t* idx, int32_t* count,
                       void* stream) {
   return compress_impl(ctx, pats, policy, batch, Hq, Hkv, d, K, token_ids, q_obs, k, v, seq_epoch, k_out, v_out, idx,
-                       count, stream, nullptr, nullptr);
+                       count, stream, nullptr, nullptr, false);
+}
+
+ta_status ta_compress_allheads(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* policy, const ta_batch* batch,
+                               int Hq, int Hkv, int d, int K, const int32_t* token_ids, ta_bf16_view q_obs,
+                               ta_bf16_view k, ta_bf16_view v, uint64_t seq_epoch, void* k_out, void* v_out,
+                               int32_t* idx, int32_t* count, void* stream) {
+  if (!policy || policy->mode != TA_MODE_SCORED) return TA_ERR_INVALID_ARG;
+  return compress_impl(ctx, pats, policy, batch, Hq, Hkv, d, K, token_ids, q_obs, k, v, seq_epoch, k_out, v_out, idx,
+                       count, stream, nullptr, nullptr, true);
 }
 
 ta_status ta_compress_scores(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* policy, const ta_batch* batch,
@@ -670,7 +697,7 @@ ta_status ta_compress_scores(ta_ctx* ctx, const ta_patterns* pats, const ta_poli
   if (policy->mode != TA_MODE_SCORED) return TA_ERR_INVALID_ARG;
   ta_bf16_view none = {};
   return compress_impl(ctx, pats, policy, batch, Hkv, Hkv, d, K, token_ids, none, k, v, seq_epoch, k_out, v_out, idx,
-                       count, stream, score, score2);
+                       count, stream, score, score2, false);
 }
 
 // ---------------------------------------------------------------------------------------------- host buffers

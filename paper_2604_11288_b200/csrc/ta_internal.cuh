@@ -117,6 +117,12 @@ cudaError_t ta_launch_select_units(const ta_select_args& a, cudaStream_t stream)
 cudaError_t ta_launch_broadcast_idx(int B, int Hkv, int K, int n_layers, const int32_t* idx_seq,
                                     const int32_t* count_seq, int32_t* idx, int32_t* count, cudaStream_t stream);
 
+// selection shared by the KV heads of a layer: head sum of the utilities, copy of the result to every head
+cudaError_t ta_launch_headsum(int n_layers, int Hkv, long long total, const float* u, float* u_all,
+                              cudaStream_t stream);
+cudaError_t ta_launch_broadcast_heads(int n_layers, int B, int Hkv, int K, const int32_t* idx_lb,
+                                      const int32_t* count_lb, int32_t* idx, int32_t* count, cudaStream_t stream);
+
 // ---- step 4 ------------------------------------------------------------------------------------------------
 struct ta_compact_args {
   ta_seq_desc seq;

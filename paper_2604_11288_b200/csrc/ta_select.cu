@@ -11,6 +11,9 @@
 //                      main pool by utility among the tokens not forced, then the ordered write of
 //                      forced + chosen positions.
 //   ta_broadcast_idx_kernel  fast mode: the per-sequence result is the same for all layers and heads.
+//   ta_headsum_kernel, ta_broadcast_heads_kernel  selection shared by the KV heads of a layer: the utilities'
+//                      attention parts are summed over the heads, one selection runs per (layer, sequence), and its
+//                      result is copied to every head.
 #include <cooperative_groups.h>
 
 #include "ta_internal.cuh"
@@ -445,6 +448,33 @@ __global__ void ta_broadcast_idx_kernel(int B, int Hkv, int K, int n_layers, con
   }
 }
 
+// u_all[l][tok] = sum over KV heads g (ascending, fp32) of u[l][g][tok]
+__global__ void ta_headsum_kernel(int n_layers, int Hkv, long long total, const float* __restrict__ u,
+                                  float* __restrict__ u_all) {
+  const long long n = (long long)n_layers * total;
+  for (long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x; t < n; t += (long long)gridDim.x * blockDim.x) {
+    const long long l = t / total, tok = t - l * total;
+    const float* src = u + l * Hkv * total + tok;
+    float acc = src[0];
+    for (int g = 1; g < Hkv; ++g) acc = __fadd_rn(acc, src[(long long)g * total]);
+    u_all[t] = acc;
+  }
+}
+
+// idx[l][b][g][:] = idx_lb[l][b][:], count[l][b][g] = count_lb[l][b]
+__global__ void ta_broadcast_heads_kernel(long long units_lb, int Hkv, int K, const int32_t* __restrict__ idx_lb,
+                                          const int32_t* __restrict__ count_lb, int32_t* __restrict__ idx,
+                                          int32_t* __restrict__ count) {
+  const long long total = units_lb * Hkv * K;
+  for (long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x; t < total;
+       t += (long long)gridDim.x * blockDim.x) {
+    const int r = (int)(t % K);
+    const long long unit = t / K, lb = unit / Hkv;
+    idx[t] = idx_lb[lb * K + r];
+    if (r == 0) count[unit] = count_lb[lb];
+  }
+}
+
 }  // namespace
 
 // Scratch layout used by the launcher (the caller carves it): forced [total] bytes, r_main [B] ints; fast mode
@@ -534,6 +564,24 @@ cudaError_t ta_launch_broadcast_idx(int B, int Hkv, int K, int n_layers, const i
   if (total == 0) return cudaSuccess;
   const int blocks = (int)((total + 255) / 256 < 4096 ? (total + 255) / 256 : 4096);
   ta_broadcast_idx_kernel<<<blocks, 256, 0, stream>>>(B, Hkv, K, n_layers, idx_seq, count_seq, idx, count);
+  return cudaGetLastError();
+}
+
+cudaError_t ta_launch_headsum(int n_layers, int Hkv, long long total, const float* u, float* u_all,
+                              cudaStream_t stream) {
+  const long long n = (long long)n_layers * total;
+  if (n == 0) return cudaSuccess;
+  const int blocks = (int)((n + 255) / 256 < 8192 ? (n + 255) / 256 : 8192);
+  ta_headsum_kernel<<<blocks, 256, 0, stream>>>(n_layers, Hkv, total, u, u_all);
+  return cudaGetLastError();
+}
+
+cudaError_t ta_launch_broadcast_heads(int n_layers, int B, int Hkv, int K, const int32_t* idx_lb,
+                                      const int32_t* count_lb, int32_t* idx, int32_t* count, cudaStream_t stream) {
+  const long long total = (long long)n_layers * B * Hkv * K;
+  if (total == 0) return cudaSuccess;
+  const int blocks = (int)((total + 255) / 256 < 4096 ? (total + 255) / 256 : 4096);
+  ta_broadcast_heads_kernel<<<blocks, 256, 0, stream>>>((long long)n_layers * B, Hkv, K, idx_lb, count_lb, idx, count);
   return cudaGetLastError();
 }
 

@@ -93,6 +93,17 @@ class Gpu:
                          self.stream)
         return ko, vo
 
+    def compress_allheads(self, Q, Kc, Vc, epoch=0):
+        w = self.w
+        idx = torch.full((self.L, w.B, w.Hkv, self.K), -7, dtype=torch.int32, device=self.dev)
+        cnt = torch.full((self.L, w.B, w.Hkv), -7, dtype=torch.int32, device=self.dev)
+        ko = torch.full((self.L, w.B, w.Hkv, self.K, w.d), 1.0, dtype=torch.bfloat16, device=self.dev)
+        vo = torch.full_like(ko, 1.0)
+        rag = not w.uniform
+        ta.ta_compress_allheads(self.ctx, self.pats, self.p, self.batch, w.Hq, w.Hkv, w.d, self.K, self.ids, ta.view(Q),
+                                ta.view(Kc, rag), ta.view(Vc, rag), epoch, ko, vo, idx, cnt, self.stream)
+        return idx, cnt, ko, vo
+
     def compress_scores(self, score, score2, Kc, Vc, epoch=0):
         w = self.w
         idx = torch.full((self.L, w.B, w.Hkv, self.K), -7, dtype=torch.int32, device=self.dev)

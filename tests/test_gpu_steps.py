@@ -384,6 +384,41 @@ def test_compress_with_external_scores_bit_exact(with_second):
         g.close()
 
 
+@pytest.mark.parametrize("preset", ["THEOREM", "SEC33"])
+def test_compress_allheads_shared_selection(preset):
+    # Eq. 1's A_i summed over all query heads of the layer: one retained set per (layer, sequence), the same for every
+    # KV head; ragged batch, two layers, a sequence shorter than the window and one shorter than the budget
+    w = _workload([1500, 20, 700, 9], [[4, 5], [9]], seed=41, Hq=8, Hkv=4, W=16)
+    K, L = 12, 2
+    pol = oracle_policy(K, preset, W=16)
+    Qh, Kh, Vh = tw.make_qkv(w, range(L))
+    g = Gpu(w, pol, K, L)
+    try:
+        idx, cnt, ko, vo = g.compress_allheads(Qh.cuda(), Kh.cuda(), Vh.cuda())
+        torch.cuda.synchronize()
+        assert g.poll() == ta.TA_OK
+        idx, cnt = idx.cpu().numpy(), cnt.cpu().numpy()
+        f_o, V_o, u0_o = oracle.sponsor_mask(w.ids, w.cu, oracle_patterns(w), pol)
+        exact = 0
+        for l in range(L):
+            for b in range(w.B):
+                o, e = int(w.cu[b]), int(w.cu[b + 1])
+                Kb = np.stack([unit_kv(w, Kh, l, b, h) for h in range(w.Hkv)])
+                A, P = oracle.attention_allheads(bf16_bits(Qh[l, b]), Kb, e - o, rho=pol.pension_rho)
+                u = oracle.utility(pol.alpha, pol.delta, A, P, u0_o[o:e])
+                io, co = oracle.select(V_o[o:e], u, K, pol.n_sink, pol.n_recent, pol.k_protected)
+                exact += bool(assert_selection_matches(idx[l, b, 0], cnt[l, b, 0], io, co, u, f"l{l} b{b}"))
+                for h in range(w.Hkv):
+                    np.testing.assert_array_equal(idx[l, b, h], idx[l, b, 0])
+                    assert cnt[l, b, h] == cnt[l, b, 0]
+                    c = int(cnt[l, b, h])
+                    np.testing.assert_array_equal(bf16_bits(ko[l, b, h]), oracle.compact(unit_kv(w, Kh, l, b, h), idx[l, b, h], c, K))
+                    np.testing.assert_array_equal(bf16_bits(vo[l, b, h]), oracle.compact(unit_kv(w, Vh, l, b, h), idx[l, b, h], c, K))
+        assert exact >= L * w.B - 1
+    finally:
+        g.close()
+
+
 def test_host_argument_checks():
     w = _workload([300], [[1, 2]], seed=1)
     pol = oracle_policy(8, fast=True)
