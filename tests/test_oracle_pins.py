@@ -461,3 +461,89 @@ def test_attention_allheads_is_sum_over_kv_heads_and_normalised():
     a, p = oracle.attention(Q[:G], K[0], n, rho=0.7)
     np.testing.assert_array_equal(A1, a)
     np.testing.assert_array_equal(P1, p)
+
+
+# ------------------------------------------------------------------ Algorithm 1 in the decode loop (streaming oracle)
+from oracle.ta_stream_oracle import StreamOracle  # noqa: E402
+
+
+def _uniform_attn(units, t):
+    return [{p: 1.0 / (len(un.pos) + 1) for p in un.pos + [t]} for un in units]
+
+
+def test_stream_vouchers_closed_form():
+    # anchor (id 2) at position 3; B = 15, L = 6: the token arriving k steps later gets 15*(0.9*0.8)^k, and every
+    # later step multiplies it by 0.9 (Algorithm 1 step 10)
+    so = StreamOracle(oracle.Patterns([[2]]), oracle.Policy(), K=64, n_units=1)
+    ids = [7, 7, 7, 2] + [5] * 10
+    for t, x in enumerate(ids):
+        so.step(x, _uniform_attn(so.units, t))
+    n = len(ids)
+    V = so.units[0].V
+    for j in range(n):
+        k = j - 3
+        want = 15.0 * (0.72 ** k) * 0.9 ** (n - j) if 1 <= k <= 6 else 0.0
+        assert float(V[j]) == pytest.approx(want, rel=2e-6, abs=1e-12), j
+    assert so.units[0].S == [0, 0, 0, 1] + [0] * 10
+
+
+def test_stream_without_decay_matches_one_shot_oracle():
+    # budget_decay = 1 and K >= n: after the last token the streamed vouchers, anchor flags and attention-free utility
+    # are the one-shot oracle's, bit for bit (multi-token patterns, overlapping spans, a prefix-only decoy)
+    rng = np.random.default_rng(9)
+    ids = rng.integers(0, 5, 120).astype(np.int32)
+    pats = oracle.Patterns([[1, 2], [3], [4, 1, 2]], budget=[15.0, 4.0, 9.0], span=[6, 3, 8])
+    pol = oracle.Policy(budget_decay=1.0, vocab_size=8)
+    so = StreamOracle(pats, pol, K=1000, n_units=1)
+    for t, x in enumerate(ids):
+        assert so.step(int(x), _uniform_attn(so.units, t)) == [-1]
+    cu = np.array([0, len(ids)], np.int32)
+    flags, V, u0 = oracle.sponsor_mask(ids, cu, pats, pol)
+    np.testing.assert_array_equal(np.array(so.units[0].V, np.float32).view(np.uint32), V.view(np.uint32))
+    np.testing.assert_array_equal(np.array(so.units[0].S, np.uint8), flags & 1)
+    np.testing.assert_array_equal(so.static_utility(0).view(np.uint32), u0.view(np.uint32))
+
+
+def test_stream_attention_only_evicts_least_accumulated():
+    # no patterns, alpha = 1 and every other weight 0, no mandatory or protected slots: each step drops the cached
+    # token with the least accumulated attention (H2O-style), latest position among equals
+    rng = np.random.default_rng(4)
+    pol = oracle.Policy(alpha=1.0, beta=0.0, gamma=0.0, delta=0.0, lam=0.0, n_sink=0, n_recent=0, k_protected=0)
+    K = 6
+    so = StreamOracle(oracle.Patterns([]), pol, K=K, n_units=2)
+    acc = [dict(), dict()]
+    for t in range(40):
+        attn = []
+        for u in range(2):
+            ps = so.units[u].pos + [t]
+            a = rng.random(len(ps)).astype(np.float32)
+            a[rng.integers(0, len(ps))] = a[0]  # some exact ties
+            attn.append({p: float(x) for p, x in zip(ps, a)})
+        ev = so.step(int(rng.integers(0, 50)), attn)
+        for u in range(2):
+            for p, x in attn[u].items():
+                acc[u][p] = np.float32(acc[u].get(p, np.float32(0)) + np.float32(x))
+            if len(acc[u]) > K:
+                lo = min(acc[u].values())
+                want = max(p for p, x in acc[u].items() if x == lo)
+                assert ev[u] == want
+                del acc[u][want]
+            else:
+                assert ev[u] == -1
+            assert sorted(acc[u]) == so.units[u].pos
+
+
+def test_stream_sponsored_span_survives_adversarial_attention():
+    # Theorem 2 in the streaming setting: budget 1 + W + L with W = 4 recents; the six tokens after the anchor are
+    # never evicted while their (decaying) vouchers exceed the largest competing utility, whatever the attention says
+    pol = oracle.Policy()  # 1 sink, 4 recent, protected = the rest
+    L, K = 6, 1 + 4 + 6
+    so = StreamOracle(oracle.Patterns([[2]]), pol, K=K, n_units=1)
+    ids = [9] * 20 + [2] + [30 + i for i in range(6)] + [9] * 6
+    for t, x in enumerate(ids):
+        un = so.units[0]
+        attn = {p: (0.0 if 21 <= p <= 26 else 1.0) for p in un.pos + [t]}  # the value tokens get no attention at all
+        so.step(x, [attn])
+        if t >= 26:
+            assert set(range(21, 27)) <= set(so.units[0].pos), t
+    assert len(so.units[0].pos) == K
