@@ -300,6 +300,51 @@ ta_status ta_compress_scores(ta_ctx* ctx, const ta_patterns* pats, const ta_poli
                              const float* score2, ta_bf16_view k, ta_bf16_view v, uint64_t seq_epoch, void* k_out,
                              void* v_out, int32_t* idx, int32_t* count, void* stream);
 
+/* ---- Algorithm 1 in the decode loop: per-step retention --------------------------------------------------------
+ * (Section 3.1: the policy selects S, |S| <= K, "after each generation step"; Algorithm 1 steps 1-10.)
+ * Every step brings one new token per sequence. Per unit (layer l, sequence b, KV head g; unit index
+ * (l*B + b)*Hkv + g) the library keeps the state of the at most K+1 cached tokens IN POSITION ORDER and decides
+ * which one to evict; it never touches key/value rows. The caller owns a cache of K+1 rows per unit: the new token's
+ * keys and values go to row next_slot[unit], and an evicted token's row is handed out as the next next_slot.
+ * What one step computes, per the readings listed in the oracle (oracle/ta_stream_oracle.py):
+ *   - the new token completes a pattern (longest wins, then lowest index) -> it becomes an anchor with that pattern's
+ *     budget and span; every cached token of the match gets S = 1;
+ *   - the new token's voucher (Eq. 2) from the anchors of the last TA_MAX_SPAN positions, whose budgets have decayed
+ *     by budget_decay once per step since detection; nearest anchor first;
+ *   - A += a and P = rho*P + (1-rho)*a for every cached token, a = this step's attention mass on it;
+ *   - u = (alpha*A + delta*P) + ((beta*R + gamma*S) - lambda*F) + V with R = (i0+1)/n, F = count(id)/n over the n
+ *     tokens seen so far; if K+1 tokens are cached, the budget partition of Section 3.3 keeps K of them
+ *     (sinks = earliest cached tokens, recents = latest);
+ *   - every voucher is multiplied by budget_decay (Algorithm 1 step 10).
+ * All arrays DEVICE, owned, allocated and zero-initialised by the caller before the first step (next_slot: 0);
+ * to continue from a prefilled cache fill them from the outputs of the one-shot calls instead (cache_len = number of
+ * cached tokens, rows 0..cache_len-1 in position order, next_slot = cache_len, n_seen / hist / rings from the prompt).
+ * Every unit holds the same number of tokens (cache_len); the call updates cache_len. policy->age_steps is ignored. */
+typedef struct ta_stream {
+  int32_t n_layers, batch, Hkv, K; /* U = n_layers*batch*Hkv units of K+1 slots; 1 <= K <= TA_MAX_BUDGET          */
+  int32_t cache_len;               /* HOST scalar: tokens cached per unit before the step, 0..K; updated          */
+  int32_t *pos, *slot, *tok;       /* [U][K+1] position, cache row and token id of the r-th cached token          */
+  float *A, *P, *V;                /* [U][K+1] accumulated attention, pension average, voucher                    */
+  uint8_t* S;                      /* [U][K+1] anchor-token indicator                                             */
+  int32_t* next_slot;              /* [U] cache row for the next new token                                        */
+  int32_t* n_seen;                 /* [B] tokens seen so far                                                      */
+  int32_t* hist;                   /* [B][vocab_size] occurrences of every token id so far                        */
+  int32_t* tok_ring;               /* [B][TA_MAX_PATTERN_LEN] the latest token ids, position t at index t % len   */
+  float* anc_B;                    /* [B][TA_MAX_SPAN] budget of the anchor at position t (index t % span), else 0 */
+  int32_t* anc_L;                  /* [B][TA_MAX_SPAN] its span, 0: no anchor                                      */
+} ta_stream;
+
+/* Context scratch one ta_stream_step needs. */
+ta_status ta_stream_scratch_bytes(const ta_stream* st, size_t* out_bytes);
+
+/*   new_ids      DEVICE int32 [B]        the new token of every sequence
+ *   attn         DEVICE float [U][K+1]   attention mass of this step's query (summed over the unit's G query heads)
+ *                                        on each CACHE ROW, the new token's own row (next_slot) included; rows that
+ *                                        hold no token are not read
+ *   evicted_pos  DEVICE int32 [U] out    position of the evicted token, -1 when nothing was evicted */
+ta_status ta_stream_step(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* policy, ta_stream* st /*HOST*/,
+                         const int32_t* new_ids, const float* attn, int32_t* evicted_pos, void* stream);
+
 /* ---- host-buffer variant of ta_compress --------------------------------------------------------------------
  * Same computation with every data pointer on the HOST (pinned memory makes the copies asynchronous):
  * token_ids, cu_seqlens (inside batch: HOST here), the q_obs / k / v views, and the four outputs. The caller lends

@@ -38,6 +38,14 @@ class ta_bf16_view(C.Structure):
                 ("stride_n", C.c_int64)]
 
 
+class ta_stream(C.Structure):
+    _fields_ = [("n_layers", C.c_int32), ("batch", C.c_int32), ("Hkv", C.c_int32), ("K", C.c_int32),
+                ("cache_len", C.c_int32), ("pos", C.c_void_p), ("slot", C.c_void_p), ("tok", C.c_void_p),
+                ("A", C.c_void_p), ("P", C.c_void_p), ("V", C.c_void_p), ("S", C.c_void_p), ("next_slot", C.c_void_p),
+                ("n_seen", C.c_void_p), ("hist", C.c_void_p), ("tok_ring", C.c_void_p), ("anc_B", C.c_void_p),
+                ("anc_L", C.c_void_p)]
+
+
 class TAError(RuntimeError):
     def __init__(self, status, what):
         self.status = status
@@ -81,6 +89,8 @@ def lib():
                                            ta_bf16_view, u64, vp, vp, vp, vp, vp]),
             "ta_compress_scores": (i32, [vp, vp, PP, PB, i32, i32, i32, vp, vp, vp, ta_bf16_view, ta_bf16_view, u64, vp,
                                          vp, vp, vp, vp]),
+            "ta_stream_scratch_bytes": (i32, [C.POINTER(ta_stream), C.POINTER(sz)]),
+            "ta_stream_step": (i32, [vp, vp, PP, C.POINTER(ta_stream), vp, vp, vp, vp]),
             "ta_compress_host_workspace_bytes": (i32, [PB, i32, i32, i32, i32, PP, C.POINTER(sz)]),
             "ta_compress_host": (i32, [vp, vp, PP, PB, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]),
         }
@@ -241,6 +251,17 @@ def ta_compress_scores(ctx, pats, policy, batch, Hkv, d, K, token_ids, score, sc
     _check(lib().ta_compress_scores(ctx, pats, C.byref(policy), C.byref(batch), Hkv, d, K, _ptr(token_ids),
                                     _ptr(score), _ptr(score2), k, v, int(seq_epoch), _ptr(k_out), _ptr(v_out),
                                     _ptr(idx), _ptr(count), stream), "ta_compress_scores")
+
+
+def ta_stream_scratch_bytes(st: ta_stream) -> int:
+    out = C.c_size_t(0)
+    _check(lib().ta_stream_scratch_bytes(C.byref(st), C.byref(out)), "ta_stream_scratch_bytes")
+    return out.value
+
+
+def ta_stream_step(ctx, pats, policy, st: ta_stream, new_ids, attn, evicted_pos, stream=None):
+    _check(lib().ta_stream_step(ctx, pats, C.byref(policy), C.byref(st), _ptr(new_ids), _ptr(attn), _ptr(evicted_pos),
+                                stream), "ta_stream_step")
 
 
 def ta_compress_host_workspace_bytes(batch, Hq, Hkv, d, K, policy) -> int:

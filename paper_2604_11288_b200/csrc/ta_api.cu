@@ -700,6 +700,128 @@ ta_status ta_compress_scores(ta_ctx* ctx, const ta_patterns* pats, const ta_poli
                        count, stream, score, score2, false);
 }
 
+// ---------------------------------------------------------------------------------------------- decode loop
+namespace {
+struct StreamLayout {
+  size_t info, u_att, u_static, vbuf, flagbuf, forced, r_main, idx, count, end;
+};
+StreamLayout stream_layout(const ta_stream& st) {
+  StreamLayout L;
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    const size_t o = off;
+    off += align_up(bytes);
+    return o;
+  };
+  const size_t U = (size_t)st.n_layers * st.batch * st.Hkv, C = (size_t)st.K + 1;
+  L.info = take((size_t)st.batch * sizeof(ta_stream_seq_info));
+  L.u_att = take(U * C * 4);
+  L.u_static = take(U * C * 4);
+  L.vbuf = take(U * C * 4);
+  L.flagbuf = take(U * C);
+  L.forced = take(U * C);
+  L.r_main = take(U * 4);
+  L.idx = take(U * st.K * 4);
+  L.count = take(U * 4);
+  L.end = off;
+  return L;
+}
+ta_status check_stream(const ta_stream* st) {
+  if (!st) return TA_ERR_INVALID_ARG;
+  if (st->n_layers < 1 || st->batch < 1 || st->Hkv < 1 || st->K < 1) return TA_ERR_INVALID_ARG;
+  if (st->K > TA_MAX_BUDGET) return TA_ERR_UNSUPPORTED;
+  if (st->cache_len < 0 || st->cache_len > st->K) return TA_ERR_INVALID_ARG;
+  if ((long long)st->n_layers * st->batch * st->Hkv * ((long long)st->K + 1) > 0x7fffffffLL) return TA_ERR_UNSUPPORTED;
+  if (!st->pos || !st->slot || !st->tok || !st->A || !st->P || !st->V || !st->S || !st->next_slot || !st->n_seen ||
+      !st->hist || !st->tok_ring || !st->anc_B || !st->anc_L)
+    return TA_ERR_INVALID_ARG;
+  return TA_OK;
+}
+}  // namespace
+
+ta_status ta_stream_scratch_bytes(const ta_stream* st, size_t* out_bytes) {
+  if (!out_bytes || !st) return TA_ERR_INVALID_ARG;
+  if (st->n_layers < 1 || st->batch < 1 || st->Hkv < 1 || st->K < 1) return TA_ERR_INVALID_ARG;
+  *out_bytes = stream_layout(*st).end + kAlign;
+  return TA_OK;
+}
+
+ta_status ta_stream_step(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* policy, ta_stream* st,
+                         const int32_t* new_ids, const float* attn, int32_t* evicted_pos, void* stream_v) {
+  if (!ctx || !pats || !new_ids || !attn || !evicted_pos) return TA_ERR_INVALID_ARG;
+  ta_status s = check_policy(policy);
+  if (s == TA_OK) s = check_stream(st);
+  if (s != TA_OK) return s;
+  if (pats->device != ctx->device) return TA_ERR_INVALID_ARG;
+  const StreamLayout L = stream_layout(*st);
+  if (L.end > ctx->scratch_bytes) return TA_ERR_SCRATCH_TOO_SMALL;
+  DeviceGuard guard(ctx->device);
+  ctx->cached_epoch = 0;  // the scratch is shared with ta_compress's per-sequence cache
+  cudaStream_t stream = (cudaStream_t)stream_v;
+  uint8_t* sc = ctx->scratch;
+  ta_stream_dev d = {};
+  d.n_layers = st->n_layers;
+  d.B = st->batch;
+  d.Hkv = st->Hkv;
+  d.K = st->K;
+  d.len = st->cache_len;
+  d.pos = st->pos;
+  d.slot = st->slot;
+  d.tok = st->tok;
+  d.next_slot = st->next_slot;
+  d.A = st->A;
+  d.P = st->P;
+  d.V = st->V;
+  d.S = st->S;
+  d.n_seen = st->n_seen;
+  d.hist = st->hist;
+  d.tok_ring = st->tok_ring;
+  d.anc_B = st->anc_B;
+  d.anc_L = st->anc_L;
+  auto* info = reinterpret_cast<ta_stream_seq_info*>(sc + L.info);
+  float* u_att = reinterpret_cast<float*>(sc + L.u_att);
+  float* u_static = reinterpret_cast<float*>(sc + L.u_static);
+  float* vbuf = reinterpret_cast<float*>(sc + L.vbuf);
+  int32_t* idx = reinterpret_cast<int32_t*>(sc + L.idx);
+  const int U = st->n_layers * st->batch * st->Hkv, C = st->K + 1;
+  const bool evict = st->cache_len + 1 > st->K;
+
+  cudaError_t e = ta_launch_stream_seq(d, pats, *policy, new_ids, info, ctx->d_status, stream);
+  if (e == cudaSuccess)
+    e = ta_launch_stream_unit(d, *policy, info, attn, u_att, u_static, vbuf, sc + L.flagbuf, ctx->d_status, stream);
+  if (e == cudaSuccess && evict) {
+    // every unit is a "sequence" of K+1 tokens in position order; one layer, one head
+    ta_select_args sel = {};
+    sel.seq.cu = nullptr;
+    sel.seq.n_uniform = C;
+    sel.seq.batch = U;
+    sel.seq.max_n = C;
+    sel.seq.total = (long long)U * C;
+    sel.n_layers = 1;
+    sel.Hkv = 1;
+    sel.K = st->K;
+    sel.n_sink = policy->n_sink;
+    sel.n_recent = policy->n_recent;
+    sel.k_protected = policy->k_protected;
+    sel.fast = 0;
+    sel.alpha = policy->alpha;
+    sel.delta = policy->delta;
+    sel.flags = sc + L.flagbuf;
+    sel.voucher = vbuf;
+    sel.u_static = u_static;
+    sel.u = u_att;
+    sel.forced = sc + L.forced;
+    sel.r_main = reinterpret_cast<int32_t*>(sc + L.r_main);
+    sel.idx = idx;
+    sel.count = reinterpret_cast<int32_t*>(sc + L.count);
+    e = ta_launch_select(sel, ctx->d_status, stream);
+  }
+  if (e == cudaSuccess) e = ta_launch_stream_evict(d, evict ? 1 : 0, idx, policy->budget_decay, evicted_pos, stream);
+  if (e != cudaSuccess) return cuda_fail(ctx, e);
+  st->cache_len = evict ? st->K : st->cache_len + 1;
+  return TA_OK;
+}
+
 // ---------------------------------------------------------------------------------------------- host buffers
 namespace {
 struct HostLayout {

@@ -123,6 +123,31 @@ cudaError_t ta_launch_headsum(int n_layers, int Hkv, long long total, const floa
 cudaError_t ta_launch_broadcast_heads(int n_layers, int B, int Hkv, int K, const int32_t* idx_lb,
                                       const int32_t* count_lb, int32_t* idx, int32_t* count, cudaStream_t stream);
 
+// ---- Algorithm 1 per decode step (ta_stream.cu) ---------------------------------------------------------------
+struct ta_stream_dev {  // the caller's ta_stream with the cached length of this step
+  int n_layers, B, Hkv, K, len;
+  int32_t *pos, *slot, *tok, *next_slot;
+  float *A, *P, *V;
+  uint8_t* S;
+  int32_t *n_seen, *hist, *tok_ring;
+  float* anc_B;
+  int32_t* anc_L;
+};
+struct ta_stream_seq_info {  // per sequence, written by the sequence kernel of a step
+  int t;          // position of the new token
+  int match_len;  // tokens t - match_len + 1 .. t belong to a pattern completed by the new token (0: none)
+  float v_new;    // voucher of the new token
+  int id;         // its token id
+};
+cudaError_t ta_launch_stream_seq(const ta_stream_dev& st, const ta_patterns* pats, const ta_policy& pol,
+                                 const int32_t* new_ids, ta_stream_seq_info* info, ta_dev_status* status,
+                                 cudaStream_t stream);
+cudaError_t ta_launch_stream_unit(const ta_stream_dev& st, const ta_policy& pol, const ta_stream_seq_info* info,
+                                  const float* attn, float* u_att, float* u_static, float* vbuf, uint8_t* flagbuf,
+                                  ta_dev_status* status, cudaStream_t stream);
+cudaError_t ta_launch_stream_evict(const ta_stream_dev& st, int evict, const int32_t* idx, float budget_decay,
+                                   int32_t* evicted_pos, cudaStream_t stream);
+
 // ---- step 4 ------------------------------------------------------------------------------------------------
 struct ta_compact_args {
   ta_seq_desc seq;
