@@ -298,6 +298,98 @@ def measure_extra(name, L, dev, steps=5, warmup=3):
         torch.cuda.empty_cache()
 
 
+def measure_variants(dev, steps=10, warmup=3):
+    """Timings of the entry points beyond the one-shot ta_compress, on synthetic inputs of the main workload's shape:
+    selection shared by the heads of a layer, a caller-supplied score, detector-confidence anchors, and the per-step
+    retention of the decode loop. Supplementary: reported next to the main line, never in place of it."""
+    import paper_2604_11288_b200 as ta
+    out = []
+    peak, _ = measured_peak_hbm()
+    w, K = build_workload("c2", 0)
+    L = w.n_layers
+    r = Runner(w, K, L, False, dev)
+    try:
+        def allheads():
+            ta.ta_compress_allheads(r.ctx, r.pats, r.p, r.batch, w.Hq, w.Hkv, w.d, K, r.ids, r.vq, r.vk, r.vv, 0, r.ko,
+                                    r.vo, r.idx, r.cnt, r.stream)
+        ms = time_steps(allheads, steps, warmup)
+        out.append({"entry": "ta_compress_allheads", "workload": f"c2, {L} layers, K={K}", "ms_per_step": ms,
+                    "value": w.total * L / (ms * 1e-3), "unit": UNIT})
+        score = torch.rand((L, w.Hkv, w.total), dtype=torch.float32, device=dev)
+
+        def scores():
+            ta.ta_compress_scores(r.ctx, r.pats, r.p, r.batch, w.Hkv, w.d, K, r.ids, score, None, r.vk, r.vv, 0, r.ko,
+                                  r.vo, r.idx, r.cnt, r.stream)
+        ms = time_steps(scores, steps, warmup)
+        out.append({"entry": "ta_compress_scores", "workload": f"c2, {L} layers, K={K}, scores resident",
+                    "ms_per_step": ms, "value": w.total * L / (ms * 1e-3), "unit": UNIT})
+    finally:
+        r.close()
+    # detector-confidence anchors on the token stream of c4 (4 x 131072 tokens)
+    w4, K4 = build_workload("c4", 0)
+    r4 = Runner(w4, K4, 1, True, dev)
+    try:
+        conf = torch.rand(w4.total, dtype=torch.float32, device=dev) * 0.4
+        conf[torch.randint(0, w4.total, (2048,), device=dev)] = 0.95
+        flags = torch.empty(w4.total, dtype=torch.uint8, device=dev)
+        V = torch.empty(w4.total, dtype=torch.float32, device=dev)
+        u0 = torch.empty_like(V)
+
+        def mask_conf():
+            ta.ta_sponsor_mask_conf(r4.ctx, r4.p, r4.batch, r4.ids, conf, 0.5, 15.0, 6, 0, flags, V, u0, r4.stream)
+        ms = time_steps(mask_conf, steps, warmup)
+        bytes_ = w4.total * (4 + 4 + 1 + 4 + 4)  # ids, conf read; flags, voucher, static utility written
+        out.append({"entry": "ta_sponsor_mask_conf", "workload": f"c4 token stream, {w4.total} tokens",
+                    "ms_per_step": ms, "GBps": bytes_ / (ms * 1e-3) / 1e9, "hbm_frac": bytes_ / (ms * 1e-3) / 1e9 / peak,
+                    "value": w4.total / (ms * 1e-3), "unit": "tokens/s"})
+    finally:
+        r4.close()
+    # decode loop: 32 layers x 16 sequences x 8 KV heads, K = 256 cached tokens per unit
+    Ls, Bs, Hs, Ks, vocab = 32, 16, 8, 256, 32000
+    U, C_ = Ls * Bs * Hs, Ks + 1
+    z = lambda shape, dt: torch.zeros(shape, dtype=dt, device=dev)
+    t = dict(pos=z((U, C_), torch.int32), slot=z((U, C_), torch.int32), tok=z((U, C_), torch.int32),
+             A=z((U, C_), torch.float32), P=z((U, C_), torch.float32), V=z((U, C_), torch.float32),
+             S=z((U, C_), torch.uint8), next_slot=z((U,), torch.int32), n_seen=z((Bs,), torch.int32),
+             hist=z((Bs, vocab), torch.int32), tok_ring=z((Bs, 8), torch.int32), anc_B=z((Bs, 64), torch.float32),
+             anc_L=z((Bs, 64), torch.int32))
+    st = ta.ta_stream()
+    st.n_layers, st.batch, st.Hkv, st.K, st.cache_len = Ls, Bs, Hs, Ks, 0
+    for k, v in t.items():
+        setattr(st, k, v.data_ptr())
+    p = ta.ta_policy_default(ta.TA_PRESET_THEOREM, Ks)
+    p.vocab_size = vocab
+    ctx = ta.ta_ctx_create(dev.index, ta.ta_stream_scratch_bytes(st))
+    pats = ta.ta_patterns_create(ctx, w.pattern_ids, w.pattern_budget, w.pattern_span)
+    try:
+        attn = torch.rand((U, C_), dtype=torch.float32, device=dev)
+        ev = torch.empty((U,), dtype=torch.int32, device=dev)
+        ids = torch.randint(0, vocab, (Ks + 64, Bs), dtype=torch.int32, device=dev)
+        stream = torch.cuda.current_stream(dev).cuda_stream
+        for i in range(Ks + 8):  # fill the caches, then a few evicting steps as warm-up
+            ta.ta_stream_step(ctx, pats, p, st, ids[i], attn, ev, stream)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n_timed = 40
+        e0.record()
+        for i in range(n_timed):
+            ta.ta_stream_step(ctx, pats, p, st, ids[Ks + 8 + i], attn, ev, stream)
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / n_timed
+        state_bytes = U * C_ * (3 * 4 + 3 * 4 + 1) * 2 + U * C_ * 4  # ordered state read + written, attention read
+        out.append({"entry": "ta_stream_step", "workload": f"{Ls} layers x {Bs} sequences x {Hs} KV heads, K={Ks}, "
+                    "steady state (one eviction per unit and step)", "ms_per_step": ms, "kernels_per_step": 5,
+                    "unit_steps_per_s": U / (ms * 1e-3), "state_GBps": state_bytes / (ms * 1e-3) / 1e9})
+        if ta.ta_ctx_poll(ctx) != 0:
+            out[-1]["error"] = "device status"
+    finally:
+        ta.ta_patterns_destroy(pats)
+        ta.ta_ctx_destroy(ctx)
+    torch.cuda.empty_cache()
+    return out
+
+
 # ------------------------------------------------------------------------------------------------ main
 def main():
     ap = argparse.ArgumentParser()
@@ -420,6 +512,10 @@ def main():
             except Exception as ex:  # supplementary only: never lose the main line
                 extra.append({"workload": name, "error": str(ex)[:200]})
         line["other_workloads"] = extra
+        try:
+            line["variants"] = measure_variants(dev)
+        except Exception as ex:
+            line["variants"] = [{"error": str(ex)[:200]}]
     print(json.dumps(line))
 
 
