@@ -128,6 +128,22 @@ def anchors_conf(conf: np.ndarray, threshold, budget, span, rank, budget_decay=0
     return atok, aend, Be, Le
 
 
+def embedding_confidence(emb: np.ndarray, concepts: np.ndarray):
+    """Embedding-based anchor detector (Section 3.2 "Anchor detection", instantiation 3): the confidence of token i is
+    the largest cosine similarity between its input embedding and the anchor-concept embeddings. emb uint16 (bf16
+    bits) [n, D], concepts uint16 [C, D]; evaluated in double, rounded to fp32; a zero vector has similarity 0.
+    Pinned by: identical vectors -> 1, opposite -> -1, orthogonal -> 0, scale invariance."""
+    def dec(a):
+        return (a.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+    e, c = dec(np.ascontiguousarray(emb)), dec(np.ascontiguousarray(concepts))
+    ne = np.sqrt((e * e).sum(-1))
+    nc = np.sqrt((c * c).sum(-1))
+    dots = e @ c.T
+    den = ne[:, None] * nc[None, :]
+    cos = np.where(den > 0, dots / np.where(den > 0, den, 1.0), 0.0)
+    return cos.max(-1).astype(np.float32)
+
+
 def vouchers(aend, Be, Le, voucher_decay=0.8):
     lib = _load()
     n = aend.shape[0]

@@ -547,3 +547,22 @@ def test_stream_sponsored_span_survives_adversarial_attention():
         if t >= 26:
             assert set(range(21, 27)) <= set(so.units[0].pos), t
     assert len(so.units[0].pos) == K
+
+
+# ----------------------------------------------------------------- embedding-based detector (Section 3.2, variant 3)
+def test_embedding_confidence_special_cases():
+    g = torch.Generator().manual_seed(2)
+    a = torch.randn(3, 64, generator=g).to(torch.bfloat16)
+    e = torch.stack([a[0], -a[1], 3.0 * a[2], torch.zeros(64).to(torch.bfloat16),
+                     torch.cat([torch.ones(32), torch.zeros(32)]).to(torch.bfloat16)])
+    conf = oracle.embedding_confidence(bf16_bits(e), bf16_bits(a))
+    assert conf[0] == pytest.approx(1.0, abs=1e-6)          # identical to concept 0
+    assert conf[2] == pytest.approx(1.0, abs=1e-6)          # a positive multiple of concept 2
+    assert conf[3] == 0.0                                   # zero vector
+    # -a[1]: similarity -1 with concept 1; the maximum is over the other two concepts, against a library routine
+    ref = torch.nn.functional.cosine_similarity(e[1].double()[None], a.double(), dim=-1).max().item()
+    assert conf[1] == pytest.approx(ref, abs=1e-6) and conf[1] < 1.0
+    # orthogonal halves
+    c2 = torch.cat([torch.zeros(32), torch.ones(32)]).to(torch.bfloat16)[None]
+    assert oracle.embedding_confidence(bf16_bits(e[4:5]), bf16_bits(c2))[0] == 0.0
+    assert oracle.embedding_confidence(bf16_bits(e[4:5]), bf16_bits(-e[4:5]))[0] == pytest.approx(-1.0, abs=1e-6)
