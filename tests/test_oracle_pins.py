@@ -553,11 +553,11 @@ def test_stream_sponsored_span_survives_adversarial_attention():
 def test_embedding_confidence_special_cases():
     g = torch.Generator().manual_seed(2)
     a = torch.randn(3, 64, generator=g).to(torch.bfloat16)
-    e = torch.stack([a[0], -a[1], 3.0 * a[2], torch.zeros(64).to(torch.bfloat16),
+    e = torch.stack([a[0], -a[1], 4.0 * a[2], torch.zeros(64).to(torch.bfloat16),
                      torch.cat([torch.ones(32), torch.zeros(32)]).to(torch.bfloat16)])
     conf = oracle.embedding_confidence(bf16_bits(e), bf16_bits(a))
     assert conf[0] == pytest.approx(1.0, abs=1e-6)          # identical to concept 0
-    assert conf[2] == pytest.approx(1.0, abs=1e-6)          # a positive multiple of concept 2
+    assert conf[2] == pytest.approx(1.0, abs=1e-6)          # concept 2 times a power of two (exact in bf16)
     assert conf[3] == 0.0                                   # zero vector
     # -a[1]: similarity -1 with concept 1; the maximum is over the other two concepts, against a library routine
     ref = torch.nn.functional.cosine_similarity(e[1].double()[None], a.double(), dim=-1).max().item()
