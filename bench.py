@@ -342,6 +342,19 @@ def measure_variants(dev, steps=10, warmup=3):
         out.append({"entry": "ta_sponsor_mask_conf", "workload": f"c4 token stream, {w4.total} tokens",
                     "ms_per_step": ms, "GBps": bytes_ / (ms * 1e-3) / 1e9, "hbm_frac": bytes_ / (ms * 1e-3) / 1e9 / peak,
                     "value": w4.total / (ms * 1e-3), "unit": "tokens/s"})
+        # embedding detector on the same token stream: 2048-wide input embeddings, 8 anchor concepts
+        D = 2048
+        emb = torch.randn((w4.total, D), dtype=torch.float32, device=dev).to(torch.bfloat16)
+        concepts = torch.randn((8, D), dtype=torch.float32, device=dev).to(torch.bfloat16)
+
+        def detect():
+            ta.ta_detect_embedding(r4.ctx, w4.total, emb, D, D, concepts, 8, conf, r4.stream)
+        ms = time_steps(detect, steps, warmup)
+        bytes_ = w4.total * (D * 2 + 4)
+        out.append({"entry": "ta_detect_embedding", "workload": f"{w4.total} tokens x {D} bf16, 8 concepts",
+                    "ms_per_step": ms, "GBps": bytes_ / (ms * 1e-3) / 1e9, "hbm_frac": bytes_ / (ms * 1e-3) / 1e9 / peak,
+                    "value": w4.total / (ms * 1e-3), "unit": "tokens/s"})
+        del emb
     finally:
         r4.close()
     # decode loop: 32 layers x 16 sequences x 8 KV heads, K = 256 cached tokens per unit

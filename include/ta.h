@@ -67,7 +67,9 @@ enum {
   TA_MAX_SCORE_ROWS = 256,  /* G * W                                                                   */
   TA_MAX_BUDGET = 4096,     /* K                                                                       */
   TA_MAX_SEQ_LEN = 1 << 20, /* tokens per sequence                                                     */
-  TA_HEAD_DIM = 128         /* d                                                                       */
+  TA_HEAD_DIM = 128,        /* d                                                                       */
+  TA_MAX_CONCEPTS = 8,      /* anchor-concept embeddings of the embedding detector                     */
+  TA_MAX_EMBED_DIM = 8192   /* embedding width of the embedding detector                               */
 };
 
 /*
@@ -181,6 +183,20 @@ void ta_patterns_destroy(ta_patterns* pats);
  * Uses B*vocab_size*4 bytes of context scratch. batch->n_layers is ignored. */
 ta_status ta_sponsor_mask(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* policy, const ta_batch* batch,
                           const int32_t* token_ids, uint8_t* flags, float* voucher, float* u_static, void* stream);
+
+/* ---- embedding-based anchor detector (Section 3.2 "Anchor detection", third instantiation; Section 5.4) ---------
+ * "Cosine similarity between input embeddings and anchor concept embeddings": conf[i] is the largest cosine
+ * similarity between token i's input embedding and the n_concepts concept embeddings (a zero vector has similarity
+ * 0 with everything; a NaN anywhere in a token's embedding gives NaN, which no threshold accepts). The result is a
+ * per-token confidence for ta_sponsor_mask_conf.
+ *   emb       DEVICE bf16, token i at emb + i*stride_tok, D contiguous values (the model's input-embedding rows of
+ *             the prompt tokens); 4-byte aligned, stride_tok even and >= D
+ *   concepts  DEVICE bf16 [n_concepts][D]
+ *   conf      DEVICE float [total_tokens] out
+ * D a multiple of 16, at most TA_MAX_EMBED_DIM; 1 <= n_concepts <= TA_MAX_CONCEPTS. bf16 products accumulated in
+ * fp32 on the tensor cores; the embeddings are read exactly once. */
+ta_status ta_detect_embedding(ta_ctx* ctx, int64_t total_tokens, const void* emb, int64_t stride_tok, int D,
+                              const void* concepts, int n_concepts, float* conf, void* stream);
 
 /* ---- step 1 with a learned anchor detector (Section 5.1, "Learned Anchor Detection") ----------------------
  * The detector itself (an MLP on hidden states, or an embedding similarity) runs in the caller's model; its

@@ -78,6 +78,7 @@ def lib():
             "ta_patterns_create": (i32, [vp, i32, vp, vp, vp, vp, C.POINTER(vp)]),
             "ta_patterns_destroy": (None, [vp]),
             "ta_sponsor_mask": (i32, [vp, vp, PP, PB, vp, vp, vp, vp, vp]),
+            "ta_detect_embedding": (i32, [vp, C.c_int64, vp, C.c_int64, i32, vp, i32, vp, vp]),
             "ta_sponsor_mask_conf": (i32, [vp, PP, PB, vp, vp, C.c_float, C.c_float, i32, i32, vp, vp, vp, vp]),
             "ta_score": (i32, [vp, PP, PB, i32, i32, i32, ta_bf16_view, ta_bf16_view, vp, vp, vp, vp]),
             "ta_select_topk": (i32, [vp, PP, PB, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]),
@@ -196,6 +197,11 @@ def ta_patterns_create(ctx, pattern_ids, budget=None, span=None):
 
 def ta_patterns_destroy(pats):
     lib().ta_patterns_destroy(pats)
+
+
+def ta_detect_embedding(ctx, total_tokens, emb, stride_tok, D, concepts, n_concepts, conf, stream=None):
+    _check(lib().ta_detect_embedding(ctx, int(total_tokens), _ptr(emb), int(stride_tok), int(D), _ptr(concepts),
+                                     int(n_concepts), _ptr(conf), stream), "ta_detect_embedding")
 
 
 def ta_sponsor_mask_conf(ctx, policy, batch, token_ids, conf, threshold, budget, span, rank_by_confidence, flags,

@@ -379,6 +379,18 @@ ta_status ta_sponsor_mask(ta_ctx* ctx, const ta_patterns* pats, const ta_policy*
   return e == cudaSuccess ? TA_OK : cuda_fail(ctx, e);
 }
 
+ta_status ta_detect_embedding(ta_ctx* ctx, int64_t total_tokens, const void* emb, int64_t stride_tok, int D,
+                              const void* concepts, int n_concepts, float* conf, void* stream) {
+  if (!ctx || !emb || !concepts || !conf || total_tokens < 0) return TA_ERR_INVALID_ARG;
+  if (D < 16 || n_concepts < 1 || stride_tok < D) return TA_ERR_INVALID_ARG;
+  if (D % 16 || D > TA_MAX_EMBED_DIM || n_concepts > TA_MAX_CONCEPTS) return TA_ERR_UNSUPPORTED;
+  if ((uintptr_t)emb % 4 || (uintptr_t)concepts % 2 || stride_tok % 2) return TA_ERR_ALIGNMENT;
+  DeviceGuard guard(ctx->device);
+  cudaError_t e = ta_launch_embed_conf(ctx->sm_count, total_tokens, emb, stride_tok, D, concepts, n_concepts, conf,
+                                       (cudaStream_t)stream);
+  return e == cudaSuccess ? TA_OK : cuda_fail(ctx, e);
+}
+
 ta_status ta_sponsor_mask_conf(ta_ctx* ctx, const ta_policy* policy, const ta_batch* batch, const int32_t* token_ids,
                                const float* conf, float threshold, float budget, int span, int rank_by_confidence,
                                uint8_t* flags, float* voucher, float* u_static, void* stream) {

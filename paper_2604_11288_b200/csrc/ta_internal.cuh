@@ -77,6 +77,10 @@ cudaError_t ta_launch_mask_conf(const ta_policy& pol, const ta_seq_desc& seq, co
                                 float threshold, float budget, int span, int rank, uint8_t* flags, float* voucher,
                                 float* u_static, int32_t* hist, ta_dev_status* status, cudaStream_t stream);
 
+// embedding-based detector: conf[i] = max over concepts of the cosine similarity (ta_detect.cu)
+cudaError_t ta_launch_embed_conf(int sm_count, long long total, const void* emb, long long stride, int D,
+                                 const void* concepts, int C, float* conf, cudaStream_t stream);
+
 // ---- step 2 ------------------------------------------------------------------------------------------------
 struct ta_score_args {
   ta_seq_desc seq;

@@ -130,6 +130,38 @@ def test_mask_from_detector_confidences_bit_exact(rank, threshold, budget, span)
         g.close()
 
 
+@pytest.mark.parametrize("D,Cn,total", [(64, 1, 5), (2048, 8, 1000), (4096, 3, 333), (8192, 8, 40)])
+def test_embedding_detector_matches_oracle(D, Cn, total):
+    # Section 3.2, third detector: largest cosine similarity to the concept embeddings. Token counts that are not a
+    # multiple of 16, a padded row stride, planted near-copies of concepts, a zero row and a NaN row.
+    g = torch.Generator().manual_seed(100 + D + Cn)
+    stride = D + 24
+    buf = torch.randn(total, stride, generator=g).to(torch.bfloat16)
+    concepts = torch.randn(Cn, D, generator=g).to(torch.bfloat16)
+    for i in range(0, total, 7):
+        buf[i, :D] = (concepts[i % Cn].float() * 2.0 + 0.05 * torch.randn(D, generator=g)).to(torch.bfloat16)
+    if total > 3:
+        buf[2, :D] = 0
+        buf[3, 5] = float("nan")
+    w = _workload([32], [[1, 2]], seed=1)
+    gp = Gpu(w, oracle_policy(4), 4, 1)
+    try:
+        conf = torch.full((total,), -7.0, dtype=torch.float32, device="cuda")
+        ta.ta_detect_embedding(gp.ctx, total, buf.cuda(), stride, D, concepts.cuda(), Cn, conf, gp.stream)
+        torch.cuda.synchronize()
+        assert gp.poll() == ta.TA_OK
+        got = conf.cpu().numpy()
+        want = oracle.embedding_confidence(bf16_bits(buf[:, :D]), bf16_bits(concepts))
+        if total > 3:
+            assert np.isnan(got[3]) and got[2] == 0.0
+            got, want = np.delete(got, 3), np.delete(want, 3)
+        # fp32 tensor-core accumulation (not rounded to nearest) of D bf16 products against double, values in [-1, 1]
+        np.testing.assert_allclose(got, want, rtol=0, atol=2e-6 + 4e-9 * D)
+        assert want.max() > 0.99
+    finally:
+        gp.close()
+
+
 def _score_case(lengths, Hq, Hkv, W, causal=1, seed=0, layers=1, permute=False, scale=0.0):
     w = _workload(lengths, [[1, 2]], seed=seed, Hq=Hq, Hkv=Hkv, W=W)
     w.n_layers = layers
