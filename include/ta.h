@@ -190,10 +190,10 @@ ta_status ta_sponsor_mask(ta_ctx* ctx, const ta_patterns* pats, const ta_policy*
  * 0 with everything; a NaN anywhere in a token's embedding gives NaN, which no threshold accepts). The result is a
  * per-token confidence for ta_sponsor_mask_conf.
  *   emb       DEVICE bf16, token i at emb + i*stride_tok, D contiguous values (the model's input-embedding rows of
- *             the prompt tokens); 4-byte aligned, stride_tok even and >= D
+ *             the prompt tokens); 16-byte aligned, stride_tok a multiple of 8 and >= D
  *   concepts  DEVICE bf16 [n_concepts][D]
  *   conf      DEVICE float [total_tokens] out
- * D a multiple of 16, at most TA_MAX_EMBED_DIM; 1 <= n_concepts <= TA_MAX_CONCEPTS. bf16 products accumulated in
+ * D a multiple of 32, at most TA_MAX_EMBED_DIM; 1 <= n_concepts <= TA_MAX_CONCEPTS. bf16 products accumulated in
  * fp32 on the tensor cores; the embeddings are read exactly once. */
 ta_status ta_detect_embedding(ta_ctx* ctx, int64_t total_tokens, const void* emb, int64_t stride_tok, int D,
                               const void* concepts, int n_concepts, float* conf, void* stream);

@@ -382,9 +382,9 @@ ta_status ta_sponsor_mask(ta_ctx* ctx, const ta_patterns* pats, const ta_policy*
 ta_status ta_detect_embedding(ta_ctx* ctx, int64_t total_tokens, const void* emb, int64_t stride_tok, int D,
                               const void* concepts, int n_concepts, float* conf, void* stream) {
   if (!ctx || !emb || !concepts || !conf || total_tokens < 0) return TA_ERR_INVALID_ARG;
-  if (D < 16 || n_concepts < 1 || stride_tok < D) return TA_ERR_INVALID_ARG;
-  if (D % 16 || D > TA_MAX_EMBED_DIM || n_concepts > TA_MAX_CONCEPTS) return TA_ERR_UNSUPPORTED;
-  if ((uintptr_t)emb % 4 || (uintptr_t)concepts % 2 || stride_tok % 2) return TA_ERR_ALIGNMENT;
+  if (D < 32 || n_concepts < 1 || stride_tok < D) return TA_ERR_INVALID_ARG;
+  if (D % 32 || D > TA_MAX_EMBED_DIM || n_concepts > TA_MAX_CONCEPTS) return TA_ERR_UNSUPPORTED;
+  if ((uintptr_t)emb % 16 || (uintptr_t)concepts % 2 || stride_tok % 8) return TA_ERR_ALIGNMENT;
   DeviceGuard guard(ctx->device);
   cudaError_t e = ta_launch_embed_conf(ctx->sm_count, total_tokens, emb, stride_tok, D, concepts, n_concepts, conf,
                                        (cudaStream_t)stream);

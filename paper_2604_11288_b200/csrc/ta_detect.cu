@@ -2,10 +2,12 @@
 // token is the largest cosine similarity between its input embedding and a handful of anchor-concept embeddings.
 //
 // The work is one pass over the embeddings (D bf16 values per token, read once; nothing else is large), so the kernel
-// is built around that stream: a warp takes 16 tokens, every lane reads its fragment of the 16 x 16 sub-tiles straight
-// from global memory with 4-byte loads that together cover whole 32-byte sectors, the dot products with the (at
-// most 8) concepts run as m16n8k16 tensor-core products against concept fragments kept in shared memory, and the
-// squared norms of the rows are accumulated from the same registers. The contraction has N = 8: far too small for a
+// is built around that stream: a warp takes 16 tokens; per 32 dimensions every lane reads 16 contiguous bytes of two
+// token rows straight from global memory (four lanes cover 64 contiguous bytes of a row: whole sectors, each fetched
+// once), the dot products with the (at most 8) concepts run as m16n8k16 tensor-core products against concept
+// fragments kept in shared memory, and the squared norms of the rows are accumulated from the same registers. The
+// order of the dimensions inside a product is free as long as both operands use the same one, so a lane's 8
+// consecutive dimensions serve as its fragment columns of two products. The contraction has N = 8: far too small for a
 // tcgen05 tile to pay; the memory stream is what bounds it (2*D bytes per token against about 20 instructions per 16
 // tokens and 16 dimensions).
 #include <cuda_bf16.h>
@@ -31,8 +33,8 @@ __global__ void __launch_bounds__(kWarps * 32)
 ta_embed_conf_kernel(long long total, const __nv_bfloat16* __restrict__ emb, long long stride, int D,
                      const __nv_bfloat16* __restrict__ concepts, int C, float* __restrict__ conf) {
   extern __shared__ __align__(16) unsigned char smem[];
-  const int ld = D + 8;  // padded row: the 8 x 4 lanes of a fragment load hit 32 different banks
-  __nv_bfloat16* s_c = reinterpret_cast<__nv_bfloat16*>(smem);           // [8][D + 8], unused concepts are zero
+  const int ld = D + 32;  // padded row: consecutive rows start 64 bytes apart modulo 128 (conflict-free 16-byte loads)
+  __nv_bfloat16* s_c = reinterpret_cast<__nv_bfloat16*>(smem);           // [8][D + 32], unused concepts are zero
   float* s_inv = reinterpret_cast<float*>(smem + (size_t)kMaxConcepts * ld * 2);  // 1 / |concept|, 0 for zero vectors
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   for (int i = tid; i < kMaxConcepts * ld; i += blockDim.x) {
@@ -57,30 +59,23 @@ ta_embed_conf_kernel(long long total, const __nv_bfloat16* __restrict__ emb, lon
   for (long long g = (long long)blockIdx.x * kWarps + warp; g < groups; g += (long long)gridDim.x * kWarps) {
     const long long t0 = g * 16 + r, t1 = t0 + 8;
     // rows past the end re-read the last token; their results are not written
-    const uint32_t* e0 = reinterpret_cast<const uint32_t*>(emb + (t0 < total ? t0 : total - 1) * stride) + q;
-    const uint32_t* e1 = reinterpret_cast<const uint32_t*>(emb + (t1 < total ? t1 : total - 1) * stride) + q;
-    const uint32_t* cb = reinterpret_cast<const uint32_t*>(s_c + (size_t)r * ld) + q;  // concept r, column pair q
+    const uint4* e0 = reinterpret_cast<const uint4*>(emb + (t0 < total ? t0 : total - 1) * stride) + q;
+    const uint4* e1 = reinterpret_cast<const uint4*>(emb + (t1 < total ? t1 : total - 1) * stride) + q;
+    const uint4* cb = reinterpret_cast<const uint4*>(s_c + (size_t)r * ld) + q;  // concept r, dimensions 8q .. 8q+7
     // two accumulator sets taken in turn: the tensor core's fp32 accumulation does not round to nearest, and its
     // error grows with the length of one accumulation chain
     float dA[4] = {0.0f, 0.0f, 0.0f, 0.0f}, dB[4] = {0.0f, 0.0f, 0.0f, 0.0f};
     float n0 = 0.0f, n1 = 0.0f;
-    auto kstep = [&](int k, float(&acc)[4]) {
-      uint32_t a[4];
-      a[0] = __ldg(e0 + (k >> 1));
-      a[1] = __ldg(e1 + (k >> 1));
-      a[2] = __ldg(e0 + (k >> 1) + 4);
-      a[3] = __ldg(e1 + (k >> 1) + 4);
-      mma_bf16_16816(acc, a, cb[k >> 1], cb[(k >> 1) + 4]);
-      n0 += sq2(a[0]) + sq2(a[2]);
-      n1 += sq2(a[1]) + sq2(a[3]);
-    };
-    int k = 0;
-#pragma unroll 2
-    for (; k + 32 <= D; k += 32) {
-      kstep(k, dA);
-      kstep(k + 16, dB);
+#pragma unroll 4
+    for (int k = 0; k < D; k += 32) {  // 32 dimensions = 4 x uint4 per row
+      const uint4 v0 = __ldg(e0 + (k >> 3)), v1 = __ldg(e1 + (k >> 3));
+      const uint4 vb = cb[k >> 3];
+      const uint32_t a0[4] = {v0.x, v1.x, v0.y, v1.y}, a1[4] = {v0.z, v1.z, v0.w, v1.w};
+      mma_bf16_16816(dA, a0, vb.x, vb.y);
+      mma_bf16_16816(dB, a1, vb.z, vb.w);
+      n0 += (sq2(v0.x) + sq2(v0.y)) + (sq2(v0.z) + sq2(v0.w));
+      n1 += (sq2(v1.x) + sq2(v1.y)) + (sq2(v1.z) + sq2(v1.w));
     }
-    if (k < D) kstep(k, dA);
     float d[4];
 #pragma unroll
     for (int x = 0; x < 4; ++x) d[x] = dA[x] + dB[x];
@@ -122,7 +117,7 @@ ta_embed_conf_kernel(long long total, const __nv_bfloat16* __restrict__ emb, lon
 cudaError_t ta_launch_embed_conf(int sm_count, long long total, const void* emb, long long stride, int D,
                                  const void* concepts, int C, float* conf, cudaStream_t stream) {
   if (total == 0) return cudaSuccess;
-  const size_t smem = (size_t)kMaxConcepts * (D + 8) * 2 + kMaxConcepts * sizeof(float);
+  const size_t smem = (size_t)kMaxConcepts * (D + 32) * 2 + kMaxConcepts * sizeof(float);
   static bool attr_set[64] = {};
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
