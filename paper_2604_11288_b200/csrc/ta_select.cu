@@ -31,6 +31,8 @@ __device__ __forceinline__ uint32_t sortable_key(float f) {
   return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
 }
 
+constexpr int kItemsLong = 32;  // keys per thread of clustered units (up to 8 * kItemsLong * kThreads elements)
+
 struct SelectResult {
   uint32_t thresh;  // key of the last element taken
   int ties;         // how many elements equal to thresh are taken (lowest positions first)
@@ -48,6 +50,12 @@ struct SelectShared {
   // alternating by pass) and every CTA's (definite, tie) totals
   uint32_t ghist[2][256];
   int totals[8][2];
+  // ordered write of a unit whose keys sit in registers: per (chunk of kThreads elements, warp) the counts of
+  // definite | tie elements (packed 16 | 16 bits, then their exclusive prefix) and the two ballots
+  uint32_t cnt[kItemsLong * kWarps];
+  uint32_t bdef[kItemsLong * kWarps], btie[kItemsLong * kWarps];
+  uint32_t wtot[kWarps];
+  uint32_t total;
 };
 constexpr int kSelectCluster = 8;  // CTAs per unit when a sequence is longer than kItems * kThreads
 
@@ -55,16 +63,17 @@ constexpr int kSelectCluster = 8;  // CTAs per unit when a sequence is longer th
 // re-read from L2 on every sweep in batches whose loads are all issued before the first use.
 constexpr int kItems = 16;
 constexpr int kBatch = 8;
+template <int ITEMS>
 struct KeyCache {
-  uint32_t key[kItems];
+  uint32_t key[ITEMS];
   uint32_t elig;  // bit `it`: element tid + it*kThreads exists and is eligible
 };
 
-template <class KeyFn>
-__device__ __forceinline__ void fill_cache(int n, KeyFn key_of, KeyCache& kc) {
+template <class KeyFn, int ITEMS>
+__device__ __forceinline__ void fill_cache(int n, KeyFn key_of, KeyCache<ITEMS>& kc) {
   kc.elig = 0;
 #pragma unroll
-  for (int it = 0; it < kItems; ++it) {
+  for (int it = 0; it < ITEMS; ++it) {
     const int i = (int)threadIdx.x + it * kThreads;
     kc.key[it] = 0;
     if (i < n && key_of(i, kc.key[it])) kc.elig |= 1u << it;
@@ -73,12 +82,12 @@ __device__ __forceinline__ void fill_cache(int n, KeyFn key_of, KeyCache& kc) {
 
 // Calls body(i, exists, eligible, key) for every element slot in ascending chunks of kThreads; every thread of the
 // block makes the same number of calls (the body may hold block-wide barriers).
-template <bool CACHED, class KeyFn, class Body>
-__device__ __forceinline__ void sweep(int n, KeyFn key_of, const KeyCache& kc, Body body) {
+template <bool CACHED, class KeyFn, class Body, int ITEMS>
+__device__ __forceinline__ void sweep(int n, KeyFn key_of, const KeyCache<ITEMS>& kc, Body body) {
   const int tid = threadIdx.x;
   if (CACHED) {
 #pragma unroll
-    for (int it = 0; it < kItems; ++it) {
+    for (int it = 0; it < ITEMS; ++it) {
       if (it * kThreads < n) {
         const int i = tid + it * kThreads;
         body(i, i < n, ((kc.elig >> it) & 1u) != 0, kc.key[it]);
@@ -107,8 +116,8 @@ __device__ __forceinline__ void sweep(int n, KeyFn key_of, const KeyCache& kc, B
 
 // Top-`want` of the eligible elements of [0, n) by key. All threads of the block must call it; the result is uniform
 // across the block.
-template <bool CACHED, int CL, class KeyFn>
-__device__ SelectResult block_radix_select(int n, int want, KeyFn key_of, const KeyCache& kc, SelectShared& sh) {
+template <bool CACHED, int CL, class KeyFn, int ITEMS>
+__device__ SelectResult block_radix_select(int n, int want, KeyFn key_of, const KeyCache<ITEMS>& kc, SelectShared& sh) {
   SelectResult r;
   r.thresh = 0;
   r.ties = 0;
@@ -201,8 +210,8 @@ __device__ SelectResult block_radix_select(int n, int want, KeyFn key_of, const 
 // Ordered pass over [0, n): classify(i, eligible, key, def, tie) marks element i `definite` (taken for sure) or a
 // `tie` (taken while ties last). Calls emit(i, rank) for every taken element with its rank in ascending position
 // order. Returns the number taken.
-template <bool CACHED, class KeyFn, class ClassFn, class EmitFn>
-__device__ int block_ordered_emit(int n, int ties_allowed, KeyFn key_of, const KeyCache& kc, ClassFn classify,
+template <bool CACHED, class KeyFn, class ClassFn, class EmitFn, int ITEMS>
+__device__ int block_ordered_emit(int n, int ties_allowed, KeyFn key_of, const KeyCache<ITEMS>& kc, ClassFn classify,
                                   EmitFn emit, SelectShared& sh, int def_base = 0, int tie_base = 0,
                                   int* def_total_out = nullptr, int* tie_total_out = nullptr) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -244,9 +253,99 @@ __device__ int block_ordered_emit(int n, int ties_allowed, KeyFn key_of, const K
 // The ordered pass for a unit split over CL CTAs (rank r owns a contiguous, ascending slice): a counting sweep
 // gives every CTA its (definite, tie) totals, the totals are exchanged through distributed shared memory, and the
 // emitting sweep starts from the sums of the lower ranks. Returns the number taken over the whole unit.
-template <bool CACHED, int CL, class KeyFn, class ClassFn, class EmitFn>
-__device__ int cluster_ordered_emit(int n, int ties_allowed, KeyFn key_of, const KeyCache& kc, ClassFn classify,
+// The ordered pass when the keys sit in registers (ITEMS chunks of kThreads elements, element tid + it*kThreads in
+// chunk it): one sweep classifies and records, per chunk and warp, the counts and ballots of definite and tie
+// elements; one block-wide exclusive scan over those (chunk-major = position order) gives every warp its base; a
+// second sweep emits. Three block barriers (and one cluster barrier for the totals of the lower ranks) instead of two
+// per chunk. classify is called exactly once per element.
+template <int CL, class ClassFn, class EmitFn, int ITEMS>
+__device__ int cached_ordered_emit(int n, int ties_allowed, const KeyCache<ITEMS>& kc, ClassFn classify, EmitFn emit,
+                                   SelectShared& sh) {
+  static_assert(ITEMS <= kItemsLong && ITEMS <= 32, "per-thread masks hold one bit per chunk");
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int chunks = (n + kThreads - 1) / kThreads;
+  uint32_t mdef = 0, mtie = 0;
+#pragma unroll
+  for (int it = 0; it < ITEMS; ++it) {
+    if (it < chunks) {
+      const int i = tid + it * kThreads;
+      bool def = false, tie = false;
+      if (i < n) classify(i, ((kc.elig >> it) & 1u) != 0, kc.key[it], def, tie);
+      const unsigned bd = __ballot_sync(0xffffffffu, def), bt = __ballot_sync(0xffffffffu, tie);
+      if (def) mdef |= 1u << it;
+      if (tie) mtie |= 1u << it;
+      if (lane == 0) {
+        sh.cnt[it * kWarps + warp] = (uint32_t)__popc(bd) | ((uint32_t)__popc(bt) << 16);
+        sh.bdef[it * kWarps + warp] = bd;
+        sh.btie[it * kWarps + warp] = bt;
+      }
+    }
+  }
+  __syncthreads();
+  // exclusive scan of the packed counts over the chunks * kWarps entries (entry tid belongs to thread tid)
+  static_assert(kItemsLong * kWarps <= kThreads, "one scan entry per thread");
+  const uint32_t mine = tid < chunks * kWarps ? sh.cnt[tid] : 0u;
+  uint32_t run = mine;
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const uint32_t o = __shfl_up_sync(0xffffffffu, run, off);
+    if (lane >= off) run += o;
+  }
+  if (lane == 31) sh.wtot[warp] = run;
+  __syncthreads();
+  uint32_t before = 0, all = 0;
+#pragma unroll
+  for (int w = 0; w < kWarps; ++w) {
+    const uint32_t t = sh.wtot[w];
+    if (w < warp) before += t;
+    all += t;
+  }
+  if (tid < chunks * kWarps) sh.cnt[tid] = before + run - mine;
+  int def_base = 0, tie_base = 0;
+  int def_all = (int)(all & 0xffffu), tie_all = (int)(all >> 16);
+  if (CL > 1) {
+    cg::cluster_group cluster = cg::this_cluster();
+    const int rank = (int)cluster.block_rank();
+    if (tid < CL) {
+      int* peer = cluster.map_shared_rank(&sh.totals[0][0], tid);
+      peer[rank * 2 + 0] = def_all;
+      peer[rank * 2 + 1] = tie_all;
+    }
+    cluster.sync();
+    def_all = 0;
+    tie_all = 0;
+#pragma unroll
+    for (int r = 0; r < CL; ++r) {
+      if (r < rank) {
+        def_base += sh.totals[r][0];
+        tie_base += sh.totals[r][1];
+      }
+      def_all += sh.totals[r][0];
+      tie_all += sh.totals[r][1];
+    }
+  } else {
+    __syncthreads();
+  }
+  const unsigned lt = (1u << lane) - 1u;
+#pragma unroll
+  for (int it = 0; it < ITEMS; ++it) {
+    if (it < chunks) {
+      const int e = it * kWarps + warp;
+      const uint32_t ex = sh.cnt[e];
+      const int def_before = def_base + (int)(ex & 0xffffu) + __popc(sh.bdef[e] & lt);
+      const int ties_seen = tie_base + (int)(ex >> 16) + __popc(sh.btie[e] & lt);
+      const int i = tid + it * kThreads;
+      if ((mdef >> it) & 1u) emit(i, def_before + min(ties_seen, ties_allowed));
+      else if (((mtie >> it) & 1u) && ties_seen < ties_allowed) emit(i, def_before + ties_seen);
+    }
+  }
+  return def_all + min(tie_all, ties_allowed);
+}
+
+template <bool CACHED, int CL, class KeyFn, class ClassFn, class EmitFn, int ITEMS>
+__device__ int cluster_ordered_emit(int n, int ties_allowed, KeyFn key_of, const KeyCache<ITEMS>& kc, ClassFn classify,
                                     EmitFn emit, SelectShared& sh) {
+  if constexpr (CACHED) return cached_ordered_emit<CL>(n, ties_allowed, kc, classify, emit, sh);
   if (CL == 1) return block_ordered_emit<CACHED>(n, ties_allowed, key_of, kc, classify, emit, sh);
   cg::cluster_group cluster = cg::this_cluster();
   const int rank = (int)cluster.block_rank();
@@ -309,7 +408,7 @@ __device__ __forceinline__ SeqInfo seq_info(const ta_seq_desc& seq, int b, int K
   return s;
 }
 
-template <bool CACHED, int CL>
+template <bool CACHED, int CL, int ITEMS = kItems>
 __global__ void __launch_bounds__(kThreads) ta_forced_kernel(ta_seq_desc seq, int K, int n_sink, int n_recent,
                                                              int k_protected, const float* __restrict__ voucher,
                                                              uint8_t* __restrict__ forced,
@@ -341,7 +440,7 @@ __global__ void __launch_bounds__(kThreads) ta_forced_kernel(ta_seq_desc seq, in
     key = sortable_key(v);
     return v > 0.0f && !mandatory(lo + il);
   };
-  KeyCache kc;
+  KeyCache<ITEMS> kc;
   if (CACHED) fill_cache(hi - lo, key_of, kc);
   const SelectResult r = block_radix_select<CACHED, CL>(hi - lo, s.p, key_of, kc, sh);
   uint8_t* f = forced + s.start + lo;
@@ -375,7 +474,7 @@ __device__ __forceinline__ float unit_utility(const UnitSrc& src, long long unit
 }
 
 // grid.x = units. scored: unit = (l*B + b)*Hkv + g; fast: unit = b.
-template <bool CACHED, int CL>
+template <bool CACHED, int CL, int ITEMS = kItems>
 __global__ void __launch_bounds__(kThreads) ta_select_kernel(ta_seq_desc seq, int n_layers, int Hkv, int K, int fast,
                                                              UnitSrc src, const uint8_t* __restrict__ forced,
                                                              const int32_t* __restrict__ r_main,
@@ -418,7 +517,7 @@ __global__ void __launch_bounds__(kThreads) ta_select_kernel(ta_seq_desc seq, in
     key = sortable_key(unit_utility(src, unit_off, (long long)start + lo + il));
     return f[il] == 0;
   };
-  KeyCache kc;
+  KeyCache<ITEMS> kc;
   if (CACHED) fill_cache(hi - lo, key_of, kc);
   const SelectResult r = block_radix_select<CACHED, CL>(hi - lo, want, key_of, kc, sh);
   auto classify = [&](int, bool elig, uint32_t key, bool& def, bool& tie) {
@@ -481,7 +580,7 @@ __global__ void ta_broadcast_heads_kernel(long long units_lb, int Hkv, int K, co
 // additionally idx_seq [B][K] and count_seq [B] (passed through a.idx / a.count by the caller when it wants the
 // per-sequence result only).
 // Sequences that fit kItems keys per thread run one CTA per unit with the keys in registers; longer ones are split
-// over a cluster of kSelectCluster CTAs (keys in registers up to kSelectCluster * kItems * kThreads elements).
+// over a cluster of kSelectCluster CTAs (keys in registers up to kSelectCluster * kItemsLong * kThreads elements).
 // Splitting pays only while the clusters of all units fit on the device about at once; with many units one CTA per
 // unit (keys re-read in batches when they do not fit in registers) keeps every SM busy without cluster barriers.
 bool split_units(int units, int max_n) {
@@ -525,6 +624,9 @@ cudaError_t ta_launch_forced(const ta_select_args& a, ta_dev_status* status, cud
   if (a.seq.max_n <= kSelectCluster * kItems * kThreads)
     return launch_clustered(ta_forced_kernel<true, kSelectCluster>, B, kSelectCluster, stream, a.seq, a.K, a.n_sink,
                             a.n_recent, a.k_protected, a.voucher, a.forced, a.r_main, status);
+  if (a.seq.max_n <= kSelectCluster * kItemsLong * kThreads)
+    return launch_clustered(ta_forced_kernel<true, kSelectCluster, kItemsLong>, B, kSelectCluster, stream, a.seq, a.K,
+                            a.n_sink, a.n_recent, a.k_protected, a.voucher, a.forced, a.r_main, status);
   return launch_clustered(ta_forced_kernel<false, kSelectCluster>, B, kSelectCluster, stream, a.seq, a.K, a.n_sink,
                           a.n_recent, a.k_protected, a.voucher, a.forced, a.r_main, status);
 }
@@ -548,6 +650,9 @@ cudaError_t ta_launch_select_units(const ta_select_args& a, cudaStream_t stream)
   if (a.seq.max_n <= kSelectCluster * kItems * kThreads)
     return launch_clustered(ta_select_kernel<true, kSelectCluster>, units, kSelectCluster, stream, a.seq, a.n_layers,
                             a.Hkv, a.K, a.fast, src, a.forced, a.r_main, a.idx, a.count);
+  if (a.seq.max_n <= kSelectCluster * kItemsLong * kThreads)
+    return launch_clustered(ta_select_kernel<true, kSelectCluster, kItemsLong>, units, kSelectCluster, stream, a.seq,
+                            a.n_layers, a.Hkv, a.K, a.fast, src, a.forced, a.r_main, a.idx, a.count);
   return launch_clustered(ta_select_kernel<false, kSelectCluster>, units, kSelectCluster, stream, a.seq, a.n_layers,
                           a.Hkv, a.K, a.fast, src, a.forced, a.r_main, a.idx, a.count);
 }
