@@ -618,6 +618,9 @@ cudaError_t ta_launch_forced(const ta_select_args& a, ta_dev_status* status, cud
   if (a.seq.max_n <= kItems * kThreads)
     return launch_clustered(ta_forced_kernel<true, 1>, B, 1, stream, a.seq, a.K, a.n_sink, a.n_recent, a.k_protected,
                             a.voucher, a.forced, a.r_main, status);
+  if (!split_units(B, a.seq.max_n) && a.seq.max_n <= kItemsLong * kThreads)
+    return launch_clustered(ta_forced_kernel<true, 1, kItemsLong>, B, 1, stream, a.seq, a.K, a.n_sink, a.n_recent,
+                            a.k_protected, a.voucher, a.forced, a.r_main, status);
   if (!split_units(B, a.seq.max_n))
     return launch_clustered(ta_forced_kernel<false, 1>, B, 1, stream, a.seq, a.K, a.n_sink, a.n_recent, a.k_protected,
                             a.voucher, a.forced, a.r_main, status);
@@ -644,6 +647,9 @@ cudaError_t ta_launch_select_units(const ta_select_args& a, cudaStream_t stream)
   if (a.seq.max_n <= kItems * kThreads)
     return launch_clustered(ta_select_kernel<true, 1>, units, 1, stream, a.seq, a.n_layers, a.Hkv, a.K, a.fast, src,
                             a.forced, a.r_main, a.idx, a.count);
+  if (!split_units(units, a.seq.max_n) && a.seq.max_n <= kItemsLong * kThreads)
+    return launch_clustered(ta_select_kernel<true, 1, kItemsLong>, units, 1, stream, a.seq, a.n_layers, a.Hkv, a.K, a.fast,
+                            src, a.forced, a.r_main, a.idx, a.count);
   if (!split_units(units, a.seq.max_n))
     return launch_clustered(ta_select_kernel<false, 1>, units, 1, stream, a.seq, a.n_layers, a.Hkv, a.K, a.fast, src,
                             a.forced, a.r_main, a.idx, a.count);
