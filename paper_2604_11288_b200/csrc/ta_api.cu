@@ -26,7 +26,7 @@ struct Carve {  // hands out aligned pieces of the context scratch
 };
 
 struct Layout {  // scratch layout of ta_compress (a superset of what the single-step entry points need)
-  size_t hist, flags, voucher, u_static, forced, r_main, idx_seq, count_seq, u, u_all, idx_lb, count_lb, end;
+  size_t hist, flags, voucher, u_static, forced, r_main, idx_seq, count_seq, u, u_all, idx_lb, count_lb, order, end;
 };
 
 Layout make_layout(const ta_batch& b, int Hkv, int K, const ta_policy& pol) {
@@ -52,6 +52,7 @@ Layout make_layout(const ta_batch& b, int Hkv, int K, const ta_policy& pol) {
   L.u_all = take(scored ? (size_t)b.n_layers * total * 4 : 0);
   L.idx_lb = take(scored ? (size_t)b.n_layers * B * K * 4 : 0);
   L.count_lb = take(scored ? (size_t)b.n_layers * B * 4 : 0);
+  L.order = take(scored && b.cu_seqlens ? (size_t)b.n_layers * B * Hkv * 4 : 0);  // unit order of the score kernel
   L.end = off;
   return L;
 }
@@ -439,6 +440,12 @@ ta_status ta_score(ta_ctx* ctx, const ta_policy* policy, const ta_batch* batch, 
   a.rho = policy->pension_rho;
   a.scale = policy->softmax_scale;
   a.causal = policy->causal;
+  // ragged batches: the unit order of the score kernel lives at the start of the context scratch when there is room
+  // (whatever ta_compress cached there is dropped)
+  if (batch->cu_seqlens && ctx->scratch_bytes >= (size_t)batch->n_layers * batch->batch * Hkv * 4) {
+    a.order_scratch = reinterpret_cast<int32_t*>(ctx->scratch);
+    ctx->cached_epoch = 0;
+  }
   cudaError_t e = ta_launch_score(ctx, a, ctx->d_status, (cudaStream_t)stream);
   return e == cudaSuccess ? TA_OK : cuda_fail(ctx, e);
 }
@@ -645,6 +652,7 @@ ta_status compress_impl(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* p
     a.scale = policy->softmax_scale;
     a.causal = policy->causal;
     a.reserve_sms = fork ? 4 : 0;
+    a.order_scratch = batch->cu_seqlens ? reinterpret_cast<int32_t*>(sc + L.order) : nullptr;
     e = ta_launch_score(ctx, a, ctx->d_status, stream);
   }
   mark(2);

@@ -94,6 +94,7 @@ struct ta_score_args {
   float alpha, delta, rho, scale;
   int causal;
   int reserve_sms;       // SMs left free for kernels running beside the (persistent) score kernel
+  int32_t* order_scratch; // nullable: n_layers*batch*Hkv ints; ragged batches then run longest sequences first
 };
 cudaError_t ta_launch_score(ta_ctx* ctx, const ta_score_args& a, ta_dev_status* status, cudaStream_t stream);
 
