@@ -481,6 +481,65 @@ def test_host_argument_checks():
         g.close()
 
 
+def test_host_argument_checks_of_the_widened_entry_points():
+    import ctypes as C
+    w = _workload([300], [[1, 2]], seed=1)
+    g = Gpu(w, oracle_policy(8), 8, 1)
+    gf = Gpu(w, oracle_policy(8, fast=True), 8, 1)
+    try:
+        L = ta.binding.lib()
+        t = w.total
+        buf = torch.zeros(max(t, 64) * 64, dtype=torch.float32, device="cuda")
+        p = buf.data_ptr()
+        conf = lambda thr, bud, span: L.ta_sponsor_mask_conf(g.ctx, C.byref(g.p), C.byref(g.batch), g.ids.data_ptr(), p,
+                                                            C.c_float(thr), C.c_float(bud), span, 0, p, p, p, None)
+        assert conf(0.5, 15.0, 0) == ta.TA_ERR_INVALID_ARG
+        assert conf(0.5, 15.0, 65) == ta.TA_ERR_UNSUPPORTED
+        assert conf(float("nan"), 15.0, 6) == ta.TA_ERR_INVALID_ARG
+        assert conf(0.5, 15.0, 6) == ta.TA_OK
+        # caller-supplied scores and the shared selection are scored-mode entry points
+        _, Kh, Vh = tw.make_qkv(w, [0], need_q=False)
+        Kd, Vd = Kh.cuda(), Vh.cuda()
+        vk, vv = ta.view(Kd, True), ta.view(Vd, True)
+        args = (g.ids.data_ptr(), p, None, vk, vv, 0, p, p, p, p, None)
+        assert L.ta_compress_scores(gf.ctx, gf.pats, C.byref(gf.p), C.byref(gf.batch), 2, 128, 8, *args) == ta.TA_ERR_INVALID_ARG
+        assert L.ta_compress_scores(g.ctx, g.pats, C.byref(g.p), C.byref(g.batch), 2, 128, 8, g.ids.data_ptr(), None,
+                                    None, vk, vv, 0, p, p, p, p, None) == ta.TA_ERR_INVALID_ARG
+        assert L.ta_compress_allheads(gf.ctx, gf.pats, C.byref(gf.p), C.byref(gf.batch), 8, 2, 128, 8,
+                                      g.ids.data_ptr(), vk, vk, vv, 0, p, p, p, p, None) == ta.TA_ERR_INVALID_ARG
+        # embedding detector: width, concept count, alignment
+        det = lambda D, Cn, ptr=p, stride=None: L.ta_detect_embedding(g.ctx, 10, ptr, D if stride is None else stride,
+                                                                      D, p, Cn, p, None)
+        assert det(48, 2) == ta.TA_ERR_UNSUPPORTED          # not a multiple of 32
+        assert det(16384, 2) == ta.TA_ERR_UNSUPPORTED
+        assert det(64, 9) == ta.TA_ERR_UNSUPPORTED
+        assert det(64, 0) == ta.TA_ERR_INVALID_ARG
+        assert det(64, 2, p + 2) == ta.TA_ERR_ALIGNMENT
+        assert det(64, 2, p, 60) == ta.TA_ERR_INVALID_ARG   # stride shorter than a row
+        # decode step: state description and scratch
+        st = ta.ta_stream()
+        st.n_layers, st.batch, st.Hkv, st.K, st.cache_len = 1, 1, 2, 8, 0
+        for k in ("pos", "slot", "tok", "A", "P", "V", "S", "next_slot", "n_seen", "hist", "tok_ring", "anc_B", "anc_L"):
+            setattr(st, k, p)
+        step = lambda: L.ta_stream_step(g.ctx, g.pats, C.byref(g.p), C.byref(st), p, p, p, None)
+        st.cache_len = 9
+        assert step() == ta.TA_ERR_INVALID_ARG
+        st.cache_len, st.K = 0, 5000
+        assert step() == ta.TA_ERR_UNSUPPORTED
+        st.K, st.hist = 8, None
+        assert step() == ta.TA_ERR_INVALID_ARG
+        st.hist = p
+        small = ta.ta_ctx_create(0, 64)
+        assert L.ta_stream_step(small, g.pats, C.byref(g.p), C.byref(st), p, p, p, None) == ta.TA_ERR_SCRATCH_TOO_SMALL
+        ta.ta_ctx_destroy(small)
+        assert st.cache_len == 0  # refused calls leave the state description alone
+        torch.cuda.synchronize()
+        assert g.poll() == ta.TA_OK
+    finally:
+        g.close()
+        gf.close()
+
+
 @pytest.mark.parametrize("fast", [False, True])
 @pytest.mark.parametrize("pinned", [True, False])
 def test_compress_host_matches_device_path(fast, pinned):
