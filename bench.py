@@ -392,7 +392,7 @@ def measure_variants(dev, steps=10, warmup=3):
         ms = e0.elapsed_time(e1) / n_timed
         state_bytes = U * C_ * (3 * 4 + 3 * 4 + 1) * 2 + U * C_ * 4  # ordered state read + written, attention read
         out.append({"entry": "ta_stream_step", "workload": f"{Ls} layers x {Bs} sequences x {Hs} KV heads, K={Ks}, "
-                    "steady state (one eviction per unit and step)", "ms_per_step": ms, "kernels_per_step": 5,
+                    "steady state (one eviction per unit and step)", "ms_per_step": ms, "kernels_per_step": 2,
                     "unit_steps_per_s": U / (ms * 1e-3), "state_GBps": state_bytes / (ms * 1e-3) / 1e9})
         if ta.ta_ctx_poll(ctx) != 0:
             out[-1]["error"] = "device status"

@@ -723,27 +723,12 @@ ta_status ta_compress_scores(ta_ctx* ctx, const ta_patterns* pats, const ta_poli
 // ---------------------------------------------------------------------------------------------- decode loop
 namespace {
 struct StreamLayout {
-  size_t info, u_att, u_static, vbuf, flagbuf, forced, r_main, idx, count, end;
+  size_t info, end;
 };
 StreamLayout stream_layout(const ta_stream& st) {
   StreamLayout L;
-  size_t off = 0;
-  auto take = [&](size_t bytes) {
-    const size_t o = off;
-    off += align_up(bytes);
-    return o;
-  };
-  const size_t U = (size_t)st.n_layers * st.batch * st.Hkv, C = (size_t)st.K + 1;
-  L.info = take((size_t)st.batch * sizeof(ta_stream_seq_info));
-  L.u_att = take(U * C * 4);
-  L.u_static = take(U * C * 4);
-  L.vbuf = take(U * C * 4);
-  L.flagbuf = take(U * C);
-  L.forced = take(U * C);
-  L.r_main = take(U * 4);
-  L.idx = take(U * st.K * 4);
-  L.count = take(U * 4);
-  L.end = off;
+  L.info = 0;
+  L.end = align_up((size_t)st.batch * sizeof(ta_stream_seq_info));
   return L;
 }
 ta_status check_stream(const ta_stream* st) {
@@ -799,44 +784,10 @@ ta_status ta_stream_step(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* 
   d.anc_B = st->anc_B;
   d.anc_L = st->anc_L;
   auto* info = reinterpret_cast<ta_stream_seq_info*>(sc + L.info);
-  float* u_att = reinterpret_cast<float*>(sc + L.u_att);
-  float* u_static = reinterpret_cast<float*>(sc + L.u_static);
-  float* vbuf = reinterpret_cast<float*>(sc + L.vbuf);
-  int32_t* idx = reinterpret_cast<int32_t*>(sc + L.idx);
-  const int U = st->n_layers * st->batch * st->Hkv, C = st->K + 1;
   const bool evict = st->cache_len + 1 > st->K;
 
   cudaError_t e = ta_launch_stream_seq(d, pats, *policy, new_ids, info, ctx->d_status, stream);
-  if (e == cudaSuccess)
-    e = ta_launch_stream_unit(d, *policy, info, attn, u_att, u_static, vbuf, sc + L.flagbuf, ctx->d_status, stream);
-  if (e == cudaSuccess && evict) {
-    // every unit is a "sequence" of K+1 tokens in position order; one layer, one head
-    ta_select_args sel = {};
-    sel.seq.cu = nullptr;
-    sel.seq.n_uniform = C;
-    sel.seq.batch = U;
-    sel.seq.max_n = C;
-    sel.seq.total = (long long)U * C;
-    sel.n_layers = 1;
-    sel.Hkv = 1;
-    sel.K = st->K;
-    sel.n_sink = policy->n_sink;
-    sel.n_recent = policy->n_recent;
-    sel.k_protected = policy->k_protected;
-    sel.fast = 0;
-    sel.alpha = policy->alpha;
-    sel.delta = policy->delta;
-    sel.flags = sc + L.flagbuf;
-    sel.voucher = vbuf;
-    sel.u_static = u_static;
-    sel.u = u_att;
-    sel.forced = sc + L.forced;
-    sel.r_main = reinterpret_cast<int32_t*>(sc + L.r_main);
-    sel.idx = idx;
-    sel.count = reinterpret_cast<int32_t*>(sc + L.count);
-    e = ta_launch_select(sel, ctx->d_status, stream);
-  }
-  if (e == cudaSuccess) e = ta_launch_stream_evict(d, evict ? 1 : 0, idx, policy->budget_decay, evicted_pos, stream);
+  if (e == cudaSuccess) e = ta_launch_stream_step(d, *policy, info, attn, evicted_pos, ctx->d_status, stream);
   if (e != cudaSuccess) return cuda_fail(ctx, e);
   st->cache_len = evict ? st->K : st->cache_len + 1;
   return TA_OK;

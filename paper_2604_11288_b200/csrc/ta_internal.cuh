@@ -147,11 +147,9 @@ struct ta_stream_seq_info {  // per sequence, written by the sequence kernel of 
 cudaError_t ta_launch_stream_seq(const ta_stream_dev& st, const ta_patterns* pats, const ta_policy& pol,
                                  const int32_t* new_ids, ta_stream_seq_info* info, ta_dev_status* status,
                                  cudaStream_t stream);
-cudaError_t ta_launch_stream_unit(const ta_stream_dev& st, const ta_policy& pol, const ta_stream_seq_info* info,
-                                  const float* attn, float* u_att, float* u_static, float* vbuf, uint8_t* flagbuf,
-                                  ta_dev_status* status, cudaStream_t stream);
-cudaError_t ta_launch_stream_evict(const ta_stream_dev& st, int evict, const int32_t* idx, float budget_decay,
-                                   int32_t* evicted_pos, cudaStream_t stream);
+cudaError_t ta_launch_stream_step(const ta_stream_dev& st, const ta_policy& pol, const ta_stream_seq_info* info,
+                                  const float* attn, int32_t* evicted_pos, ta_dev_status* status,
+                                  cudaStream_t stream);
 
 // ---- step 4 ------------------------------------------------------------------------------------------------
 struct ta_compact_args {

@@ -1,23 +1,20 @@
 // Algorithm 1 in the decode loop: one new token per sequence and step, at most K cached tokens per unit afterwards.
 // (Section 3.1: a retention policy selects S, |S| <= K, "after each generation step"; Algorithm 1 steps 1-10.)
 //
-// Per step three small kernels run around the selection kernels of ta_select.cu:
+// Per step two kernels run:
 //   ta_stream_seq_kernel    one warp per sequence: token histogram, pattern match ending at the new token (longest
 //                           pattern wins, then the lowest index), the new token's voucher from the anchors of the last
 //                           TA_MAX_SPAN positions (Eq. 2 with budgets that decayed once per step since detection)
-//   ta_stream_unit_kernel   one block per unit: appends the new token to the position-ordered state, adds this step's
-//                           attention mass to A, updates the pension average P, and writes the two parts of the utility
-//                           of Eq. 1 for the K+1 cached tokens
-//   (selection of K of the K+1 tokens: ta_forced_kernel + ta_select_kernel, each unit taken as a sequence of K+1 tokens)
-//   ta_stream_evict_kernel  one block per unit: removes the evicted token from the ordered state (4-byte entries move;
-//                           key/value rows never do: the freed cache row is handed to the next token), then decays
-//                           every voucher by budget_decay (Algorithm 1 step 10)
+//   ta_stream_step_kernel   one block per unit with the unit's K+1 entries in shared memory: appends the new token to
+//                           the position-ordered state, adds this step's attention mass to A, updates the pension
+//                           average P, forms the utility of Eq. 1, applies the budget partition of Section 3.3 to the
+//                           K+1 cached tokens (exactly one token loses), removes it from the ordered state (4-byte
+//                           entries move; key/value rows never do: the freed cache row is handed to the next token) and
+//                           decays every voucher by budget_decay (Algorithm 1 step 10)
 // All arithmetic that decides the selection is fp32 with one rounding per operation, in the order the CPU oracle uses.
 #include "ta_internal.cuh"
 
 namespace {
-
-constexpr int kUnitThreads = 256;
 
 __device__ __forceinline__ void report(ta_dev_status* st, int code, int where, int d0, int d1) {
   if (atomicCAS(&st->code, 0, code) == 0) {
@@ -94,123 +91,216 @@ __global__ void __launch_bounds__(32) ta_stream_seq_kernel(ta_stream_dev st, con
   }
 }
 
-__global__ void __launch_bounds__(kUnitThreads)
-ta_stream_unit_kernel(ta_stream_dev st, const ta_stream_seq_info* __restrict__ info, const float* __restrict__ attn,
-                      int vocab, float alpha, float beta, float gamma, float delta, float lambda, float rho,
-                      float* __restrict__ u_att, float* __restrict__ u_static, float* __restrict__ vbuf,
-                      uint8_t* __restrict__ flagbuf, ta_dev_status* status) {
-  const int u = blockIdx.x;
+__device__ __forceinline__ uint32_t sortable_key(float f) {
+  uint32_t b = __float_as_uint(f);
+  if ((b << 1) == 0u) b = 0u;  // -0 == +0
+  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+
+// One block per unit; the unit's K+1 entries live in shared memory for the whole step. Thread t owns the contiguous
+// entries [t*per, (t+1)*per), so everything that depends on position order is a block-wide scan of per-thread counts.
+// Selection (Section 3.3 on the K+1 cached tokens): mandatory sinks and recents; the protected pool = the sponsored,
+// non-mandatory tokens with the largest vouchers (lower position first among equals), found with a 4-pass radix
+// select on the voucher keys when there are more candidates than protected slots; exactly one token is then not
+// forced and loses: the one with the smallest utility, the latest position among equals.
+__global__ void ta_stream_step_kernel(ta_stream_dev st, const ta_stream_seq_info* __restrict__ info,
+                                      const float* __restrict__ attn, int vocab, float alpha, float beta, float gamma,
+                                      float delta, float lambda, float rho, float budget_decay, int n_sink,
+                                      int n_recent, int k_protected, int32_t* __restrict__ evicted_pos,
+                                      ta_dev_status* status) {
+  extern __shared__ __align__(16) unsigned char smem[];
+  const int u = blockIdx.x, tid = threadIdx.x, nt = blockDim.x;
   const int b = (u / st.Hkv) % st.B;
-  const int C = st.K + 1, len = st.len;
+  const int K = st.K, C = K + 1, len = st.len, n = len + 1;
   const size_t base = (size_t)u * C;
+  int32_t* s_pos = reinterpret_cast<int32_t*>(smem);
+  int32_t* s_slot = s_pos + C;
+  int32_t* s_tok = s_slot + C;
+  float* s_A = reinterpret_cast<float*>(s_tok + C);
+  float* s_P = s_A + C;
+  float* s_V = s_P + C;
+  uint32_t* s_ku = reinterpret_cast<uint32_t*>(s_V + C);  // sortable key of the utility
+  uint8_t* s_S = reinterpret_cast<uint8_t*>(s_ku + C);
+  uint8_t* s_forced = s_S + C;
+  __shared__ uint32_t hist[256];
+  __shared__ uint32_t scan[512];
+  __shared__ unsigned long long best;
+  __shared__ uint32_t sel_prefix, sel_mask;
+  __shared__ int sel_remaining, cand_total;
+
   const ta_stream_seq_info si = info[b];
   const int t = si.t;
   const float nf = (float)(t + 1);
   const float omr = __fsub_rn(1.0f, rho);
-  for (int r = threadIdx.x; r < C; r += kUnitThreads) {
-    float vu = 0.0f, us = 0.0f, vv = 0.0f;
-    uint8_t fl = 0;
-    if (r <= len) {
-      int p, row, id;
-      float A, P, V;
-      int S;
-      if (r < len) {
-        p = st.pos[base + r];
-        row = st.slot[base + r];
-        id = st.tok[base + r];
-        A = st.A[base + r];
-        P = st.P[base + r];
-        V = st.V[base + r];
-        S = st.S[base + r];
-      } else {
-        p = t;
-        row = st.next_slot[u];
-        id = si.id;
-        A = 0.0f;
-        P = 0.0f;
-        V = si.v_new;
-        S = 0;
-        st.pos[base + r] = p;
-        st.slot[base + r] = row;
-        st.tok[base + r] = id;
-        st.V[base + r] = V;
-      }
-      float a = 0.0f;
-      if (row >= 0 && row < C) a = attn[base + row];
-      else report(status, TA_ERR_DEVICE_BOUNDS, 6, u, row);
-      A = __fadd_rn(A, a);
-      P = __fadd_rn(__fmul_rn(rho, P), __fmul_rn(omr, a));
-      if (p >= t - si.match_len + 1) S = 1;
-      st.A[base + r] = A;
-      st.P[base + r] = P;
-      st.S[base + r] = (uint8_t)S;
-      const int c = (id >= 0 && id < vocab) ? st.hist[(size_t)b * vocab + id] : 0;
-      const float R = __fdiv_rn((float)(p + 1), nf);
-      const float F = __fdiv_rn((float)c, nf);
-      const float t0 = __fadd_rn(__fmul_rn(beta, R), __fmul_rn(gamma, S ? 1.0f : 0.0f));
-      const float t1 = __fsub_rn(t0, __fmul_rn(lambda, F));
-      us = __fadd_rn(t1, V);
-      vu = __fadd_rn(__fmul_rn(alpha, A), __fmul_rn(delta, P));
-      vv = V;
-      fl = (uint8_t)((S ? TA_FLAG_ANCHOR_TOKEN : 0) | (V > 0.0f ? TA_FLAG_SPONSORED : 0));
+  // ---- append, attention update, utility
+  for (int r = tid; r < n; r += nt) {
+    int p, row, id, S;
+    float A, P, V;
+    if (r < len) {
+      p = st.pos[base + r];
+      row = st.slot[base + r];
+      id = st.tok[base + r];
+      A = st.A[base + r];
+      P = st.P[base + r];
+      V = st.V[base + r];
+      S = st.S[base + r];
+    } else {
+      p = t;
+      row = st.next_slot[u];
+      id = si.id;
+      A = 0.0f;
+      P = 0.0f;
+      V = si.v_new;
+      S = 0;
     }
-    u_att[base + r] = vu;
-    u_static[base + r] = us;
-    vbuf[base + r] = vv;
-    flagbuf[base + r] = fl;
-  }
-}
-
-// Moves entries (from, to] of one per-unit array down by one, 256 at a time in ascending order: a chunk is read by
-// all threads before any of them writes it one place lower.
-template <class T>
-__device__ __forceinline__ void shift_down(T* a, int from, int to) {
-  for (int r0 = from + 1; r0 <= to; r0 += kUnitThreads) {
-    const int r = r0 + threadIdx.x;
-    T v = T();
-    if (r <= to) v = a[r];
-    __syncthreads();
-    if (r <= to) a[r - 1] = v;
-    __syncthreads();
-  }
-}
-
-__global__ void __launch_bounds__(kUnitThreads)
-ta_stream_evict_kernel(ta_stream_dev st, int evict, const int32_t* __restrict__ idx, float budget_decay,
-                       int32_t* __restrict__ evicted_pos) {
-  __shared__ int e_sh;
-  const int u = blockIdx.x;
-  const int C = st.K + 1, K = st.K, len = st.len;  // len + 1 tokens are cached when this kernel starts
-  const size_t base = (size_t)u * C;
-  int kept = len + 1;
-  if (evict) {
-    if (threadIdx.x == 0) e_sh = K;  // all of idx[0..K) in place: the last entry goes
-    __syncthreads();
-    for (int r = threadIdx.x; r < K; r += kUnitThreads)
-      if (idx[(size_t)u * K + r] != r) atomicMin(&e_sh, r);
-    __syncthreads();
-    const int e = e_sh;
-    const int freed = st.slot[base + e];
-    const int gone = st.pos[base + e];
-    __syncthreads();
-    shift_down(st.pos + base, e, K);
-    shift_down(st.slot + base, e, K);
-    shift_down(st.tok + base, e, K);
-    shift_down(st.A + base, e, K);
-    shift_down(st.P + base, e, K);
-    shift_down(st.V + base, e, K);
-    shift_down(st.S + base, e, K);
-    if (threadIdx.x == 0) {
-      st.next_slot[u] = freed;
-      evicted_pos[u] = gone;
-    }
-    kept = K;
-  } else if (threadIdx.x == 0) {
-    st.next_slot[u] = len + 1;  // rows fill up in order until the cache is full
-    evicted_pos[u] = -1;
+    float a = 0.0f;
+    if (row >= 0 && row < C) a = attn[base + row];
+    else report(status, TA_ERR_DEVICE_BOUNDS, 6, u, row);
+    A = __fadd_rn(A, a);
+    P = __fadd_rn(__fmul_rn(rho, P), __fmul_rn(omr, a));
+    if (p >= t - si.match_len + 1) S = 1;
+    const int c = (id >= 0 && id < vocab) ? st.hist[(size_t)b * vocab + id] : 0;
+    const float R = __fdiv_rn((float)(p + 1), nf);
+    const float F = __fdiv_rn((float)c, nf);
+    const float t0 = __fadd_rn(__fmul_rn(beta, R), __fmul_rn(gamma, S ? 1.0f : 0.0f));
+    const float t1 = __fsub_rn(t0, __fmul_rn(lambda, F));
+    const float us = __fadd_rn(t1, V);
+    const float ua = __fadd_rn(__fmul_rn(alpha, A), __fmul_rn(delta, P));
+    s_pos[r] = p;
+    s_slot[r] = row;
+    s_tok[r] = id;
+    s_A[r] = A;
+    s_P[r] = P;
+    s_V[r] = V;
+    s_S[r] = (uint8_t)S;
+    s_ku[r] = sortable_key(__fadd_rn(ua, us));
   }
   __syncthreads();
-  for (int r = threadIdx.x; r < kept; r += kUnitThreads) st.V[base + r] = __fmul_rn(st.V[base + r], budget_decay);
+  int e = -1;  // entry to evict
+  if (n > K) {
+    // ---- budget partition on n = K + 1 tokens
+    int p = k_protected < 0 ? K - n_sink - n_recent : k_protected;
+    p = max(0, min(p, K));
+    const int K_main = K - p;
+    const int sinks = min(n_sink, n);
+    const int recents = max(0, min(n_recent, n - sinks));
+    const int s_take = min(sinks, K_main);
+    const int r_take = min(recents, K_main - s_take);
+    auto mandatory = [&](int i) { return i < s_take || i >= n - r_take; };
+    const int per = (n + nt - 1) / nt;
+    const int lo = min(n, tid * per), hi = min(n, lo + per);
+    // candidates of the protected pool
+    int my_c = 0;
+    for (int i = lo; i < hi; ++i) my_c += (s_V[i] > 0.0f && !mandatory(i));
+    if (tid == 0) cand_total = 0;
+    __syncthreads();
+    if (my_c) atomicAdd(&cand_total, my_c);
+    __syncthreads();
+    const int cs = cand_total;
+    uint32_t thresh = 0;
+    int ties = 0;
+    const bool all_protected = cs <= p;
+    if (!all_protected && p > 0) {
+      if (tid == 0) {
+        sel_prefix = 0;
+        sel_mask = 0;
+        sel_remaining = p;
+      }
+      for (int pass = 0; pass < 4; ++pass) {
+        const int shift = 24 - 8 * pass;
+        for (int k = tid; k < 256; k += nt) hist[k] = 0;
+        __syncthreads();
+        const uint32_t prefix = sel_prefix, mask = sel_mask;
+        for (int i = lo; i < hi; ++i) {
+          const float v = s_V[i];
+          if (v > 0.0f && !mandatory(i)) {
+            const uint32_t key = sortable_key(v);
+            if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+          }
+        }
+        __syncthreads();
+        if (tid == 0) {
+          int remaining = sel_remaining;
+          uint32_t cum = 0;
+          int bin = 255;
+          for (; bin > 0; --bin) {
+            if (cum + hist[bin] >= (uint32_t)remaining) break;
+            cum += hist[bin];
+          }
+          sel_remaining = remaining - (int)cum;
+          sel_prefix = prefix | ((uint32_t)bin << shift);
+          sel_mask = mask | (255u << shift);
+        }
+        __syncthreads();
+      }
+      thresh = sel_prefix;
+      ties = sel_remaining;
+    }
+    // ---- forced set: mandatory, vouchers above the threshold, and the first `ties` of the vouchers equal to it
+    int my_ties = 0;
+    for (int i = lo; i < hi; ++i) {
+      const float v = s_V[i];
+      const bool cand = v > 0.0f && !mandatory(i);
+      bool f = mandatory(i);
+      if (cand && p > 0) {
+        if (all_protected) f = true;
+        else {
+          const uint32_t key = sortable_key(v);
+          if (key > thresh) f = true;
+          else if (key == thresh) ++my_ties;
+        }
+      }
+      s_forced[i] = f ? 1 : 0;
+    }
+    if (!all_protected && p > 0) {
+      // exclusive scan of the per-thread tie counts (thread order = position order)
+      scan[tid] = (uint32_t)my_ties;
+      __syncthreads();
+      for (int off = 1; off < nt; off <<= 1) {
+        const uint32_t add = tid >= off ? scan[tid - off] : 0u;
+        __syncthreads();
+        scan[tid] += add;
+        __syncthreads();
+      }
+      int seen = (int)scan[tid] - my_ties;
+      for (int i = lo; i < hi; ++i) {
+        const float v = s_V[i];
+        if (v > 0.0f && !mandatory(i) && sortable_key(v) == thresh) {
+          if (seen < ties) s_forced[i] = 1;
+          ++seen;
+        }
+      }
+    }
+    if (tid == 0) best = ~0ull;
+    __syncthreads();
+    // ---- the loser: smallest utility among the tokens that are not forced, latest position among equals
+    unsigned long long mine = ~0ull;
+    for (int i = lo; i < hi; ++i)
+      if (!s_forced[i]) {
+        const unsigned long long cnd = ((unsigned long long)s_ku[i] << 32) | (uint32_t)(~(uint32_t)i);
+        mine = cnd < mine ? cnd : mine;
+      }
+    if (mine != ~0ull) atomicMin(&best, mine);
+    __syncthreads();
+    e = (int)(~(uint32_t)(best & 0xffffffffull));
+    if (best == ~0ull) e = K;  // cannot happen: K + 1 tokens and at most K forced
+  }
+  // ---- write the state back without the evicted entry; vouchers decay (Algorithm 1 step 10)
+  const int kept = e >= 0 ? K : n;
+  for (int r = tid; r < kept; r += nt) {
+    const int src = (e >= 0 && r >= e) ? r + 1 : r;
+    st.pos[base + r] = s_pos[src];
+    st.slot[base + r] = s_slot[src];
+    st.tok[base + r] = s_tok[src];
+    st.A[base + r] = s_A[src];
+    st.P[base + r] = s_P[src];
+    st.V[base + r] = __fmul_rn(s_V[src], budget_decay);
+    st.S[base + r] = s_S[src];
+  }
+  if (tid == 0) {
+    st.next_slot[u] = e >= 0 ? s_slot[e] : n;  // rows fill up in order until the cache is full
+    evicted_pos[u] = e >= 0 ? s_pos[e] : -1;
+  }
 }
 
 }  // namespace
@@ -224,19 +314,23 @@ cudaError_t ta_launch_stream_seq(const ta_stream_dev& st, const ta_patterns* pat
   return cudaGetLastError();
 }
 
-cudaError_t ta_launch_stream_unit(const ta_stream_dev& st, const ta_policy& pol, const ta_stream_seq_info* info,
-                                  const float* attn, float* u_att, float* u_static, float* vbuf, uint8_t* flagbuf,
-                                  ta_dev_status* status, cudaStream_t stream) {
-  const int U = st.n_layers * st.B * st.Hkv;
-  ta_stream_unit_kernel<<<U, kUnitThreads, 0, stream>>>(st, info, attn, pol.vocab_size, pol.alpha, pol.beta, pol.gamma,
-                                                       pol.delta, pol.lambda, pol.pension_rho, u_att, u_static, vbuf,
-                                                       flagbuf, status);
-  return cudaGetLastError();
-}
-
-cudaError_t ta_launch_stream_evict(const ta_stream_dev& st, int evict, const int32_t* idx, float budget_decay,
-                                   int32_t* evicted_pos, cudaStream_t stream) {
-  const int U = st.n_layers * st.B * st.Hkv;
-  ta_stream_evict_kernel<<<U, kUnitThreads, 0, stream>>>(st, evict, idx, budget_decay, evicted_pos);
+cudaError_t ta_launch_stream_step(const ta_stream_dev& st, const ta_policy& pol, const ta_stream_seq_info* info,
+                                  const float* attn, int32_t* evicted_pos, ta_dev_status* status,
+                                  cudaStream_t stream) {
+  const int U = st.n_layers * st.B * st.Hkv, C = st.K + 1;
+  const int threads = C <= 512 ? 128 : 512;
+  const size_t smem = (size_t)C * (7 * 4 + 2) + 16;
+  static bool attr_set[64] = {};
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (!attr_set[dev & 63]) {
+    e = cudaFuncSetAttribute(ta_stream_step_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
+    if (e != cudaSuccess) return e;
+    attr_set[dev & 63] = true;
+  }
+  ta_stream_step_kernel<<<U, threads, smem, stream>>>(st, info, attn, pol.vocab_size, pol.alpha, pol.beta, pol.gamma,
+                                                      pol.delta, pol.lambda, pol.pension_rho, pol.budget_decay,
+                                                      pol.n_sink, pol.n_recent, pol.k_protected, evicted_pos, status);
   return cudaGetLastError();
 }
