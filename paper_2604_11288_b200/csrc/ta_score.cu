@@ -357,23 +357,34 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
       const int Wp = min(p.W, n);
 
       if (p.two_pass) {
-        // ---- pass 1: per row, sum of exp2(s*c - ref) against a reference `ref` that trails the running maximum:
-        // the exponentials of a chunk use the reference left by the previous chunks, so they do not wait for the
-        // chunk's own maximum; only when the maximum jumps by more than 2^8 is the chunk redone with a new reference.
+        // ---- pass 1: per row, sum of exp2(s*c - ref) against a reference `ref` that only has to keep the sum inside
+        // the fp32 range (the result does not depend on it). Two forms, chosen by what measured faster:
+        //  * one row block per job (MB 1): ref is the largest of the first 16 keys the row sees; after that a key
+        //    costs one multiply-add, one ex2 and one add, and no maximum is tracked. A tile whose sum leaves the safe
+        //    range (a score more than 2^60 above ref) is redone against its own maximum. That check must not wait
+        //    for the tile's last exponentials (the accumulator stage is released right after it, and the group's next
+        //    product waits for the release): it uses the sum without the last 16 keys and, for those, their largest
+        //    score.
+        //  * two row blocks per job (MB 2; there the form above came out 6-10 % slower, with the redo path merely
+        //    present): ref trails the running maximum; the exponentials of a tile use the reference left by the
+        //    previous tiles, and only when the tile's maximum is more than 2^8 ahead of it is the tile redone.
         float ref_c[MB], z_run[MB];
         int lim_row[MB];
 #pragma unroll
         for (int mb = 0; mb < MB; ++mb) {
-          ref_c[mb] = -1e30f;
           z_run[mb] = 0.0f;
           const int pos = n - p.W + my_t[mb];
           lim_row[mb] = (my_t[mb] >= 0 && pos >= 0) ? (p.causal ? pos : n - 1) : -1;
+          // rows that see no key (padding) get a reference that turns every exponential into 0
+          ref_c[mb] = lim_row[mb] >= 0 ? -1e30f : 1e30f;
         }
-        // 16 keys of one row (half of a 32-key chunk): adds exp2(s*c - rc) to `sum`, tracks the largest s*c.
-        // Masked tiles (cold) drop keys beyond `lim`.
-        auto half1 = [&](auto masked_tag, const float(&cur)[16], float rc, float& sum, float& mx, int kbase,
-                         int lim) {
+        constexpr float kSumLimit = 1.0e18f;  // about 2^60
+        // 16 keys of one row (half of a 32-key chunk): adds exp2(s*c - rc) to `sum`; with `track_tag` set also
+        // tracks the largest s in `mx`. Masked tiles (cold) drop keys beyond `lim`.
+        auto half1 = [&](auto masked_tag, auto track_tag, const float(&cur)[16], float rc, float& sum, float& mx,
+                         int kbase, int lim) {
           constexpr bool masked = decltype(masked_tag)::value;
+          constexpr bool track = decltype(track_tag)::value;
           float v[16];
 #pragma unroll
           for (int q = 0; q < 16; ++q) v[q] = cur[q];
@@ -390,11 +401,26 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             a2 += ex2(fmaf(v[q + 2], c, -rc));
             a3 += ex2(fmaf(v[q + 3], c, -rc));
           }
+          if (track) {
+            float t4[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) t4[q] = fmaxf(fmaxf(v[4 * q], v[4 * q + 1]), fmaxf(v[4 * q + 2], v[4 * q + 3]));
+            mx = fmaxf(mx, fmaxf(fmaxf(t4[0], t4[1]), fmaxf(t4[2], t4[3])));
+          }
+          sum += (a0 + a1) + (a2 + a3);
+        };
+        // largest of 16 keys of one row
+        auto max16 = [&](auto masked_tag, const float(&cur)[16], float& mx, int kbase, int lim) {
+          constexpr bool masked = decltype(masked_tag)::value;
           float t4[4];
 #pragma unroll
-          for (int q = 0; q < 4; ++q) t4[q] = fmaxf(fmaxf(v[4 * q], v[4 * q + 1]), fmaxf(v[4 * q + 2], v[4 * q + 3]));
+          for (int q = 0; q < 4; ++q) {
+            float w[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) w[e] = (masked && kbase + 4 * q + e > lim) ? -INFINITY : cur[4 * q + e];
+            t4[q] = fmaxf(fmaxf(w[0], w[1]), fmaxf(w[2], w[3]));
+          }
           mx = fmaxf(mx, fmaxf(fmaxf(t4[0], t4[1]), fmaxf(t4[2], t4[3])));
-          sum += (a0 + a1) + (a2 + a3);
         };
         float ra[16], rb[16];
         int j = (grp - jg % NG + NG) % NG;  // first job of this pass that belongs to the group
@@ -404,53 +430,115 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         }
         // One job: the accumulator in 32-column chunks, each fetched as two 16-column loads (ra, rb) so that one
         // load is always in flight; the next job's first load is issued before the last half-chunk is computed.
-        // The exponentials of the whole tile use the reference left by the previous tiles; only after the tile is
-        // it checked whether its maximum ran more than 2^8 ahead of that reference, in which case the tile is
-        // read again (the accumulator stage is released after the check) with its own maximum as the new reference.
+        // On entry of every row block the load of its first 16 columns is in flight in `ra`.
         auto job1 = [&](auto masked_tag, int j) {
           const int jj = jg + j;
           const int key0 = (ui.t_begin + j) * kTileN;
           const uint32_t abase = acc_addr(jj);
 #pragma unroll
           for (int mb = 0; mb < MB; ++mb) {
-            const int lim = lim_row[mb];
-            const float rc = ref_c[mb];
-            float sum = 0.0f, mx = -INFINITY;
-#pragma unroll 1
-            for (int c4 = 0; c4 < 4; ++c4) {
-              const uint32_t col = (uint32_t)(mb * 128 + c4 * 32);
-              tmem_ld_wait(ra);
-              tmem_ld16_issue(abase + col + 16, rb);
-              half1(masked_tag, ra, rc, sum, mx, key0 + c4 * 32, lim);
-              tmem_ld_wait(rb);
-              if (mb == MB - 1 && c4 == 3) {
-                // with more than one stage per group the next job's accumulator is a different stage: fetch ahead
-                if (kAhead && j + NG < T) {
-                  wait_full(jj + NG, 30);
-                  tmem_ld16_issue(acc_addr(jj + NG), ra);
+            if constexpr (MB == 1) {
+              const int lim = lim_row[mb];
+              float rc = ref_c[mb];
+              const bool first = rc < -1e29f;
+              if (__any_sync(0xffffffffu, first)) {  // the row has no reference yet: take it from the 16 keys in flight
+                float mx = -INFINITY;
+                tmem_ld_wait(ra);
+                max16(masked_tag, ra, mx, key0, lim);
+                if (first && mx > -INFINITY) {
+                  rc = mx * c;
+                  ref_c[mb] = rc;
                 }
-              } else {
-                tmem_ld16_issue(abase + col + 32, ra);
               }
-              half1(masked_tag, rb, rc, sum, mx, key0 + c4 * 32 + 16, lim);
-            }
-            const float mx_c = mx * c;
-            const bool jump = mx_c > rc + 8.0f;
-            if (__any_sync(0xffffffffu, jump)) {  // rare: first tiles of a unit, or a score far above all before
-              float sum2 = 0.0f, mx2 = -INFINITY;
+              float sum = 0.0f, sum_head = 0.0f, mx_tail = -INFINITY, unused = 0.0f;
 #pragma unroll 1
-              for (int h = 0; h < 8; ++h) {
-                tmem_ld16_issue(abase + (uint32_t)(mb * 128 + h * 16), rb);
+              for (int c4 = 0; c4 < 4; ++c4) {
+                const uint32_t col = (uint32_t)(mb * 128 + c4 * 32);
+                tmem_ld_wait(ra);
+                tmem_ld16_issue(abase + col + 16, rb);
+                half1(masked_tag, std::false_type{}, ra, rc, sum, unused, key0 + c4 * 32, lim);
                 tmem_ld_wait(rb);
-                half1(masked_tag, rb, jump ? mx_c : rc, sum2, mx2, key0 + h * 16, lim);
+                if (mb == MB - 1 && c4 == 3) {
+                  // with more than one stage per group the next job's accumulator is a different stage: fetch ahead
+                  if (kAhead && j + NG < T) {
+                    wait_full(jj + NG, 30);
+                    tmem_ld16_issue(acc_addr(jj + NG), ra);
+                  }
+                } else {
+                  tmem_ld16_issue(abase + col + 32, ra);
+                }
+                if (c4 < 3) {
+                  half1(masked_tag, std::false_type{}, rb, rc, sum, unused, key0 + c4 * 32 + 16, lim);
+                } else {
+                  sum_head = sum;
+                  half1(masked_tag, std::true_type{}, rb, rc, sum, mx_tail, key0 + c4 * 32 + 16, lim);
+                }
               }
-              if (jump) {
-                z_run[mb] *= ex2(rc - mx_c);
-                ref_c[mb] = mx_c;
-                sum = sum2;
+              // also true for inf and NaN sums
+              const bool over = !(sum_head < kSumLimit) || fmaf(mx_tail, c, -rc) > 60.0f;
+              if (__any_sync(0xffffffffu, over)) {   // rare: a score far above the reference
+                float mx = -INFINITY;
+#pragma unroll 1
+                for (int h = 0; h < 8; ++h) {
+                  tmem_ld16_issue(abase + (uint32_t)(mb * 128 + h * 16), rb);
+                  tmem_ld_wait(rb);
+                  max16(masked_tag, rb, mx, key0 + h * 16, lim);
+                }
+                const float mx_c = mx * c;
+                float sum2 = 0.0f;
+#pragma unroll 1
+                for (int h = 0; h < 8; ++h) {
+                  tmem_ld16_issue(abase + (uint32_t)(mb * 128 + h * 16), rb);
+                  tmem_ld_wait(rb);
+                  half1(masked_tag, std::false_type{}, rb, over ? mx_c : rc, sum2, unused, key0 + h * 16, lim);
+                }
+                if (over) {
+                  z_run[mb] *= ex2(rc - mx_c);
+                  ref_c[mb] = mx_c;
+                  sum = sum2;
+                }
               }
+              z_run[mb] += sum;
+            } else {
+              const int lim = lim_row[mb];
+              const float rc = ref_c[mb];
+              float sum = 0.0f, mx = -INFINITY;
+#pragma unroll 1
+              for (int c4 = 0; c4 < 4; ++c4) {
+                const uint32_t col = (uint32_t)(mb * 128 + c4 * 32);
+                tmem_ld_wait(ra);
+                tmem_ld16_issue(abase + col + 16, rb);
+                half1(masked_tag, std::true_type{}, ra, rc, sum, mx, key0 + c4 * 32, lim);
+                tmem_ld_wait(rb);
+                if (mb == MB - 1 && c4 == 3) {
+                  // with more than one stage per group the next job's accumulator is a different stage: fetch ahead
+                  if (kAhead && j + NG < T) {
+                    wait_full(jj + NG, 30);
+                    tmem_ld16_issue(acc_addr(jj + NG), ra);
+                  }
+                } else {
+                  tmem_ld16_issue(abase + col + 32, ra);
+                }
+                half1(masked_tag, std::true_type{}, rb, rc, sum, mx, key0 + c4 * 32 + 16, lim);
+              }
+              const float mx_c = mx * c;
+              const bool jump = mx_c > rc + 8.0f;
+              if (__any_sync(0xffffffffu, jump)) {  // rare: first tiles of a unit, or a score far above all before
+                float sum2 = 0.0f, mx2 = -INFINITY;
+#pragma unroll 1
+                for (int h = 0; h < 8; ++h) {
+                  tmem_ld16_issue(abase + (uint32_t)(mb * 128 + h * 16), rb);
+                  tmem_ld_wait(rb);
+                  half1(masked_tag, std::true_type{}, rb, jump ? mx_c : rc, sum2, mx2, key0 + h * 16, lim);
+                }
+                if (jump) {
+                  z_run[mb] *= ex2(rc - mx_c);
+                  ref_c[mb] = mx_c;
+                  sum = sum2;
+                }
+              }
+              z_run[mb] += sum;
             }
-            z_run[mb] += sum;
           }
           release(jj);
           if (!kAhead && j + NG < T) {  // one stage per group: the next job can only be fetched once this one is released

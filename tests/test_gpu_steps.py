@@ -162,11 +162,13 @@ def test_embedding_detector_matches_oracle(D, Cn, total):
         gp.close()
 
 
-def _score_case(lengths, Hq, Hkv, W, causal=1, seed=0, layers=1, permute=False, scale=0.0):
+def _score_case(lengths, Hq, Hkv, W, causal=1, seed=0, layers=1, permute=False, scale=0.0, edit=None):
     w = _workload(lengths, [[1, 2]], seed=seed, Hq=Hq, Hkv=Hkv, W=W)
     w.n_layers = layers
     pol = oracle_policy(4, W=W, causal=causal, softmax_scale=scale)
     Qh, Kh, _ = tw.make_qkv(w, range(layers))
+    if edit is not None:
+        edit(w, Qh, Kh)
     g = Gpu(w, pol, 4, layers)
     try:
         Qd = Qh.cuda()
@@ -229,6 +231,25 @@ def test_score_cluster_sizes():
     *_, g = _score_case([2048 + 5], 4, 1, 32)
     g.close()
     *_, g = _score_case([8192 - 77], 4, 1, 32, seed=2)
+    g.close()
+
+
+@pytest.mark.parametrize("W", [32, 64])
+def test_score_scores_far_above_and_below_the_first_keys(W):
+    # keys aligned with one query row score about 68 nats (98 in base 2) above the rest: the running normaliser of
+    # that row must survive a jump far beyond anything the row's first keys suggested, early and late in the sequence;
+    # and a row whose first 16 keys score far below the rest
+    def edit(w, Qh, Kh):
+        G = w.Hq // w.Hkv
+        q = Qh[0, 0, 1, W - 1].float()           # query head 1 reads KV head 0; the last window row sees every key
+        for j in (40, 700, 1290):
+            Kh[0, 0, j] = (6.0 * q).to(torch.bfloat16)
+        q2 = Qh[0, 0, G + 2, W - 3].float()      # KV head 1
+        Kh[0, 1, 0:16] = (-6.0 * q2).to(torch.bfloat16)
+        q3 = Qh[0, 1, 0, 5].float()              # second sequence: a spike in its last, masked tile
+        Kh[0, 0, int(w.cu[2]) - W + 2] = (6.0 * q3).to(torch.bfloat16)
+
+    *_, g = _score_case([1300, 300], 8, 2, W, seed=7, edit=edit)
     g.close()
 
 
