@@ -205,9 +205,16 @@ class Runner:
         self.ta.ta_compress(self.ctx, self.pats, self.p, self.batch, w.Hq, w.Hkv, w.d, self.K, self.ids, self.vq,
                             self.vk, self.vv, 0, self.ko, self.vo, self.idx, self.cnt, self.stream)
 
+    def fused_gather(self):
+        # with a budget of at most 64 the scored selection kernel gathers the rows itself when it runs one block per
+        # unit (the library's rule, restated)
+        w = self.w
+        units = self.L * w.B * w.Hkv
+        return (not self.fast) and self.K <= 64 and (int(w.max_n) <= 8192 or units * 8 > 2 * 148)
+
     def kernels_per_step(self):
-        # mask + static utility, [score], forced + select, [broadcast], gather
-        return 2 + (0 if self.fast else 1) + 2 + (1 if self.fast else 0) + 1
+        # mask + static utility, [score], forced + select, [broadcast], [gather]
+        return 2 + (0 if self.fast else 1) + 2 + (1 if self.fast else 0) + (0 if self.fused_gather() else 1)
 
     def close(self):
         self.ta.ta_patterns_destroy(self.pats)
@@ -290,7 +297,9 @@ def measure_extra(name, L, dev, steps=5, warmup=3):
         if not fast and br[1] > 0:
             out["score_hbm_frac"] = score_kernel_bytes(w, L) / (br[1] * 1e-3) / 1e9 / peak
             out["score_tflops"] = 2.0 * (w.Hq // w.Hkv) * w.W * w.d * w.total * w.Hkv * L / (br[1] * 1e-3) / 1e12
-        if br[3] > 0:
+        if r.fused_gather():
+            out["gather_fused_into_select"] = True
+        elif br[3] > 0:
             out["compact_hbm_frac"] = ab["gather"] / (br[3] * 1e-3) / 1e9 / peak
         return out
     finally:
@@ -499,6 +508,8 @@ def main():
                 "traffic": None if fast else recorded_traffic(w.name, L),
                 "ms_per_launch": stage[dom], "stage_ms": stage,
                 "step_algorithmic_bytes": ab["total"], "step_frac": ab["total"] / (ms * 1e-3) / 1e9 / peak}
+    if r.fused_gather():
+        roofline["gather_fused_into_select"] = True
     if not fast:
         roofline["tensor_tflops"] = 2.0 * (w.Hq // w.Hkv) * w.W * w.d * w.total * w.Hkv * L / (stage[dom] * 1e-3) / 1e12
 

@@ -607,7 +607,13 @@ ta_status compress_impl(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* p
     sel.u = u_all;
     sel.idx = idx_lb;
     sel.count = count_lb;
+  } else if (!fast) {  // small budgets: the selecting block gathers the unit's rows itself
+    sel.gather_k = k;
+    sel.gather_v = v;
+    sel.gather_k_out = k_out;
+    sel.gather_v_out = v_out;
   }
+  const bool select_gathers = ta_select_gathers(sel);
 
   // Per-sequence work (anchor mask, vouchers, static utility, forced set) does not depend on Q/K: in scored mode it
   // runs on the context's side stream beside the score kernel and joins before the per-unit selection.
@@ -664,7 +670,7 @@ ta_status compress_impl(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* p
   if (e == cudaSuccess && fast)
     e = ta_launch_broadcast_idx(batch->batch, Hkv, K, batch->n_layers, idx_seq, count_seq, idx, count, stream);
   mark(3);
-  if (e == cudaSuccess) {
+  if (e == cudaSuccess && !select_gathers) {
     ta_compact_args a = {};
     a.seq = seq;
     a.n_layers = batch->n_layers;

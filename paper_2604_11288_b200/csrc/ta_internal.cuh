@@ -115,7 +115,12 @@ struct ta_select_args {
   int32_t* r_main;     // scratch [B]   main-pool picks per sequence (-1: keep everything)
   int32_t* idx;        // [L][B][Hkv][K]
   int32_t* count;      // [L][B][Hkv]
+  // optional: the select kernel also gathers the retained rows (small K, one block per unit; see ta_select_gathers)
+  ta_bf16_view gather_k, gather_v;
+  void* gather_k_out;  // null: no gather
+  void* gather_v_out;
 };
+bool ta_select_gathers(const ta_select_args& a);  // whether ta_launch_select_units will do the gather itself
 cudaError_t ta_launch_select(const ta_select_args& a, ta_dev_status* status, cudaStream_t stream);  // both below
 cudaError_t ta_launch_forced(const ta_select_args& a, ta_dev_status* status, cudaStream_t stream);
 cudaError_t ta_launch_select_units(const ta_select_args& a, cudaStream_t stream);

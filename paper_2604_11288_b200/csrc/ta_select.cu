@@ -473,12 +473,45 @@ __device__ __forceinline__ float unit_utility(const UnitSrc& src, long long unit
   return __fadd_rn(__fadd_rn(aA, dP), u0);
 }
 
+// Small budgets: the block that selected a unit also moves its retained K and V rows (Algorithm 1 step 9), which
+// saves the launch of the gather kernel where that launch costs more than the copy. Same result as ta_compact_kernel:
+// rows at and beyond the retained count, and rows whose index lies outside the sequence, are zero.
+struct GatherDst {
+  ta_bf16_view k, v;
+  uint4* k_out;
+  uint4* v_out;
+  int on;
+};
+constexpr int kGatherMaxK = 64;
+
+__device__ __forceinline__ void gather_unit(const GatherDst& gd, const ta_seq_desc& seq, int unit, int l, int b, int g,
+                                            int n, int K, const int32_t* out, int taken) {
+  constexpr int kLanesPerRow = TA_HEAD_DIM * 2 / 16;
+  __syncthreads();  // the unit's indices were written by other threads of this block
+  for (int t = threadIdx.x; t < K * 2 * kLanesPerRow; t += kThreads) {
+    const int r = t / (2 * kLanesPerRow), which = (t / kLanesPerRow) & 1, lane16 = t % kLanesPerRow;
+    const ta_bf16_view& src = which ? gd.v : gd.k;
+    uint4 val = make_uint4(0u, 0u, 0u, 0u);
+    if (r < taken) {
+      const int i = out[r];
+      if (i >= 0 && i < n) {
+        const long long base = (long long)l * src.stride_l + (long long)g * src.stride_h +
+                               (seq.cu ? (long long)seq.cu[b] * src.stride_n : (long long)b * src.stride_b);
+        val = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const uint16_t*>(src.ptr) + base +
+                                                   (long long)i * src.stride_n) + lane16);
+      }
+    }
+    (which ? gd.v_out : gd.k_out)[((long long)unit * K + r) * kLanesPerRow + lane16] = val;
+  }
+}
+
 // grid.x = units. scored: unit = (l*B + b)*Hkv + g; fast: unit = b.
 template <bool CACHED, int CL, int ITEMS = kItems>
 __global__ void __launch_bounds__(kThreads) ta_select_kernel(ta_seq_desc seq, int n_layers, int Hkv, int K, int fast,
                                                              UnitSrc src, const uint8_t* __restrict__ forced,
                                                              const int32_t* __restrict__ r_main,
-                                                             int32_t* __restrict__ idx, int32_t* __restrict__ count) {
+                                                             int32_t* __restrict__ idx, int32_t* __restrict__ count,
+                                                             GatherDst gd) {
   __shared__ SelectShared sh;
   const int unit = blockIdx.x / CL;
   const bool lead = blockIdx.x % CL == 0;
@@ -500,6 +533,7 @@ __global__ void __launch_bounds__(kThreads) ta_select_kernel(ta_seq_desc seq, in
       for (int r = tid; r < K; r += kThreads) out[r] = -1;
       if (tid == 0) count[unit] = 0;
     }
+    if (CL == 1 && gd.on) gather_unit(gd, seq, unit, l, b, g, n, K, out, 0);
     return;
   }
   if (want == -1) {  // K >= n: keep everything
@@ -507,6 +541,7 @@ __global__ void __launch_bounds__(kThreads) ta_select_kernel(ta_seq_desc seq, in
       for (int r = tid; r < K; r += kThreads) out[r] = r < n ? r : -1;
       if (tid == 0) count[unit] = n;
     }
+    if (CL == 1 && gd.on) gather_unit(gd, seq, unit, l, b, g, n, K, out, n);
     return;
   }
   const long long unit_off = fast ? 0 : ((long long)l * Hkv + g) * seq.total;
@@ -531,6 +566,7 @@ __global__ void __launch_bounds__(kThreads) ta_select_kernel(ta_seq_desc seq, in
   if (!lead) return;
   for (int q = taken + tid; q < K; q += kThreads) out[q] = -1;
   if (tid == 0) count[unit] = taken;
+  if (CL == 1 && gd.on) gather_unit(gd, seq, unit, l, b, g, n, K, out, min(taken, K));
 }
 
 __global__ void ta_broadcast_idx_kernel(int B, int Hkv, int K, int n_layers, const int32_t* __restrict__ idx_seq,
@@ -634,6 +670,13 @@ cudaError_t ta_launch_forced(const ta_select_args& a, ta_dev_status* status, cud
                           a.n_recent, a.k_protected, a.voucher, a.forced, a.r_main, status);
 }
 
+bool ta_select_gathers(const ta_select_args& a) {
+  if (!a.gather_k_out || a.fast || a.K > kGatherMaxK) return false;
+  const int units = a.n_layers * a.seq.batch * a.Hkv;
+  // only the variants that keep a unit in one block
+  return a.seq.max_n <= kItems * kThreads || !split_units(units, a.seq.max_n);
+}
+
 cudaError_t ta_launch_select_units(const ta_select_args& a, cudaStream_t stream) {
   if (a.seq.batch == 0 || a.n_layers == 0) return cudaSuccess;
   UnitSrc src;
@@ -644,23 +687,31 @@ cudaError_t ta_launch_select_units(const ta_select_args& a, cudaStream_t stream)
   src.alpha = a.alpha;
   src.delta = a.delta;
   const int units = a.fast ? a.seq.batch : a.n_layers * a.seq.batch * a.Hkv;
+  GatherDst gd = {};
+  if (ta_select_gathers(a)) {
+    gd.k = a.gather_k;
+    gd.v = a.gather_v;
+    gd.k_out = reinterpret_cast<uint4*>(a.gather_k_out);
+    gd.v_out = reinterpret_cast<uint4*>(a.gather_v_out);
+    gd.on = 1;
+  }
   if (a.seq.max_n <= kItems * kThreads)
     return launch_clustered(ta_select_kernel<true, 1>, units, 1, stream, a.seq, a.n_layers, a.Hkv, a.K, a.fast, src,
-                            a.forced, a.r_main, a.idx, a.count);
+                            a.forced, a.r_main, a.idx, a.count, gd);
   if (!split_units(units, a.seq.max_n) && a.seq.max_n <= kItemsLong * kThreads)
     return launch_clustered(ta_select_kernel<true, 1, kItemsLong>, units, 1, stream, a.seq, a.n_layers, a.Hkv, a.K, a.fast,
-                            src, a.forced, a.r_main, a.idx, a.count);
+                            src, a.forced, a.r_main, a.idx, a.count, gd);
   if (!split_units(units, a.seq.max_n))
     return launch_clustered(ta_select_kernel<false, 1>, units, 1, stream, a.seq, a.n_layers, a.Hkv, a.K, a.fast, src,
-                            a.forced, a.r_main, a.idx, a.count);
+                            a.forced, a.r_main, a.idx, a.count, gd);
   if (a.seq.max_n <= kSelectCluster * kItems * kThreads)
     return launch_clustered(ta_select_kernel<true, kSelectCluster>, units, kSelectCluster, stream, a.seq, a.n_layers,
-                            a.Hkv, a.K, a.fast, src, a.forced, a.r_main, a.idx, a.count);
+                            a.Hkv, a.K, a.fast, src, a.forced, a.r_main, a.idx, a.count, gd);
   if (a.seq.max_n <= kSelectCluster * kItemsLong * kThreads)
     return launch_clustered(ta_select_kernel<true, kSelectCluster, kItemsLong>, units, kSelectCluster, stream, a.seq,
-                            a.n_layers, a.Hkv, a.K, a.fast, src, a.forced, a.r_main, a.idx, a.count);
+                            a.n_layers, a.Hkv, a.K, a.fast, src, a.forced, a.r_main, a.idx, a.count, gd);
   return launch_clustered(ta_select_kernel<false, kSelectCluster>, units, kSelectCluster, stream, a.seq, a.n_layers,
-                          a.Hkv, a.K, a.fast, src, a.forced, a.r_main, a.idx, a.count);
+                          a.Hkv, a.K, a.fast, src, a.forced, a.r_main, a.idx, a.count, gd);
 }
 
 cudaError_t ta_launch_select(const ta_select_args& a, ta_dev_status* status, cudaStream_t stream) {
