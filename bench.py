@@ -206,11 +206,12 @@ class Runner:
                             self.vk, self.vv, 0, self.ko, self.vo, self.idx, self.cnt, self.stream)
 
     def fused_gather(self):
-        # with a budget of at most 64 the scored selection kernel gathers the rows itself when it runs one block per
-        # unit (the library's rule, restated)
+        # with a budget of at most 16, sequences of at most 8192 tokens and at most 4 units per SM the scored
+        # selection kernel gathers the rows itself (the library's rule, restated)
         w = self.w
         units = self.L * w.B * w.Hkv
-        return (not self.fast) and self.K <= 64 and (int(w.max_n) <= 8192 or units * 8 > 2 * 148)
+        sms = torch.cuda.get_device_properties(self.dev).multi_processor_count
+        return (not self.fast) and self.K <= 16 and int(w.max_n) <= 8192 and units <= 4 * sms
 
     def kernels_per_step(self):
         # mask + static utility, [score], forced + select, [broadcast], [gather]

@@ -473,16 +473,15 @@ __device__ __forceinline__ float unit_utility(const UnitSrc& src, long long unit
   return __fadd_rn(__fadd_rn(aA, dP), u0);
 }
 
-// Small budgets: the block that selected a unit also moves its retained K and V rows (Algorithm 1 step 9), which
-// saves the launch of the gather kernel where that launch costs more than the copy. Same result as ta_compact_kernel:
+// Small budgets and few units: the block that selected a unit also moves its retained K and V rows (Algorithm 1
+// step 9), which saves the launch of the gather kernel where that launch costs more than the copy. Same result as ta_compact_kernel:
 // rows at and beyond the retained count, and rows whose index lies outside the sequence, are zero.
 struct GatherDst {
   ta_bf16_view k, v;
   uint4* k_out;
   uint4* v_out;
-  int on;
 };
-constexpr int kGatherMaxK = 64;
+constexpr int kGatherMaxK = 16;  // one 16-byte piece per thread
 
 __device__ __forceinline__ void gather_unit(const GatherDst& gd, const ta_seq_desc& seq, int unit, int l, int b, int g,
                                             int n, int K, const int32_t* out, int taken) {
@@ -506,7 +505,7 @@ __device__ __forceinline__ void gather_unit(const GatherDst& gd, const ta_seq_de
 }
 
 // grid.x = units. scored: unit = (l*B + b)*Hkv + g; fast: unit = b.
-template <bool CACHED, int CL, int ITEMS = kItems>
+template <bool CACHED, int CL, int ITEMS = kItems, bool GATHER = false>
 __global__ void __launch_bounds__(kThreads) ta_select_kernel(ta_seq_desc seq, int n_layers, int Hkv, int K, int fast,
                                                              UnitSrc src, const uint8_t* __restrict__ forced,
                                                              const int32_t* __restrict__ r_main,
@@ -533,7 +532,7 @@ __global__ void __launch_bounds__(kThreads) ta_select_kernel(ta_seq_desc seq, in
       for (int r = tid; r < K; r += kThreads) out[r] = -1;
       if (tid == 0) count[unit] = 0;
     }
-    if (CL == 1 && gd.on) gather_unit(gd, seq, unit, l, b, g, n, K, out, 0);
+    if constexpr (GATHER) gather_unit(gd, seq, unit, l, b, g, n, K, out, 0);
     return;
   }
   if (want == -1) {  // K >= n: keep everything
@@ -541,7 +540,7 @@ __global__ void __launch_bounds__(kThreads) ta_select_kernel(ta_seq_desc seq, in
       for (int r = tid; r < K; r += kThreads) out[r] = r < n ? r : -1;
       if (tid == 0) count[unit] = n;
     }
-    if (CL == 1 && gd.on) gather_unit(gd, seq, unit, l, b, g, n, K, out, n);
+    if constexpr (GATHER) gather_unit(gd, seq, unit, l, b, g, n, K, out, n);
     return;
   }
   const long long unit_off = fast ? 0 : ((long long)l * Hkv + g) * seq.total;
@@ -566,7 +565,7 @@ __global__ void __launch_bounds__(kThreads) ta_select_kernel(ta_seq_desc seq, in
   if (!lead) return;
   for (int q = taken + tid; q < K; q += kThreads) out[q] = -1;
   if (tid == 0) count[unit] = taken;
-  if (CL == 1 && gd.on) gather_unit(gd, seq, unit, l, b, g, n, K, out, min(taken, K));
+  if constexpr (GATHER) gather_unit(gd, seq, unit, l, b, g, n, K, out, min(taken, K));
 }
 
 __global__ void ta_broadcast_idx_kernel(int B, int Hkv, int K, int n_layers, const int32_t* __restrict__ idx_seq,
@@ -672,9 +671,15 @@ cudaError_t ta_launch_forced(const ta_select_args& a, ta_dev_status* status, cud
 
 bool ta_select_gathers(const ta_select_args& a) {
   if (!a.gather_k_out || a.fast || a.K > kGatherMaxK) return false;
+  // The gather adds one dependent load chain (index -> row -> store, about 2 us) to every block, the separate kernel
+  // costs one launch (about 8 us for so few rows): fusing pays only while the blocks run in a few waves. Short units
+  // (keys in 16 registers: two blocks per SM) only.
   const int units = a.n_layers * a.seq.batch * a.Hkv;
-  // only the variants that keep a unit in one block
-  return a.seq.max_n <= kItems * kThreads || !split_units(units, a.seq.max_n);
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1)
+    sms = 148;
+  return a.seq.max_n <= kItems * kThreads && units <= 4 * sms;
 }
 
 cudaError_t ta_launch_select_units(const ta_select_args& a, cudaStream_t stream) {
@@ -688,12 +693,13 @@ cudaError_t ta_launch_select_units(const ta_select_args& a, cudaStream_t stream)
   src.delta = a.delta;
   const int units = a.fast ? a.seq.batch : a.n_layers * a.seq.batch * a.Hkv;
   GatherDst gd = {};
-  if (ta_select_gathers(a)) {
+  if (ta_select_gathers(a)) {  // implies the first variant below
     gd.k = a.gather_k;
     gd.v = a.gather_v;
     gd.k_out = reinterpret_cast<uint4*>(a.gather_k_out);
     gd.v_out = reinterpret_cast<uint4*>(a.gather_v_out);
-    gd.on = 1;
+    return launch_clustered(ta_select_kernel<true, 1, kItems, true>, units, 1, stream, a.seq, a.n_layers, a.Hkv, a.K,
+                            a.fast, src, a.forced, a.r_main, a.idx, a.count, gd);
   }
   if (a.seq.max_n <= kItems * kThreads)
     return launch_clustered(ta_select_kernel<true, 1>, units, 1, stream, a.seq, a.n_layers, a.Hkv, a.K, a.fast, src,

@@ -362,10 +362,11 @@ def test_compact_strided_and_zero_fill():
         g.close()
 
 
-@pytest.mark.parametrize("fast", [False, True])
-def test_compress_equals_steps_and_oracle(fast):
+@pytest.mark.parametrize("fast,K", [(False, 24), (True, 24), (False, 12)])
+def test_compress_equals_steps_and_oracle(fast, K):
+    # K = 12 in scored mode: the selection kernel gathers the rows itself (also for the sequence shorter than K)
     w = _workload([900, 2100, 64, 10], [[4, 5], [6]], seed=12, Hq=8, Hkv=2, W=32)
-    K, L = 24, 2
+    L = 2
     pol = oracle_policy(K, "THEOREM", fast=fast, W=32)
     Qh, Kh, Vh = tw.make_qkv(w, range(L))
     g = Gpu(w, pol, K, L)
