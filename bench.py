@@ -335,6 +335,27 @@ def measure_variants(dev, steps=10, warmup=3):
                     "ms_per_step": ms, "value": w.total * L / (ms * 1e-3), "unit": UNIT})
     finally:
         r.close()
+    # budgets per layer (a pyramid from 64 down to 16 tokens in 8 levels) on the same scores
+    Kmax = 64
+    rb = Runner(w, Kmax, L, False, dev)
+    try:
+        levels = np.linspace(64, 16, 8).round().astype(np.int32)
+        budgets = np.repeat(levels[(np.arange(L) * 8) // L][:, None], w.Hkv, axis=1).astype(np.int32).copy()
+        ctxb = ta.ta_ctx_create(dev.index, ta.ta_scratch_bytes_budgets(rb.batch, w.Hkv, Kmax, rb.p, 8))
+        patsb = ta.ta_patterns_create(ctxb, w.pattern_ids, w.pattern_budget, w.pattern_span)
+        score = torch.rand((L, w.Hkv, w.total), dtype=torch.float32, device=dev)
+
+        def budgeted():
+            ta.ta_compress_scores_budgets(ctxb, patsb, rb.p, rb.batch, w.Hkv, w.d, Kmax, budgets, rb.ids, score, None,
+                                          rb.vk, rb.vv, rb.ko, rb.vo, rb.idx, rb.cnt, rb.stream)
+        ms = time_steps(budgeted, steps, warmup)
+        out.append({"entry": "ta_compress_scores_budgets",
+                    "workload": f"c2, {L} layers, budgets 64..16 by layer (8 levels), scores resident",
+                    "ms_per_step": ms, "value": w.total * L / (ms * 1e-3), "unit": UNIT})
+        ta.ta_patterns_destroy(patsb)
+        ta.ta_ctx_destroy(ctxb)
+    finally:
+        rb.close()
     # detector-confidence anchors on the token stream of c4 (4 x 131072 tokens)
     w4, K4 = build_workload("c4", 0)
     r4 = Runner(w4, K4, 1, True, dev)

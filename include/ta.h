@@ -316,6 +316,25 @@ ta_status ta_compress_scores(ta_ctx* ctx, const ta_patterns* pats, const ta_poli
                              const float* score2, ta_bf16_view k, ta_bf16_view v, uint64_t seq_epoch, void* k_out,
                              void* v_out, int32_t* idx, int32_t* count, void* stream);
 
+/* Composition with methods that give every layer or every head its own budget (Section 2 names PyramidKV, whose
+ * budgets shrink from layer to layer, and Ada-KV, which sets one per head; Section 4.5 claims TA composes with
+ * them): as ta_compress_scores, but (layer l, KV head g) keeps budgets[l*Hkv + g] tokens of every sequence.
+ *   budgets  HOST int32 [n_layers][Hkv], each in 1..K_max; at most TA_MAX_BUDGET_CLASSES distinct values and
+ *            n_layers*Hkv <= 4096 (else TA_ERR_UNSUPPORTED). Read before the call returns.
+ *   K_max    stride of the outputs: idx [L][B][Hkv][K_max], k_out/v_out [L][B][Hkv][K_max][d]; rows at and beyond a
+ *            unit's count = min(budget, n) are -1 / zero as in ta_compress.
+ * The budget partition of Section 3.3 (sinks, recents, protected pool) is taken per budget value, so a unit's result
+ * equals that of ta_compress_scores called with K = its own budget. The per-sequence step is not cached between
+ * calls. Scratch: ta_scratch_bytes_budgets (n_budget_classes = number of distinct budget values, or an upper bound). */
+#define TA_MAX_BUDGET_CLASSES 64
+ta_status ta_scratch_bytes_budgets(const ta_batch* batch, int Hkv, int K_max, const ta_policy* policy,
+                                   int n_budget_classes, size_t* out_bytes);
+ta_status ta_compress_scores_budgets(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* policy,
+                                     const ta_batch* batch, int Hkv, int d, int K_max, const int32_t* budgets,
+                                     const int32_t* token_ids, const float* score, const float* score2,
+                                     ta_bf16_view k, ta_bf16_view v, void* k_out, void* v_out, int32_t* idx,
+                                     int32_t* count, void* stream);
+
 /* ---- Algorithm 1 in the decode loop: per-step retention --------------------------------------------------------
  * (Section 3.1: the policy selects S, |S| <= K, "after each generation step"; Algorithm 1 steps 1-10.)
  * Every step brings one new token per sequence. Per unit (layer l, sequence b, KV head g; unit index

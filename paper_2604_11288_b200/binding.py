@@ -90,6 +90,9 @@ def lib():
                                            ta_bf16_view, u64, vp, vp, vp, vp, vp]),
             "ta_compress_scores": (i32, [vp, vp, PP, PB, i32, i32, i32, vp, vp, vp, ta_bf16_view, ta_bf16_view, u64, vp,
                                          vp, vp, vp, vp]),
+            "ta_scratch_bytes_budgets": (i32, [PB, i32, i32, PP, i32, C.POINTER(sz)]),
+            "ta_compress_scores_budgets": (i32, [vp, vp, PP, PB, i32, i32, i32, vp, vp, vp, vp, ta_bf16_view,
+                                                 ta_bf16_view, vp, vp, vp, vp, vp]),
             "ta_stream_scratch_bytes": (i32, [C.POINTER(ta_stream), C.POINTER(sz)]),
             "ta_stream_step": (i32, [vp, vp, PP, C.POINTER(ta_stream), vp, vp, vp, vp]),
             "ta_compress_host_workspace_bytes": (i32, [PB, i32, i32, i32, i32, PP, C.POINTER(sz)]),
@@ -257,6 +260,21 @@ def ta_compress_scores(ctx, pats, policy, batch, Hkv, d, K, token_ids, score, sc
     _check(lib().ta_compress_scores(ctx, pats, C.byref(policy), C.byref(batch), Hkv, d, K, _ptr(token_ids),
                                     _ptr(score), _ptr(score2), k, v, int(seq_epoch), _ptr(k_out), _ptr(v_out),
                                     _ptr(idx), _ptr(count), stream), "ta_compress_scores")
+
+
+def ta_scratch_bytes_budgets(batch: ta_batch, Hkv, K_max, policy: ta_policy, n_budget_classes) -> int:
+    out = C.c_size_t(0)
+    _check(lib().ta_scratch_bytes_budgets(C.byref(batch), Hkv, K_max, C.byref(policy), n_budget_classes, C.byref(out)),
+           "ta_scratch_bytes_budgets")
+    return out.value
+
+
+def ta_compress_scores_budgets(ctx, pats, policy, batch, Hkv, d, K_max, budgets, token_ids, score, score2,
+                               k: ta_bf16_view, v: ta_bf16_view, k_out, v_out, idx, count, stream=None):
+    """budgets: host int32 array [n_layers][Hkv] (numpy or a CPU tensor)."""
+    _check(lib().ta_compress_scores_budgets(ctx, pats, C.byref(policy), C.byref(batch), Hkv, d, K_max, _ptr(budgets),
+                                            _ptr(token_ids), _ptr(score), _ptr(score2), k, v, _ptr(k_out), _ptr(v_out),
+                                            _ptr(idx), _ptr(count), stream), "ta_compress_scores_budgets")
 
 
 def ta_stream_scratch_bytes(st: ta_stream) -> int:

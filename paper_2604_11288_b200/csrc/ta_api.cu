@@ -26,10 +26,12 @@ struct Carve {  // hands out aligned pieces of the context scratch
 };
 
 struct Layout {  // scratch layout of ta_compress (a superset of what the single-step entry points need)
-  size_t hist, flags, voucher, u_static, forced, r_main, idx_seq, count_seq, u, u_all, idx_lb, count_lb, order, end;
+  size_t hist, flags, voucher, u_static, forced, r_main, idx_seq, count_seq, u, u_all, idx_lb, count_lb, order;
+  size_t forced_cls, r_main_cls, class_K, class_of;  // budgets per (layer, head) only (n_classes > 0)
+  size_t end;
 };
 
-Layout make_layout(const ta_batch& b, int Hkv, int K, const ta_policy& pol) {
+Layout make_layout(const ta_batch& b, int Hkv, int K, const ta_policy& pol, int n_classes = 0) {
   Layout L;
   size_t off = 0;
   auto take = [&](size_t bytes) {
@@ -53,6 +55,10 @@ Layout make_layout(const ta_batch& b, int Hkv, int K, const ta_policy& pol) {
   L.idx_lb = take(scored ? (size_t)b.n_layers * B * K * 4 : 0);
   L.count_lb = take(scored ? (size_t)b.n_layers * B * 4 : 0);
   L.order = take(scored && b.cu_seqlens ? (size_t)b.n_layers * B * Hkv * 4 : 0);  // unit order of the score kernel
+  L.forced_cls = take((size_t)n_classes * total);
+  L.r_main_cls = take((size_t)n_classes * B * 4);
+  L.class_K = take((size_t)n_classes * 4);
+  L.class_of = take(n_classes > 0 ? (size_t)b.n_layers * Hkv * 4 : 0);
   L.end = off;
   return L;
 }
@@ -233,6 +239,18 @@ ta_status ta_scratch_bytes(const ta_batch* batch, int Hq, int Hkv, int d, int K,
   if (s != TA_OK) return s;
   if (K < 1 || Hkv < 1) return TA_ERR_INVALID_ARG;
   *out_bytes = make_layout(*batch, Hkv, K, *policy).end + kAlign;
+  return TA_OK;
+}
+
+ta_status ta_scratch_bytes_budgets(const ta_batch* batch, int Hkv, int K_max, const ta_policy* policy,
+                                   int n_budget_classes, size_t* out_bytes) {
+  if (!out_bytes) return TA_ERR_INVALID_ARG;
+  ta_status s = check_batch(batch);
+  if (s == TA_OK) s = check_policy(policy);
+  if (s != TA_OK) return s;
+  if (K_max < 1 || Hkv < 1 || n_budget_classes < 1) return TA_ERR_INVALID_ARG;
+  if (n_budget_classes > TA_MAX_BUDGET_CLASSES) return TA_ERR_UNSUPPORTED;
+  *out_bytes = make_layout(*batch, Hkv, K_max, *policy, n_budget_classes).end + kAlign;
   return TA_OK;
 }
 
@@ -534,7 +552,8 @@ namespace {
 ta_status compress_impl(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* policy, const ta_batch* batch, int Hq,
                         int Hkv, int d, int K, const int32_t* token_ids, ta_bf16_view q_obs, ta_bf16_view k,
                         ta_bf16_view v, uint64_t seq_epoch, void* k_out, void* v_out, int32_t* idx, int32_t* count,
-                        void* stream_v, const float* ext_A, const float* ext_P, bool share_heads) {
+                        void* stream_v, const float* ext_A, const float* ext_P, bool share_heads,
+                        const int32_t* budgets = nullptr) {
   if (!ctx || !pats || !token_ids || !k_out || !v_out || !idx || !count) return TA_ERR_INVALID_ARG;
   ta_status s = check_batch(batch);
   if (s == TA_OK) s = check_policy(policy);
@@ -554,7 +573,27 @@ ta_status compress_impl(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* p
   if (K > TA_MAX_BUDGET) return TA_ERR_UNSUPPORTED;
   if ((uintptr_t)k_out % 16 || (uintptr_t)v_out % 16) return TA_ERR_ALIGNMENT;
   if (pats->device != ctx->device) return TA_ERR_INVALID_ARG;
-  const Layout L = make_layout(*batch, Hkv, K, *policy);
+  // budgets per (layer, KV head): pairs with equal budgets form a class (HOST work on at most kMaxPairs entries)
+  constexpr int kMaxPairs = 4096;
+  int n_classes = 0;
+  int32_t class_K_h[TA_MAX_BUDGET_CLASSES];
+  int32_t class_of_h[kMaxPairs];
+  if (budgets) {
+    if (fast || share_heads) return TA_ERR_INVALID_ARG;
+    const long long pairs = (long long)batch->n_layers * Hkv;
+    if (pairs > kMaxPairs) return TA_ERR_UNSUPPORTED;
+    for (int i = 0; i < (int)pairs; ++i) {
+      if (budgets[i] < 1 || budgets[i] > K) return TA_ERR_INVALID_ARG;
+      int c = 0;
+      while (c < n_classes && class_K_h[c] != budgets[i]) ++c;
+      if (c == n_classes) {
+        if (n_classes == TA_MAX_BUDGET_CLASSES) return TA_ERR_UNSUPPORTED;
+        class_K_h[n_classes++] = budgets[i];
+      }
+      class_of_h[i] = c;
+    }
+  }
+  const Layout L = make_layout(*batch, Hkv, K, *policy, n_classes);
   if (L.end > ctx->scratch_bytes) return TA_ERR_SCRATCH_TOO_SMALL;
 
   DeviceGuard guard(ctx->device);
@@ -579,8 +618,9 @@ ta_status compress_impl(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* p
     if (timing && e == cudaSuccess) e = cudaEventRecord(ctx->ev[i], stream);
   };
 
-  const bool reuse = seq_epoch != 0 && seq_epoch == ctx->cached_epoch && ctx->cached_total == batch->total_tokens &&
-                     ctx->cached_batch == batch->batch && ctx->cached_K == K;
+  // (with budget classes the forced sets live elsewhere and depend on the budgets: nothing is reused or cached)
+  const bool reuse = !budgets && seq_epoch != 0 && seq_epoch == ctx->cached_epoch &&
+                     ctx->cached_total == batch->total_tokens && ctx->cached_batch == batch->batch && ctx->cached_K == K;
   ta_select_args sel = {};
   sel.seq = seq;
   sel.n_layers = batch->n_layers;
@@ -612,6 +652,17 @@ ta_status compress_impl(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* p
     sel.gather_v = v;
     sel.gather_k_out = k_out;
     sel.gather_v_out = v_out;
+  }
+  if (budgets) {
+    sel.n_classes = n_classes;
+    sel.forced = sc + L.forced_cls;
+    sel.r_main = reinterpret_cast<int32_t*>(sc + L.r_main_cls);
+    sel.class_K = reinterpret_cast<const int32_t*>(sc + L.class_K);
+    sel.class_of = reinterpret_cast<const int32_t*>(sc + L.class_of);
+    // the host arrays are pageable: the copies are staged before the calls return
+    e = cudaMemcpyAsync(sc + L.class_K, class_K_h, (size_t)n_classes * 4, cudaMemcpyHostToDevice, stream);
+    if (e == cudaSuccess)
+      e = cudaMemcpyAsync(sc + L.class_of, class_of_h, (size_t)batch->n_layers * Hkv * 4, cudaMemcpyHostToDevice, stream);
   }
   const bool select_gathers = ta_select_gathers(sel);
 
@@ -690,7 +741,7 @@ ta_status compress_impl(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* p
     return cuda_fail(ctx, e);
   }
   ctx->timing_valid = timing ? 1 : 0;
-  ctx->cached_epoch = seq_epoch;
+  ctx->cached_epoch = budgets ? 0 : seq_epoch;
   ctx->cached_total = batch->total_tokens;
   ctx->cached_batch = batch->batch;
   ctx->cached_K = K;
@@ -724,6 +775,18 @@ ta_status ta_compress_scores(ta_ctx* ctx, const ta_patterns* pats, const ta_poli
   ta_bf16_view none = {};
   return compress_impl(ctx, pats, policy, batch, Hkv, Hkv, d, K, token_ids, none, k, v, seq_epoch, k_out, v_out, idx,
                        count, stream, score, score2, false);
+}
+
+ta_status ta_compress_scores_budgets(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* policy,
+                                     const ta_batch* batch, int Hkv, int d, int K_max, const int32_t* budgets,
+                                     const int32_t* token_ids, const float* score, const float* score2,
+                                     ta_bf16_view k, ta_bf16_view v, void* k_out, void* v_out, int32_t* idx,
+                                     int32_t* count, void* stream) {
+  if (!score || !policy || !budgets) return TA_ERR_INVALID_ARG;
+  if (policy->mode != TA_MODE_SCORED) return TA_ERR_INVALID_ARG;
+  ta_bf16_view none = {};
+  return compress_impl(ctx, pats, policy, batch, Hkv, Hkv, d, K_max, token_ids, none, k, v, 0, k_out, v_out, idx, count,
+                       stream, score, score2, false, budgets);
 }
 
 // ---------------------------------------------------------------------------------------------- decode loop

@@ -115,6 +115,12 @@ struct ta_select_args {
   int32_t* r_main;     // scratch [B]   main-pool picks per sequence (-1: keep everything)
   int32_t* idx;        // [L][B][Hkv][K]
   int32_t* count;      // [L][B][Hkv]
+  // optional: budgets that differ between (layer, KV head) pairs. Pairs with the same budget form a class; the forced
+  // set is computed once per (class, sequence): forced [n_classes][total], r_main [n_classes][B]. K is then the
+  // largest budget (the stride of idx).
+  int n_classes;            // 0: one budget K for all units
+  const int32_t* class_K;   // DEVICE [n_classes]
+  const int32_t* class_of;  // DEVICE [n_layers][Hkv]
   // optional: the select kernel also gathers the retained rows (small K, one block per unit; see ta_select_gathers)
   ta_bf16_view gather_k, gather_v;
   void* gather_k_out;  // null: no gather

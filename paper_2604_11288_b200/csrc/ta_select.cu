@@ -412,9 +412,17 @@ template <bool CACHED, int CL, int ITEMS = kItems>
 __global__ void __launch_bounds__(kThreads) ta_forced_kernel(ta_seq_desc seq, int K, int n_sink, int n_recent,
                                                              int k_protected, const float* __restrict__ voucher,
                                                              uint8_t* __restrict__ forced,
-                                                             int32_t* __restrict__ r_main, ta_dev_status* status) {
+                                                             int32_t* __restrict__ r_main, ta_dev_status* status,
+                                                             const int32_t* __restrict__ class_K) {
   __shared__ SelectShared sh;
-  const int b = blockIdx.x / CL;
+  // grid.x = classes * sequences * CL; without budget classes there is one class and K is the argument
+  const int b = (blockIdx.x / CL) % seq.batch;
+  if (class_K) {
+    const int cls = (blockIdx.x / CL) / seq.batch;
+    K = class_K[cls];
+    forced += (long long)cls * seq.total;
+    r_main += cls * seq.batch;
+  }
   const SeqInfo s = seq_info(seq, b, K, n_sink, n_recent, k_protected);
   if (s.n > seq.max_n || s.n < 0) {
     if (threadIdx.x == 0) {
@@ -510,7 +518,7 @@ __global__ void __launch_bounds__(kThreads) ta_select_kernel(ta_seq_desc seq, in
                                                              UnitSrc src, const uint8_t* __restrict__ forced,
                                                              const int32_t* __restrict__ r_main,
                                                              int32_t* __restrict__ idx, int32_t* __restrict__ count,
-                                                             GatherDst gd) {
+                                                             GatherDst gd, const int32_t* __restrict__ class_of) {
   __shared__ SelectShared sh;
   const int unit = blockIdx.x / CL;
   const bool lead = blockIdx.x % CL == 0;
@@ -521,6 +529,11 @@ __global__ void __launch_bounds__(kThreads) ta_select_kernel(ta_seq_desc seq, in
     g = unit % Hkv;
     b = (unit / Hkv) % seq.batch;
     l = unit / (Hkv * seq.batch);
+  }
+  if (class_of) {  // budgets per (layer, head): the forced set and the main-pool size of this pair's class
+    const int cls = class_of[l * Hkv + g];
+    forced += (long long)cls * seq.total;
+    r_main += cls * seq.batch;
   }
   const int start = ta_seq_begin(seq, b);
   const int n = (seq.cu ? seq.cu[b + 1] : start + seq.n_uniform) - start;
@@ -649,24 +662,25 @@ cudaError_t launch_clustered(Kern kern, int units, int cl, cudaStream_t stream, 
 
 cudaError_t ta_launch_forced(const ta_select_args& a, ta_dev_status* status, cudaStream_t stream) {
   if (a.seq.batch == 0 || a.n_layers == 0) return cudaSuccess;
-  const int B = a.seq.batch;
+  const int B = a.seq.batch * (a.n_classes > 0 ? a.n_classes : 1);  // blocks: (class, sequence)
+  const int32_t* ck = a.n_classes > 0 ? a.class_K : nullptr;
   if (a.seq.max_n <= kItems * kThreads)
     return launch_clustered(ta_forced_kernel<true, 1>, B, 1, stream, a.seq, a.K, a.n_sink, a.n_recent, a.k_protected,
-                            a.voucher, a.forced, a.r_main, status);
+                            a.voucher, a.forced, a.r_main, status, ck);
   if (!split_units(B, a.seq.max_n) && a.seq.max_n <= kItemsLong * kThreads)
     return launch_clustered(ta_forced_kernel<true, 1, kItemsLong>, B, 1, stream, a.seq, a.K, a.n_sink, a.n_recent,
-                            a.k_protected, a.voucher, a.forced, a.r_main, status);
+                            a.k_protected, a.voucher, a.forced, a.r_main, status, ck);
   if (!split_units(B, a.seq.max_n))
     return launch_clustered(ta_forced_kernel<false, 1>, B, 1, stream, a.seq, a.K, a.n_sink, a.n_recent, a.k_protected,
-                            a.voucher, a.forced, a.r_main, status);
+                            a.voucher, a.forced, a.r_main, status, ck);
   if (a.seq.max_n <= kSelectCluster * kItems * kThreads)
     return launch_clustered(ta_forced_kernel<true, kSelectCluster>, B, kSelectCluster, stream, a.seq, a.K, a.n_sink,
-                            a.n_recent, a.k_protected, a.voucher, a.forced, a.r_main, status);
+                            a.n_recent, a.k_protected, a.voucher, a.forced, a.r_main, status, ck);
   if (a.seq.max_n <= kSelectCluster * kItemsLong * kThreads)
     return launch_clustered(ta_forced_kernel<true, kSelectCluster, kItemsLong>, B, kSelectCluster, stream, a.seq, a.K,
-                            a.n_sink, a.n_recent, a.k_protected, a.voucher, a.forced, a.r_main, status);
+                            a.n_sink, a.n_recent, a.k_protected, a.voucher, a.forced, a.r_main, status, ck);
   return launch_clustered(ta_forced_kernel<false, kSelectCluster>, B, kSelectCluster, stream, a.seq, a.K, a.n_sink,
-                          a.n_recent, a.k_protected, a.voucher, a.forced, a.r_main, status);
+                          a.n_recent, a.k_protected, a.voucher, a.forced, a.r_main, status, ck);
 }
 
 bool ta_select_gathers(const ta_select_args& a) {
@@ -692,6 +706,7 @@ cudaError_t ta_launch_select_units(const ta_select_args& a, cudaStream_t stream)
   src.alpha = a.alpha;
   src.delta = a.delta;
   const int units = a.fast ? a.seq.batch : a.n_layers * a.seq.batch * a.Hkv;
+  const int32_t* co = a.n_classes > 0 ? a.class_of : nullptr;
   GatherDst gd = {};
   if (ta_select_gathers(a)) {  // implies the first variant below
     gd.k = a.gather_k;
@@ -699,25 +714,25 @@ cudaError_t ta_launch_select_units(const ta_select_args& a, cudaStream_t stream)
     gd.k_out = reinterpret_cast<uint4*>(a.gather_k_out);
     gd.v_out = reinterpret_cast<uint4*>(a.gather_v_out);
     return launch_clustered(ta_select_kernel<true, 1, kItems, true>, units, 1, stream, a.seq, a.n_layers, a.Hkv, a.K,
-                            a.fast, src, a.forced, a.r_main, a.idx, a.count, gd);
+                            a.fast, src, a.forced, a.r_main, a.idx, a.count, gd, co);
   }
   if (a.seq.max_n <= kItems * kThreads)
     return launch_clustered(ta_select_kernel<true, 1>, units, 1, stream, a.seq, a.n_layers, a.Hkv, a.K, a.fast, src,
-                            a.forced, a.r_main, a.idx, a.count, gd);
+                            a.forced, a.r_main, a.idx, a.count, gd, co);
   if (!split_units(units, a.seq.max_n) && a.seq.max_n <= kItemsLong * kThreads)
     return launch_clustered(ta_select_kernel<true, 1, kItemsLong>, units, 1, stream, a.seq, a.n_layers, a.Hkv, a.K, a.fast,
-                            src, a.forced, a.r_main, a.idx, a.count, gd);
+                            src, a.forced, a.r_main, a.idx, a.count, gd, co);
   if (!split_units(units, a.seq.max_n))
     return launch_clustered(ta_select_kernel<false, 1>, units, 1, stream, a.seq, a.n_layers, a.Hkv, a.K, a.fast, src,
-                            a.forced, a.r_main, a.idx, a.count, gd);
+                            a.forced, a.r_main, a.idx, a.count, gd, co);
   if (a.seq.max_n <= kSelectCluster * kItems * kThreads)
     return launch_clustered(ta_select_kernel<true, kSelectCluster>, units, kSelectCluster, stream, a.seq, a.n_layers,
-                            a.Hkv, a.K, a.fast, src, a.forced, a.r_main, a.idx, a.count, gd);
+                            a.Hkv, a.K, a.fast, src, a.forced, a.r_main, a.idx, a.count, gd, co);
   if (a.seq.max_n <= kSelectCluster * kItemsLong * kThreads)
     return launch_clustered(ta_select_kernel<true, kSelectCluster, kItemsLong>, units, kSelectCluster, stream, a.seq,
-                            a.n_layers, a.Hkv, a.K, a.fast, src, a.forced, a.r_main, a.idx, a.count, gd);
+                            a.n_layers, a.Hkv, a.K, a.fast, src, a.forced, a.r_main, a.idx, a.count, gd, co);
   return launch_clustered(ta_select_kernel<false, kSelectCluster>, units, kSelectCluster, stream, a.seq, a.n_layers,
-                          a.Hkv, a.K, a.fast, src, a.forced, a.r_main, a.idx, a.count, gd);
+                          a.Hkv, a.K, a.fast, src, a.forced, a.r_main, a.idx, a.count, gd, co);
 }
 
 cudaError_t ta_launch_select(const ta_select_args& a, ta_dev_status* status, cudaStream_t stream) {

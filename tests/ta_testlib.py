@@ -32,7 +32,7 @@ def gpu_policy(pol: oracle.Policy) -> ta.ta_policy:
 class Gpu:
     """Owns a context, a pattern set and the device copies of one workload's per-sequence inputs."""
 
-    def __init__(self, w, pol: oracle.Policy, K, n_layers, device="cuda:0"):
+    def __init__(self, w, pol: oracle.Policy, K, n_layers, device="cuda:0", n_budget_classes=0):
         self.w, self.pol, self.K, self.L = w, pol, K, n_layers
         self.dev = torch.device(device)
         self.p = gpu_policy(pol)
@@ -41,6 +41,8 @@ class Gpu:
         n_uni = int(w.lengths[0]) if w.uniform else 0
         self.batch = ta.make_batch(n_layers, w.B, n_uni, w.max_n, w.total, self.cu)
         need = ta.ta_scratch_bytes(self.batch, w.Hq, w.Hkv, w.d, K, self.p)
+        if n_budget_classes:
+            need = max(need, ta.ta_scratch_bytes_budgets(self.batch, w.Hkv, K, self.p, n_budget_classes))
         self.ctx = ta.ta_ctx_create(self.dev.index or 0, need)
         self.pats = ta.ta_patterns_create(self.ctx, w.pattern_ids, w.pattern_budget, w.pattern_span)
         self.stream = torch.cuda.current_stream(self.dev).cuda_stream
@@ -113,6 +115,17 @@ class Gpu:
         rag = not w.uniform
         ta.ta_compress_scores(self.ctx, self.pats, self.p, self.batch, w.Hkv, w.d, self.K, self.ids, score, score2,
                               ta.view(Kc, rag), ta.view(Vc, rag), epoch, ko, vo, idx, cnt, self.stream)
+        return idx, cnt, ko, vo
+
+    def compress_scores_budgets(self, budgets, score, score2, Kc, Vc):
+        w = self.w
+        idx = torch.full((self.L, w.B, w.Hkv, self.K), -7, dtype=torch.int32, device=self.dev)
+        cnt = torch.full((self.L, w.B, w.Hkv), -7, dtype=torch.int32, device=self.dev)
+        ko = torch.full((self.L, w.B, w.Hkv, self.K, w.d), 1.0, dtype=torch.bfloat16, device=self.dev)
+        vo = torch.full_like(ko, 1.0)
+        rag = not w.uniform
+        ta.ta_compress_scores_budgets(self.ctx, self.pats, self.p, self.batch, w.Hkv, w.d, self.K, budgets, self.ids,
+                                      score, score2, ta.view(Kc, rag), ta.view(Vc, rag), ko, vo, idx, cnt, self.stream)
         return idx, cnt, ko, vo
 
     def compress(self, Q, Kc, Vc, epoch=0):

@@ -438,6 +438,59 @@ def test_compress_with_external_scores_bit_exact(with_second):
         g.close()
 
 
+def test_compress_with_budgets_per_layer_and_head_bit_exact():
+    # Section 4.5 with a provider that sets its own budget per layer (pyramid) and per head: every unit must come out
+    # as if the whole call had used that unit's budget (sinks, recents and protected pool sized from it)
+    w = _workload([1500, 90, 12, 700], [[4, 5], [9]], seed=33, Hq=8, Hkv=2, W=32)
+    L, K_max = 3, 40
+    budgets = np.array([[40, 24], [24, 9], [16, 40]], np.int32)  # 5 distinct values; 9 and 16 < a short sequence's n
+    pol = oracle_policy(K_max, "THEOREM", W=32)
+    Qh, Kh, Vh = tw.make_qkv(w, range(L))
+    rng = np.random.default_rng(4)
+    score = rng.random((L, w.Hkv, w.total)).astype(np.float32)
+    score[:, :, ::7] = 0.5  # ties
+    g = Gpu(w, pol, K_max, L, n_budget_classes=5)
+    try:
+        idx, cnt, ko, vo = g.compress_scores_budgets(budgets, torch.from_numpy(score).cuda(), None, Kh.cuda(), Vh.cuda())
+        torch.cuda.synchronize()
+        assert g.poll() == ta.TA_OK
+        idx, cnt = idx.cpu().numpy(), cnt.cpu().numpy()
+        f_o, V_o, u0_o = oracle.sponsor_mask(w.ids, w.cu, oracle_patterns(w), pol)
+        for l in range(L):
+            for b in range(w.B):
+                o, e = int(w.cu[b]), int(w.cu[b + 1])
+                for h in range(w.Hkv):
+                    Ku = int(budgets[l, h])
+                    u = oracle.utility(pol.alpha, pol.delta, score[l, h, o:e], None, u0_o[o:e])
+                    io, co = oracle.select(V_o[o:e], u, Ku, pol.n_sink, pol.n_recent, pol.k_protected)
+                    assert cnt[l, b, h] == co == min(Ku, e - o)
+                    np.testing.assert_array_equal(idx[l, b, h, :Ku], io, err_msg=f"l{l} b{b} h{h}")
+                    assert (idx[l, b, h, Ku:] == -1).all()
+                    for out, src in ((ko, Kh), (vo, Vh)):
+                        got = bf16_bits(out[l, b, h])
+                        np.testing.assert_array_equal(got[:Ku], oracle.compact(unit_kv(w, src, l, b, h), io, co, Ku))
+                        assert not got[Ku:].any()
+        # the same call twice, and after a call of another entry point on the same context: same result
+        idx2, cnt2, ko2, vo2 = g.compress_scores_budgets(budgets, torch.from_numpy(score).cuda(), None, Kh.cuda(), Vh.cuda())
+        torch.cuda.synchronize()
+        assert np.array_equal(idx2.cpu().numpy(), idx) and torch.equal(ko2, ko) and torch.equal(vo2, vo)
+        # argument checks on the host
+        bad = budgets.copy()
+        bad[0, 0] = K_max + 1
+        with pytest.raises(ta.TAError) as ei:
+            g.compress_scores_budgets(bad, torch.from_numpy(score).cuda(), None, Kh.cuda(), Vh.cuda())
+        assert ei.value.status == ta.TA_ERR_INVALID_ARG
+        small = Gpu(w, pol, K_max, L)  # scratch without room for budget classes
+        try:
+            with pytest.raises(ta.TAError) as ei:
+                small.compress_scores_budgets(budgets, torch.from_numpy(score).cuda(), None, Kh.cuda(), Vh.cuda())
+            assert ei.value.status == ta.TA_ERR_SCRATCH_TOO_SMALL
+        finally:
+            small.close()
+    finally:
+        g.close()
+
+
 @pytest.mark.parametrize("preset", ["THEOREM", "SEC33"])
 def test_compress_allheads_shared_selection(preset):
     # Eq. 1's A_i summed over all query heads of the layer: one retained set per (layer, sequence), the same for every
