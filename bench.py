@@ -445,7 +445,8 @@ def main():
     ap.add_argument("--budget", type=int, default=0, help="K (default: the workload's first budget)")
     ap.add_argument("--mode", default="", choices=["", "scored", "fast"])
     ap.add_argument("--layers", type=int, default=0, help="layers per call (default: the workload's layer count)")
-    ap.add_argument("--no-extra", action="store_true", help="skip the supplementary workloads")
+    ap.add_argument("--no-extra", action="store_true", help="skip the supplementary workloads and entry points")
+    ap.add_argument("--no-other", action="store_true", help="skip the supplementary workloads, keep the entry points")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     a = ap.parse_args()
@@ -551,7 +552,7 @@ def main():
     if not a.no_extra and world == 1:
         extra = []
         for name, layers in (("c3", 2), ("c4", 16), ("c5", 2)):
-            if name == a.workload:
+            if name == a.workload or a.no_other:
                 continue
             try:
                 extra.append(measure_extra(name, layers, dev))
