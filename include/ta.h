@@ -334,6 +334,12 @@ ta_status ta_compress_scores_budgets(ta_ctx* ctx, const ta_patterns* pats, const
                                      const int32_t* token_ids, const float* score, const float* score2,
                                      ta_bf16_view k, ta_bf16_view v, void* k_out, void* v_out, int32_t* idx,
                                      int32_t* count, void* stream);
+/* The same budgets with TA's own attention terms (scored mode of ta_compress: A_i and P_i of Eq. 1 from q_obs and k).
+ * Scratch: ta_scratch_bytes_budgets (it covers what ta_compress needs). */
+ta_status ta_compress_budgets(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* policy, const ta_batch* batch,
+                              int Hq, int Hkv, int d, int K_max, const int32_t* budgets, const int32_t* token_ids,
+                              ta_bf16_view q_obs, ta_bf16_view k, ta_bf16_view v, void* k_out, void* v_out,
+                              int32_t* idx, int32_t* count, void* stream);
 
 /* ---- Algorithm 1 in the decode loop: per-step retention --------------------------------------------------------
  * (Section 3.1: the policy selects S, |S| <= K, "after each generation step"; Algorithm 1 steps 1-10.)

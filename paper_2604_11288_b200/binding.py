@@ -93,6 +93,8 @@ def lib():
             "ta_scratch_bytes_budgets": (i32, [PB, i32, i32, PP, i32, C.POINTER(sz)]),
             "ta_compress_scores_budgets": (i32, [vp, vp, PP, PB, i32, i32, i32, vp, vp, vp, vp, ta_bf16_view,
                                                  ta_bf16_view, vp, vp, vp, vp, vp]),
+            "ta_compress_budgets": (i32, [vp, vp, PP, PB, i32, i32, i32, i32, vp, vp, ta_bf16_view, ta_bf16_view,
+                                          ta_bf16_view, vp, vp, vp, vp, vp]),
             "ta_stream_scratch_bytes": (i32, [C.POINTER(ta_stream), C.POINTER(sz)]),
             "ta_stream_step": (i32, [vp, vp, PP, C.POINTER(ta_stream), vp, vp, vp, vp]),
             "ta_compress_host_workspace_bytes": (i32, [PB, i32, i32, i32, i32, PP, C.POINTER(sz)]),
@@ -275,6 +277,14 @@ def ta_compress_scores_budgets(ctx, pats, policy, batch, Hkv, d, K_max, budgets,
     _check(lib().ta_compress_scores_budgets(ctx, pats, C.byref(policy), C.byref(batch), Hkv, d, K_max, _ptr(budgets),
                                             _ptr(token_ids), _ptr(score), _ptr(score2), k, v, _ptr(k_out), _ptr(v_out),
                                             _ptr(idx), _ptr(count), stream), "ta_compress_scores_budgets")
+
+
+def ta_compress_budgets(ctx, pats, policy, batch, Hq, Hkv, d, K_max, budgets, token_ids, q_obs: ta_bf16_view,
+                        k: ta_bf16_view, v: ta_bf16_view, k_out, v_out, idx, count, stream=None):
+    """budgets: host int32 array [n_layers][Hkv] (numpy or a CPU tensor)."""
+    _check(lib().ta_compress_budgets(ctx, pats, C.byref(policy), C.byref(batch), Hq, Hkv, d, K_max, _ptr(budgets),
+                                     _ptr(token_ids), q_obs, k, v, _ptr(k_out), _ptr(v_out), _ptr(idx), _ptr(count),
+                                     stream), "ta_compress_budgets")
 
 
 def ta_stream_scratch_bytes(st: ta_stream) -> int:

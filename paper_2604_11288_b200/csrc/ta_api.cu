@@ -789,6 +789,16 @@ ta_status ta_compress_scores_budgets(ta_ctx* ctx, const ta_patterns* pats, const
                        stream, score, score2, false, budgets);
 }
 
+ta_status ta_compress_budgets(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* policy, const ta_batch* batch,
+                              int Hq, int Hkv, int d, int K_max, const int32_t* budgets, const int32_t* token_ids,
+                              ta_bf16_view q_obs, ta_bf16_view k, ta_bf16_view v, void* k_out, void* v_out,
+                              int32_t* idx, int32_t* count, void* stream) {
+  if (!policy || !budgets) return TA_ERR_INVALID_ARG;
+  if (policy->mode != TA_MODE_SCORED) return TA_ERR_INVALID_ARG;
+  return compress_impl(ctx, pats, policy, batch, Hq, Hkv, d, K_max, token_ids, q_obs, k, v, 0, k_out, v_out, idx, count,
+                       stream, nullptr, nullptr, false, budgets);
+}
+
 // ---------------------------------------------------------------------------------------------- decode loop
 namespace {
 struct StreamLayout {

@@ -128,6 +128,17 @@ class Gpu:
                                       score, score2, ta.view(Kc, rag), ta.view(Vc, rag), ko, vo, idx, cnt, self.stream)
         return idx, cnt, ko, vo
 
+    def compress_budgets(self, budgets, Q, Kc, Vc):
+        w = self.w
+        idx = torch.full((self.L, w.B, w.Hkv, self.K), -7, dtype=torch.int32, device=self.dev)
+        cnt = torch.full((self.L, w.B, w.Hkv), -7, dtype=torch.int32, device=self.dev)
+        ko = torch.full((self.L, w.B, w.Hkv, self.K, w.d), 1.0, dtype=torch.bfloat16, device=self.dev)
+        vo = torch.full_like(ko, 1.0)
+        rag = not w.uniform
+        ta.ta_compress_budgets(self.ctx, self.pats, self.p, self.batch, w.Hq, w.Hkv, w.d, self.K, budgets, self.ids,
+                               ta.view(Q), ta.view(Kc, rag), ta.view(Vc, rag), ko, vo, idx, cnt, self.stream)
+        return idx, cnt, ko, vo
+
     def compress(self, Q, Kc, Vc, epoch=0):
         w = self.w
         idx = torch.full((self.L, w.B, w.Hkv, self.K), -7, dtype=torch.int32, device=self.dev)

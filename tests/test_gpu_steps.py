@@ -491,6 +491,38 @@ def test_compress_with_budgets_per_layer_and_head_bit_exact():
         g.close()
 
 
+def test_compress_budgets_with_own_attention_scores():
+    # budgets per (layer, head) with TA's own attention terms: every unit as the one-budget path with K = its budget
+    w = _workload([1100, 200, 2300], [[4, 5], [9]], seed=35, Hq=8, Hkv=2, W=32)
+    L, K_max = 2, 48
+    budgets = np.array([[48, 12], [20, 48]], np.int32)
+    pol = oracle_policy(K_max, "THEOREM", W=32)
+    Qh, Kh, Vh = tw.make_qkv(w, range(L))
+    g = Gpu(w, pol, K_max, L, n_budget_classes=3)
+    try:
+        idx, cnt, ko, vo = g.compress_budgets(budgets, Qh.cuda(), Kh.cuda(), Vh.cuda())
+        torch.cuda.synchronize()
+        assert g.poll() == ta.TA_OK
+        idx, cnt = idx.cpu().numpy(), cnt.cpu().numpy()
+        f_o, V_o, u0_o = oracle.sponsor_mask(w.ids, w.cu, oracle_patterns(w), pol)
+        exact = 0
+        for l in range(L):
+            for b in range(w.B):
+                for h in range(w.Hkv):
+                    Ku = int(budgets[l, h])
+                    A, P, u, io, co = oracle_unit(w, pol, Ku, Qh, Kh, l, b, h, V_o, u0_o)
+                    exact += assert_selection_matches(idx[l, b, h, :Ku], cnt[l, b, h], io, co, u, f"l{l} b{b} h{h}")
+                    assert (idx[l, b, h, Ku:] == -1).all()
+                    sel, c = idx[l, b, h, :Ku], int(cnt[l, b, h])
+                    for out, src in ((ko, Kh), (vo, Vh)):
+                        got = bf16_bits(out[l, b, h])
+                        np.testing.assert_array_equal(got[:Ku], oracle.compact(unit_kv(w, src, l, b, h), sel, c, Ku))
+                        assert not got[Ku:].any()
+        assert exact >= 0.9 * L * w.B * w.Hkv
+    finally:
+        g.close()
+
+
 @pytest.mark.parametrize("preset", ["THEOREM", "SEC33"])
 def test_compress_allheads_shared_selection(preset):
     # Eq. 1's A_i summed over all query heads of the layer: one retained set per (layer, sequence), the same for every
