@@ -139,13 +139,16 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
   // direction (the cluster that got the longest unit of one round gets the shortest of the next), which evens out the
   // clusters' totals; a position past the end of the list is an empty unit.
   auto get_unit = [&](int walk) {
+    // every cluster makes the same number of rounds; walk positions at and beyond the number of units are empty
     int u = walk;
-    bool empty = false;
+    bool empty = walk >= p.units;
     if (p.order) {
       const int round = walk / n_clusters;
       const int w = (round & 1) ? round * n_clusters + (n_clusters - 1 - cluster_id) : walk;
       empty = w >= p.units;
       u = empty ? 0 : p.order[w];
+    } else if (empty) {
+      u = 0;
     }
     UnitInfo ui;
     ui.g = u % p.Hkv;

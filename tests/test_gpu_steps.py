@@ -226,6 +226,37 @@ def test_score_layers_and_strided_keys():
     g.close()
 
 
+def test_score_more_units_than_ctas_stays_inside_its_outputs():
+    # 160 units of one tile-row each on a persistent grid of fewer CTAs: the grid walks the units in rounds, and the
+    # positions of the last round that lie beyond the last unit must do nothing (guard layers behind A and P stay
+    # untouched)
+    L, guard = 20, 16
+    w = _workload([300], [[1, 2]], seed=3, Hq=32, Hkv=8, W=32)
+    w.n_layers = L
+    pol = oracle_policy(4, W=32)
+    Qh, Kh, _ = tw.make_qkv(w, range(L))
+    g = Gpu(w, pol, 4, L)
+    try:
+        A = torch.full((L + guard, w.Hkv, w.total), float("nan"), dtype=torch.float32, device="cuda")
+        P = torch.full_like(A, float("nan"))
+        Qd, Kd = Qh.cuda(), Kh.cuda()  # held until the kernel has run: a view is only a pointer
+        ta.ta_score(g.ctx, g.p, g.batch, w.Hq, w.Hkv, w.d, ta.view(Qd), ta.view(Kd, not w.uniform), None, A, P,
+                    g.stream)
+        torch.cuda.synchronize()
+        assert g.poll() == ta.TA_OK
+        assert torch.isnan(A[L:]).all() and torch.isnan(P[L:]).all()
+        assert not torch.isnan(A[:L]).any() and not torch.isnan(P[:L]).any()
+        G = w.Hq // w.Hkv
+        for l in (0, 7, L - 1):
+            for h in range(w.Hkv):
+                Ao, Po = oracle.attention(bf16_bits(Qh[l, 0, h * G:(h + 1) * G]), unit_kv(w, Kh, l, 0, h), 300,
+                                          scale=0.0, causal=1, rho=pol.pension_rho)
+                assert_scores_close(A[l, h].cpu().numpy(), Ao, f"A l{l} h{h}")
+                assert_scores_close(P[l, h].cpu().numpy(), Po, f"P l{l} h{h}")
+    finally:
+        g.close()
+
+
 def test_score_cluster_sizes():
     # 16, 32 and 64 tiles: clusters of 4 and 8 CTAs per unit
     *_, g = _score_case([2048 + 5], 4, 1, 32)
