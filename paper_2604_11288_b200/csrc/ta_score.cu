@@ -574,36 +574,42 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           float z = 0.0f;
 #pragma unroll
           for (int gq = 0; gq < NG; ++gq) z += sm.part_z[gq][st] * ex2(sm.part_m[gq][st] - m);
-          sm.mine_m[up][st] = m;
-          sm.mine_z[up][st] = z;
-        }
-        softmax_bar<NG>();
-        // one thread per peer tells that peer that this CTA's statistics of the unit are in place
-        if (st < p.cluster) {
-          fence_cluster();
-          mbar_arrive_remote(smem_u32(&sm.xchg_full[up]), (uint32_t)st);
-        }
-        if (st < kRowsPad) {
-          mbar_wait_cluster(smem_u32(&sm.xchg_full[up]), (uint32_t)(it >> 1) & 1u, abort_flag, p.status, 32);
-          float pm[kMaxCluster], pz[kMaxCluster];
-#pragma unroll
-          for (int r = 0; r < kMaxCluster; ++r) {
-            pm[r] = -1e30f;
-            pz[r] = 0.0f;
-            if (r < p.cluster) {
-              pm[r] = ld_cluster_f32(smem_u32(&sm.mine_m[up][st]), (uint32_t)r);
-              pz[r] = ld_cluster_f32(smem_u32(&sm.mine_z[up][st]), (uint32_t)r);
-            }
+          if (p.cluster == 1) {  // nothing to exchange: the CTA's statistics are the unit's
+            sm.lse2[up][st] = (z > 0.0f) ? m + log2f(z) : INFINITY;
+          } else {
+            sm.mine_m[up][st] = m;
+            sm.mine_z[up][st] = z;
           }
-          float m = pm[0];
-#pragma unroll
-          for (int r = 1; r < kMaxCluster; ++r) m = fmaxf(m, pm[r]);
-          float z = 0.0f;
-#pragma unroll
-          for (int r = 0; r < kMaxCluster; ++r) z += pz[r] * ex2(pm[r] - m);
-          sm.lse2[up][st] = (z > 0.0f) ? m + log2f(z) : INFINITY;
         }
         softmax_bar<NG>();
+        if (p.cluster > 1) {
+          // one thread per peer tells that peer that this CTA's statistics of the unit are in place
+          if (st < p.cluster) {
+            fence_cluster();
+            mbar_arrive_remote(smem_u32(&sm.xchg_full[up]), (uint32_t)st);
+          }
+          if (st < kRowsPad) {
+            mbar_wait_cluster(smem_u32(&sm.xchg_full[up]), (uint32_t)(it >> 1) & 1u, abort_flag, p.status, 32);
+            float pm[kMaxCluster], pz[kMaxCluster];
+#pragma unroll
+            for (int r = 0; r < kMaxCluster; ++r) {
+              pm[r] = -1e30f;
+              pz[r] = 0.0f;
+              if (r < p.cluster) {
+                pm[r] = ld_cluster_f32(smem_u32(&sm.mine_m[up][st]), (uint32_t)r);
+                pz[r] = ld_cluster_f32(smem_u32(&sm.mine_z[up][st]), (uint32_t)r);
+              }
+            }
+            float m = pm[0];
+#pragma unroll
+            for (int r = 1; r < kMaxCluster; ++r) m = fmaxf(m, pm[r]);
+            float z = 0.0f;
+#pragma unroll
+            for (int r = 0; r < kMaxCluster; ++r) z += pz[r] * ex2(pm[r] - m);
+            sm.lse2[up][st] = (z > 0.0f) ? m + log2f(z) : INFINITY;
+          }
+          softmax_bar<NG>();
+        }
       } else {
         if (st < kRowsPad) {
           float lse2 = INFINITY;
