@@ -45,11 +45,15 @@ constexpr int kMaxCluster = 8;
 // NG softmax warpgroups (4 warps each) plus one warpgroup holding the TMA producer warp, the MMA issuer warp and
 // two idle warps. Register split after set-up (setmaxnreg); the shares must fit in threads x registers at launch:
 //   NG = 2: 384 threads x 168 = 64512 = 8*32*216 + 4*32*72        NG = 3: 512 threads x 128 = 65536 = 12*32*152 + 4*32*56
+//   NG = 4: 640 threads x  96 = 61440 = 16*32*112 + 4*32*32
+// The softmax warps wait on the chain accumulator load -> multiply-add -> ex2 -> add rather than on issue slots, so one
+// more warp per scheduler pays where the loops fit its smaller register share: sweep 2 with the pension term then adds
+// every exponential straight into two sums (PM 3) instead of keeping 32 per-position partial sums in registers.
 template <int NG>
 struct GroupCfg {
   static constexpr int kThreads = (NG + 1) * 128;
-  static constexpr int kRegsSoftmax = NG == 2 ? 216 : 152;
-  static constexpr int kRegsOther = NG == 2 ? 72 : 56;
+  static constexpr int kRegsSoftmax = NG == 2 ? 216 : NG == 3 ? 152 : 112;
+  static constexpr int kRegsOther = NG == 2 ? 72 : NG == 3 ? 56 : 32;
   static constexpr int kRegsNeeded = (NG * 4 * kRegsSoftmax + 4 * kRegsOther) * 32;
 };
 
@@ -82,7 +86,7 @@ struct ScoreCfg {
   static constexpr int kRowsPad = MB * 128;
   // accumulator stages in tensor memory (at most 512 columns): two per softmax group when they fit (the group can
   // then fetch its next job before releasing the current one), else one per group
-  static constexpr int kAcc = MB == 1 ? (NG == 2 ? 4 : 3) : 2;
+  static constexpr int kAcc = MB == 1 ? (NG == 3 ? 3 : 4) : 2;
 };
 
 template <int MB, int NG>
@@ -925,14 +929,14 @@ cudaError_t ta_launch_score(ta_ctx* ctx, const ta_score_args& a, ta_dev_status* 
     const uint32_t box[5] = {64, (uint32_t)kTileN, 1, 1, 1};
     if (encode_5d(ctx->encode_tiled, &mk, a.k.ptr, dims, str, box) != CUDA_SUCCESS) return cudaErrorInvalidValue;
   }
-  // how the pension term is accumulated: 0 none, 1 W divides 32, 2 W == 64, 3 any W (per-element weights)
+  // how the pension term is accumulated: 0 none, 1 W divides 32, 2 W == 64, 3 any W (per-element weights);
+  // one row block: four softmax groups with per-element weights whenever the term is needed
   const bool need_p = a.P != nullptr || (a.u != nullptr && a.delta != 0.0f);
   const int pm = !need_p ? 0 : (32 % a.W == 0) ? 1 : (a.W == 64 && rows == 256) ? 2 : 3;
   if (MB == 1) {
     switch (pm) {
       case 0: return launch_variant<1, 0, 3>(ctx, mq, mk, sp, tiles_max, a.reserve_sms, stream);
-      case 1: return launch_variant<1, 1, 3>(ctx, mq, mk, sp, tiles_max, a.reserve_sms, stream);
-      default: return launch_variant<1, 3, 3>(ctx, mq, mk, sp, tiles_max, a.reserve_sms, stream);
+      default: return launch_variant<1, 3, 4>(ctx, mq, mk, sp, tiles_max, a.reserve_sms, stream);
     }
   }
   switch (pm) {
