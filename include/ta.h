@@ -58,7 +58,7 @@ enum {
   TA_FLAG_SPONSORED = 4     /* V_i > 0                                                                */
 };
 
-/* hard limits of this build (validated on every call) */
+/* hard limits of the library (validated on every call) */
 enum {
   TA_MAX_PATTERNS = 256,    /* patterns in one set                                                     */
   TA_MAX_PATTERN_LEN = 8,   /* token ids per pattern                                                   */
