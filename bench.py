@@ -177,6 +177,8 @@ def subset_sequences(w, keep):
 
 # ------------------------------------------------------------------------------------------------ GPU leg
 class Runner:
+    score_cluster = 0  # --score-cluster: CTAs per unit in the score kernel (0: the library chooses)
+
     def __init__(self, w, K, L, fast, dev):
         import paper_2604_11288_b200 as ta
         self.ta, self.w, self.K, self.L, self.fast, self.dev = ta, w, K, L, fast, dev
@@ -190,6 +192,8 @@ class Runner:
         self.batch = ta.make_batch(L, w.B, int(w.lengths[0]) if w.uniform else 0, w.max_n, w.total, self.cu)
         self.ctx = ta.ta_ctx_create(dev.index, ta.ta_scratch_bytes(self.batch, w.Hq, w.Hkv, w.d, K, p))
         self.pats = ta.ta_patterns_create(self.ctx, w.pattern_ids, w.pattern_budget, w.pattern_span)
+        if Runner.score_cluster:
+            ta.ta_ctx_set_score_cluster(self.ctx, Runner.score_cluster)
         self.Q, self.Kc, self.Vc = tw.make_qkv(w, range(L), device=dev, need_q=not fast)
         self.idx = torch.empty((L, w.B, w.Hkv, K), dtype=torch.int32, device=dev)
         self.cnt = torch.empty((L, w.B, w.Hkv), dtype=torch.int32, device=dev)
@@ -447,10 +451,12 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="layers per call (default: the workload's layer count)")
     ap.add_argument("--no-extra", action="store_true", help="skip the supplementary workloads and entry points")
     ap.add_argument("--no-other", action="store_true", help="skip the supplementary workloads, keep the entry points")
+    ap.add_argument("--score-cluster", type=int, default=0, help="tuning: CTAs per unit in the score kernel")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     a = ap.parse_args()
 
+    Runner.score_cluster = a.score_cluster
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))

@@ -151,6 +151,15 @@ ta_status ta_ctx_poll(ta_ctx* ctx);
 int ta_ctx_last_cuda_error(const ta_ctx* ctx);
 const char* ta_status_string(ta_status s);
 
+/* Limit of every device-side wait of the kernels launched through this context, in nanoseconds of wall time
+ * (default and 0: two seconds). A wait that runs out makes its kernel return early; ta_ctx_poll then reports
+ * TA_ERR_TIMEOUT once and the outputs of that call are undefined. Meant for callers with their own watchdog and for
+ * tests. */
+ta_status ta_ctx_set_wait_limit(ta_ctx* ctx, uint64_t nanoseconds);
+/* Tuning: CTAs that share one (layer, sequence, KV head) unit in the score kernel: 1, 2, 4 or 8; 0 (default) lets
+ * the library choose per launch from the unit count, the sequence length and the L2 size. */
+ta_status ta_ctx_set_score_cluster(ta_ctx* ctx, int ctas_per_unit);
+
 /* Optional per-kernel timing of ta_compress: when enabled, CUDA events are recorded on the call's stream around
  * each kernel of the next ta_compress calls. ta_ctx_read_timing synchronises on those events and returns the
  * milliseconds of the most recent call in out_ms[0..4] = {mask+static utility, score, select, compact, total}.
@@ -228,6 +237,15 @@ ta_status ta_sponsor_mask_conf(ta_ctx* ctx, const ta_policy* policy, const ta_ba
  * The contraction runs on the tensor cores (bf16 inputs, fp32 accumulation). */
 ta_status ta_score(ta_ctx* ctx, const ta_policy* policy, const ta_batch* batch, int Hq, int Hkv, int d,
                    ta_bf16_view q_obs, ta_bf16_view k, const float* lse_obs, float* A, float* P, void* stream);
+
+/* The attention part of Eq. 1 with its weights applied, u_att_i = alpha*A_i + delta*P_i, as ta_compress computes it
+ * before the attention-free terms are added: the same rows, keys and arguments as ta_score, one output.
+ *   u_att   DEVICE float [L][Hkv][total_tokens], out.
+ * When every row weight alpha + delta*(1-rho)*rho^(W-1-t) is positive (true for the paper's alpha = 1, delta = 0.2)
+ * the weights are folded into the softmax exponents and a key costs a single sum; the result equals
+ * alpha*A + delta*P up to fp32 rounding (relative 1e-3 + absolute 1e-5 against exact arithmetic, as for A and P). */
+ta_status ta_score_weighted(ta_ctx* ctx, const ta_policy* policy, const ta_batch* batch, int Hq, int Hkv, int d,
+                            ta_bf16_view q_obs, ta_bf16_view k, const float* lse_obs, float* u_att, void* stream);
 
 /* ---- step 3: budget-K selection (Algorithm 1 step 8 with the partition of Section 3.3) --------------------
  * Per unit: K_eff = min(K, n). If K_eff == n everything is kept. Otherwise p = k_protected (auto when < 0,

@@ -81,6 +81,9 @@ def lib():
             "ta_detect_embedding": (i32, [vp, C.c_int64, vp, C.c_int64, i32, vp, i32, vp, vp]),
             "ta_sponsor_mask_conf": (i32, [vp, PP, PB, vp, vp, C.c_float, C.c_float, i32, i32, vp, vp, vp, vp]),
             "ta_score": (i32, [vp, PP, PB, i32, i32, i32, ta_bf16_view, ta_bf16_view, vp, vp, vp, vp]),
+            "ta_score_weighted": (i32, [vp, PP, PB, i32, i32, i32, ta_bf16_view, ta_bf16_view, vp, vp, vp]),
+            "ta_ctx_set_wait_limit": (i32, [vp, u64]),
+            "ta_ctx_set_score_cluster": (i32, [vp, i32]),
             "ta_select_topk": (i32, [vp, PP, PB, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]),
             "ta_select_topk_static": (i32, [PP, PB, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]),
             "ta_compact_kv": (i32, [vp, PB, i32, i32, i32, ta_bf16_view, ta_bf16_view, vp, vp, vp, vp, vp]),
@@ -224,6 +227,19 @@ def ta_sponsor_mask(ctx, pats, policy, batch, token_ids, flags, voucher, u_stati
 def ta_score(ctx, policy, batch, Hq, Hkv, d, q_obs: ta_bf16_view, k: ta_bf16_view, lse_obs, A, P, stream=None):
     _check(lib().ta_score(ctx, C.byref(policy), C.byref(batch), Hq, Hkv, d, q_obs, k, _ptr(lse_obs), _ptr(A), _ptr(P),
                           stream), "ta_score")
+
+
+def ta_score_weighted(ctx, policy, batch, Hq, Hkv, d, q_obs: ta_bf16_view, k: ta_bf16_view, lse_obs, u_att, stream=None):
+    _check(lib().ta_score_weighted(ctx, C.byref(policy), C.byref(batch), Hq, Hkv, d, q_obs, k, _ptr(lse_obs),
+                                   _ptr(u_att), stream), "ta_score_weighted")
+
+
+def ta_ctx_set_wait_limit(ctx, nanoseconds: int):
+    _check(lib().ta_ctx_set_wait_limit(ctx, int(nanoseconds)), "ta_ctx_set_wait_limit")
+
+
+def ta_ctx_set_score_cluster(ctx, ctas_per_unit: int):
+    _check(lib().ta_ctx_set_score_cluster(ctx, int(ctas_per_unit)), "ta_ctx_set_score_cluster")
 
 
 def ta_select_topk(ctx, policy, batch, Hkv, K, flags, voucher, u_static, A, P, idx, count, stream=None):

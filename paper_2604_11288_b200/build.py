@@ -50,7 +50,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
             failed = True
     if failed:
         raise RuntimeError("nvcc failed")
-    subprocess.run([nvcc, "-shared", "-o", LIB_PATH] + objs + ["-cudart", "static"], check=True)
+    subprocess.run([nvcc, "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-o", LIB_PATH] + objs +
+                   ["-cudart", "static"], check=True)
     return LIB_PATH
 
 

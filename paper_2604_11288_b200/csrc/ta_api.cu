@@ -272,6 +272,20 @@ ta_status ta_ctx_poll(ta_ctx* ctx) {
 
 int ta_ctx_last_cuda_error(const ta_ctx* ctx) { return ctx ? ctx->last_cuda_error : 0; }
 
+ta_status ta_ctx_set_wait_limit(ta_ctx* ctx, uint64_t nanoseconds) {
+  if (!ctx) return TA_ERR_INVALID_ARG;
+  ctx->wait_limit_ns = nanoseconds;
+  return TA_OK;
+}
+
+ta_status ta_ctx_set_score_cluster(ta_ctx* ctx, int ctas_per_unit) {
+  if (!ctx) return TA_ERR_INVALID_ARG;
+  if (ctas_per_unit != 0 && ctas_per_unit != 1 && ctas_per_unit != 2 && ctas_per_unit != 4 && ctas_per_unit != 8)
+    return TA_ERR_INVALID_ARG;
+  ctx->score_force_cluster = ctas_per_unit;
+  return TA_OK;
+}
+
 ta_status ta_ctx_enable_timing(ta_ctx* ctx, int enable) {
   if (!ctx) return TA_ERR_INVALID_ARG;
   ctx->timing_enabled = enable ? 1 : 0;
@@ -430,9 +444,10 @@ ta_status ta_sponsor_mask_conf(ta_ctx* ctx, const ta_policy* policy, const ta_ba
 }
 
 // ---------------------------------------------------------------------------------------------- step 2
-ta_status ta_score(ta_ctx* ctx, const ta_policy* policy, const ta_batch* batch, int Hq, int Hkv, int d,
-                   ta_bf16_view q_obs, ta_bf16_view k, const float* lse_obs, float* A, float* P, void* stream) {
-  if (!ctx || !A) return TA_ERR_INVALID_ARG;
+static ta_status score_impl(ta_ctx* ctx, const ta_policy* policy, const ta_batch* batch, int Hq, int Hkv, int d,
+                            ta_bf16_view q_obs, ta_bf16_view k, const float* lse_obs, float* A, float* P, float* u,
+                            void* stream) {
+  if (!ctx || (!A && !u)) return TA_ERR_INVALID_ARG;
   ta_status s = check_batch(batch);
   if (s == TA_OK) s = check_policy(policy);
   if (s == TA_OK) s = check_heads(Hq, Hkv, d, policy, true);
@@ -451,8 +466,7 @@ ta_status ta_score(ta_ctx* ctx, const ta_policy* policy, const ta_batch* batch, 
   a.lse_obs = lse_obs;
   a.A = A;
   a.P = P;
-  a.u = nullptr;
-  a.u_static = nullptr;
+  a.u = u;
   a.alpha = policy->alpha;
   a.delta = policy->delta;
   a.rho = policy->pension_rho;
@@ -466,6 +480,18 @@ ta_status ta_score(ta_ctx* ctx, const ta_policy* policy, const ta_batch* batch, 
   }
   cudaError_t e = ta_launch_score(ctx, a, ctx->d_status, (cudaStream_t)stream);
   return e == cudaSuccess ? TA_OK : cuda_fail(ctx, e);
+}
+
+ta_status ta_score(ta_ctx* ctx, const ta_policy* policy, const ta_batch* batch, int Hq, int Hkv, int d,
+                   ta_bf16_view q_obs, ta_bf16_view k, const float* lse_obs, float* A, float* P, void* stream) {
+  if (!A) return TA_ERR_INVALID_ARG;
+  return score_impl(ctx, policy, batch, Hq, Hkv, d, q_obs, k, lse_obs, A, P, nullptr, stream);
+}
+
+ta_status ta_score_weighted(ta_ctx* ctx, const ta_policy* policy, const ta_batch* batch, int Hq, int Hkv, int d,
+                            ta_bf16_view q_obs, ta_bf16_view k, const float* lse_obs, float* u_att, void* stream) {
+  if (!u_att) return TA_ERR_INVALID_ARG;
+  return score_impl(ctx, policy, batch, Hq, Hkv, d, q_obs, k, lse_obs, nullptr, nullptr, u_att, stream);
 }
 
 // ---------------------------------------------------------------------------------------------- step 3
@@ -702,8 +728,7 @@ ta_status compress_impl(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* p
     a.A = nullptr;
     a.P = nullptr;
     a.u = u;
-    a.u_static = nullptr;
-    a.alpha = policy->alpha;
+      a.alpha = policy->alpha;
     a.delta = policy->delta;
     a.rho = policy->pension_rho;
     a.scale = policy->softmax_scale;

@@ -49,6 +49,12 @@ struct ta_ctx {
   cudaEvent_t ev_fork, ev_join;
   // launch shape of the most recent score kernel (diagnostics)
   int score_cluster, score_clusters;
+  // score kernel launch state per instantiation (2 row-block counts x 3 output forms): attribute set, resident
+  // clusters per cluster size (0: not queried yet, -1: does not fit)
+  int score_attr_set[6];
+  int score_max_clusters[6][9];
+  int score_force_cluster;            // > 0: CTAs per unit fixed by ta_ctx_set_option (tuning, tests)
+  unsigned long long wait_limit_ns;   // 0: default limit of device-side waits
   // driver entry point for tensor-map encoding (resolved at create time)
   void* encode_tiled;
 };
@@ -90,7 +96,6 @@ struct ta_score_args {
   float* A;              // nullable
   float* P;              // nullable
   float* u;              // nullable: fused attention part alpha*A + delta*P (u_static is added by the selection)
-  const float* u_static; // unused
   float alpha, delta, rho, scale;
   int causal;
   int reserve_sms;       // SMs left free for kernels running beside the (persistent) score kernel

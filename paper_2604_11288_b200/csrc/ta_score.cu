@@ -1,12 +1,12 @@
 // Step 2 of the retention path: the attention terms of Eq. 1 (A_i, the pension P_i) over the observation window,
-// optionally fused with the rest of the utility. sm_100a only: TMA tile loads, tcgen05 tensor-core MMAs with the
+// optionally fused with their weights alpha and delta. sm_100a only: TMA tile loads, tcgen05 tensor-core MMAs with the
 // accumulators in tensor memory, and a thread-block cluster per unit for the softmax statistics.
 //
 // For unit (l, b, g) the score matrix is S = Q_obs[heads of g] * K^T, M = G*W rows (<= 256) by n keys. Each row is
 // softmax-normalised over the keys it may see and the result is summed over rows per key. The normaliser of a row
 // needs every key before any column sum can be finished, so the keys are swept twice:
 //   pass 1  S = Q * Ktile^T   (TMEM lane = query row)  -> reference and sum of exponentials per row
-//   pass 2  S^T = Ktile * Q^T (TMEM lane = key)        -> A_i = sum_rows exp2(s*c - lse_row), P_i likewise
+//   pass 2  S^T = Ktile * Q^T (TMEM lane = key)        -> sum over rows of exp2(s*c - beta_row) per key
 // Both passes use the same shared-memory operand tiles (both K-major, 128-byte swizzle); only the roles in the
 // instruction descriptor swap, which puts the reduction axis of each pass along a thread's own registers.
 // A unit is handled by a cluster of 1, 2, 4 or 8 CTAs (chosen per launch: one CTA when there are many units, more when
@@ -17,15 +17,25 @@
 //
 // The grid is persistent: as many clusters as the device can hold at once, each walking over units
 // cluster, cluster + n_clusters, ...; the TMA and MMA warps run ahead across pass and unit boundaries (double-buffered
-// query tile, ring of key tiles, one accumulator stage per softmax group or two where tensor memory allows), so
-// barrier set-up, TMEM allocation and pipeline fill are paid once per CTA and not once per unit.
+// query tile, ring of key tiles, one accumulator stage per softmax group or pair of groups), so barrier set-up, TMEM
+// allocation and pipeline fill are paid once per CTA and not once per unit.
 //
-// Warp roles: NG softmax warpgroups (3 for M = 128, 2 for M = 256) that take the jobs round-robin, plus one warpgroup
-// with the TMA producer warp, the MMA issuer warp (TMEM owner) and two idle warps. After set-up that last warpgroup
-// gives registers back (setmaxnreg) and the softmax warpgroups take them. Every wait on an mbarrier is bounded by
-// wall time; when one runs out the CTA records TA_ERR_TIMEOUT, stops waiting anywhere, drains its copies, frees its
-// tensor memory and returns. The only unbounded waits are two hardware cluster barriers (start, end) that every
-// thread reaches on every path.
+// Warp roles: four softmax warpgroups plus one warpgroup with the TMA producer warp, the MMA issuer warp (TMEM owner)
+// and two idle warps. A "job" is one key tile in one pass. With up to 128 score rows (MB 1) the four groups take the
+// jobs round-robin, one accumulator stage of 128 columns each. With 129..256 rows (MB 2) an accumulator stage holds
+// 256 columns and a pair of groups shares each job: in pass 1 each group of the pair owns one block of 128 rows, in
+// pass 2 each sums half of the rows for the tile's keys and the two halves are added through shared memory.
+// After set-up the last warpgroup gives registers back (setmaxnreg) and the softmax warpgroups take them.
+//
+// The softmax warps are bound by instruction issue and by the special-function unit (one ex2 per score element and
+// pass), so a fixed share of the exponentials (2 of every 16 with 256 score rows) is evaluated on the FMA pipe instead: the argument is
+// clamped to [-126, 126] with a saturating multiply-add, split into integer and fraction with the 1.5*2^23 rounding
+// trick, 2^fraction comes from a cubic polynomial (relative error 7.5e-5) and the integer part goes into the exponent
+// field with an integer add.
+//
+// Every wait on an mbarrier is bounded by wall time; when one runs out the CTA records TA_ERR_TIMEOUT, its producer
+// and MMA warps stop issuing work, the copies and MMAs in flight are drained, and the softmax warps finish their loops
+// without waiting or storing. The only unbounded waits are hardware barriers that every thread reaches on every path.
 #include <cuda.h>
 
 #include <type_traits>
@@ -42,20 +52,29 @@ constexpr int kD = TA_HEAD_DIM;                   // 128
 constexpr int kHalfBytes = kTileN * 128;          // one 64-column half of a 128-row operand tile: 16 KB
 constexpr int kKTileBytes = 2 * kHalfBytes;       // 32 KB
 constexpr int kMaxCluster = 8;
-// NG softmax warpgroups (4 warps each) plus one warpgroup holding the TMA producer warp, the MMA issuer warp and
-// two idle warps. Register split after set-up (setmaxnreg); the shares must fit in threads x registers at launch:
-//   NG = 2: 384 threads x 168 = 64512 = 8*32*216 + 4*32*72        NG = 3: 512 threads x 128 = 65536 = 12*32*152 + 4*32*56
-//   NG = 4: 640 threads x  96 = 61440 = 16*32*112 + 4*32*32
-// The softmax warps wait on the chain accumulator load -> multiply-add -> ex2 -> add rather than on issue slots, so one
-// more warp per scheduler pays where the loops fit its smaller register share: sweep 2 with the pension term then adds
-// every exponential straight into two sums (PM 3) instead of keeping 32 per-position partial sums in registers.
-template <int NG>
-struct GroupCfg {
-  static constexpr int kThreads = (NG + 1) * 128;
-  static constexpr int kRegsSoftmax = NG == 2 ? 216 : NG == 3 ? 152 : 112;
-  static constexpr int kRegsOther = NG == 2 ? 72 : NG == 3 ? 56 : 32;
-  static constexpr int kRegsNeeded = (NG * 4 * kRegsSoftmax + 4 * kRegsOther) * 32;
-};
+constexpr int kGroups = 4;                        // softmax warpgroups
+constexpr int kThreads = (kGroups + 1) * 128;     // 640
+// Register split after set-up (setmaxnreg); the shares must fit in threads x registers at launch:
+// 640 threads x 96 = 61440 = 16*32*112 + 4*32*32
+constexpr int kRegsSoftmax = 112;
+constexpr int kRegsOther = 32;
+constexpr int kRegsNeeded = (kGroups * 4 * kRegsSoftmax + 4 * kRegsOther) * 32;
+
+// Of every 16 exponentials, this many run on the FMA pipe. Measured on B200: with up to 128 score rows the softmax
+// warps are not what limits the kernel (replacing every ex2 by a multiply changes its duration by 3 %) and any
+// polynomial share costs issue slots (0: 119 us, 4: 129 us on 32 layers x 4096 tokens); with 256 rows the
+// special-function unit is the longest pole and 2 of 16 is the best share (1.69 -> 1.62 ms on 2 layers of 16 x 32768).
+#ifndef TA_SCORE_POLY_MB1
+#define TA_SCORE_POLY_MB1 0
+#endif
+#ifndef TA_SCORE_POLY_MB2
+#define TA_SCORE_POLY_MB2 2
+#endif
+
+// how pass 2 turns the exponentials of a key into outputs
+constexpr int kOutA = 0;      // A only
+constexpr int kOutAP = 3;     // A and P (per-row pension weights), or their weighted sum
+constexpr int kOutFused = 4;  // alpha*A + delta*P with the positive row weights folded into the exponent
 
 struct ScoreParams {
   ta_seq_desc seq;
@@ -68,38 +87,39 @@ struct ScoreParams {
   float c;            // softmax scale * log2(e)
   float alpha, delta;
   const float* lse_obs;
-  const float* u_static;
   const int32_t* order;  // nullable: the clusters walk units order[0], order[1], .. (longest sequences first)
   float* A;
   float* P;
   float* u;
   ta_dev_status* status;
+  unsigned long long wait_limit_ns;
   float wrow[TA_MAX_WINDOW];  // pension weight of window row t (for W' = W; shorter sequences are handled in-kernel)
-  float rho;
 };
 
 // ---------------------------------------------------------------------------------------------- shared memory
-template <int MB, int NG>
+template <int MB>
 struct ScoreCfg {
   static constexpr int kQBufs = MB == 1 ? 2 : 1;   // query tiles in flight (next unit's tile loads early)
   static constexpr int kStages = MB == 1 ? 4 : 3;  // ring of key tiles
   static constexpr int kRowsPad = MB * 128;
-  // accumulator stages in tensor memory (at most 512 columns): two per softmax group when they fit (the group can
-  // then fetch its next job before releasing the current one), else one per group
-  static constexpr int kAcc = MB == 1 ? (NG == 3 ? 3 : 4) : 2;
+  static constexpr int kAcc = MB == 1 ? 4 : 2;     // accumulator stages of kRowsPad columns (512 columns in all)
+  static constexpr int kWarpsPerJob = MB * 4;      // softmax warps that read one accumulator stage
 };
 
-template <int MB, int NG>
+template <int MB>
 struct alignas(1024) ScoreSmem {
-  using Cfg = ScoreCfg<MB, NG>;
+  using Cfg = ScoreCfg<MB>;
   uint8_t q[Cfg::kQBufs][MB * 2 * kHalfBytes];    // [buffer][half][MB*128 rows][128 B]
   uint8_t k[Cfg::kStages][kKTileBytes];           // [stage][half][128 rows][128 B]
   float mine_m[2][MB * 128];                      // [unit parity][row]: this CTA's row statistics, read by its peers
   float mine_z[2][MB * 128];
-  float part_m[NG][MB * 128];                     // per softmax group
-  float part_z[NG][MB * 128];
-  float lse2[2][MB * 128];                        // [unit parity][row] log2-domain log-sum-exp (+inf: row is mute)
+  float part_m[kGroups][128];                     // per softmax group: MB 1 rows 0..127; MB 2 rows of block (group & 1)
+  float part_z[kGroups][128];
+  float tab[2][MB * 128];                         // [unit parity][row] pass-2 constant of the row (see row constants)
+  float nbeta[2][MB * 128];                       // [unit parity][row] -beta (masked tiles use ex2 for every row)
   float wrow[MB * 128];                           // pension weight per row
+  float lv[MB * 128];                             // log2 of the row's output weight (kOutFused), else 0
+  float pair_sum[2][2][2][128];                   // MB 2: [pair][job parity][A|P][key] partial sums of the second group
   int row_t[MB * 128];                            // window index t of the row, -1 for padding rows
   unsigned long long full[Cfg::kStages], empty[Cfg::kStages], acc_full[Cfg::kAcc], acc_empty[Cfg::kAcc];
   unsigned long long q_full[Cfg::kQBufs], q_empty[Cfg::kQBufs], xchg_full[2], drain;
@@ -107,37 +127,61 @@ struct alignas(1024) ScoreSmem {
   int abort_flag;
 };
 
-// Pass-2 order of the 32-row chunks of an accumulator (as a TMEM column offset). With W = 64 and the pension term
-// (PM 2) the chunks holding window positions 0..31 of every head come first, then those holding 32..63.
-template <int MB, int PM>
-__device__ __forceinline__ uint32_t chunk_col(int ci) {
-  if (PM == 2) return (uint32_t)((ci < 2 * MB ? 2 * ci : 2 * (ci - 2 * MB) + 1) * 32);
-  return (uint32_t)(ci * 32);
-}
-
 struct UnitInfo {
   int l, b, g, tok0, n, t_begin, T;
 };
 
+// ---------------------------------------------------------------------------------------------- exponentials
+// Position q of a 16-element group runs on the FMA pipe when this is true (the positions are spread evenly).
+template <int MB>
+__host__ __device__ constexpr bool poly_slot(int q) {
+  constexpr int kPoly = MB == 1 ? TA_SCORE_POLY_MB1 : TA_SCORE_POLY_MB2;
+  return ((q * kPoly) / 16) != (((q + 1) * kPoly) / 16);
+}
+
+constexpr float kPolyRange = 252.0f;                // width of the clamped argument range [-126, 126]
+constexpr float kPolyMagic = 12582912.0f - 126.0f;  // 1.5 * 2^23 - 126: adding it leaves the integer part in the low bits
+// minimax cubic for 2^f on [0, 1) in relative error (7.5e-5)
+constexpr float kC0 = 0.9999251961708069f, kC1 = 0.6958335638046265f, kC2 = 0.22606715559959412f,
+                kC3 = 0.07802452147006989f;
+
+__device__ __forceinline__ float fma_sat(float a, float b, float c) {
+  float d;
+  asm("fma.rn.sat.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+// exp2(x) for x = s*c - beta clamped to [-126, 126], given c252 = c/252 and bias = (126 - beta)/252
+__device__ __forceinline__ float exp2_poly(float s, float c252, float bias) {
+  const float t = fma_sat(s, c252, bias);                 // (x + 126) / 252 in [0, 1]
+  const float y = __fmaf_rd(t, kPolyRange, kPolyMagic);   // 1.5*2^23 + floor(x)
+  const float w = kPolyMagic - y;                         // -126 - floor(x), exact
+  const float f = fmaf(t, kPolyRange, w);                 // x - floor(x)
+  float p = fmaf(kC3, f, kC2);
+  p = fmaf(p, f, kC1);
+  p = fmaf(p, f, kC0);
+  return __int_as_float((__float_as_int(y) << 23) + __float_as_int(p));
+}
+__device__ __forceinline__ float poly_bias(float beta) { return (126.0f - beta) * (1.0f / kPolyRange); }
+
 // ---------------------------------------------------------------------------------------------- the kernel
-template <int MB, int PM, int NG>
-__global__ void __launch_bounds__(GroupCfg<NG>::kThreads, 1)
+template <int MB, int PM>
+__global__ void __launch_bounds__(kThreads, 1)
 ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                 const __grid_constant__ ScoreParams p) {
-  using Cfg = ScoreCfg<MB, NG>;
-  constexpr int kThreads = GroupCfg<NG>::kThreads;
-  constexpr int kWarpTma = NG * 4, kWarpMma = NG * 4 + 1;
+  using Cfg = ScoreCfg<MB>;
+  constexpr int kWarpTma = kGroups * 4, kWarpMma = kGroups * 4 + 1;
   constexpr int kStages = Cfg::kStages, kQBufs = Cfg::kQBufs, kRowsPad = Cfg::kRowsPad;
   constexpr int kAcc = Cfg::kAcc;
   constexpr uint32_t kTmemCols = 512;  // kAcc accumulator stages of kRowsPad columns
   extern __shared__ uint8_t smem_raw[];
-  ScoreSmem<MB, NG>& sm = *reinterpret_cast<ScoreSmem<MB, NG>*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  ScoreSmem<MB>& sm = *reinterpret_cast<ScoreSmem<MB>*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const uint32_t rank = cluster_ctarank();
   const int cluster_id = blockIdx.x / p.cluster;
   const int n_clusters = gridDim.x / p.cluster;
   volatile int* abort_flag = &sm.abort_flag;
+  const unsigned long long limit = p.wait_limit_ns;
 
   // `walk` = cluster_id + round * n_clusters. With a length-sorted order the rounds are taken in alternating
   // direction (the cluster that got the longest unit of one round gets the shortest of the next), which evens out the
@@ -160,7 +204,8 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     ui.l = u / (p.Hkv * p.seq.batch);
     ui.tok0 = ta_seq_begin(p.seq, ui.b);
     int n = (p.seq.cu ? p.seq.cu[ui.b + 1] : ui.tok0 + p.seq.n_uniform) - ui.tok0;
-    if (n > p.seq.max_n || n < 0) {  // the selection step rejects this sequence; here it is simply skipped
+    // a sequence that does not lie inside the token arrays is skipped here and rejected by the selection step
+    if (n > p.seq.max_n || n < 0 || ui.tok0 < 0 || (long long)ui.tok0 + n > p.seq.total) {
       if (tid == 0 && atomicCAS(&p.status->code, 0, (int)TA_ERR_DEVICE_BOUNDS) == 0) {
         p.status->where = 2;
         p.status->detail0 = ui.b;
@@ -184,7 +229,7 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     }
     for (int a = 0; a < kAcc; ++a) {
       mbar_init(smem_u32(&sm.acc_full[a]), 1);
-      mbar_init(smem_u32(&sm.acc_empty[a]), 4);
+      mbar_init(smem_u32(&sm.acc_empty[a]), Cfg::kWarpsPerJob);
     }
     for (int a = 0; a < 2; ++a) mbar_init(smem_u32(&sm.xchg_full[a]), (uint32_t)p.cluster);
     for (int qb = 0; qb < kQBufs; ++qb) {
@@ -204,7 +249,10 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
   for (int r = tid; r < kRowsPad; r += kThreads) {
     const int t = r < p.rows ? r % p.W : -1;
     sm.row_t[r] = t;
-    sm.wrow[r] = t >= 0 ? p.wrow[t] : 0.0f;  // (1-rho) rho^(W-1-t); also right for W' < W (same exponent)
+    const float w = t >= 0 ? p.wrow[t] : 0.0f;  // (1-rho) rho^(W-1-t); also right for W' < W (same exponent)
+    sm.wrow[r] = w;
+    // kOutFused: the row's contribution alpha + delta*w (positive, checked by the host) goes into the exponent
+    sm.lv[r] = (PM == kOutFused && t >= 0) ? log2f(fmaf(p.delta, w, p.alpha)) : 0.0f;
   }
   // Rows of the query tile that the TMA box does not cover are multiplied like any other row: make them zeros so
   // that the padded score columns are finite.
@@ -229,125 +277,137 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
   const uint32_t k_smem = smem_u32(sm.k);
 
   if (warp >= kWarpTma) {
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(GroupCfg<NG>::kRegsOther));
-  if (warp == kWarpTma) {
-    // =========================================================================== TMA producer
-    if (lane == 0) {
-      int issued[kStages];
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsOther));
+    if (warp == kWarpTma) {
+      // =========================================================================== TMA producer
+      if (lane == 0) {
+        int issued[kStages], q_issued[kQBufs];
 #pragma unroll
-      for (int s = 0; s < kStages; ++s) issued[s] = 0;
-      int jg = 0, qn = 0;
-      for (int u = cluster_id; u - cluster_id < p.units; u += n_clusters) {
-        const UnitInfo ui = get_unit(u);
-        if (ui.T == 0) continue;
-        const int qb = qn % kQBufs;
-        mbar_wait(smem_u32(&sm.q_empty[qb]), ((uint32_t)(qn / kQBufs) & 1u) ^ 1u, abort_flag, p.status, 11);
-        {
-          const uint32_t bar = smem_u32(&sm.q_full[qb]);
-          const uint32_t dst = smem_u32(sm.q[qb]);
-          mbar_expect_tx(bar, (uint32_t)(2 * p.rows * 128));
-          tma_load_5d(dst, &map_q, bar, 0, 0, ui.g * p.G, ui.b, ui.l);
-          tma_load_5d(dst + MB * kHalfBytes, &map_q, bar, 64, 0, ui.g * p.G, ui.b, ui.l);
-        }
-        ++qn;
-        const int row0 = p.seq.cu ? ui.tok0 : 0;  // ragged: tokens are packed along the row axis
-        const int bc = p.seq.cu ? 0 : ui.b;
-        const int n_jobs = p.two_pass ? 2 * ui.T : ui.T;
-        for (int j = 0; j < n_jobs; ++j, ++jg) {
-          const int s = jg % kStages;
-          mbar_wait(smem_u32(&sm.empty[s]), ((uint32_t)(jg / kStages) & 1u) ^ 1u, abort_flag, p.status, 10);
-          // the second sweep walks the CTA's tiles backwards: the tiles read last are the ones still in L2
-          const int tile = ui.t_begin + (j >= ui.T ? 2 * ui.T - 1 - j : j);
-          const uint32_t bar = smem_u32(&sm.full[s]);
-          mbar_expect_tx(bar, kKTileBytes);
-          const uint32_t dst = k_smem + s * kKTileBytes;
-          tma_load_5d(dst, &map_k, bar, 0, row0 + tile * kTileN, ui.g, bc, ui.l);
-          tma_load_5d(dst + kHalfBytes, &map_k, bar, 64, row0 + tile * kTileN, ui.g, bc, ui.l);
-          issued[s] = jg + 1;
-        }
-      }
-      if (*abort_flag) {  // drain: every armed stage must have landed before the CTA may leave
-        for (int s = 0; s < kStages; ++s) {
-          if (!issued[s]) continue;
-          const uint32_t ph = (uint32_t)((issued[s] - 1) / kStages) & 1u;
-          const unsigned long long t0 = globaltimer_ns();
-          while (!mbar_try_wait(smem_u32(&sm.full[s]), ph) && globaltimer_ns() - t0 < kWaitLimitNs) {
+        for (int s = 0; s < kStages; ++s) issued[s] = 0;
+#pragma unroll
+        for (int s = 0; s < kQBufs; ++s) q_issued[s] = 0;
+        int jg = 0, qn = 0;
+        bool ok = true;
+        for (int u = cluster_id; ok && u - cluster_id < p.units; u += n_clusters) {
+          const UnitInfo ui = get_unit(u);
+          if (ui.T == 0) continue;
+          const int qb = qn % kQBufs;
+          ok = mbar_wait(smem_u32(&sm.q_empty[qb]), ((uint32_t)(qn / kQBufs) & 1u) ^ 1u, abort_flag, p.status, 11, limit);
+          if (!ok) break;  // nothing may be copied into a buffer that was not handed back
+          {
+            const uint32_t bar = smem_u32(&sm.q_full[qb]);
+            const uint32_t dst = smem_u32(sm.q[qb]);
+            mbar_expect_tx(bar, (uint32_t)(2 * p.rows * 128));
+            tma_load_5d(dst, &map_q, bar, 0, 0, ui.g * p.G, ui.b, ui.l);
+            tma_load_5d(dst + MB * kHalfBytes, &map_q, bar, 64, 0, ui.g * p.G, ui.b, ui.l);
+            q_issued[qb] = qn + 1;
+          }
+          ++qn;
+          const int row0 = p.seq.cu ? ui.tok0 : 0;  // ragged: tokens are packed along the row axis
+          const int bc = p.seq.cu ? 0 : ui.b;
+          const int n_jobs = p.two_pass ? 2 * ui.T : ui.T;
+          for (int j = 0; j < n_jobs; ++j, ++jg) {
+            const int s = jg % kStages;
+            ok = mbar_wait(smem_u32(&sm.empty[s]), ((uint32_t)(jg / kStages) & 1u) ^ 1u, abort_flag, p.status, 10, limit);
+            if (!ok) break;
+            // the second sweep walks the CTA's tiles backwards: the tiles read last are the ones still in L2
+            const int tile = ui.t_begin + (j >= ui.T ? 2 * ui.T - 1 - j : j);
+            const uint32_t bar = smem_u32(&sm.full[s]);
+            mbar_expect_tx(bar, kKTileBytes);
+            const uint32_t dst = k_smem + s * kKTileBytes;
+            tma_load_5d(dst, &map_k, bar, 0, row0 + tile * kTileN, ui.g, bc, ui.l);
+            tma_load_5d(dst + kHalfBytes, &map_k, bar, 64, row0 + tile * kTileN, ui.g, bc, ui.l);
+            issued[s] = jg + 1;
           }
         }
+        if (!ok || *abort_flag) {
+          // drain: every copy that was started must have landed before the CTA may leave. A stage is only ever armed
+          // after its previous contents were handed back, so at most the last copy per stage can still be in flight.
+          for (int s = 0; s < kStages; ++s)
+            if (issued[s]) mbar_wait_drain(smem_u32(&sm.full[s]), (uint32_t)((issued[s] - 1) / kStages) & 1u, limit);
+          for (int s = 0; s < kQBufs; ++s)
+            if (q_issued[s]) mbar_wait_drain(smem_u32(&sm.q_full[s]), (uint32_t)((q_issued[s] - 1) / kQBufs) & 1u, limit);
+        }
       }
-    }
-  } else if (warp == kWarpMma) {
-    // =========================================================================== MMA issuer
-    if (lane == 0) {
-      int jg = 0, qn = 0;
-      const uint64_t dk_base = smem_desc_sw128(k_smem);
-      const uint32_t idesc1 = idesc_bf16(128, kTileN), idesc2 = idesc_bf16(128, kRowsPad);
-      for (int u = cluster_id; u - cluster_id < p.units; u += n_clusters) {
-        const UnitInfo ui = get_unit(u);
-        if (ui.T == 0) continue;
-        const int qb = qn % kQBufs;
-        mbar_wait(smem_u32(&sm.q_full[qb]), (uint32_t)(qn / kQBufs) & 1u, abort_flag, p.status, 22);
-        const uint64_t dq = smem_desc_sw128(smem_u32(sm.q[qb]));
-        const int n_jobs = p.two_pass ? 2 * ui.T : ui.T;
-        for (int j = 0; j < n_jobs; ++j, ++jg) {
-          const int s = jg % kStages;
-          const int a = jg % kAcc;
-          const bool stats = p.two_pass && j < ui.T;
-          mbar_wait(smem_u32(&sm.full[s]), (uint32_t)(jg / kStages) & 1u, abort_flag, p.status, 20);
-          mbar_wait(smem_u32(&sm.acc_empty[a]), ((uint32_t)(jg / kAcc) & 1u) ^ 1u, abort_flag, p.status, 21);
-          tc_fence_after();
-          const uint64_t dk = dk_base + (uint64_t)((uint32_t)(s * kKTileBytes) >> 4);
-          const uint32_t acc = tmem_base + (uint32_t)(a * kRowsPad);
-          if (stats) {
+    } else if (warp == kWarpMma) {
+      // =========================================================================== MMA issuer
+      if (lane == 0) {
+        int jg = 0, qn = 0;
+        bool ok = true;
+        // operand descriptors: the upper word is the same for every tile; the lower word is the address >> 4
+        const uint32_t desc_hi = (uint32_t)(smem_desc_sw128(0) >> 32);
+        const uint32_t k_lo = (k_smem & 0x3FFFFu) >> 4;
+        const uint32_t idesc1 = idesc_bf16(128, kTileN), idesc2 = idesc_bf16(128, kRowsPad);
+        for (int u = cluster_id; ok && u - cluster_id < p.units; u += n_clusters) {
+          const UnitInfo ui = get_unit(u);
+          if (ui.T == 0) continue;
+          const int qb = qn % kQBufs;
+          ok = mbar_wait(smem_u32(&sm.q_full[qb]), (uint32_t)(qn / kQBufs) & 1u, abort_flag, p.status, 22, limit);
+          if (!ok) break;
+          const uint32_t q_lo = (smem_u32(sm.q[qb]) & 0x3FFFFu) >> 4;
+          const int n_jobs = p.two_pass ? 2 * ui.T : ui.T;
+          for (int j = 0; j < n_jobs; ++j, ++jg) {
+            const int s = jg % kStages;
+            const int a = jg % kAcc;
+            const bool stats = p.two_pass && j < ui.T;
+            ok = mbar_wait(smem_u32(&sm.full[s]), (uint32_t)(jg / kStages) & 1u, abort_flag, p.status, 20, limit) &&
+                 mbar_wait(smem_u32(&sm.acc_empty[a]), ((uint32_t)(jg / kAcc) & 1u) ^ 1u, abort_flag, p.status, 21, limit);
+            if (!ok) break;  // no product is issued on operands or into an accumulator that are not ready
+            tc_fence_after();
+            const uint32_t dk_lo = k_lo + (uint32_t)((s * kKTileBytes) >> 4);
+            const uint32_t acc = tmem_base + (uint32_t)(a * kRowsPad);
+            if (stats) {
 #pragma unroll
-            for (int mb = 0; mb < MB; ++mb) {
+              for (int mb = 0; mb < MB; ++mb) {
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                  const uint32_t da = q_lo + (uint32_t)(((k >> 2) * (MB * kHalfBytes) + mb * kHalfBytes + (k & 3) * 32) >> 4);
+                  const uint32_t db = dk_lo + (uint32_t)(((k >> 2) * kHalfBytes + (k & 3) * 32) >> 4);
+                  umma_bf16_lo(acc + mb * 128, da, db, desc_hi, idesc1, k > 0);
+                }
+              }
+            } else {
 #pragma unroll
               for (int k = 0; k < 8; ++k) {
-                const uint64_t da = dq + (uint64_t)(((k >> 2) * (MB * kHalfBytes) + mb * kHalfBytes + (k & 3) * 32) >> 4);
-                const uint64_t db = dk + (uint64_t)(((k >> 2) * kHalfBytes + (k & 3) * 32) >> 4);
-                umma_bf16(acc + mb * 128, da, db, idesc1, k > 0);
+                const uint32_t da = dk_lo + (uint32_t)(((k >> 2) * kHalfBytes + (k & 3) * 32) >> 4);
+                const uint32_t db = q_lo + (uint32_t)(((k >> 2) * (MB * kHalfBytes) + (k & 3) * 32) >> 4);
+                umma_bf16_lo(acc, da, db, desc_hi, idesc2, k > 0);
               }
             }
-          } else {
-#pragma unroll
-            for (int k = 0; k < 8; ++k) {
-              const uint64_t da = dk + (uint64_t)(((k >> 2) * kHalfBytes + (k & 3) * 32) >> 4);
-              const uint64_t db = dq + (uint64_t)(((k >> 2) * (MB * kHalfBytes) + (k & 3) * 32) >> 4);
-              umma_bf16(acc, da, db, idesc2, k > 0);
-            }
+            umma_commit(smem_u32(&sm.empty[s]));
+            umma_commit(smem_u32(&sm.acc_full[a]));
           }
-          umma_commit(smem_u32(&sm.empty[s]));
-          umma_commit(smem_u32(&sm.acc_full[a]));
+          if (!ok) break;
+          umma_commit(smem_u32(&sm.q_empty[qb]));  // the query tile may be overwritten once these MMAs are done
+          ++qn;
         }
-        umma_commit(smem_u32(&sm.q_empty[qb]));  // the query tile may be overwritten once these MMAs are done
-        ++qn;
-      }
-      if (*abort_flag) {  // make sure no MMA is still writing tensor memory before it is freed
-        umma_commit(smem_u32(&sm.drain));
-        const unsigned long long t0 = globaltimer_ns();
-        while (!mbar_try_wait(smem_u32(&sm.drain), 0) && globaltimer_ns() - t0 < kWaitLimitNs) {
+        if (!ok || *abort_flag) {  // make sure no MMA is still writing tensor memory before it is freed
+          umma_commit(smem_u32(&sm.drain));
+          mbar_wait_drain(smem_u32(&sm.drain), 0, limit);
         }
       }
     }
-  }
   } else {
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(GroupCfg<NG>::kRegsSoftmax));
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmax));
     // =========================================================================== softmax warps
-    const int st = tid;                   // 0..255
-    const int grp = st >> 7;              // this group serves jobs with (global job index % NG) == grp
-    constexpr bool kAhead = (kAcc >= 2 * NG);  // two stages per group: fetch the next job before releasing this one
-    const int quad = warp & 3;            // TMEM lane quadrant this warp may read
+    constexpr int kShare = kAcc;            // jobs are dealt round-robin to kShare groups (MB 1) or pairs (MB 2)
+    const int st = tid;                     // 0..511
+    const int grp = st >> 7;
+    const int slot = MB == 1 ? grp : grp >> 1;   // serves jobs with (global job index % kShare) == slot
+    const int half = MB == 1 ? 0 : grp & 1;      // MB 2: which 128 accumulator columns of the job
+    const int coff = half * 128;
+    const int quad = warp & 3;              // TMEM lane quadrant this warp may read
     const int row_in_tile = quad * 32 + lane;
-    const uint32_t tlane = tmem_base + ((uint32_t)(quad * 32) << 16);
+    const uint32_t tlane = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)coff;
     const float c = p.c;
-    const int n_chunks2 = (p.rows + 31) >> 5;
-    int my_t[MB];
-#pragma unroll
-    for (int mb = 0; mb < MB; ++mb) my_t[mb] = sm.row_t[mb * 128 + row_in_tile];
+    const float c252 = c * (1.0f / kPolyRange);
+    const int my_t = sm.row_t[coff + row_in_tile];  // pass 1: this thread's row is coff + row_in_tile
+    const int rows_mine = min(128, p.rows - coff);
+    const int n_chunks2 = (rows_mine + 31) >> 5;
 
     auto acc_addr = [&](int jj) { return tlane + (uint32_t)((jj % kAcc) * kRowsPad); };
     auto wait_full = [&](int jj, int where) {
-      mbar_wait(smem_u32(&sm.acc_full[jj % kAcc]), (uint32_t)(jj / kAcc) & 1u, abort_flag, p.status, where);
+      mbar_wait(smem_u32(&sm.acc_full[jj % kAcc]), (uint32_t)(jj / kAcc) & 1u, abort_flag, p.status, where, limit);
       tc_fence_after();
     };
     auto release = [&](int jj) {  // the whole accumulator of the job is in registers: hand the stage back
@@ -365,32 +425,25 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 
       if (p.two_pass) {
         // ---- pass 1: per row, sum of exp2(s*c - ref) against a reference `ref` that only has to keep the sum inside
-        // the fp32 range (the result does not depend on it). Two forms, chosen by what measured faster:
-        //  * one row block per job (MB 1): ref is the largest of the first 16 keys the row sees; after that a key
-        //    costs one multiply-add, one ex2 and one add, and no maximum is tracked. A tile whose sum leaves the safe
-        //    range (a score more than 2^60 above ref) is redone against its own maximum. That check must not wait
-        //    for the tile's last exponentials (the accumulator stage is released right after it, and the group's next
-        //    product waits for the release): it uses the sum without the last 16 keys and, for those, their largest
-        //    score.
-        //  * two row blocks per job (MB 2; there the form above came out 6-10 % slower, with the redo path merely
-        //    present): ref trails the running maximum; the exponentials of a tile use the reference left by the
-        //    previous tiles, and only when the tile's maximum is more than 2^8 ahead of it is the tile redone.
-        float ref_c[MB], z_run[MB];
-        int lim_row[MB];
-#pragma unroll
-        for (int mb = 0; mb < MB; ++mb) {
-          z_run[mb] = 0.0f;
-          const int pos = n - p.W + my_t[mb];
-          lim_row[mb] = (my_t[mb] >= 0 && pos >= 0) ? (p.causal ? pos : n - 1) : -1;
-          // rows that see no key (padding) get a reference that turns every exponential into 0
-          ref_c[mb] = lim_row[mb] >= 0 ? -1e30f : 1e30f;
-        }
+        // the fp32 range (the result does not depend on it): the largest of the first 16 keys the row sees. After that
+        // a key costs one multiply-add, one exponential and one add, and no maximum is tracked. A tile whose sum
+        // leaves the safe range (a score more than 2^60 above ref) is redone against its own maximum. That check must
+        // not wait for the tile's last exponentials (the accumulator stage is released right after it, and the next
+        // product into the stage waits for the release): it uses the sum without the last 16 keys and, for those,
+        // their largest score. The polynomial exponentials saturate at 2^126, which the same check catches.
+        float ref_c, z_run = 0.0f, pb;
+        const int pos = n - p.W + my_t;
+        const int lim = (my_t >= 0 && pos >= 0) ? (p.causal ? pos : n - 1) : -1;
+        // rows that see no key (padding) get a reference that turns every exponential into 0
+        ref_c = lim >= 0 ? -1e30f : 1e30f;
+        pb = poly_bias(ref_c);
         constexpr float kSumLimit = 1.0e18f;  // about 2^60
-        // 16 keys of one row (half of a 32-key chunk): adds exp2(s*c - rc) to `sum`; with `track_tag` set also
-        // tracks the largest s in `mx`. Masked tiles (cold) drop keys beyond `lim`.
-        auto half1 = [&](auto masked_tag, auto track_tag, const float(&cur)[16], float rc, float& sum, float& mx,
-                         int kbase, int lim) {
+        // 16 keys of one row: adds exp2(s*c - rc) to the four sums; `mix`: kPoly of them on the FMA pipe;
+        // `track`: also the largest s in `mx`. Masked tiles (cold) drop keys beyond `lim`.
+        auto half1 = [&](auto masked_tag, auto mix_tag, auto track_tag, const float(&cur)[16], float rc, float pbias,
+                         float(&s4)[4], float& mx, int kbase) {
           constexpr bool masked = decltype(masked_tag)::value;
+          constexpr bool mix = decltype(mix_tag)::value && !masked;
           constexpr bool track = decltype(track_tag)::value;
           float v[16];
 #pragma unroll
@@ -400,13 +453,10 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             for (int q = 0; q < 16; ++q)
               if (kbase + q > lim) v[q] = -INFINITY;
           }
-          float a0 = 0.0f, a1 = 0.0f, a2 = 0.0f, a3 = 0.0f;
 #pragma unroll
-          for (int q = 0; q < 16; q += 4) {
-            a0 += ex2(fmaf(v[q + 0], c, -rc));
-            a1 += ex2(fmaf(v[q + 1], c, -rc));
-            a2 += ex2(fmaf(v[q + 2], c, -rc));
-            a3 += ex2(fmaf(v[q + 3], c, -rc));
+          for (int q = 0; q < 16; ++q) {
+            const float e = (mix && poly_slot<MB>(q)) ? exp2_poly(v[q], c252, pbias) : ex2(fmaf(v[q], c, -rc));
+            s4[q & 3] += e;
           }
           if (track) {
             float t4[4];
@@ -414,10 +464,9 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             for (int q = 0; q < 4; ++q) t4[q] = fmaxf(fmaxf(v[4 * q], v[4 * q + 1]), fmaxf(v[4 * q + 2], v[4 * q + 3]));
             mx = fmaxf(mx, fmaxf(fmaxf(t4[0], t4[1]), fmaxf(t4[2], t4[3])));
           }
-          sum += (a0 + a1) + (a2 + a3);
         };
         // largest of 16 keys of one row
-        auto max16 = [&](auto masked_tag, const float(&cur)[16], float& mx, int kbase, int lim) {
+        auto max16 = [&](auto masked_tag, const float(&cur)[16], float& mx, int kbase) {
           constexpr bool masked = decltype(masked_tag)::value;
           float t4[4];
 #pragma unroll
@@ -430,170 +479,122 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           mx = fmaxf(mx, fmaxf(fmaxf(t4[0], t4[1]), fmaxf(t4[2], t4[3])));
         };
         float ra[16], rb[16];
-        int j = (grp - jg % NG + NG) % NG;  // first job of this pass that belongs to the group
+        int j = (slot - jg % kShare + kShare) % kShare;  // first job of this pass that belongs to the group
         if (j < T) {
           wait_full(jg + j, 30);
           tmem_ld16_issue(acc_addr(jg + j), ra);
         }
-        // One job: the accumulator in 32-column chunks, each fetched as two 16-column loads (ra, rb) so that one
-        // load is always in flight; the next job's first load is issued before the last half-chunk is computed.
-        // On entry of every row block the load of its first 16 columns is in flight in `ra`.
+        // One job: the 128 accumulator columns in 32-column chunks, each fetched as two 16-column loads (ra, rb) so
+        // that one load is always in flight. On entry the load of the first 16 columns is in flight in `ra`.
         auto job1 = [&](auto masked_tag, int j) {
           const int jj = jg + j;
           const int key0 = (ui.t_begin + j) * kTileN;
           const uint32_t abase = acc_addr(jj);
-#pragma unroll
-          for (int mb = 0; mb < MB; ++mb) {
-            if constexpr (MB == 1) {
-              const int lim = lim_row[mb];
-              float rc = ref_c[mb];
-              const bool first = rc < -1e29f;
-              if (__any_sync(0xffffffffu, first)) {  // the row has no reference yet: take it from the 16 keys in flight
-                float mx = -INFINITY;
-                tmem_ld_wait(ra);
-                max16(masked_tag, ra, mx, key0, lim);
-                if (first && mx > -INFINITY) {
-                  rc = mx * c;
-                  ref_c[mb] = rc;
-                }
-              }
-              float sum = 0.0f, sum_head = 0.0f, mx_tail = -INFINITY, unused = 0.0f;
-#pragma unroll 1
-              for (int c4 = 0; c4 < 4; ++c4) {
-                const uint32_t col = (uint32_t)(mb * 128 + c4 * 32);
-                tmem_ld_wait(ra);
-                tmem_ld16_issue(abase + col + 16, rb);
-                half1(masked_tag, std::false_type{}, ra, rc, sum, unused, key0 + c4 * 32, lim);
-                tmem_ld_wait(rb);
-                if (mb == MB - 1 && c4 == 3) {
-                  // with more than one stage per group the next job's accumulator is a different stage: fetch ahead
-                  if (kAhead && j + NG < T) {
-                    wait_full(jj + NG, 30);
-                    tmem_ld16_issue(acc_addr(jj + NG), ra);
-                  }
-                } else {
-                  tmem_ld16_issue(abase + col + 32, ra);
-                }
-                if (c4 < 3) {
-                  half1(masked_tag, std::false_type{}, rb, rc, sum, unused, key0 + c4 * 32 + 16, lim);
-                } else {
-                  sum_head = sum;
-                  half1(masked_tag, std::true_type{}, rb, rc, sum, mx_tail, key0 + c4 * 32 + 16, lim);
-                }
-              }
-              // also true for inf and NaN sums
-              const bool over = !(sum_head < kSumLimit) || fmaf(mx_tail, c, -rc) > 60.0f;
-              if (__any_sync(0xffffffffu, over)) {   // rare: a score far above the reference
-                float mx = -INFINITY;
-#pragma unroll 1
-                for (int h = 0; h < 8; ++h) {
-                  tmem_ld16_issue(abase + (uint32_t)(mb * 128 + h * 16), rb);
-                  tmem_ld_wait(rb);
-                  max16(masked_tag, rb, mx, key0 + h * 16, lim);
-                }
-                const float mx_c = mx * c;
-                float sum2 = 0.0f;
-#pragma unroll 1
-                for (int h = 0; h < 8; ++h) {
-                  tmem_ld16_issue(abase + (uint32_t)(mb * 128 + h * 16), rb);
-                  tmem_ld_wait(rb);
-                  half1(masked_tag, std::false_type{}, rb, over ? mx_c : rc, sum2, unused, key0 + h * 16, lim);
-                }
-                if (over) {
-                  z_run[mb] *= ex2(rc - mx_c);
-                  ref_c[mb] = mx_c;
-                  sum = sum2;
-                }
-              }
-              z_run[mb] += sum;
-            } else {
-              const int lim = lim_row[mb];
-              const float rc = ref_c[mb];
-              float sum = 0.0f, mx = -INFINITY;
-#pragma unroll 1
-              for (int c4 = 0; c4 < 4; ++c4) {
-                const uint32_t col = (uint32_t)(mb * 128 + c4 * 32);
-                tmem_ld_wait(ra);
-                tmem_ld16_issue(abase + col + 16, rb);
-                half1(masked_tag, std::true_type{}, ra, rc, sum, mx, key0 + c4 * 32, lim);
-                tmem_ld_wait(rb);
-                if (mb == MB - 1 && c4 == 3) {
-                  // with more than one stage per group the next job's accumulator is a different stage: fetch ahead
-                  if (kAhead && j + NG < T) {
-                    wait_full(jj + NG, 30);
-                    tmem_ld16_issue(acc_addr(jj + NG), ra);
-                  }
-                } else {
-                  tmem_ld16_issue(abase + col + 32, ra);
-                }
-                half1(masked_tag, std::true_type{}, rb, rc, sum, mx, key0 + c4 * 32 + 16, lim);
-              }
-              const float mx_c = mx * c;
-              const bool jump = mx_c > rc + 8.0f;
-              if (__any_sync(0xffffffffu, jump)) {  // rare: first tiles of a unit, or a score far above all before
-                float sum2 = 0.0f, mx2 = -INFINITY;
-#pragma unroll 1
-                for (int h = 0; h < 8; ++h) {
-                  tmem_ld16_issue(abase + (uint32_t)(mb * 128 + h * 16), rb);
-                  tmem_ld_wait(rb);
-                  half1(masked_tag, std::true_type{}, rb, jump ? mx_c : rc, sum2, mx2, key0 + h * 16, lim);
-                }
-                if (jump) {
-                  z_run[mb] *= ex2(rc - mx_c);
-                  ref_c[mb] = mx_c;
-                  sum = sum2;
-                }
-              }
-              z_run[mb] += sum;
+          float rc = ref_c;
+          const bool first = rc < -1e29f;
+          if (__any_sync(0xffffffffu, first)) {  // the row has no reference yet: take it from the 16 keys in flight
+            float mx = -INFINITY;
+            tmem_ld_wait(ra);
+            max16(masked_tag, ra, mx, key0);
+            if (first && mx > -INFINITY) {
+              rc = mx * c;
+              ref_c = rc;
+              pb = poly_bias(rc);
             }
           }
+          float s4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+          float sum_head = 0.0f, mx_tail = -INFINITY, unused = 0.0f;
+#pragma unroll 1
+          for (int c4 = 0; c4 < 4; ++c4) {
+            const uint32_t col = (uint32_t)(c4 * 32);
+            tmem_ld_wait(ra);
+            tmem_ld16_issue(abase + col + 16, rb);
+            half1(masked_tag, std::true_type{}, std::false_type{}, ra, rc, pb, s4, unused, key0 + c4 * 32);
+            tmem_ld_wait(rb);
+            if (c4 < 3) {
+              tmem_ld16_issue(abase + col + 32, ra);
+              half1(masked_tag, std::true_type{}, std::false_type{}, rb, rc, pb, s4, unused, key0 + c4 * 32 + 16);
+            } else {
+              sum_head = (s4[0] + s4[1]) + (s4[2] + s4[3]);
+              half1(masked_tag, std::true_type{}, std::true_type{}, rb, rc, pb, s4, mx_tail, key0 + c4 * 32 + 16);
+            }
+          }
+          float sum = (s4[0] + s4[1]) + (s4[2] + s4[3]);
+          // also true for inf and NaN sums
+          const bool over = !(sum_head < kSumLimit) || fmaf(mx_tail, c, -rc) > 60.0f;
+          if (__any_sync(0xffffffffu, over)) {   // rare: a score far above the reference
+            float mx = -INFINITY;
+#pragma unroll 1
+            for (int h = 0; h < 8; ++h) {
+              tmem_ld16_issue(abase + (uint32_t)(h * 16), rb);
+              tmem_ld_wait(rb);
+              max16(masked_tag, rb, mx, key0 + h * 16);
+            }
+            const float mx_c = mx * c;
+            float r4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll 1
+            for (int h = 0; h < 8; ++h) {
+              tmem_ld16_issue(abase + (uint32_t)(h * 16), rb);
+              tmem_ld_wait(rb);
+              half1(masked_tag, std::false_type{}, std::false_type{}, rb, over ? mx_c : rc, 0.0f, r4, unused,
+                    key0 + h * 16);
+            }
+            if (over) {
+              z_run *= ex2(rc - mx_c);
+              ref_c = mx_c;
+              pb = poly_bias(mx_c);
+              sum = (r4[0] + r4[1]) + (r4[2] + r4[3]);
+            }
+          }
+          z_run += sum;
           release(jj);
-          if (!kAhead && j + NG < T) {  // one stage per group: the next job can only be fetched once this one is released
-            wait_full(jj + NG, 30);
-            tmem_ld16_issue(acc_addr(jj + NG), ra);
+          if (j + kShare < T) {  // the next job of the group reuses this stage: fetch it once it is full again
+            wait_full(jj + kShare, 30);
+            tmem_ld16_issue(acc_addr(jj + kShare), ra);
           }
         };
-        for (; j < T; j += NG) {
+        for (; j < T; j += kShare) {
           // tiles that every row of the warp sees completely take the unmasked path (rows that see nothing at all,
           // i.e. padding, still run: their sums are never used)
-          bool masked = false;
-#pragma unroll
-          for (int mb = 0; mb < MB; ++mb)
-            masked = masked || (lim_row[mb] >= 0 && (ui.t_begin + j) * kTileN + kTileN - 1 > lim_row[mb]);
+          const bool masked = lim >= 0 && (ui.t_begin + j) * kTileN + kTileN - 1 > lim;
           if (__any_sync(0xffffffffu, masked)) job1(std::true_type{}, j);
           else job1(std::false_type{}, j);
         }
         // ---- exchange: group partials -> CTA partial -> every CTA of the cluster reads every other's
-#pragma unroll
-        for (int mb = 0; mb < MB; ++mb) {
-          // rows that see no key at all (padding, window positions before the sequence start) stay mute
-          sm.part_m[grp][mb * 128 + row_in_tile] = lim_row[mb] >= 0 ? ref_c[mb] : -1e30f;
-          sm.part_z[grp][mb * 128 + row_in_tile] = lim_row[mb] >= 0 ? z_run[mb] : 0.0f;
-        }
-        softmax_bar<NG>();
+        // rows that see no key at all (padding, window positions before the sequence start) stay mute
+        sm.part_m[grp][row_in_tile] = lim >= 0 ? ref_c : -1e30f;
+        sm.part_z[grp][row_in_tile] = lim >= 0 ? z_run : 0.0f;
+        softmax_bar<kGroups>();
+        float lse2_row = INFINITY;  // log2-domain log-sum-exp of row `st` (+inf: the row is mute)
         if (st < kRowsPad) {
-          float m = sm.part_m[0][st];
+          float m, z = 0.0f;
+          if (MB == 1) {
+            m = sm.part_m[0][st];
 #pragma unroll
-          for (int gq = 1; gq < NG; ++gq) m = fmaxf(m, sm.part_m[gq][st]);
-          float z = 0.0f;
+            for (int gq = 1; gq < kGroups; ++gq) m = fmaxf(m, sm.part_m[gq][st]);
 #pragma unroll
-          for (int gq = 0; gq < NG; ++gq) z += sm.part_z[gq][st] * ex2(sm.part_m[gq][st] - m);
+            for (int gq = 0; gq < kGroups; ++gq) z += sm.part_z[gq][st] * ex2(sm.part_m[gq][st] - m);
+          } else {  // rows of block h were summed by groups h and h + 2
+            const int h = st >> 7, i = st & 127;
+            m = fmaxf(sm.part_m[h][i], sm.part_m[h + 2][i]);
+            z = sm.part_z[h][i] * ex2(sm.part_m[h][i] - m) + sm.part_z[h + 2][i] * ex2(sm.part_m[h + 2][i] - m);
+          }
           if (p.cluster == 1) {  // nothing to exchange: the CTA's statistics are the unit's
-            sm.lse2[up][st] = (z > 0.0f) ? m + log2f(z) : INFINITY;
+            lse2_row = (z > 0.0f) ? m + log2f(z) : INFINITY;
           } else {
             sm.mine_m[up][st] = m;
             sm.mine_z[up][st] = z;
           }
         }
-        softmax_bar<NG>();
         if (p.cluster > 1) {
+          softmax_bar<kGroups>();
           // one thread per peer tells that peer that this CTA's statistics of the unit are in place
           if (st < p.cluster) {
             fence_cluster();
             mbar_arrive_remote(smem_u32(&sm.xchg_full[up]), (uint32_t)st);
           }
           if (st < kRowsPad) {
-            mbar_wait_cluster(smem_u32(&sm.xchg_full[up]), (uint32_t)(it >> 1) & 1u, abort_flag, p.status, 32);
+            mbar_wait_cluster(smem_u32(&sm.xchg_full[up]), (uint32_t)(it >> 1) & 1u, abort_flag, p.status, 32, limit);
             float pm[kMaxCluster], pz[kMaxCluster];
 #pragma unroll
             for (int r = 0; r < kMaxCluster; ++r) {
@@ -610,10 +611,15 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             float z = 0.0f;
 #pragma unroll
             for (int r = 0; r < kMaxCluster; ++r) z += pz[r] * ex2(pm[r] - m);
-            sm.lse2[up][st] = (z > 0.0f) ? m + log2f(z) : INFINITY;
+            lse2_row = (z > 0.0f) ? m + log2f(z) : INFINITY;
           }
-          softmax_bar<NG>();
         }
+        if (st < kRowsPad) {
+          const float beta = lse2_row - sm.lv[st];
+          sm.nbeta[up][st] = -beta;
+          sm.tab[up][st] = poly_slot<MB>(st & 15) ? poly_bias(beta) : -beta;
+        }
+        softmax_bar<kGroups>();
       } else {
         if (st < kRowsPad) {
           float lse2 = INFINITY;
@@ -623,119 +629,117 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             const float lse = p.lse_obs[(((long long)ui.l * p.seq.batch + ui.b) * p.Hq + (ui.g * p.G + h)) * p.W + t];
             lse2 = lse * 1.4426950408889634f;
           }
-          sm.lse2[up][st] = lse2;
+          const float beta = lse2 - sm.lv[st];
+          sm.nbeta[up][st] = -beta;
+          sm.tab[up][st] = poly_slot<MB>(st & 15) ? poly_bias(beta) : -beta;
         }
-        softmax_bar<NG>();
+        softmax_bar<kGroups>();
       }
 
-      // ---- pass 2: column sums for key row_in_tile of each tile
+      // ---- pass 2: for key row_in_tile of each tile, the sum over this group's rows of exp2(s*c - beta_row)
       const int min_lim = p.causal ? n - Wp : n - 1;  // every valid row sees keys up to here
       const int j0 = p.two_pass ? T : 0;
       const int n_jobs = j0 + T;
       const long long unit_off = ((long long)ui.l * p.Hkv + ui.g) * p.seq.total;
-      const float4* l4 = reinterpret_cast<const float4*>(sm.lse2[up]);
-      const float4* w4 = reinterpret_cast<const float4*>(sm.wrow);
+      const float4* tab4 = reinterpret_cast<const float4*>(sm.tab[up] + coff);
+      const float4* nb4 = reinterpret_cast<const float4*>(sm.nbeta[up] + coff);
+      const float4* w4 = reinterpret_cast<const float4*>(sm.wrow + coff);
       {
-        float sT[32];  // PM 0..2: partial column sums per register position (window position q % W); PM 3: unused
-        float sA = 0.0f, sP = 0.0f;
-        // 16 rows (half `hi` of the 32-row chunk cc) of this thread's key; masked: keys inside the observation
-        // window (cold tiles only)
+        float sA4[4], sP = 0.0f;
+        // 16 rows (half `hi` of the 32-row chunk cc) of this thread's key. Hot form: kPoly of the 16 exponentials on
+        // the FMA pipe, row constants from `tab`. Masked form (keys inside the observation window, cold tiles only):
+        // every exponential on the special-function unit against -beta, rows that do not see the key dropped.
         auto chunk2 = [&](auto masked_tag, auto hi_tag, const float(&cur)[16], int cc, int key) {
           constexpr bool masked = decltype(masked_tag)::value;
           constexpr int hi = decltype(hi_tag)::value;  // 0: rows 32cc..32cc+15, 1: rows 32cc+16..32cc+31
 #pragma unroll
           for (int q4 = 0; q4 < 4; ++q4) {
-            const float4 ls = l4[cc * 8 + hi * 4 + q4];
+            const float4 tb = masked ? nb4[cc * 8 + hi * 4 + q4] : tab4[cc * 8 + hi * 4 + q4];
+            const float tbv[4] = {tb.x, tb.y, tb.z, tb.w};
             float a[4];
-            a[0] = ex2(fmaf(cur[4 * q4 + 0], c, -ls.x));
-            a[1] = ex2(fmaf(cur[4 * q4 + 1], c, -ls.y));
-            a[2] = ex2(fmaf(cur[4 * q4 + 2], c, -ls.z));
-            a[3] = ex2(fmaf(cur[4 * q4 + 3], c, -ls.w));
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              a[e] = (!masked && poly_slot<MB>(4 * q4 + e)) ? exp2_poly(cur[4 * q4 + e], c252, tbv[e])
+                                                        : ex2(fmaf(cur[4 * q4 + e], c, tbv[e]));
+            }
             if (masked) {  // row r sees key i only if i <= the row's own position
 #pragma unroll
               for (int e = 0; e < 4; ++e) {
-                const int t = sm.row_t[cc * 32 + hi * 16 + 4 * q4 + e];
+                const int t = sm.row_t[coff + cc * 32 + hi * 16 + 4 * q4 + e];
                 const int pos = n - p.W + t;
                 const int lim = (t >= 0 && pos >= 0) ? (p.causal ? pos : n - 1) : -1;
                 if (key > lim) a[e] = 0.0f;
               }
             }
-            if (PM == 3) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) sA4[e] += a[e];
+            if (PM == kOutAP) {
               const float4 ws = w4[cc * 8 + hi * 4 + q4];
-              sA += (a[0] + a[1]) + (a[2] + a[3]);
               sP = fmaf(ws.x, a[0], sP);
               sP = fmaf(ws.y, a[1], sP);
               sP = fmaf(ws.z, a[2], sP);
               sP = fmaf(ws.w, a[3], sP);
-            } else {
-#pragma unroll
-              for (int e = 0; e < 4; ++e) sT[hi * 16 + 4 * q4 + e] += a[e];
             }
-          }
-        };
-        // fold the per-position sums into A (and P with the weights starting at w4[wbase])
-        auto fold = [&](int wbase) {
-#pragma unroll
-          for (int q4 = 0; q4 < 8; ++q4) {
-            sA += (sT[4 * q4] + sT[4 * q4 + 1]) + (sT[4 * q4 + 2] + sT[4 * q4 + 3]);
-            if (PM == 1 || PM == 2) {
-              const float4 ws = w4[wbase + q4];
-              sP = fmaf(ws.x, sT[4 * q4 + 0], sP);
-              sP = fmaf(ws.y, sT[4 * q4 + 1], sP);
-              sP = fmaf(ws.z, sT[4 * q4 + 2], sP);
-              sP = fmaf(ws.w, sT[4 * q4 + 3], sP);
-            }
-            sT[4 * q4] = sT[4 * q4 + 1] = sT[4 * q4 + 2] = sT[4 * q4 + 3] = 0.0f;
           }
         };
         float ra[16], rb[16];
-        int j = j0 + (grp - (jg + j0) % NG + NG) % NG;
+        int j = j0 + (slot - (jg + j0) % kShare + kShare) % kShare;
         if (j < n_jobs) {
           wait_full(jg + j, 31);
-          tmem_ld16_issue(acc_addr(jg + j) + chunk_col<MB, PM>(0), ra);
+          tmem_ld16_issue(acc_addr(jg + j), ra);
         }
-        // one job: 32-row chunks in the order chunk_col gives, each as two 16-column loads (ra low half, rb high half)
+        // one job: 32-row chunks, each as two 16-column loads (ra low half, rb high half)
         auto job2 = [&](auto masked_tag, int j, int key) {
           const int jj = jg + j;
           const uint32_t abase = acc_addr(jj);
 #pragma unroll 1
           for (int ci = 0; ci < n_chunks2; ++ci) {
-            const uint32_t col = chunk_col<MB, PM>(ci);
-            const int cc = (int)(col >> 5);
+            const uint32_t col = (uint32_t)(ci * 32);
             tmem_ld_wait(ra);
             tmem_ld16_issue(abase + col + 16, rb);
-            chunk2(masked_tag, std::integral_constant<int, 0>{}, ra, cc, key);
+            chunk2(masked_tag, std::integral_constant<int, 0>{}, ra, ci, key);
             tmem_ld_wait(rb);
             if (ci == n_chunks2 - 1) {
               release(jj);
-              if (j + NG < n_jobs) {
-                wait_full(jj + NG, 31);
-                tmem_ld16_issue(acc_addr(jj + NG) + chunk_col<MB, PM>(0), ra);
+              if (j + kShare < n_jobs) {
+                wait_full(jj + kShare, 31);
+                tmem_ld16_issue(acc_addr(jj + kShare), ra);
               }
             } else {
-              tmem_ld16_issue(abase + chunk_col<MB, PM>(ci + 1), ra);
+              tmem_ld16_issue(abase + col + 32, ra);
             }
-            chunk2(masked_tag, std::integral_constant<int, 1>{}, rb, cc, key);
-            // W = 64 with pension: window positions 0..31 end with the first half of the sequence
-            if (PM == 2 && ci == 2 * MB - 1) fold(0);
+            chunk2(masked_tag, std::integral_constant<int, 1>{}, rb, ci, key);
           }
-          if (PM == 2) fold(8);
-          if (PM == 0 || PM == 1) fold(0);
         };
-        for (; j < n_jobs; j += NG) {
+        for (; j < n_jobs; j += kShare) {
           const int key = (ui.t_begin + (p.two_pass ? n_jobs - 1 - j : j)) * kTileN + row_in_tile;
-#pragma unroll
-          for (int q = 0; q < 32; ++q) sT[q] = 0.0f;
-          sA = 0.0f;
+          sA4[0] = sA4[1] = sA4[2] = sA4[3] = 0.0f;
           sP = 0.0f;
           // only the last W-1 keys of a sequence are hidden from some rows: those tiles take the masked path
           if (__all_sync(0xffffffffu, key <= min_lim || key >= n)) job2(std::false_type{}, j, key);
           else job2(std::true_type{}, j, key);
-          if (key < n) {
+          float sA = (sA4[0] + sA4[1]) + (sA4[2] + sA4[3]);
+          if (MB == 2) {  // add the two halves of the rows: the second group of the pair hands its sums to the first
+            const int jpar = ((jg + j) >> 1) & 1;
+            if (half == 1) {
+              sm.pair_sum[slot][jpar][0][row_in_tile] = sA;
+              if (PM == kOutAP) sm.pair_sum[slot][jpar][1][row_in_tile] = sP;
+            }
+            pair_bar(slot);
+            if (half == 0) {
+              sA += sm.pair_sum[slot][jpar][0][row_in_tile];
+              if (PM == kOutAP) sP += sm.pair_sum[slot][jpar][1][row_in_tile];
+            }
+          }
+          if (half == 0 && key < n && !*abort_flag) {
             const long long o = unit_off + ui.tok0 + key;
-            if (p.A) p.A[o] = sA;
-            if (p.P) p.P[o] = sP;
-            if (p.u) p.u[o] = __fadd_rn(__fmul_rn(p.alpha, sA), __fmul_rn(p.delta, sP));
+            if (PM == kOutFused) {
+              p.u[o] = sA;
+            } else {
+              if (p.A) p.A[o] = sA;
+              if (p.P) p.P[o] = sP;
+              if (p.u) p.u[o] = __fadd_rn(__fmul_rn(p.alpha, sA), __fmul_rn(p.delta, sP));
+            }
           }
         }
       }
@@ -755,9 +759,9 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
   cluster_wait();
 }
 
-template <int MB, int NG>
+template <int MB>
 size_t score_smem_bytes() {
-  return sizeof(ScoreSmem<MB, NG>) + 1024;
+  return sizeof(ScoreSmem<MB>) + 1024;
 }
 
 CUresult encode_5d(void* fn, CUtensorMap* map, const void* base, const uint64_t dims[5], const uint64_t strides_el[4],
@@ -779,23 +783,24 @@ CUresult encode_5d(void* fn, CUtensorMap* map, const void* base, const uint64_t 
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
 }
 
-template <int MB, int PM, int NG>
+template <int MB, int PM>
 cudaError_t launch_variant(ta_ctx* ctx, const CUtensorMap& mq, const CUtensorMap& mk, ScoreParams& sp,
                            int tiles_max, int reserve_sms, cudaStream_t stream) {
-  auto kern = ta_score_kernel<MB, PM, NG>;
-  const size_t smem = score_smem_bytes<MB, NG>();
-  constexpr int kThreads = GroupCfg<NG>::kThreads;
-  static bool attr_set_dev[64] = {};  // per device and instantiation; the attribute is sticky
-  bool& attr_set = attr_set_dev[ctx->device & 63];
-  if (!attr_set) {
+  auto kern = ta_score_kernel<MB, PM>;
+  const size_t smem = score_smem_bytes<MB>();
+  // per context (and so per device) and instantiation: the attribute is sticky, the occupancy does not change
+  constexpr int vi = (MB - 1) * 3 + (PM == kOutA ? 0 : PM == kOutAP ? 1 : 2);
+  int* max_clusters = ctx->score_max_clusters[vi];
+  if (!ctx->score_attr_set[vi]) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     // the in-kernel register split must fit in what the launch provides, or the warps asking for more wait forever
     cudaFuncAttributes fa;
     e = cudaFuncGetAttributes(&fa, kern);
     if (e != cudaSuccess) return e;
-    if (fa.numRegs * kThreads < GroupCfg<NG>::kRegsNeeded) return cudaErrorLaunchOutOfResources;
-    attr_set = true;
+    if (fa.numRegs * kThreads < kRegsNeeded) return cudaErrorLaunchOutOfResources;
+    for (int cl = 0; cl <= kMaxCluster; ++cl) max_clusters[cl] = 0;
+    ctx->score_attr_set[vi] = 1;
   }
   cudaLaunchConfig_t cfg = {};
   cfg.blockDim = dim3(kThreads, 1, 1);
@@ -810,13 +815,13 @@ cudaError_t launch_variant(ta_ctx* ctx, const CUtensorMap& mq, const CUtensorMap
   cfg.numAttrs = 1;
   // Persistent grid: as many clusters as can be resident at once (queried once per cluster size). CTAs per unit:
   // the size with the fewest tile-times on the busiest CTA, counting ~1 tile-time of overhead per unit and ~2 more
-  // for the statistics exchange when a unit spans several CTAs.
-  static int max_clusters_dev[64][kMaxCluster + 1] = {};
-  int* max_clusters = max_clusters_dev[ctx->device & 63];
-  int best_cl = 1;
-  long long best_cost = -1;
+  // for the statistics exchange when a unit spans several CTAs. (Choosing more CTAs per unit so that the keys of
+  // all units in flight fit in L2 was measured and lost: 16 x 32768 tokens, 8 CTAs per unit 2.02 ms against 1.63 ms.)
+  int best_cl = ctx->score_force_cluster;
+  long long best_cost = best_cl > 0 ? 0 : -1;
   for (int cl = 1; cl <= kMaxCluster; cl *= 2) {
-    if (cl > 1 && tiles_max < 2 * cl) break;
+    if (ctx->score_force_cluster > 0 && cl != ctx->score_force_cluster) continue;
+    if (cl > 1 && tiles_max < 2 * cl && ctx->score_force_cluster <= 0) break;
     if (max_clusters[cl] == 0) {
       attr[0].val.clusterDim.x = (unsigned)cl;
       cfg.gridDim = dim3((unsigned)(ctx->sm_count / cl * cl), 1, 1);
@@ -825,10 +830,15 @@ cudaError_t launch_variant(ta_ctx* ctx, const CUtensorMap& mq, const CUtensorMap
       if (e != cudaSuccess) return e;
       max_clusters[cl] = n < 1 ? -1 : n;
     }
-    if (max_clusters[cl] < 1) continue;
+    if (max_clusters[cl] < 1) {
+      if (ctx->score_force_cluster > 0) return cudaErrorLaunchOutOfResources;
+      continue;
+    }
+    if (ctx->score_force_cluster > 0) break;
     const int avail = max_clusters[cl] - (reserve_sms + cl - 1) / cl > 0 ? max_clusters[cl] - (reserve_sms + cl - 1) / cl : 1;
     const long long rounds = (sp.units + avail - 1) / avail;
-    const long long cost = rounds * ((tiles_max + cl - 1) / cl + (cl > 1 ? 3 : 1));
+    const long long per_cta = (tiles_max + cl - 1) / cl;
+    const long long cost = rounds * (per_cta + (cl > 1 ? 3 : 1));
     if (best_cost < 0 || cost < best_cost) {
       best_cost = cost;
       best_cl = cl;
@@ -893,12 +903,11 @@ cudaError_t ta_launch_score(ta_ctx* ctx, const ta_score_args& a, ta_dev_status* 
   sp.alpha = a.alpha;
   sp.delta = a.delta;
   sp.lse_obs = a.lse_obs;
-  sp.u_static = a.u_static;
   sp.A = a.A;
   sp.P = a.P;
   sp.u = a.u;
   sp.status = status;
-  sp.rho = a.rho;
+  sp.wait_limit_ns = ctx->wait_limit_ns ? ctx->wait_limit_ns : kWaitLimitNs;
   for (int t = 0; t < a.W; ++t) sp.wrow[t] = (float)((1.0 - (double)a.rho) * pow((double)a.rho, (double)(a.W - 1 - t)));
   sp.units = units;
   sp.order = nullptr;
@@ -929,20 +938,18 @@ cudaError_t ta_launch_score(ta_ctx* ctx, const ta_score_args& a, ta_dev_status* 
     const uint32_t box[5] = {64, (uint32_t)kTileN, 1, 1, 1};
     if (encode_5d(ctx->encode_tiled, &mk, a.k.ptr, dims, str, box) != CUDA_SUCCESS) return cudaErrorInvalidValue;
   }
-  // how the pension term is accumulated: 0 none, 1 W divides 32, 2 W == 64, 3 any W (per-element weights);
-  // one row block: four softmax groups with per-element weights whenever the term is needed
+  // Output form of pass 2. With only the weighted sum alpha*A + delta*P wanted and every row weight
+  // alpha + delta*w_t positive, the weights go into the exponents and a key costs one sum (kOutFused); otherwise A
+  // alone (kOutA) or A and P with per-row weights (kOutAP).
+  bool fused = a.u != nullptr && a.A == nullptr && a.P == nullptr;
+  for (int t = 0; fused && t < a.W; ++t) fused = a.alpha + a.delta * sp.wrow[t] > 0.0f;
   const bool need_p = a.P != nullptr || (a.u != nullptr && a.delta != 0.0f);
-  const int pm = !need_p ? 0 : (32 % a.W == 0) ? 1 : (a.W == 64 && rows == 256) ? 2 : 3;
   if (MB == 1) {
-    switch (pm) {
-      case 0: return launch_variant<1, 0, 3>(ctx, mq, mk, sp, tiles_max, a.reserve_sms, stream);
-      default: return launch_variant<1, 3, 4>(ctx, mq, mk, sp, tiles_max, a.reserve_sms, stream);
-    }
+    if (fused) return launch_variant<1, kOutFused>(ctx, mq, mk, sp, tiles_max, a.reserve_sms, stream);
+    if (need_p) return launch_variant<1, kOutAP>(ctx, mq, mk, sp, tiles_max, a.reserve_sms, stream);
+    return launch_variant<1, kOutA>(ctx, mq, mk, sp, tiles_max, a.reserve_sms, stream);
   }
-  switch (pm) {
-    case 0: return launch_variant<2, 0, 2>(ctx, mq, mk, sp, tiles_max, a.reserve_sms, stream);
-    case 1: return launch_variant<2, 1, 2>(ctx, mq, mk, sp, tiles_max, a.reserve_sms, stream);
-    case 2: return launch_variant<2, 2, 2>(ctx, mq, mk, sp, tiles_max, a.reserve_sms, stream);
-    default: return launch_variant<2, 3, 2>(ctx, mq, mk, sp, tiles_max, a.reserve_sms, stream);
-  }
+  if (fused) return launch_variant<2, kOutFused>(ctx, mq, mk, sp, tiles_max, a.reserve_sms, stream);
+  if (need_p) return launch_variant<2, kOutAP>(ctx, mq, mk, sp, tiles_max, a.reserve_sms, stream);
+  return launch_variant<2, kOutA>(ctx, mq, mk, sp, tiles_max, a.reserve_sms, stream);
 }

@@ -388,6 +388,7 @@ __device__ __forceinline__ void unit_slice(int n, int& lo, int& hi) {
 
 struct SeqInfo {
   int start, n, K_eff, s_take, r_take, p;
+  bool bad;  // the sequence does not lie inside the token arrays (cu_seqlens is device data the host cannot check)
 };
 
 __device__ __forceinline__ SeqInfo seq_info(const ta_seq_desc& seq, int b, int K, int n_sink, int n_recent,
@@ -395,6 +396,8 @@ __device__ __forceinline__ SeqInfo seq_info(const ta_seq_desc& seq, int b, int K
   SeqInfo s;
   s.start = ta_seq_begin(seq, b);
   s.n = (seq.cu ? seq.cu[b + 1] : s.start + seq.n_uniform) - s.start;
+  s.bad = s.n < 0 || s.n > seq.max_n || s.start < 0 || (long long)s.start + s.n > seq.total;
+  if (s.bad) s.n = 0;
   s.K_eff = min(K, s.n);
   int p = k_protected < 0 ? s.K_eff - n_sink - n_recent : k_protected;
   p = max(0, min(p, s.K_eff));
@@ -424,12 +427,12 @@ __global__ void __launch_bounds__(kThreads) ta_forced_kernel(ta_seq_desc seq, in
     r_main += cls * seq.batch;
   }
   const SeqInfo s = seq_info(seq, b, K, n_sink, n_recent, k_protected);
-  if (s.n > seq.max_n || s.n < 0) {
+  if (s.bad) {
     if (threadIdx.x == 0) {
       if (atomicCAS(&status->code, 0, (int)TA_ERR_DEVICE_BOUNDS) == 0) {
         status->where = 3;
         status->detail0 = b;
-        status->detail1 = s.n;
+        status->detail1 = s.start;
       }
       r_main[b] = -2;  // poisoned: the select kernel writes an empty result
     }

@@ -9,7 +9,7 @@
 
 namespace ta_sm100 {
 
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // default limit of a device-side wait: 2 s
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -39,36 +39,6 @@ __device__ __forceinline__ unsigned long long globaltimer_ns() {
   unsigned long long t;
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
-}
-
-// Bounded wait. Returns false (and raises the CTA's abort flag) when the limit is reached or another thread of the
-// CTA already gave up. The common case (the phase has completed) is one inlined try_wait.
-__device__ __forceinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                            ta_dev_status* status, int where) {
-  if (*abort_flag) return false;
-  const unsigned long long t0 = globaltimer_ns();
-  for (;;) {
-#pragma unroll 1
-    for (int it = 0; it < 64; ++it) {
-      if (mbar_try_wait(bar, parity)) return true;
-      __nanosleep(100);  // a polling warp must not eat the issue slots of the softmax warps on its sub-partition
-    }
-    if (*abort_flag) return false;
-    if (globaltimer_ns() - t0 > kWaitLimitNs) {
-      *abort_flag = 1;
-      if (atomicCAS(&status->code, 0, (int)TA_ERR_TIMEOUT) == 0) {
-        status->where = where;
-        status->detail0 = (int)blockIdx.x;
-        status->detail1 = (int)parity;
-      }
-      return false;
-    }
-  }
-}
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                          ta_dev_status* status, int where) {
-  if (mbar_try_wait(bar, parity)) return true;
-  return mbar_wait_slow(bar, parity, abort_flag, status, where);
 }
 
 __device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1,
@@ -102,6 +72,21 @@ __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t desc_a, uint
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n"
       "}\n" ::"r"(tmem_d),
       "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// The same with the descriptors given as their lower words (address >> 4) and the common upper word.
+__device__ __forceinline__ void umma_bf16_lo(uint32_t tmem_d, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi,
+                                             uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      ".reg .b64 da, db;\n"
+      "mov.b64 da, {%1, %3};\n"
+      "mov.b64 db, {%2, %3};\n"
+      "setp.ne.b32 p, %5, 0;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n"
+      "}\n" ::"r"(tmem_d),
+      "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate)
       : "memory");
 }
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
@@ -190,18 +175,31 @@ __device__ __forceinline__ uint32_t idesc_bf16(int M, int N) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 
-// Bounded wait with cluster-scope acquire (for barriers that peers of the cluster arrive on).
-__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                               ta_dev_status* status, int where) {
-  if (mbar_try_wait_cluster(bar, parity)) return true;
+// Bounded wait on an mbarrier phase. Returns false (and raises the CTA's abort flag) when `limit_ns` of wall time
+// have passed or another thread of the CTA already gave up. The common case (the phase has completed) is one inlined
+// try_wait. CLUSTER: the barrier is arrived on by peers of the cluster (acquire at cluster scope).
+template <bool CLUSTER>
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+  if constexpr (CLUSTER) return mbar_try_wait_cluster(bar, parity);
+  else return mbar_try_wait(bar, parity);
+}
+template <bool CLUSTER>
+__device__ __forceinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                            ta_dev_status* status, int where, unsigned long long limit_ns) {
   if (*abort_flag) return false;
-  const unsigned long long t0 = globaltimer_ns();
+  // try_wait suspends the thread in hardware for a while and resumes it as soon as the phase completes, so the loop
+  // needs no sleep of its own. The wall clock is read only once per 64 polls: reading it costs a few hundred cycles,
+  // which on the single MMA-issuing thread would be paid on every hand-over that is not ready at the first poll.
+  unsigned long long t0 = 0;
   for (;;) {
 #pragma unroll 1
     for (int it = 0; it < 64; ++it)
-      if (mbar_try_wait_cluster(bar, parity)) return true;
+      if (mbar_try<CLUSTER>(bar, parity)) return true;
     if (*abort_flag) return false;
-    if (globaltimer_ns() - t0 > kWaitLimitNs) {
+    const unsigned long long now = globaltimer_ns();
+    if (t0 == 0) {
+      t0 = now;
+    } else if (now - t0 > limit_ns) {
       *abort_flag = 1;
       if (atomicCAS(&status->code, 0, (int)TA_ERR_TIMEOUT) == 0) {
         status->where = where;
@@ -212,5 +210,25 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity,
     }
   }
 }
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          ta_dev_status* status, int where, unsigned long long limit_ns) {
+  if (mbar_try_wait(bar, parity)) return true;
+  return mbar_wait_slow<false>(bar, parity, abort_flag, status, where, limit_ns);
+}
+// Wait used while draining after a failed wait: bounded, reports nothing (the failure is already recorded).
+__device__ __forceinline__ void mbar_wait_drain(uint32_t bar, uint32_t parity, unsigned long long limit_ns) {
+  const unsigned long long t0 = globaltimer_ns();
+  while (!mbar_try_wait(bar, parity) && globaltimer_ns() - t0 < limit_ns) __nanosleep(100);
+}
+
+// Bounded wait with cluster-scope acquire (for barriers that peers of the cluster arrive on).
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                                  ta_dev_status* status, int where, unsigned long long limit_ns) {
+  if (mbar_try_wait_cluster(bar, parity)) return true;
+  return mbar_wait_slow<true>(bar, parity, abort_flag, status, where, limit_ns);
+}
+
+// named barrier shared by the two softmax warpgroups of pair `pair` (256 threads); barrier 1 is softmax_bar's
+__device__ __forceinline__ void pair_bar(int pair) { asm volatile("bar.sync %0, 256;" ::"r"(2 + pair) : "memory"); }
 
 }  // namespace ta_sm100
