@@ -156,6 +156,11 @@ const char* ta_status_string(ta_status s);
  * TA_ERR_TIMEOUT once and the outputs of that call are undefined. Meant for callers with their own watchdog and for
  * tests. */
 ta_status ta_ctx_set_wait_limit(ta_ctx* ctx, uint64_t nanoseconds);
+/* Diagnostic for the time-out path: enqueues a kernel of one warp that waits, with a limit of limit_ns (at most one
+ * second), on a barrier that nothing completes, with no copy or tensor-core operation in flight. The kernel returns
+ * when the limit is reached, sets bit 2 of *outcome (DEVICE int32; bits 0 and 1 would mean a wait succeeded), and
+ * the next ta_ctx_poll reports TA_ERR_TIMEOUT once. The context stays usable. */
+ta_status ta_ctx_selftest_wait(ta_ctx* ctx, uint64_t limit_ns, int32_t* outcome, void* stream);
 /* Tuning: CTAs that share one (layer, sequence, KV head) unit in the score kernel: 1, 2, 4 or 8; 0 (default) lets
  * the library choose per launch from the unit count, the sequence length and the L2 size. */
 ta_status ta_ctx_set_score_cluster(ta_ctx* ctx, int ctas_per_unit);

@@ -286,6 +286,13 @@ ta_status ta_ctx_set_score_cluster(ta_ctx* ctx, int ctas_per_unit) {
   return TA_OK;
 }
 
+ta_status ta_ctx_selftest_wait(ta_ctx* ctx, uint64_t limit_ns, int32_t* outcome, void* stream) {
+  if (!ctx || !outcome || limit_ns == 0 || limit_ns > 1000000000ull) return TA_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->device);
+  cudaError_t e = ta_launch_wait_selftest(ctx->d_status, limit_ns, outcome, (cudaStream_t)stream);
+  return e == cudaSuccess ? TA_OK : cuda_fail(ctx, e);
+}
+
 ta_status ta_ctx_enable_timing(ta_ctx* ctx, int enable) {
   if (!ctx) return TA_ERR_INVALID_ARG;
   ctx->timing_enabled = enable ? 1 : 0;

@@ -103,6 +103,11 @@ struct ta_score_args {
 };
 cudaError_t ta_launch_score(ta_ctx* ctx, const ta_score_args& a, ta_dev_status* status, cudaStream_t stream);
 
+// diagnostic: one warp runs into the limit of a bounded wait (TA_ERR_TIMEOUT in `status`); *outcome gets bit 2 set when
+// the kernel ran to its end, bits 0/1 when a wait unexpectedly succeeded
+cudaError_t ta_launch_wait_selftest(ta_dev_status* status, unsigned long long limit_ns, int* outcome,
+                                    cudaStream_t stream);
+
 // ---- step 3 ------------------------------------------------------------------------------------------------
 struct ta_select_args {
   ta_seq_desc seq;

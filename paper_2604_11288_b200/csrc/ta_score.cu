@@ -875,7 +875,33 @@ __global__ void ta_unit_order_kernel(ta_seq_desc seq, int n_layers, int Hkv, int
   }
 }
 
+// One warp that waits, with the bounded waits of the score kernel, on a barrier nothing ever completes: first the CTA-scope
+// form, then (with the abort flag lowered again) the cluster-scope form. Nothing else is in flight.
+__global__ void ta_wait_selftest_kernel(ta_dev_status* status, unsigned long long limit_ns, int* outcome) {
+  __shared__ unsigned long long bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncwarp();
+  volatile int* af = &abort_flag;
+  const bool a = mbar_wait(smem_u32(&bar), 0, af, status, 90, limit_ns);
+  __syncwarp();
+  if (threadIdx.x == 0) abort_flag = 0;
+  __syncwarp();
+  const bool b = mbar_wait_cluster(smem_u32(&bar), 0, af, status, 91, limit_ns);
+  if (threadIdx.x == 0 && outcome) *outcome = (a ? 1 : 0) | (b ? 2 : 0) | 4;  // 4: the kernel ran to its end
+}
+
 }  // namespace
+
+cudaError_t ta_launch_wait_selftest(ta_dev_status* status, unsigned long long limit_ns, int* outcome,
+                                    cudaStream_t stream) {
+  ta_wait_selftest_kernel<<<1, 32, 0, stream>>>(status, limit_ns, outcome);
+  return cudaGetLastError();
+}
 
 // A stride that multiplies a coordinate which is always 0 still has to be a valid tensor-map stride.
 static uint64_t safe_stride(int64_t s, uint64_t dim) { return (dim <= 1 || s <= 0) ? 128 : (uint64_t)s; }
