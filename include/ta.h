@@ -165,6 +165,11 @@ ta_status ta_ctx_selftest_wait(ta_ctx* ctx, uint64_t limit_ns, int32_t* outcome,
  * the library choose per launch from the unit count, the sequence length and the L2 size. */
 ta_status ta_ctx_set_score_cluster(ta_ctx* ctx, int ctas_per_unit);
 
+/* What the most recent ta_compress (or variant) call on this context launched: out[0] = CTAs per unit of the score
+ * kernel, out[1] = its clusters, out[2] = 1 when the selection kernel gathered the retained rows itself (small
+ * budgets; no separate gather kernel), out[3] = kernels of this library the call enqueued. */
+ta_status ta_ctx_last_launch_info(const ta_ctx* ctx, int32_t out[4] /*HOST*/);
+
 /* Optional per-kernel timing of ta_compress: when enabled, CUDA events are recorded on the call's stream around
  * each kernel of the next ta_compress calls. ta_ctx_read_timing synchronises on those events and returns the
  * milliseconds of the most recent call in out_ms[0..4] = {mask+static utility, score, select, compact, total}.

@@ -85,6 +85,7 @@ def lib():
             "ta_ctx_set_wait_limit": (i32, [vp, u64]),
             "ta_ctx_set_score_cluster": (i32, [vp, i32]),
             "ta_ctx_selftest_wait": (i32, [vp, u64, vp, vp]),
+            "ta_ctx_last_launch_info": (i32, [vp, C.POINTER(C.c_int32)]),
             "ta_select_topk": (i32, [vp, PP, PB, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]),
             "ta_select_topk_static": (i32, [PP, PB, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]),
             "ta_compact_kv": (i32, [vp, PB, i32, i32, i32, ta_bf16_view, ta_bf16_view, vp, vp, vp, vp, vp]),
@@ -237,6 +238,13 @@ def ta_score_weighted(ctx, policy, batch, Hq, Hkv, d, q_obs: ta_bf16_view, k: ta
 
 def ta_ctx_set_wait_limit(ctx, nanoseconds: int):
     _check(lib().ta_ctx_set_wait_limit(ctx, int(nanoseconds)), "ta_ctx_set_wait_limit")
+
+
+def ta_ctx_last_launch_info(ctx):
+    """(CTAs per unit of the score kernel, its clusters, selection gathered the rows itself, kernels enqueued)."""
+    out = (C.c_int32 * 4)()
+    _check(lib().ta_ctx_last_launch_info(ctx, out), "ta_ctx_last_launch_info")
+    return list(out)
 
 
 def ta_ctx_selftest_wait(ctx, limit_ns: int, outcome, stream=None):

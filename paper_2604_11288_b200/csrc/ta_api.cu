@@ -293,6 +293,15 @@ ta_status ta_ctx_selftest_wait(ta_ctx* ctx, uint64_t limit_ns, int32_t* outcome,
   return e == cudaSuccess ? TA_OK : cuda_fail(ctx, e);
 }
 
+ta_status ta_ctx_last_launch_info(const ta_ctx* ctx, int32_t out[4]) {
+  if (!ctx || !out) return TA_ERR_INVALID_ARG;
+  out[0] = ctx->score_cluster;
+  out[1] = ctx->score_clusters;
+  out[2] = ctx->last_select_gathered;
+  out[3] = ctx->last_kernel_launches;
+  return TA_OK;
+}
+
 ta_status ta_ctx_enable_timing(ta_ctx* ctx, int enable) {
   if (!ctx) return TA_ERR_INVALID_ARG;
   ctx->timing_enabled = enable ? 1 : 0;
@@ -698,6 +707,8 @@ ta_status compress_impl(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* p
       e = cudaMemcpyAsync(sc + L.class_of, class_of_h, (size_t)batch->n_layers * Hkv * 4, cudaMemcpyHostToDevice, stream);
   }
   const bool select_gathers = ta_select_gathers(sel);
+  ctx->last_select_gathered = select_gathers ? 1 : 0;
+  int launches = 0;  // kernels of this library enqueued by this call
 
   // Per-sequence work (anchor mask, vouchers, static utility, forced set) does not depend on Q/K: in scored mode it
   // runs on the context's side stream beside the score kernel and joins before the per-unit selection.
@@ -715,6 +726,7 @@ ta_status compress_impl(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* p
     if (e == cudaSuccess)
       e = ta_launch_mask(pats, *policy, seq, token_ids, flags, voucher, u_static, hist, ctx->d_status, seq_stream);
     if (e == cudaSuccess) e = ta_launch_forced(sel, ctx->d_status, seq_stream);
+    launches += 3;  // mask, static utility, forced set
     if (timing && e == cudaSuccess) {
       e = cudaEventRecord(ctx->ev[6], seq_stream);
       ctx->ev_ran[0] = 1;
@@ -743,11 +755,13 @@ ta_status compress_impl(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* p
     a.reserve_sms = fork ? 4 : 0;
     a.order_scratch = batch->cu_seqlens ? reinterpret_cast<int32_t*>(sc + L.order) : nullptr;
     e = ta_launch_score(ctx, a, ctx->d_status, stream);
+    launches += a.order_scratch && batch->batch > 1 ? 2 : 1;  // (unit order of a ragged batch,) score
   }
   mark(2);
   if (fork && e == cudaSuccess) e = cudaStreamWaitEvent(stream, ctx->ev_join, 0);
   if (e == cudaSuccess && share_heads) e = ta_launch_headsum(batch->n_layers, Hkv, batch->total_tokens, u, u_all, stream);
   if (e == cudaSuccess && !(fast && reuse)) e = ta_launch_select_units(sel, stream);
+  launches += (share_heads ? 2 : 0) + (fast && reuse ? 0 : 1) + (fast ? 1 : 0) + (select_gathers ? 0 : 1);
   if (e == cudaSuccess && share_heads)
     e = ta_launch_broadcast_heads(batch->n_layers, batch->batch, Hkv, K, idx_lb, count_lb, idx, count, stream);
   if (e == cudaSuccess && fast)
@@ -773,6 +787,7 @@ ta_status compress_impl(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* p
     return cuda_fail(ctx, e);
   }
   ctx->timing_valid = timing ? 1 : 0;
+  ctx->last_kernel_launches = launches;
   ctx->cached_epoch = budgets ? 0 : seq_epoch;
   ctx->cached_total = batch->total_tokens;
   ctx->cached_batch = batch->batch;

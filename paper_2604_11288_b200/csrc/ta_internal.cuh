@@ -53,6 +53,8 @@ struct ta_ctx {
   // clusters per cluster size (0: not queried yet, -1: does not fit)
   int score_attr_set[6];
   int score_max_clusters[6][9];
+  int last_select_gathered;           // the most recent ta_compress let the selection kernel gather the rows
+  int last_kernel_launches;           // kernels enqueued by the most recent ta_compress
   int score_force_cluster;            // > 0: CTAs per unit fixed by ta_ctx_set_option (tuning, tests)
   unsigned long long wait_limit_ns;   // 0: default limit of device-side waits
   // driver entry point for tensor-map encoding (resolved at create time)

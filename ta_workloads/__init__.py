@@ -234,18 +234,17 @@ def make_qkv(w: Workload, layers, device="cpu", need_q=True, need_kv=True):
     """
     layers = list(layers)
     L = len(layers)
-    qs, ks, vs = [], [], []
-    for l in layers:
+    kv_shape = (w.B, w.Hkv, int(w.lengths[0]), w.d) if w.uniform else (w.Hkv, w.total, w.d)
+    # the outputs are allocated once and filled layer by layer (no second copy of a 30 GB cache while stacking)
+    Q = torch.empty((L, w.B, w.Hq, w.W, w.d), dtype=torch.bfloat16, device=device) if need_q else None
+    K = torch.empty((L,) + kv_shape, dtype=torch.bfloat16, device=device) if need_kv else None
+    V = torch.empty((L,) + kv_shape, dtype=torch.bfloat16, device=device) if need_kv else None
+    for i, l in enumerate(layers):
         g = torch.Generator(device=device)
         g.manual_seed(w.seed * 1000 + l)
         if need_q:
-            qs.append(torch.randn((w.B, w.Hq, w.W, w.d), generator=g, device=device, dtype=torch.float32)
-                      .to(torch.bfloat16))
+            Q[i].copy_(torch.randn((w.B, w.Hq, w.W, w.d), generator=g, device=device, dtype=torch.float32))
         if need_kv:
-            shape = (w.B, w.Hkv, int(w.lengths[0]), w.d) if w.uniform else (w.Hkv, w.total, w.d)
-            ks.append(torch.randn(shape, generator=g, device=device, dtype=torch.bfloat16))
-            vs.append(torch.randn(shape, generator=g, device=device, dtype=torch.bfloat16))
-    Q = torch.stack(qs) if need_q else None
-    K = torch.stack(ks) if need_kv else None
-    V = torch.stack(vs) if need_kv else None
+            torch.randn(kv_shape, generator=g, device=device, dtype=torch.bfloat16, out=K[i])
+            torch.randn(kv_shape, generator=g, device=device, dtype=torch.bfloat16, out=V[i])
     return Q, K, V
