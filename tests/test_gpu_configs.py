@@ -152,3 +152,88 @@ def test_config5_ragged_batch():
         _check_units(w, pol, K, Q, Kc, Vc, idx, cnt, ko, vo, V_o, u0_o, units, None)
     finally:
         g.close()
+
+
+def _units_over_rounds(w, L, grid, per_round, extra=()):
+    """Units spread over the rounds a persistent grid of `grid` CTAs makes (unit index = (l*B + b)*Hkv + g), taken
+    from the start, the middle and the end of every round, plus `extra`."""
+    total = L * w.B * w.Hkv
+    picks = set(extra)
+    for r in range((total + grid - 1) // grid):
+        lo, hi = r * grid, min(total, (r + 1) * grid) - 1
+        for u in sorted({lo, (lo + hi) // 2, hi})[:per_round]:
+            picks.add((u // (w.B * w.Hkv), (u // w.Hkv) % w.B, u % w.Hkv))
+    return sorted(picks)
+
+
+def test_config3_several_rounds_of_the_persistent_grid():
+    # the shape the benchmark times (many more units than CTAs, 256 score rows, 256 tiles per unit), at three layers:
+    # 384 units make three rounds; units from every round and from both ends of the batch are recomputed on the host
+    w = tw.config3()
+    K, L = w.K_list[0], 3
+    pol = oracle_policy(K, "THEOREM", W=w.W)
+    Q, Kc, Vc = tw.make_qkv(w, range(L), device="cuda")
+    g = Gpu(w, pol, K, L)
+    try:
+        f_o, V_o, u0_o = oracle.sponsor_mask(w.ids, w.cu, oracle_patterns(w), pol)
+        idx, cnt, ko, vo = g.compress(Q, Kc, Vc)
+        torch.cuda.synchronize()
+        assert g.poll() == ta.TA_OK
+        assert (cnt == K).all()
+        units = _units_over_rounds(w, L, 144, 3, extra=[(0, 0, 0), (L - 1, w.B - 1, w.Hkv - 1)])
+        assert len(units) >= 8
+        _check_units(w, pol, K, Q, Kc, Vc, idx, cnt, ko, vo, V_o, u0_o, units, None)
+    finally:
+        g.close()
+
+
+def test_config5_two_layers_sorted_walk():
+    # two layers of the ragged batch: 1024 units walk the length-sorted order in alternating directions over several
+    # rounds; the longest and the shortest sequences (first and last entries of that order) are checked in both layers
+    w = tw.config5()
+    K, L = w.K_list[0], 2
+    pol = oracle_policy(K, "THEOREM", W=w.W)
+    Q, Kc, Vc = tw.make_qkv(w, range(L), device="cuda")
+    g = Gpu(w, pol, K, L)
+    try:
+        f_o, V_o, u0_o = oracle.sponsor_mask(w.ids, w.cu, oracle_patterns(w), pol)
+        idx, cnt, ko, vo = g.compress(Q, Kc, Vc)
+        torch.cuda.synchronize()
+        assert g.poll() == ta.TA_OK
+        order = np.argsort(-w.lengths, kind="stable")
+        ends = [int(order[0]), int(order[1]), int(order[-2]), int(order[-1])]
+        units = [(l, b, h) for l in range(L) for b in ends for h in (0, w.Hkv - 1)]
+        units += _sample_units(w, L, 4, 11)
+        assert len(set(units)) >= 16
+        _check_units(w, pol, K, Q, Kc, Vc, idx, cnt, ko, vo, V_o, u0_o, sorted(set(units)), None)
+    finally:
+        g.close()
+
+
+def test_long_units_two_row_blocks_more_units_than_ctas():
+    # 168 units of 33-40 tiles with 256 score rows on a grid of fewer CTAs (two rounds), ragged, with guard layers
+    # behind every output
+    rng = np.random.default_rng(77)
+    lengths = rng.integers(4200, 5100, size=21).astype(np.int32)
+    from test_gpu_steps import _workload
+    w = _workload(lengths, [[3, 4], [9]], seed=31, Hq=32, Hkv=8, W=64)
+    K, L, guard = 96, 1, 2
+    pol = oracle_policy(K, "THEOREM", W=64)
+    Q, Kc, Vc = tw.make_qkv(w, range(L))
+    g = Gpu(w, pol, K, L)
+    try:
+        f_o, V_o, u0_o = oracle.sponsor_mask(w.ids, w.cu, oracle_patterns(w), pol)
+        idx = torch.full((L + guard, w.B, w.Hkv, K), -7, dtype=torch.int32, device="cuda")
+        cnt = torch.full((L + guard, w.B, w.Hkv), -7, dtype=torch.int32, device="cuda")
+        ko = torch.full((L + guard, w.B, w.Hkv, K, w.d), 1.0, dtype=torch.bfloat16, device="cuda")
+        vo = torch.full_like(ko, 1.0)
+        Qd, Kd, Vd = Q.cuda(), Kc.cuda(), Vc.cuda()
+        ta.ta_compress(g.ctx, g.pats, g.p, g.batch, w.Hq, w.Hkv, w.d, K, g.ids, ta.view(Qd), ta.view(Kd, True),
+                       ta.view(Vd, True), 0, ko, vo, idx, cnt, g.stream)
+        torch.cuda.synchronize()
+        assert g.poll() == ta.TA_OK
+        assert (idx[L:] == -7).all() and (cnt[L:] == -7).all() and (ko[L:] == 1.0).all() and (vo[L:] == 1.0).all()
+        units = _units_over_rounds(w, L, 144, 3)
+        _check_units(w, pol, K, Q, Kc, Vc, idx[:L], cnt[:L], ko[:L], vo[:L], V_o, u0_o, units, None)
+    finally:
+        g.close()
