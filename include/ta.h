@@ -329,6 +329,23 @@ ta_status ta_compress_allheads(ta_ctx* ctx, const ta_patterns* pats, const ta_po
                                ta_bf16_view k, ta_bf16_view v, uint64_t seq_epoch, void* k_out, void* v_out,
                                int32_t* idx, int32_t* count, void* stream);
 
+/* The same for a layer whose heads are sharded over several GPUs (tensor-parallel attention), as a pair of calls
+ * with the caller's all-reduce in between (Eq. 1 and Appendix A Definition 1: A_i is summed "across heads"):
+ *   ta_score_headsum          u_heads[l][tok] = sum over THIS shard's KV heads g (ascending, fp32) of
+ *                             alpha*A_g + delta*P_g; Hq and Hkv are the shard's head counts, q_obs and k its views.
+ *                             u_heads is DEVICE float [L][total_tokens], out.
+ *   (caller)                  sums u_heads over the shards, e.g. an fp32 sum all-reduce of L*total_tokens floats
+ *   ta_compress_from_headsum  adds the attention-free terms, selects once per (layer, sequence) exactly as
+ *                             ta_compress_allheads does, and gathers the rows of this shard's Hkv heads.
+ * Every shard passes the same token ids, patterns, policy and K and therefore retains the same positions. The
+ * library performs no communication itself. */
+ta_status ta_score_headsum(ta_ctx* ctx, const ta_policy* policy, const ta_batch* batch, int Hq, int Hkv, int d,
+                           ta_bf16_view q_obs, ta_bf16_view k, float* u_heads, void* stream);
+ta_status ta_compress_from_headsum(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* policy,
+                                   const ta_batch* batch, int Hkv, int d, int K, const int32_t* token_ids,
+                                   const float* u_heads, ta_bf16_view k, ta_bf16_view v, uint64_t seq_epoch,
+                                   void* k_out, void* v_out, int32_t* idx, int32_t* count, void* stream);
+
 /* ---- composition with another eviction score (Section 4.5 "Composability") ---------------------------------
  * TA changes the scoring function, not the eviction policy: sponsorship is added on top of whatever importance
  * score a pipeline already has (accumulated attention of H2O, the pooled prefill-window attention of SnapKV, a

@@ -93,6 +93,9 @@ def lib():
                                   u64, vp, vp, vp, vp, vp]),
             "ta_compress_allheads": (i32, [vp, vp, PP, PB, i32, i32, i32, i32, vp, ta_bf16_view, ta_bf16_view,
                                            ta_bf16_view, u64, vp, vp, vp, vp, vp]),
+            "ta_score_headsum": (i32, [vp, PP, PB, i32, i32, i32, ta_bf16_view, ta_bf16_view, vp, vp]),
+            "ta_compress_from_headsum": (i32, [vp, vp, PP, PB, i32, i32, i32, vp, vp, ta_bf16_view, ta_bf16_view, u64,
+                                               vp, vp, vp, vp, vp]),
             "ta_compress_scores": (i32, [vp, vp, PP, PB, i32, i32, i32, vp, vp, vp, ta_bf16_view, ta_bf16_view, u64, vp,
                                          vp, vp, vp, vp]),
             "ta_scratch_bytes_budgets": (i32, [PB, i32, i32, PP, i32, C.POINTER(sz)]),
@@ -238,6 +241,18 @@ def ta_score_weighted(ctx, policy, batch, Hq, Hkv, d, q_obs: ta_bf16_view, k: ta
 
 def ta_ctx_set_wait_limit(ctx, nanoseconds: int):
     _check(lib().ta_ctx_set_wait_limit(ctx, int(nanoseconds)), "ta_ctx_set_wait_limit")
+
+
+def ta_score_headsum(ctx, policy, batch, Hq, Hkv, d, q_obs: ta_bf16_view, k: ta_bf16_view, u_heads, stream=None):
+    _check(lib().ta_score_headsum(ctx, C.byref(policy), C.byref(batch), Hq, Hkv, d, q_obs, k, _ptr(u_heads), stream),
+           "ta_score_headsum")
+
+
+def ta_compress_from_headsum(ctx, pats, policy, batch, Hkv, d, K, token_ids, u_heads, k: ta_bf16_view,
+                             v: ta_bf16_view, seq_epoch, k_out, v_out, idx, count, stream=None):
+    _check(lib().ta_compress_from_headsum(ctx, pats, C.byref(policy), C.byref(batch), Hkv, d, K, _ptr(token_ids),
+                                          _ptr(u_heads), k, v, seq_epoch, _ptr(k_out), _ptr(v_out), _ptr(idx),
+                                          _ptr(count), stream), "ta_compress_from_headsum")
 
 
 def ta_ctx_last_launch_info(ctx):

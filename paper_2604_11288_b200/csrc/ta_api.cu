@@ -595,15 +595,17 @@ ta_status compress_impl(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* p
                         int Hkv, int d, int K, const int32_t* token_ids, ta_bf16_view q_obs, ta_bf16_view k,
                         ta_bf16_view v, uint64_t seq_epoch, void* k_out, void* v_out, int32_t* idx, int32_t* count,
                         void* stream_v, const float* ext_A, const float* ext_P, bool share_heads,
-                        const int32_t* budgets = nullptr) {
+                        const int32_t* budgets = nullptr, const float* ext_u_all = nullptr) {
   if (!ctx || !pats || !token_ids || !k_out || !v_out || !idx || !count) return TA_ERR_INVALID_ARG;
   ta_status s = check_batch(batch);
   if (s == TA_OK) s = check_policy(policy);
   if (s != TA_OK) return s;
   const bool fast = policy->mode == TA_MODE_FAST;
-  const bool external = ext_A != nullptr;
+  // ext_u_all: the head-summed attention part comes from the caller (head-sharded layers); implies share_heads
+  const bool external = ext_A != nullptr || ext_u_all != nullptr;
   if ((external || share_heads) && fast) return TA_ERR_INVALID_ARG;
-  if (external && share_heads) return TA_ERR_INVALID_ARG;
+  if (ext_A && share_heads) return TA_ERR_INVALID_ARG;
+  if (ext_u_all && (!share_heads || budgets)) return TA_ERR_INVALID_ARG;
   const bool uniform = batch->cu_seqlens == nullptr;
   s = check_heads(Hq, Hkv, d, policy, !fast && !external);
   if (s == TA_OK && !fast && !external) s = check_view(q_obs, true);
@@ -686,7 +688,7 @@ ta_status compress_impl(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* p
   sel.count = fast ? count_seq : count;
   if (share_heads) {  // one selection per (layer, sequence) on the head sums
     sel.Hkv = 1;
-    sel.u = u_all;
+    sel.u = ext_u_all ? ext_u_all : u_all;
     sel.idx = idx_lb;
     sel.count = count_lb;
   } else if (!fast) {  // small budgets: the selecting block gathers the unit's rows itself
@@ -759,7 +761,8 @@ ta_status compress_impl(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* p
   }
   mark(2);
   if (fork && e == cudaSuccess) e = cudaStreamWaitEvent(stream, ctx->ev_join, 0);
-  if (e == cudaSuccess && share_heads) e = ta_launch_headsum(batch->n_layers, Hkv, batch->total_tokens, u, u_all, stream);
+  if (e == cudaSuccess && share_heads && !ext_u_all)
+    e = ta_launch_headsum(batch->n_layers, Hkv, batch->total_tokens, u, u_all, stream);
   if (e == cudaSuccess && !(fast && reuse)) e = ta_launch_select_units(sel, stream);
   launches += (share_heads ? 2 : 0) + (fast && reuse ? 0 : 1) + (fast ? 1 : 0) + (select_gathers ? 0 : 1);
   if (e == cudaSuccess && share_heads)
@@ -811,6 +814,53 @@ ta_status ta_compress_allheads(ta_ctx* ctx, const ta_patterns* pats, const ta_po
   if (!policy || policy->mode != TA_MODE_SCORED) return TA_ERR_INVALID_ARG;
   return compress_impl(ctx, pats, policy, batch, Hq, Hkv, d, K, token_ids, q_obs, k, v, seq_epoch, k_out, v_out, idx,
                        count, stream, nullptr, nullptr, true);
+}
+
+ta_status ta_score_headsum(ta_ctx* ctx, const ta_policy* policy, const ta_batch* batch, int Hq, int Hkv, int d,
+                           ta_bf16_view q_obs, ta_bf16_view k, float* u_heads, void* stream_v) {
+  if (!ctx || !u_heads) return TA_ERR_INVALID_ARG;
+  ta_status s = check_batch(batch);
+  if (s == TA_OK) s = check_policy(policy);
+  if (s == TA_OK && policy->mode != TA_MODE_SCORED) s = TA_ERR_INVALID_ARG;
+  if (s == TA_OK) s = check_heads(Hq, Hkv, d, policy, true);
+  if (s == TA_OK) s = check_view(q_obs, true);
+  if (s == TA_OK) s = check_view(k, batch->cu_seqlens == nullptr);
+  if (s != TA_OK) return s;
+  const Layout L = make_layout(*batch, Hkv, 1, *policy);
+  if (L.end > ctx->scratch_bytes) return TA_ERR_SCRATCH_TOO_SMALL;
+  DeviceGuard guard(ctx->device);
+  cudaStream_t stream = (cudaStream_t)stream_v;
+  ctx->cached_epoch = 0;  // the per-unit utilities share the scratch with ta_compress's cache
+  float* u = reinterpret_cast<float*>(ctx->scratch + L.u);
+  ta_score_args a = {};
+  a.seq = seq_desc(*batch);
+  a.n_layers = batch->n_layers;
+  a.Hq = Hq;
+  a.Hkv = Hkv;
+  a.W = policy->obs_window;
+  a.q = q_obs;
+  a.k = k;
+  a.u = u;
+  a.alpha = policy->alpha;
+  a.delta = policy->delta;
+  a.rho = policy->pension_rho;
+  a.scale = policy->softmax_scale;
+  a.causal = policy->causal;
+  a.order_scratch = batch->cu_seqlens ? reinterpret_cast<int32_t*>(ctx->scratch + L.order) : nullptr;
+  cudaError_t e = ta_launch_score(ctx, a, ctx->d_status, stream);
+  if (e == cudaSuccess) e = ta_launch_headsum(batch->n_layers, Hkv, batch->total_tokens, u, u_heads, stream);
+  return e == cudaSuccess ? TA_OK : cuda_fail(ctx, e);
+}
+
+ta_status ta_compress_from_headsum(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* policy,
+                                   const ta_batch* batch, int Hkv, int d, int K, const int32_t* token_ids,
+                                   const float* u_heads, ta_bf16_view k, ta_bf16_view v, uint64_t seq_epoch,
+                                   void* k_out, void* v_out, int32_t* idx, int32_t* count, void* stream) {
+  if (!policy || !u_heads) return TA_ERR_INVALID_ARG;
+  if (policy->mode != TA_MODE_SCORED) return TA_ERR_INVALID_ARG;
+  ta_bf16_view none = {};
+  return compress_impl(ctx, pats, policy, batch, Hkv, Hkv, d, K, token_ids, none, k, v, seq_epoch, k_out, v_out, idx,
+                       count, stream, nullptr, nullptr, true, nullptr, u_heads);
 }
 
 ta_status ta_compress_scores(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* policy, const ta_batch* batch,

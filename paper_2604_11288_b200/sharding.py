@@ -45,3 +45,21 @@ def sum_over_ranks(value: float, device=None) -> float:
     t = torch.tensor([float(value)], dtype=torch.float64, device=device)
     dist.all_reduce(t, op=dist.ReduceOp.SUM)
     return float(t.item())
+
+
+def head_shard(Hq: int, Hkv: int, rank: int, world_size: int):
+    """Head-sharded (tensor-parallel) layer: the half-open ranges of KV heads and of query heads that `rank` holds.
+    KV heads are split contiguously and a KV head's query heads stay with it."""
+    if Hkv % world_size or Hq % Hkv:
+        raise ValueError("the KV heads must divide evenly over the ranks and the query heads over the KV heads")
+    per, G = Hkv // world_size, Hq // Hkv
+    return (rank * per, (rank + 1) * per), (rank * per * G, (rank + 1) * per * G)
+
+
+def allreduce_headsum(u_heads):
+    """The exchange between ta_score_headsum and ta_compress_from_headsum: an fp32 SUM all-reduce of the per-shard
+    head sums [L][total_tokens] over the default process group, in place (a no-op without one)."""
+    import torch.distributed as dist
+    if dist.is_available() and dist.is_initialized():
+        dist.all_reduce(u_heads, op=dist.ReduceOp.SUM)
+    return u_heads

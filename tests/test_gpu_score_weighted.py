@@ -178,3 +178,70 @@ def test_sequence_offsets_outside_the_token_arrays_are_rejected_on_the_device():
         assert (c[0] == K).all() and (c[1] == K).all()
     finally:
         g.close()
+
+
+@pytest.mark.parametrize("preset", ["THEOREM", "SEC33"])
+def test_head_sharded_allheads_selection(preset):
+    # A layer whose 4 KV heads (8 query heads) live on two shards: each shard sums its own heads' weighted attention,
+    # a plain fp32 add stands in for the all-reduce between the two calls, and each shard then selects and gathers
+    # its own heads. Every head of both shards must retain what the oracle's all-heads selection retains.
+    from paper_2604_11288_b200 import sharding
+    from ta_testlib import assert_selection_matches, oracle_patterns
+    w = _workload([1500, 20, 700, 9, 2300], [[4, 5], [9]], seed=41, Hq=8, Hkv=4, W=16)
+    K, L, shards = 12, 2, 2
+    pol = oracle_policy(K, preset, W=16)
+    Qh, Kh, Vh = tw.make_qkv(w, range(L))
+    Qd, Kd, Vd = Qh.cuda(), Kh.cuda(), Vh.cuda()
+    g = Gpu(w, pol, K, L)
+    try:
+        part, views = [], []
+        for r in range(shards):
+            (k0, k1), (q0, q1) = sharding.head_shard(w.Hq, w.Hkv, r, shards)
+            Qs, Ks, Vs = Qd[:, :, q0:q1], Kd[:, k0:k1], Vd[:, k0:k1]   # strided views of the shard's heads
+            views.append((k0, k1, q0, q1, Qs, Ks, Vs))
+            u = torch.full((L, w.total), float("nan"), dtype=torch.float32, device="cuda")
+            ta.ta_score_headsum(g.ctx, g.p, g.batch, q1 - q0, k1 - k0, w.d, ta.view(Qs), ta.view(Ks, True), u, g.stream)
+            part.append(u)
+        u_all = part[0] + part[1]  # the caller's all-reduce
+        idx = torch.full((L, w.B, w.Hkv, K), -7, dtype=torch.int32, device="cuda")
+        cnt = torch.full((L, w.B, w.Hkv), -7, dtype=torch.int32, device="cuda")
+        ko = torch.full((L, w.B, w.Hkv, K, w.d), 1.0, dtype=torch.bfloat16, device="cuda")
+        vo = torch.full_like(ko, 1.0)
+        for (k0, k1, q0, q1, Qs, Ks, Vs) in views:
+            n_h = k1 - k0
+            i_s = torch.full((L, w.B, n_h, K), -7, dtype=torch.int32, device="cuda")
+            c_s = torch.full((L, w.B, n_h), -7, dtype=torch.int32, device="cuda")
+            ko_s = torch.full((L, w.B, n_h, K, w.d), 1.0, dtype=torch.bfloat16, device="cuda")
+            vo_s = torch.full_like(ko_s, 1.0)
+            ta.ta_compress_from_headsum(g.ctx, g.pats, g.p, g.batch, n_h, w.d, K, g.ids, u_all, ta.view(Ks, True),
+                                        ta.view(Vs, True), 0, ko_s, vo_s, i_s, c_s, g.stream)
+            idx[:, :, k0:k1], cnt[:, :, k0:k1], ko[:, :, k0:k1], vo[:, :, k0:k1] = i_s, c_s, ko_s, vo_s
+        torch.cuda.synchronize()
+        assert g.poll() == ta.TA_OK
+        idx, cnt = idx.cpu().numpy(), cnt.cpu().numpy()
+        f_o, V_o, u0_o = oracle.sponsor_mask(w.ids, w.cu, oracle_patterns(w), pol)
+        exact = 0
+        for l in range(L):
+            for b in range(w.B):
+                o, e = int(w.cu[b]), int(w.cu[b + 1])
+                Kb = np.stack([unit_kv(w, Kh, l, b, h) for h in range(w.Hkv)])
+                A, P = oracle.attention_allheads(bf16_bits(Qh[l, b]), Kb, e - o, rho=pol.pension_rho)
+                u = oracle.utility(pol.alpha, pol.delta, A, P, u0_o[o:e])
+                io, co = oracle.select(V_o[o:e], u, K, pol.n_sink, pol.n_recent, pol.k_protected)
+                exact += bool(assert_selection_matches(idx[l, b, 0], cnt[l, b, 0], io, co, u, f"l{l} b{b}"))
+                for h in range(w.Hkv):
+                    np.testing.assert_array_equal(idx[l, b, h], idx[l, b, 0])
+                    assert cnt[l, b, h] == cnt[l, b, 0]
+                    c = int(cnt[l, b, h])
+                    np.testing.assert_array_equal(bf16_bits(ko[l, b, h]),
+                                                  oracle.compact(unit_kv(w, Kh, l, b, h), idx[l, b, h], c, K))
+                    np.testing.assert_array_equal(bf16_bits(vo[l, b, h]),
+                                                  oracle.compact(unit_kv(w, Vh, l, b, h), idx[l, b, h], c, K))
+        assert exact >= L * w.B - 1
+        # and the same retained sets as the single-GPU all-heads call
+        i1, c1, _, _ = g.compress_allheads(Qd, Kd, Vd)
+        torch.cuda.synchronize()
+        same = (i1.cpu().numpy() == idx).all(axis=-1).mean()
+        assert same >= 0.9 and (c1.cpu().numpy() == cnt).all()
+    finally:
+        g.close()
