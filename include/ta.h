@@ -170,6 +170,9 @@ ta_status ta_ctx_set_score_cluster(ta_ctx* ctx, int ctas_per_unit);
  * budgets; no separate gather kernel), out[3] = kernels of this library the call enqueued. */
 ta_status ta_ctx_last_launch_info(const ta_ctx* ctx, int32_t out[4] /*HOST*/);
 
+/* Every entry point that enqueues work opens an NVTX range of its own name around its host side (visible in timeline
+ * tools; free when no tool is attached). */
+
 /* Optional per-kernel timing of ta_compress: when enabled, CUDA events are recorded on the call's stream around
  * each kernel of the next ta_compress calls. ta_ctx_read_timing synchronises on those events and returns the
  * milliseconds of the most recent call in out_ms[0..4] = {mask+static utility, score, select, compact, total}.
@@ -309,8 +312,9 @@ ta_status ta_compact_kv(ta_ctx* ctx, const ta_batch* batch, int Hkv, int d, int 
  * Steps 1-4 for batch->n_layers layers. The per-sequence results of step 1 (and, in fast mode, of step 3, which
  * then does not depend on layer or head) are kept in the context and reused when seq_epoch is non-zero and equal
  * to the previous call's: pass the same non-zero epoch for successive layers of one batch, a new one (or 0:
- * never reuse) for a new batch. In scored mode the utilities stay in context scratch; A and P are not
- * materialised. q_obs and k are not read in fast mode (their ptr may be NULL). */
+ * never reuse) for a new batch. Under one epoch the token ids and cu_seqlens must stay the same; a change of the
+ * pattern set, of K, of the mode or of any policy field that the per-sequence steps read is noticed and recomputed.
+ * In scored mode the utilities stay in context scratch; A and P are not materialised. q_obs and k are not read in fast mode (their ptr may be NULL). */
 ta_status ta_compress(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* policy, const ta_batch* batch, int Hq,
                       int Hkv, int d, int K, const int32_t* token_ids, ta_bf16_view q_obs, ta_bf16_view k,
                       ta_bf16_view v, uint64_t seq_epoch, void* k_out, void* v_out, int32_t* idx, int32_t* count,
@@ -392,7 +396,12 @@ ta_status ta_compress_budgets(ta_ctx* ctx, const ta_patterns* pats, const ta_pol
  * (l*B + b)*Hkv + g) the library keeps the state of the at most K+1 cached tokens IN POSITION ORDER and decides
  * which one to evict; it never touches key/value rows. The caller owns a cache of K+1 rows per unit: the new token's
  * keys and values go to row next_slot[unit], and an evicted token's row is handed out as the next next_slot.
- * What one step computes, per the readings listed in the oracle (oracle/ta_stream_oracle.py):
+ * The paper does not say what persists between steps; this library takes these readings: an anchor is detected
+ * once, when the token that completes a pattern arrives (Algorithm 1 step 1 on the stream of ids: evicted tokens were
+ * seen); a token's voucher is fixed at its arrival (Eq. 2, steps 2-6) and afterwards only decays (step 10); A_i
+ * accumulates and P_i averages the per-step attention mass (Eq. 1; Appendix A Definition 1); R_i and F_i use the count
+ * of tokens seen so far; nothing is evicted while at most K tokens are cached (Section 3.1).
+ * What one step computes:
  *   - the new token completes a pattern (longest wins, then lowest index) -> it becomes an anchor with that pattern's
  *     budget and span; every cached token of the match gets S = 1;
  *   - the new token's voucher (Eq. 2) from the anchors of the last TA_MAX_SPAN positions, whose budgets have decayed

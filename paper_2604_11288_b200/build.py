@@ -51,7 +51,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     if failed:
         raise RuntimeError("nvcc failed")
     subprocess.run([nvcc, "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-o", LIB_PATH] + objs +
-                   ["-cudart", "static"], check=True)
+                   ["-cudart", "static", "-ldl"], check=True)
     return LIB_PATH
 
 

@@ -3,6 +3,7 @@
 // ta_select.cu and ta_compact.cu.
 #include <cuda.h>
 #include <math.h>
+#include <nvtx3/nvToolsExt.h>
 #include <new>
 #include <string.h>
 
@@ -120,6 +121,34 @@ ta_seq_desc seq_desc(const ta_batch& b) {
 ta_status cuda_fail(ta_ctx* ctx, cudaError_t e) {
   ctx->last_cuda_error = (int)e;
   return TA_ERR_CUDA;
+}
+
+struct Range {  // NVTX range around the host side of an entry point (what a timeline tool shows per call)
+  explicit Range(const char* name) { nvtxRangePushA(name); }
+  ~Range() { nvtxRangePop(); }
+};
+
+// What the per-sequence results cached under a seq_epoch depend on besides the token ids: every policy field that
+// the mask, the static utility and the forced set read, and the pattern set.
+uint64_t reuse_key(const ta_policy& p, const ta_patterns* pats) {
+  uint64_t h = 1469598103934665603ull;
+  auto mix = [&](const void* data, size_t n) {
+    const unsigned char* b = static_cast<const unsigned char*>(data);
+    for (size_t i = 0; i < n; ++i) h = (h ^ b[i]) * 1099511628211ull;
+  };
+  mix(&p.beta, sizeof p.beta);
+  mix(&p.gamma, sizeof p.gamma);
+  mix(&p.lambda, sizeof p.lambda);
+  mix(&p.voucher_decay, sizeof p.voucher_decay);
+  mix(&p.budget_decay, sizeof p.budget_decay);
+  mix(&p.age_steps, sizeof p.age_steps);
+  mix(&p.n_sink, sizeof p.n_sink);
+  mix(&p.n_recent, sizeof p.n_recent);
+  mix(&p.k_protected, sizeof p.k_protected);
+  mix(&p.mode, sizeof p.mode);
+  mix(&p.vocab_size, sizeof p.vocab_size);
+  mix(&pats, sizeof pats);
+  return h;
 }
 
 struct DeviceGuard {  // makes the context's device current for the duration of a call
@@ -414,6 +443,7 @@ void ta_patterns_destroy(ta_patterns* P) {
 // ---------------------------------------------------------------------------------------------- step 1
 ta_status ta_sponsor_mask(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* policy, const ta_batch* batch,
                           const int32_t* token_ids, uint8_t* flags, float* voucher, float* u_static, void* stream) {
+  Range range("ta_sponsor_mask");
   if (!ctx || !pats || !token_ids || !flags || !voucher || !u_static) return TA_ERR_INVALID_ARG;
   ta_status s = check_batch(batch);
   if (s == TA_OK) s = check_policy(policy);
@@ -430,6 +460,7 @@ ta_status ta_sponsor_mask(ta_ctx* ctx, const ta_patterns* pats, const ta_policy*
 
 ta_status ta_detect_embedding(ta_ctx* ctx, int64_t total_tokens, const void* emb, int64_t stride_tok, int D,
                               const void* concepts, int n_concepts, float* conf, void* stream) {
+  Range range("ta_detect_embedding");
   if (!ctx || !emb || !concepts || !conf || total_tokens < 0) return TA_ERR_INVALID_ARG;
   if (D < 32 || n_concepts < 1 || stride_tok < D) return TA_ERR_INVALID_ARG;
   if (D % 32 || D > TA_MAX_EMBED_DIM || n_concepts > TA_MAX_CONCEPTS) return TA_ERR_UNSUPPORTED;
@@ -443,6 +474,7 @@ ta_status ta_detect_embedding(ta_ctx* ctx, int64_t total_tokens, const void* emb
 ta_status ta_sponsor_mask_conf(ta_ctx* ctx, const ta_policy* policy, const ta_batch* batch, const int32_t* token_ids,
                                const float* conf, float threshold, float budget, int span, int rank_by_confidence,
                                uint8_t* flags, float* voucher, float* u_static, void* stream) {
+  Range range("ta_sponsor_mask_conf");
   if (!ctx || !token_ids || !conf || !flags || !voucher || !u_static) return TA_ERR_INVALID_ARG;
   ta_status s = check_batch(batch);
   if (s == TA_OK) s = check_policy(policy);
@@ -463,6 +495,7 @@ ta_status ta_sponsor_mask_conf(ta_ctx* ctx, const ta_policy* policy, const ta_ba
 static ta_status score_impl(ta_ctx* ctx, const ta_policy* policy, const ta_batch* batch, int Hq, int Hkv, int d,
                             ta_bf16_view q_obs, ta_bf16_view k, const float* lse_obs, float* A, float* P, float* u,
                             void* stream) {
+  Range range("ta_score");
   if (!ctx || (!A && !u)) return TA_ERR_INVALID_ARG;
   ta_status s = check_batch(batch);
   if (s == TA_OK) s = check_policy(policy);
@@ -514,6 +547,7 @@ ta_status ta_score_weighted(ta_ctx* ctx, const ta_policy* policy, const ta_batch
 ta_status ta_select_topk(ta_ctx* ctx, const ta_policy* policy, const ta_batch* batch, int Hkv, int K,
                          const uint8_t* flags, const float* voucher, const float* u_static, const float* A,
                          const float* P, int32_t* idx, int32_t* count, void* stream) {
+  Range range("ta_select_topk");
   if (!ctx || !flags || !voucher || !u_static || !idx || !count) return TA_ERR_INVALID_ARG;
   ta_status s = check_batch(batch);
   if (s == TA_OK) s = check_policy(policy);
@@ -539,6 +573,7 @@ ta_status ta_select_topk(ta_ctx* ctx, const ta_policy* policy, const ta_batch* b
   a.n_recent = policy->n_recent;
   a.k_protected = policy->k_protected;
   a.fast = fast;
+  a.sm_count = ctx->sm_count;
   a.alpha = policy->alpha;
   a.delta = policy->delta;
   a.flags = flags;
@@ -561,6 +596,7 @@ ta_status ta_select_topk(ta_ctx* ctx, const ta_policy* policy, const ta_batch* b
 // ---------------------------------------------------------------------------------------------- step 4
 ta_status ta_compact_kv(ta_ctx* ctx, const ta_batch* batch, int Hkv, int d, int K, ta_bf16_view k, ta_bf16_view v,
                         const int32_t* idx, const int32_t* count, void* k_out, void* v_out, void* stream) {
+  Range range("ta_compact_kv");
   if (!ctx || !idx || !count || !k_out || !v_out) return TA_ERR_INVALID_ARG;
   ta_status s = check_batch(batch);
   if (s != TA_OK) return s;
@@ -596,6 +632,7 @@ ta_status compress_impl(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* p
                         ta_bf16_view v, uint64_t seq_epoch, void* k_out, void* v_out, int32_t* idx, int32_t* count,
                         void* stream_v, const float* ext_A, const float* ext_P, bool share_heads,
                         const int32_t* budgets = nullptr, const float* ext_u_all = nullptr) {
+  Range range("ta_compress");
   if (!ctx || !pats || !token_ids || !k_out || !v_out || !idx || !count) return TA_ERR_INVALID_ARG;
   ta_status s = check_batch(batch);
   if (s == TA_OK) s = check_policy(policy);
@@ -663,7 +700,8 @@ ta_status compress_impl(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* p
   };
 
   // (with budget classes the forced sets live elsewhere and depend on the budgets: nothing is reused or cached)
-  const bool reuse = !budgets && seq_epoch != 0 && seq_epoch == ctx->cached_epoch &&
+  const uint64_t key = reuse_key(*policy, pats);
+  const bool reuse = !budgets && seq_epoch != 0 && seq_epoch == ctx->cached_epoch && key == ctx->cached_key &&
                      ctx->cached_total == batch->total_tokens && ctx->cached_batch == batch->batch && ctx->cached_K == K;
   ta_select_args sel = {};
   sel.seq = seq;
@@ -674,6 +712,7 @@ ta_status compress_impl(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* p
   sel.n_recent = policy->n_recent;
   sel.k_protected = policy->k_protected;
   sel.fast = fast;
+  sel.sm_count = ctx->sm_count;
   sel.alpha = policy->alpha;
   sel.delta = policy->delta;
   sel.flags = flags;
@@ -795,6 +834,7 @@ ta_status compress_impl(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* p
   ctx->cached_total = batch->total_tokens;
   ctx->cached_batch = batch->batch;
   ctx->cached_K = K;
+  ctx->cached_key = key;
   return TA_OK;
 }
 }  // namespace
@@ -818,6 +858,7 @@ ta_status ta_compress_allheads(ta_ctx* ctx, const ta_patterns* pats, const ta_po
 
 ta_status ta_score_headsum(ta_ctx* ctx, const ta_policy* policy, const ta_batch* batch, int Hq, int Hkv, int d,
                            ta_bf16_view q_obs, ta_bf16_view k, float* u_heads, void* stream_v) {
+  Range range("ta_score_headsum");
   if (!ctx || !u_heads) return TA_ERR_INVALID_ARG;
   ta_status s = check_batch(batch);
   if (s == TA_OK) s = check_policy(policy);
@@ -929,6 +970,7 @@ ta_status ta_stream_scratch_bytes(const ta_stream* st, size_t* out_bytes) {
 
 ta_status ta_stream_step(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* policy, ta_stream* st,
                          const int32_t* new_ids, const float* attn, int32_t* evicted_pos, void* stream_v) {
+  Range range("ta_stream_step");
   if (!ctx || !pats || !new_ids || !attn || !evicted_pos) return TA_ERR_INVALID_ARG;
   ta_status s = check_policy(policy);
   if (s == TA_OK) s = check_stream(st);
@@ -1018,6 +1060,7 @@ ta_status ta_compress_host(ta_ctx* ctx, const ta_patterns* pats, const ta_policy
                            int Hq, int Hkv, int d, int K, const int32_t* token_ids, const void* q_obs, const void* k,
                            const void* v, void* k_out, void* v_out, int32_t* idx, int32_t* count, void* workspace,
                            size_t workspace_bytes, void* stream_v) {
+  Range range("ta_compress_host");
   if (!ctx || !pats || !token_ids || !k || !v || !k_out || !v_out || !idx || !count || !workspace)
     return TA_ERR_INVALID_ARG;
   ta_status s = check_batch(batch);

@@ -36,6 +36,7 @@ struct ta_ctx {
   ta_dev_status* d_status;  // device
   // cache of per-sequence results inside scratch (ta_compress)
   uint64_t cached_epoch;
+  uint64_t cached_key;  // policy fields and pattern set the cached results were computed with
   int64_t cached_total;
   int cached_batch;
   int cached_K;
@@ -116,6 +117,7 @@ struct ta_select_args {
   int n_layers, Hkv, K;
   int n_sink, n_recent, k_protected;
   int fast;
+  int sm_count;  // of the device the launch goes to (0: ask the runtime about the current device)
   float alpha, delta;
   const uint8_t* flags;
   const float* voucher;

@@ -634,16 +634,19 @@ __global__ void ta_broadcast_heads_kernel(long long units_lb, int Hkv, int K, co
 // over a cluster of kSelectCluster CTAs (keys in registers up to kSelectCluster * kItemsLong * kThreads elements).
 // Splitting pays only while the clusters of all units fit on the device about at once; with many units one CTA per
 // unit (keys re-read in batches when they do not fit in registers) keeps every SM busy without cluster barriers.
-bool split_units(int units, int max_n) {
+bool split_units(int units, int max_n, int sms) {
   if (max_n <= kItems * kThreads) return false;
-  static int sms = 0;
-  if (sms == 0) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess ||
-        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1)
-      sms = 148;
-  }
   return units * kSelectCluster <= 2 * sms;
+}
+
+// SM count of the device the launch goes to: the caller's (a context knows its device), else the current device's
+int sm_count_of(const ta_select_args& a) {
+  if (a.sm_count > 0) return a.sm_count;
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1)
+    sms = 148;
+  return sms;
 }
 
 template <class Kern, class... Args>
@@ -667,13 +670,14 @@ cudaError_t ta_launch_forced(const ta_select_args& a, ta_dev_status* status, cud
   if (a.seq.batch == 0 || a.n_layers == 0) return cudaSuccess;
   const int B = a.seq.batch * (a.n_classes > 0 ? a.n_classes : 1);  // blocks: (class, sequence)
   const int32_t* ck = a.n_classes > 0 ? a.class_K : nullptr;
+  const int sms = sm_count_of(a);
   if (a.seq.max_n <= kItems * kThreads)
     return launch_clustered(ta_forced_kernel<true, 1>, B, 1, stream, a.seq, a.K, a.n_sink, a.n_recent, a.k_protected,
                             a.voucher, a.forced, a.r_main, status, ck);
-  if (!split_units(B, a.seq.max_n) && a.seq.max_n <= kItemsLong * kThreads)
+  if (!split_units(B, a.seq.max_n, sms) && a.seq.max_n <= kItemsLong * kThreads)
     return launch_clustered(ta_forced_kernel<true, 1, kItemsLong>, B, 1, stream, a.seq, a.K, a.n_sink, a.n_recent,
                             a.k_protected, a.voucher, a.forced, a.r_main, status, ck);
-  if (!split_units(B, a.seq.max_n))
+  if (!split_units(B, a.seq.max_n, sms))
     return launch_clustered(ta_forced_kernel<false, 1>, B, 1, stream, a.seq, a.K, a.n_sink, a.n_recent, a.k_protected,
                             a.voucher, a.forced, a.r_main, status, ck);
   if (a.seq.max_n <= kSelectCluster * kItems * kThreads)
@@ -692,11 +696,7 @@ bool ta_select_gathers(const ta_select_args& a) {
   // costs one launch (about 8 us for so few rows): fusing pays only while the blocks run in a few waves. Short units
   // (keys in 16 registers: two blocks per SM) only.
   const int units = a.n_layers * a.seq.batch * a.Hkv;
-  int dev = 0, sms = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess ||
-      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1)
-    sms = 148;
-  return a.seq.max_n <= kItems * kThreads && units <= 4 * sms;
+  return a.seq.max_n <= kItems * kThreads && units <= 4 * sm_count_of(a);
 }
 
 cudaError_t ta_launch_select_units(const ta_select_args& a, cudaStream_t stream) {
@@ -710,6 +710,7 @@ cudaError_t ta_launch_select_units(const ta_select_args& a, cudaStream_t stream)
   src.delta = a.delta;
   const int units = a.fast ? a.seq.batch : a.n_layers * a.seq.batch * a.Hkv;
   const int32_t* co = a.n_classes > 0 ? a.class_of : nullptr;
+  const int sms = sm_count_of(a);
   GatherDst gd = {};
   if (ta_select_gathers(a)) {  // implies the first variant below
     gd.k = a.gather_k;
@@ -722,10 +723,10 @@ cudaError_t ta_launch_select_units(const ta_select_args& a, cudaStream_t stream)
   if (a.seq.max_n <= kItems * kThreads)
     return launch_clustered(ta_select_kernel<true, 1>, units, 1, stream, a.seq, a.n_layers, a.Hkv, a.K, a.fast, src,
                             a.forced, a.r_main, a.idx, a.count, gd, co);
-  if (!split_units(units, a.seq.max_n) && a.seq.max_n <= kItemsLong * kThreads)
+  if (!split_units(units, a.seq.max_n, sms) && a.seq.max_n <= kItemsLong * kThreads)
     return launch_clustered(ta_select_kernel<true, 1, kItemsLong>, units, 1, stream, a.seq, a.n_layers, a.Hkv, a.K, a.fast,
                             src, a.forced, a.r_main, a.idx, a.count, gd, co);
-  if (!split_units(units, a.seq.max_n))
+  if (!split_units(units, a.seq.max_n, sms))
     return launch_clustered(ta_select_kernel<false, 1>, units, 1, stream, a.seq, a.n_layers, a.Hkv, a.K, a.fast, src,
                             a.forced, a.r_main, a.idx, a.count, gd, co);
   if (a.seq.max_n <= kSelectCluster * kItems * kThreads)

@@ -12,6 +12,8 @@
 //                           entries move; key/value rows never do: the freed cache row is handed to the next token) and
 //                           decays every voucher by budget_decay (Algorithm 1 step 10)
 // All arithmetic that decides the selection is fp32 with one rounding per operation, in the order the CPU oracle uses.
+#include <atomic>
+
 #include "ta_internal.cuh"
 
 namespace {
@@ -320,14 +322,15 @@ cudaError_t ta_launch_stream_step(const ta_stream_dev& st, const ta_policy& pol,
   const int U = st.n_layers * st.B * st.Hkv, C = st.K + 1;
   const int threads = C <= 512 ? 128 : 512;
   const size_t smem = (size_t)C * (7 * 4 + 2) + 16;
-  static bool attr_set[64] = {};
+  // per device; setting the (sticky) attribute twice from two threads is harmless, the flag only saves the call
+  static std::atomic<bool> attr_set[64];
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
-  if (!attr_set[dev & 63]) {
+  if (!attr_set[dev & 63].load(std::memory_order_acquire)) {
     e = cudaFuncSetAttribute(ta_stream_step_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
     if (e != cudaSuccess) return e;
-    attr_set[dev & 63] = true;
+    attr_set[dev & 63].store(true, std::memory_order_release);
   }
   ta_stream_step_kernel<<<U, threads, smem, stream>>>(st, info, attn, pol.vocab_size, pol.alpha, pol.beta, pol.gamma,
                                                       pol.delta, pol.lambda, pol.pension_rho, pol.budget_decay,

@@ -245,3 +245,35 @@ def test_head_sharded_allheads_selection(preset):
         assert same >= 0.9 and (c1.cpu().numpy() == cnt).all()
     finally:
         g.close()
+
+
+def test_epoch_reuse_notices_a_changed_policy():
+    # same non-zero epoch, scored call then fast call then another preset: nothing stale may be reused
+    from ta_testlib import assert_selection_matches, gpu_policy, oracle_patterns, oracle_unit
+    w = _workload([900, 300], [[4, 5]], seed=16, Hq=8, Hkv=2, W=32)
+    K = 10
+    Qh, Kh, Vh = tw.make_qkv(w, [0])
+    Qd, Kd, Vd = Qh.cuda(), Kh.cuda(), Vh.cuda()
+    g = Gpu(w, oracle_policy(K, "THEOREM", W=32), K, 1)
+    try:
+        for pol in (oracle_policy(K, "THEOREM", W=32), oracle_policy(K, "THEOREM", W=32, fast=True),
+                    oracle_policy(K, "SEC33", W=32, fast=True), oracle_policy(K, "SEC33", W=32)):
+            g.pol, g.p = pol, gpu_policy(pol)
+            idx, cnt, ko, vo = g.compress(Qd, Kd, Vd, epoch=77)
+            torch.cuda.synchronize()
+            assert g.poll() == ta.TA_OK
+            idx, cnt = idx.cpu().numpy(), cnt.cpu().numpy()
+            f_o, V_o, u0_o = oracle.sponsor_mask(w.ids, w.cu, oracle_patterns(w), pol)
+            for b in range(w.B):
+                for h in range(w.Hkv):
+                    A, P, u, io, co = oracle_unit(w, pol, K, Qh, Kh, 0, b, h, V_o, u0_o)
+                    assert_selection_matches(idx[0, b, h], cnt[0, b, h], io, co, u, f"fast={pol.fast} b{b} h{h}")
+    finally:
+        g.close()
+
+
+@pytest.mark.parametrize("W", [1, 5, 33, 63])
+def test_weighted_odd_windows(W):
+    # windows that are not a multiple of 8: G*W rows that end inside a 16-row group of the accumulator
+    _weighted_case([700, 40, 3], 4, 1, W, seed=20 + W)
+    _weighted_case([1400], 8, 2, W, seed=40 + W)
