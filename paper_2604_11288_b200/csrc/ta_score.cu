@@ -21,10 +21,10 @@
 // allocation and pipeline fill are paid once per CTA and not once per unit.
 //
 // Warp roles: four softmax warpgroups plus one warpgroup with the TMA producer warp, the MMA issuer warp (TMEM owner)
-// and two idle warps. A "job" is one key tile in one pass. With up to 128 score rows (MB 1) the four groups take the
-// jobs round-robin, one accumulator stage of 128 columns each. With 129..256 rows (MB 2) an accumulator stage holds
-// 256 columns and a pair of groups shares each job: in pass 1 each group of the pair owns one block of 128 rows, in
-// pass 2 each sums half of the rows for the tile's keys and the two halves are added through shared memory.
+// and two idle warps. A "job" is one block of up to 128 score rows of one key tile in one pass. With up to 128 score rows (MB 1) the four groups take the
+// jobs round-robin, one accumulator stage of 128 columns each. With 129..256 rows (MB 2) every tile is two jobs, one
+// per block of 128 rows, again one group and one stage each: in pass 1 a group owns the rows of its block, in pass 2
+// it sums its block's rows for the tile's keys and the two partial sums meet in a small shared-memory ring.
 // After set-up the last warpgroup gives registers back (setmaxnreg) and the softmax warpgroups take them.
 //
 // The softmax warps are bound by instruction issue and by the special-function unit (one ex2 per score element and
@@ -102,8 +102,9 @@ struct ScoreCfg {
   static constexpr int kQBufs = MB == 1 ? 2 : 1;   // query tiles in flight (next unit's tile loads early)
   static constexpr int kStages = MB == 1 ? 4 : 3;  // ring of key tiles
   static constexpr int kRowsPad = MB * 128;
-  static constexpr int kAcc = MB == 1 ? 4 : 2;     // accumulator stages of kRowsPad columns (512 columns in all)
-  static constexpr int kWarpsPerJob = MB * 4;      // softmax warps that read one accumulator stage
+  static constexpr int kAcc = 4;                   // accumulator stages of 128 columns (512 columns in all)
+  static constexpr int kWarpsPerJob = 4;           // softmax warps that read one accumulator stage
+  static constexpr int kRing = 4;                  // MB 2: partial sums in flight between the two groups of a pair
 };
 
 template <int MB>
@@ -119,10 +120,11 @@ struct alignas(1024) ScoreSmem {
   float nbeta[2][MB * 128];                       // [unit parity][row] -beta (masked tiles use ex2 for every row)
   float wrow[MB * 128];                           // pension weight per row
   float lv[MB * 128];                             // log2 of the row's output weight (kOutFused), else 0
-  float pair_sum[2][2][2][128];                   // MB 2: [pair][job parity][A|P][key] partial sums of the second group
+  float psum[2][Cfg::kRing][2][128];              // MB 2: [pair][ring slot][A|P][key] partial sums of row block 0
   int row_t[MB * 128];                            // window index t of the row, -1 for padding rows
   unsigned long long full[Cfg::kStages], empty[Cfg::kStages], acc_full[Cfg::kAcc], acc_empty[Cfg::kAcc];
   unsigned long long q_full[Cfg::kQBufs], q_empty[Cfg::kQBufs], xchg_full[2], drain;
+  unsigned long long pfull[2][Cfg::kRing], pfree[2][Cfg::kRing];
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -172,7 +174,7 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
   constexpr int kWarpTma = kGroups * 4, kWarpMma = kGroups * 4 + 1;
   constexpr int kStages = Cfg::kStages, kQBufs = Cfg::kQBufs, kRowsPad = Cfg::kRowsPad;
   constexpr int kAcc = Cfg::kAcc;
-  constexpr uint32_t kTmemCols = 512;  // kAcc accumulator stages of kRowsPad columns
+  constexpr uint32_t kTmemCols = 512;  // kAcc accumulator stages of 128 columns
   extern __shared__ uint8_t smem_raw[];
   ScoreSmem<MB>& sm = *reinterpret_cast<ScoreSmem<MB>*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
 
@@ -237,6 +239,11 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
       mbar_init(smem_u32(&sm.q_empty[qb]), 1);
     }
     mbar_init(smem_u32(&sm.drain), 1);
+    for (int pr = 0; pr < 2; ++pr)
+      for (int r = 0; r < Cfg::kRing; ++r) {
+        mbar_init(smem_u32(&sm.pfull[pr][r]), 4);
+        mbar_init(smem_u32(&sm.pfree[pr][r]), 4);
+      }
     // a wait that ran out in an earlier CTA or call (not yet polled) makes the remaining CTAs skip their waits
     sm.abort_flag = (*reinterpret_cast<volatile int*>(&p.status->code) == (int)TA_ERR_TIMEOUT) ? 1 : 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -332,12 +339,12 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     } else if (warp == kWarpMma) {
       // =========================================================================== MMA issuer
       if (lane == 0) {
-        int jg = 0, qn = 0;
+        int jg = 0, tg = 0, qn = 0;
         bool ok = true;
         // operand descriptors: the upper word is the same for every tile; the lower word is the address >> 4
         const uint32_t desc_hi = (uint32_t)(smem_desc_sw128(0) >> 32);
         const uint32_t k_lo = (k_smem & 0x3FFFFu) >> 4;
-        const uint32_t idesc1 = idesc_bf16(128, kTileN), idesc2 = idesc_bf16(128, kRowsPad);
+        const uint32_t idesc = idesc_bf16(128, 128);
         for (int u = cluster_id; ok && u - cluster_id < p.units; u += n_clusters) {
           const UnitInfo ui = get_unit(u);
           if (ui.T == 0) continue;
@@ -345,37 +352,33 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           ok = mbar_wait(smem_u32(&sm.q_full[qb]), (uint32_t)(qn / kQBufs) & 1u, abort_flag, p.status, 22, limit);
           if (!ok) break;
           const uint32_t q_lo = (smem_u32(sm.q[qb]) & 0x3FFFFu) >> 4;
-          const int n_jobs = p.two_pass ? 2 * ui.T : ui.T;
-          for (int j = 0; j < n_jobs; ++j, ++jg) {
-            const int s = jg % kStages;
-            const int a = jg % kAcc;
-            const bool stats = p.two_pass && j < ui.T;
-            ok = mbar_wait(smem_u32(&sm.full[s]), (uint32_t)(jg / kStages) & 1u, abort_flag, p.status, 20, limit) &&
-                 mbar_wait(smem_u32(&sm.acc_empty[a]), ((uint32_t)(jg / kAcc) & 1u) ^ 1u, abort_flag, p.status, 21, limit);
-            if (!ok) break;  // no product is issued on operands or into an accumulator that are not ready
-            tc_fence_after();
+          // A tile's product is issued as MB jobs, one per block of 128 score rows, each into its own accumulator
+          // stage of 128 columns: S = Q_block * Ktile^T in pass 1, S^T = Ktile * Q_block^T in pass 2.
+          const int n_tiles = p.two_pass ? 2 * ui.T : ui.T;
+          for (int jt = 0; ok && jt < n_tiles; ++jt, ++tg) {
+            const int s = tg % kStages;
+            const bool stats = p.two_pass && jt < ui.T;
+            ok = mbar_wait(smem_u32(&sm.full[s]), (uint32_t)(tg / kStages) & 1u, abort_flag, p.status, 20, limit);
+            if (!ok) break;  // no product is issued on operands that are not ready
             const uint32_t dk_lo = k_lo + (uint32_t)((s * kKTileBytes) >> 4);
-            const uint32_t acc = tmem_base + (uint32_t)(a * kRowsPad);
-            if (stats) {
 #pragma unroll
-              for (int mb = 0; mb < MB; ++mb) {
+            for (int rb = 0; rb < MB; ++rb, ++jg) {
+              const int a = jg % kAcc;
+              ok = ok && mbar_wait(smem_u32(&sm.acc_empty[a]), ((uint32_t)(jg / kAcc) & 1u) ^ 1u, abort_flag, p.status,
+                                   21, limit);
+              if (ok) {  // (nor into an accumulator that was not handed back)
+                tc_fence_after();
+                const uint32_t acc = tmem_base + (uint32_t)(a * 128);
 #pragma unroll
                 for (int k = 0; k < 8; ++k) {
-                  const uint32_t da = q_lo + (uint32_t)(((k >> 2) * (MB * kHalfBytes) + mb * kHalfBytes + (k & 3) * 32) >> 4);
-                  const uint32_t db = dk_lo + (uint32_t)(((k >> 2) * kHalfBytes + (k & 3) * 32) >> 4);
-                  umma_bf16_lo(acc + mb * 128, da, db, desc_hi, idesc1, k > 0);
+                  const uint32_t dq = q_lo + (uint32_t)(((k >> 2) * (MB * kHalfBytes) + rb * kHalfBytes + (k & 3) * 32) >> 4);
+                  const uint32_t dk = dk_lo + (uint32_t)(((k >> 2) * kHalfBytes + (k & 3) * 32) >> 4);
+                  umma_bf16_lo(acc, stats ? dq : dk, stats ? dk : dq, desc_hi, idesc, k > 0);
                 }
-              }
-            } else {
-#pragma unroll
-              for (int k = 0; k < 8; ++k) {
-                const uint32_t da = dk_lo + (uint32_t)(((k >> 2) * kHalfBytes + (k & 3) * 32) >> 4);
-                const uint32_t db = q_lo + (uint32_t)(((k >> 2) * (MB * kHalfBytes) + (k & 3) * 32) >> 4);
-                umma_bf16_lo(acc, da, db, desc_hi, idesc2, k > 0);
+                if (rb == MB - 1) umma_commit(smem_u32(&sm.empty[s]));
+                umma_commit(smem_u32(&sm.acc_full[a]));
               }
             }
-            umma_commit(smem_u32(&sm.empty[s]));
-            umma_commit(smem_u32(&sm.acc_full[a]));
           }
           if (!ok) break;
           umma_commit(smem_u32(&sm.q_empty[qb]));  // the query tile may be overwritten once these MMAs are done
@@ -390,22 +393,25 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
   } else {
     asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmax));
     // =========================================================================== softmax warps
-    constexpr int kShare = kAcc;            // jobs are dealt round-robin to kShare groups (MB 1) or pairs (MB 2)
+    // A job is one block of 128 score rows of one key tile in one pass; jobs are dealt round-robin to the four
+    // groups. With two row blocks (MB 2) a tile is two consecutive jobs, every unit has an even number of jobs, and
+    // group g therefore always gets row block g & 1.
+    constexpr int kShare = kAcc;
     const int st = tid;                     // 0..511
     const int grp = st >> 7;
-    const int slot = MB == 1 ? grp : grp >> 1;   // serves jobs with (global job index % kShare) == slot
-    const int half = MB == 1 ? 0 : grp & 1;      // MB 2: which 128 accumulator columns of the job
-    const int coff = half * 128;
+    const int slot = grp;                   // serves jobs with (global job index % kShare) == slot
+    const int blk = MB == 1 ? 0 : grp & 1;  // the row block of every job this group gets
+    const int coff = blk * 128;              // first score row of that block
     const int quad = warp & 3;              // TMEM lane quadrant this warp may read
     const int row_in_tile = quad * 32 + lane;
-    const uint32_t tlane = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)coff;
+    const uint32_t tlane = tmem_base + ((uint32_t)(quad * 32) << 16);
     const float c = p.c;
     const float c252 = c * (1.0f / kPolyRange);
     const int my_t = sm.row_t[coff + row_in_tile];  // pass 1: this thread's row is coff + row_in_tile
     const int rows_mine = min(128, p.rows - coff);
     const int n_chunks2 = (rows_mine + 31) >> 5;
 
-    auto acc_addr = [&](int jj) { return tlane + (uint32_t)((jj % kAcc) * kRowsPad); };
+    auto acc_addr = [&](int jj) { return tlane + (uint32_t)((jj % kAcc) * 128); };
     auto wait_full = [&](int jj, int where) {
       mbar_wait(smem_u32(&sm.acc_full[jj % kAcc]), (uint32_t)(jj / kAcc) & 1u, abort_flag, p.status, where, limit);
       tc_fence_after();
@@ -417,6 +423,7 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     };
 
     int jg = 0, it = 0;
+    int pc = 0;  // MB 2: tiles of pass 2 this group has handled (same count in both groups of a pair)
     for (int u = cluster_id; u - cluster_id < p.units; u += n_clusters, ++it) {
       const UnitInfo ui = get_unit(u);
       const int n = ui.n, T = ui.T;
@@ -480,7 +487,7 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         };
         float ra[16], rb[16];
         int j = (slot - jg % kShare + kShare) % kShare;  // first job of this pass that belongs to the group
-        if (j < T) {
+        if (j < MB * T) {
           wait_full(jg + j, 30);
           tmem_ld16_issue(acc_addr(jg + j), ra);
         }
@@ -488,7 +495,7 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         // that one load is always in flight. On entry the load of the first 16 columns is in flight in `ra`.
         auto job1 = [&](auto masked_tag, int j) {
           const int jj = jg + j;
-          const int key0 = (ui.t_begin + j) * kTileN;
+          const int key0 = (ui.t_begin + j / MB) * kTileN;
           const uint32_t abase = acc_addr(jj);
           float rc = ref_c;
           const bool first = rc < -1e29f;
@@ -548,15 +555,15 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           }
           z_run += sum;
           release(jj);
-          if (j + kShare < T) {  // the next job of the group reuses this stage: fetch it once it is full again
+          if (j + kShare < MB * T) {  // the next job of the group reuses this stage: fetch it once it is full again
             wait_full(jj + kShare, 30);
             tmem_ld16_issue(acc_addr(jj + kShare), ra);
           }
         };
-        for (; j < T; j += kShare) {
+        for (; j < MB * T; j += kShare) {
           // tiles that every row of the warp sees completely take the unmasked path (rows that see nothing at all,
           // i.e. padding, still run: their sums are never used)
-          const bool masked = lim >= 0 && (ui.t_begin + j) * kTileN + kTileN - 1 > lim;
+          const bool masked = lim >= 0 && (ui.t_begin + j / MB) * kTileN + kTileN - 1 > lim;
           if (__any_sync(0xffffffffu, masked)) job1(std::true_type{}, j);
           else job1(std::false_type{}, j);
         }
@@ -638,8 +645,8 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 
       // ---- pass 2: for key row_in_tile of each tile, the sum over this group's rows of exp2(s*c - beta_row)
       const int min_lim = p.causal ? n - Wp : n - 1;  // every valid row sees keys up to here
-      const int j0 = p.two_pass ? T : 0;
-      const int n_jobs = j0 + T;
+      const int j0 = p.two_pass ? MB * T : 0;
+      const int n_jobs = j0 + MB * T;
       const long long unit_off = ((long long)ui.l * p.Hkv + ui.g) * p.seq.total;
       const float4* tab4 = reinterpret_cast<const float4*>(sm.tab[up] + coff);
       const float4* nb4 = reinterpret_cast<const float4*>(sm.nbeta[up] + coff);
@@ -712,26 +719,36 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           }
         };
         for (; j < n_jobs; j += kShare) {
-          const int key = (ui.t_begin + (p.two_pass ? n_jobs - 1 - j : j)) * kTileN + row_in_tile;
+          const int tl = (j - j0) / MB;  // the pass walks the CTA's tiles backwards after a first pass
+          const int key = (ui.t_begin + (p.two_pass ? T - 1 - tl : tl)) * kTileN + row_in_tile;
           sA4[0] = sA4[1] = sA4[2] = sA4[3] = 0.0f;
           sP = 0.0f;
           // only the last W-1 keys of a sequence are hidden from some rows: those tiles take the masked path
           if (__all_sync(0xffffffffu, key <= min_lim || key >= n)) job2(std::false_type{}, j, key);
           else job2(std::true_type{}, j, key);
           float sA = (sA4[0] + sA4[1]) + (sA4[2] + sA4[3]);
-          if (MB == 2) {  // add the two halves of the rows: the second group of the pair hands its sums to the first
-            const int jpar = ((jg + j) >> 1) & 1;
-            if (half == 1) {
-              sm.pair_sum[slot][jpar][0][row_in_tile] = sA;
-              if (PM == kOutAP) sm.pair_sum[slot][jpar][1][row_in_tile] = sP;
-            }
-            pair_bar(slot);
-            if (half == 0) {
-              sA += sm.pair_sum[slot][jpar][0][row_in_tile];
-              if (PM == kOutAP) sP += sm.pair_sum[slot][jpar][1][row_in_tile];
+          if (MB == 2) {
+            // The two row blocks of a tile are consecutive jobs of two different groups. The group of block 0 leaves
+            // its sums in a ring slot and goes on; the group of block 1, which gets its job later, picks them up, adds
+            // its own and stores. Neither waits for the other unless the ring is full (block 0 four tiles ahead).
+            const int pr = grp >> 1, r = pc % Cfg::kRing;
+            const uint32_t ph = (uint32_t)(pc / Cfg::kRing) & 1u;
+            ++pc;
+            if (blk == 0) {
+              mbar_wait(smem_u32(&sm.pfree[pr][r]), ph ^ 1u, abort_flag, p.status, 33, limit);
+              sm.psum[pr][r][0][row_in_tile] = sA;
+              if (PM == kOutAP) sm.psum[pr][r][1][row_in_tile] = sP;
+              __syncwarp();
+              if (lane == 0) mbar_arrive(smem_u32(&sm.pfull[pr][r]));
+            } else {
+              mbar_wait(smem_u32(&sm.pfull[pr][r]), ph, abort_flag, p.status, 34, limit);
+              sA += sm.psum[pr][r][0][row_in_tile];
+              if (PM == kOutAP) sP += sm.psum[pr][r][1][row_in_tile];
+              __syncwarp();
+              if (lane == 0) mbar_arrive(smem_u32(&sm.pfree[pr][r]));
             }
           }
-          if (half == 0 && key < n && !*abort_flag) {
+          if (blk == MB - 1 && key < n && !*abort_flag) {
             const long long o = unit_off + ui.tok0 + key;
             if (PM == kOutFused) {
               p.u[o] = sA;
