@@ -756,7 +756,12 @@ ta_status compress_impl(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* p
   mark(0);
   ctx->ev_ran[0] = 0;
   cudaStream_t seq_stream = stream;
-  const bool fork = !reuse && !fast && !external;
+  // ...but only while the score kernel is short. It is persistent, so kernels beside it need SMs of their own (4 are
+  // left free); a long score kernel gains more from those SMs than the step gains from hiding the per-sequence work,
+  // which then simply runs first.
+  const long long score_jobs = 2LL * batch->n_layers * batch->batch * Hkv * ((batch->max_n + 127) / 128) *
+                               (((Hq / Hkv) * policy->obs_window + 127) / 128);
+  const bool fork = !reuse && !fast && !external && score_jobs <= 400LL * ctx->sm_count;
   if (fork) {
     seq_stream = ctx->side;
     e = cudaEventRecord(ctx->ev_fork, stream);
