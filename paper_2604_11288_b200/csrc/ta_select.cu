@@ -20,569 +20,20 @@
 
 namespace cg = cooperative_groups;
 
+#define TA_SEL_THREADS 512
+#define TA_SEL_NS sel512
+#include "ta_select_core.cuh"
+#undef TA_SEL_THREADS
+#undef TA_SEL_NS
+#define TA_SEL_THREADS 1024
+#define TA_SEL_NS sel1024
+#include "ta_select_core.cuh"
+#undef TA_SEL_THREADS
+#undef TA_SEL_NS
+
 namespace {
 
-constexpr int kThreads = 512;
-constexpr int kWarps = kThreads / 32;
-
-__device__ __forceinline__ uint32_t sortable_key(float f) {
-  uint32_t b = __float_as_uint(f);
-  if ((b << 1) == 0u) b = 0u;  // -0 == +0
-  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
-}
-
-constexpr int kItemsLong = 32;  // keys per thread of clustered units (up to 8 * kItemsLong * kThreads elements)
-
-struct SelectResult {
-  uint32_t thresh;  // key of the last element taken
-  int ties;         // how many elements equal to thresh are taken (lowest positions first)
-  int all;          // 1: every eligible element is taken (fewer eligible than requested)
-  int none;         // 1: nothing is taken
-};
-
-struct SelectShared {
-  uint32_t hist[256];
-  uint32_t prefix, mask;
-  int remaining;
-  int done_all;
-  __align__(16) uint32_t warp_cnt[kWarps];  // per warp: definite count (low 16 bits) | tie count (high 16 bits)
-  // long sequences are split over the CTAs of a cluster: histogram of the whole unit (on rank 0, two buffers
-  // alternating by pass) and every CTA's (definite, tie) totals
-  uint32_t ghist[2][256];
-  int totals[8][2];
-  // ordered write of a unit whose keys sit in registers: per (chunk of kThreads elements, warp) the counts of
-  // definite | tie elements (packed 16 | 16 bits, then their exclusive prefix) and the two ballots
-  uint32_t cnt[kItemsLong * kWarps];
-  uint32_t bdef[kItemsLong * kWarps], btie[kItemsLong * kWarps];
-  uint32_t wtot[kWarps];
-  uint32_t total;
-};
-constexpr int kSelectCluster = 8;  // CTAs per unit when a sequence is longer than kItems * kThreads
-
-// Keys of a unit are read once into registers when the unit is short enough (kItems per thread), else they are
-// re-read from L2 on every sweep in batches whose loads are all issued before the first use.
-constexpr int kItems = 16;
-constexpr int kBatch = 8;
-template <int ITEMS>
-struct KeyCache {
-  uint32_t key[ITEMS];
-  uint32_t elig;  // bit `it`: element tid + it*kThreads exists and is eligible
-};
-
-template <class KeyFn, int ITEMS>
-__device__ __forceinline__ void fill_cache(int n, KeyFn key_of, KeyCache<ITEMS>& kc) {
-  kc.elig = 0;
-#pragma unroll
-  for (int it = 0; it < ITEMS; ++it) {
-    const int i = (int)threadIdx.x + it * kThreads;
-    kc.key[it] = 0;
-    if (i < n && key_of(i, kc.key[it])) kc.elig |= 1u << it;
-  }
-}
-
-// Calls body(i, exists, eligible, key) for every element slot in ascending chunks of kThreads; every thread of the
-// block makes the same number of calls (the body may hold block-wide barriers).
-template <bool CACHED, class KeyFn, class Body, int ITEMS>
-__device__ __forceinline__ void sweep(int n, KeyFn key_of, const KeyCache<ITEMS>& kc, Body body) {
-  const int tid = threadIdx.x;
-  if (CACHED) {
-#pragma unroll
-    for (int it = 0; it < ITEMS; ++it) {
-      if (it * kThreads < n) {
-        const int i = tid + it * kThreads;
-        body(i, i < n, ((kc.elig >> it) & 1u) != 0, kc.key[it]);
-      }
-    }
-  } else {
-    for (int base = 0; base < n; base += kBatch * kThreads) {
-      uint32_t k[kBatch];
-      uint32_t e = 0;
-#pragma unroll
-      for (int b = 0; b < kBatch; ++b) {
-        const int i = base + b * kThreads + tid;
-        k[b] = 0;
-        if (i < n && key_of(i, k[b])) e |= 1u << b;
-      }
-#pragma unroll
-      for (int b = 0; b < kBatch; ++b) {
-        if (base + b * kThreads < n) {
-          const int i = base + b * kThreads + tid;
-          body(i, i < n, ((e >> b) & 1u) != 0, k[b]);
-        }
-      }
-    }
-  }
-}
-
-// Top-`want` of the eligible elements of [0, n) by key. All threads of the block must call it; the result is uniform
-// across the block.
-template <bool CACHED, int CL, class KeyFn, int ITEMS>
-__device__ SelectResult block_radix_select(int n, int want, KeyFn key_of, const KeyCache<ITEMS>& kc, SelectShared& sh) {
-  SelectResult r;
-  r.thresh = 0;
-  r.ties = 0;
-  r.all = 0;
-  r.none = (want <= 0);
-  if (r.none) return r;
-  const int tid = threadIdx.x, lane = tid & 31;
-  if (tid == 0) {
-    sh.prefix = 0;
-    sh.mask = 0;
-    sh.remaining = want;
-    sh.done_all = 0;
-  }
-  uint32_t* ghist0 = nullptr;
-  if (CL > 1) ghist0 = cg::this_cluster().map_shared_rank(&sh.ghist[0][0], 0);
-  for (int pass = 0; pass < 4; ++pass) {
-    const int shift = 24 - 8 * pass;
-    if (tid < 256) {
-      sh.hist[tid] = 0;
-      if (CL > 1) sh.ghist[pass & 1][tid] = 0;  // only rank 0's copy is used; its readers of two passes ago are done
-    }
-    if (CL > 1) cg::this_cluster().sync();
-    else __syncthreads();
-    const uint32_t prefix = sh.prefix, mask = sh.mask;
-    sweep<CACHED>(n, key_of, kc, [&](int, bool, bool elig, uint32_t key) {
-      const int bin = (elig && (key & mask) == prefix) ? (int)((key >> shift) & 255u) : -1;
-      const unsigned peers = __match_any_sync(0xffffffffu, bin);
-      if (bin >= 0 && lane == __ffs(peers) - 1) atomicAdd(&sh.hist[bin], (uint32_t)__popc(peers));
-    });
-    __syncthreads();
-    const uint32_t* hist = sh.hist;
-    if (CL > 1) {  // merge the slices' histograms on rank 0, then every CTA takes the same decision from the sum
-      uint32_t* gh = ghist0 + (pass & 1) * 256;
-      if (tid < 256 && sh.hist[tid]) atomicAdd(&gh[tid], sh.hist[tid]);
-      cg::this_cluster().sync();
-      hist = gh;
-    }
-    if (tid < 32) {
-      // lane l owns bins [8l, 8l+8); walk from the top bin down until `remaining` elements are covered
-      uint32_t hl[8];
-#pragma unroll
-      for (int k = 0; k < 8; ++k) hl[k] = hist[8 * lane + k];
-      uint32_t tot = 0;
-#pragma unroll
-      for (int k = 0; k < 8; ++k) tot += hl[k];
-      uint32_t above = 0;  // elements in lanes above this one
-      {
-        uint32_t run = tot;
-#pragma unroll
-        for (int off = 1; off < 32; off <<= 1) {
-          const uint32_t o = __shfl_down_sync(0xffffffffu, run, off);
-          if (lane + off < 32) run += o;
-        }
-        above = run - tot;
-      }
-      const int remaining = sh.remaining;
-      const uint32_t total = __shfl_sync(0xffffffffu, above + tot, 0);
-      if (pass == 0 && total < (uint32_t)remaining) {
-        if (lane == 0) sh.done_all = 1;
-      } else {
-        const bool mine = above < (uint32_t)remaining && (uint32_t)remaining <= above + tot;
-        if (mine) {
-          uint32_t cum = above;
-          int k = 7;
-#pragma unroll
-          for (int kk = 7; kk > 0; --kk) {
-            if (k == kk && cum + hl[kk] < (uint32_t)remaining) {
-              cum += hl[kk];
-              k = kk - 1;
-            }
-          }
-          const int bin = 8 * lane + k;
-          sh.remaining = remaining - (int)cum;
-          sh.prefix = prefix | ((uint32_t)bin << shift);
-          sh.mask = mask | (255u << shift);
-        }
-      }
-    }
-    __syncthreads();
-    if (sh.done_all) {
-      r.all = 1;
-      return r;
-    }
-  }
-  r.thresh = sh.prefix;
-  r.ties = sh.remaining;
-  return r;
-}
-
-// Ordered pass over [0, n): classify(i, eligible, key, def, tie) marks element i `definite` (taken for sure) or a
-// `tie` (taken while ties last). Calls emit(i, rank) for every taken element with its rank in ascending position
-// order. Returns the number taken.
-template <bool CACHED, class KeyFn, class ClassFn, class EmitFn, int ITEMS>
-__device__ int block_ordered_emit(int n, int ties_allowed, KeyFn key_of, const KeyCache<ITEMS>& kc, ClassFn classify,
-                                  EmitFn emit, SelectShared& sh, int def_base = 0, int tie_base = 0,
-                                  int* def_total_out = nullptr, int* tie_total_out = nullptr) {
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int def0 = def_base, tie0 = tie_base;
-  sweep<CACHED>(n, key_of, kc, [&](int i, bool exists, bool elig, uint32_t key) {
-    bool def = false, tie = false;
-    if (exists) classify(i, elig, key, def, tie);
-    const unsigned bd = __ballot_sync(0xffffffffu, def), bt = __ballot_sync(0xffffffffu, tie);
-    const unsigned lt = (1u << lane) - 1u;
-    if (lane == 0) sh.warp_cnt[warp] = (uint32_t)__popc(bd) | ((uint32_t)__popc(bt) << 16);
-    __syncthreads();
-    uint32_t before = 0, total = 0;
-    const uint4* wc = reinterpret_cast<const uint4*>(sh.warp_cnt);
-#pragma unroll
-    for (int q = 0; q < kWarps / 4; ++q) {
-      const uint4 c4 = wc[q];
-      const uint32_t cs[4] = {c4.x, c4.y, c4.z, c4.w};
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        total += cs[e];
-        if (4 * q + e < warp) before += cs[e];
-      }
-    }
-    const int def_before = (int)(before & 0xffffu) + __popc(bd & lt);
-    const int ties_seen = tie_base + (int)(before >> 16) + __popc(bt & lt);
-    if (def)
-      emit(i, def_base + def_before + min(ties_seen, ties_allowed));
-    else if (tie && ties_seen < ties_allowed)
-      emit(i, def_base + def_before + ties_seen);
-    def_base += (int)(total & 0xffffu);
-    tie_base += (int)(total >> 16);
-    __syncthreads();
-  });
-  if (def_total_out) *def_total_out = def_base - def0;
-  if (tie_total_out) *tie_total_out = tie_base - tie0;
-  return def_base + min(tie_base, ties_allowed);
-}
-
-// The ordered pass for a unit split over CL CTAs (rank r owns a contiguous, ascending slice): a counting sweep
-// gives every CTA its (definite, tie) totals, the totals are exchanged through distributed shared memory, and the
-// emitting sweep starts from the sums of the lower ranks. Returns the number taken over the whole unit.
-// The ordered pass when the keys sit in registers (ITEMS chunks of kThreads elements, element tid + it*kThreads in
-// chunk it): one sweep classifies and records, per chunk and warp, the counts and ballots of definite and tie
-// elements; one block-wide exclusive scan over those (chunk-major = position order) gives every warp its base; a
-// second sweep emits. Three block barriers (and one cluster barrier for the totals of the lower ranks) instead of two
-// per chunk. classify is called exactly once per element.
-template <int CL, class ClassFn, class EmitFn, int ITEMS>
-__device__ int cached_ordered_emit(int n, int ties_allowed, const KeyCache<ITEMS>& kc, ClassFn classify, EmitFn emit,
-                                   SelectShared& sh) {
-  static_assert(ITEMS <= kItemsLong && ITEMS <= 32, "per-thread masks hold one bit per chunk");
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int chunks = (n + kThreads - 1) / kThreads;
-  uint32_t mdef = 0, mtie = 0;
-#pragma unroll
-  for (int it = 0; it < ITEMS; ++it) {
-    if (it < chunks) {
-      const int i = tid + it * kThreads;
-      bool def = false, tie = false;
-      if (i < n) classify(i, ((kc.elig >> it) & 1u) != 0, kc.key[it], def, tie);
-      const unsigned bd = __ballot_sync(0xffffffffu, def), bt = __ballot_sync(0xffffffffu, tie);
-      if (def) mdef |= 1u << it;
-      if (tie) mtie |= 1u << it;
-      if (lane == 0) {
-        sh.cnt[it * kWarps + warp] = (uint32_t)__popc(bd) | ((uint32_t)__popc(bt) << 16);
-        sh.bdef[it * kWarps + warp] = bd;
-        sh.btie[it * kWarps + warp] = bt;
-      }
-    }
-  }
-  __syncthreads();
-  // exclusive scan of the packed counts over the chunks * kWarps entries (entry tid belongs to thread tid)
-  static_assert(kItemsLong * kWarps <= kThreads, "one scan entry per thread");
-  const uint32_t mine = tid < chunks * kWarps ? sh.cnt[tid] : 0u;
-  uint32_t run = mine;
-#pragma unroll
-  for (int off = 1; off < 32; off <<= 1) {
-    const uint32_t o = __shfl_up_sync(0xffffffffu, run, off);
-    if (lane >= off) run += o;
-  }
-  if (lane == 31) sh.wtot[warp] = run;
-  __syncthreads();
-  uint32_t before = 0, all = 0;
-#pragma unroll
-  for (int w = 0; w < kWarps; ++w) {
-    const uint32_t t = sh.wtot[w];
-    if (w < warp) before += t;
-    all += t;
-  }
-  if (tid < chunks * kWarps) sh.cnt[tid] = before + run - mine;
-  int def_base = 0, tie_base = 0;
-  int def_all = (int)(all & 0xffffu), tie_all = (int)(all >> 16);
-  if (CL > 1) {
-    cg::cluster_group cluster = cg::this_cluster();
-    const int rank = (int)cluster.block_rank();
-    if (tid < CL) {
-      int* peer = cluster.map_shared_rank(&sh.totals[0][0], tid);
-      peer[rank * 2 + 0] = def_all;
-      peer[rank * 2 + 1] = tie_all;
-    }
-    cluster.sync();
-    def_all = 0;
-    tie_all = 0;
-#pragma unroll
-    for (int r = 0; r < CL; ++r) {
-      if (r < rank) {
-        def_base += sh.totals[r][0];
-        tie_base += sh.totals[r][1];
-      }
-      def_all += sh.totals[r][0];
-      tie_all += sh.totals[r][1];
-    }
-  } else {
-    __syncthreads();
-  }
-  const unsigned lt = (1u << lane) - 1u;
-#pragma unroll
-  for (int it = 0; it < ITEMS; ++it) {
-    if (it < chunks) {
-      const int e = it * kWarps + warp;
-      const uint32_t ex = sh.cnt[e];
-      const int def_before = def_base + (int)(ex & 0xffffu) + __popc(sh.bdef[e] & lt);
-      const int ties_seen = tie_base + (int)(ex >> 16) + __popc(sh.btie[e] & lt);
-      const int i = tid + it * kThreads;
-      if ((mdef >> it) & 1u) emit(i, def_before + min(ties_seen, ties_allowed));
-      else if (((mtie >> it) & 1u) && ties_seen < ties_allowed) emit(i, def_before + ties_seen);
-    }
-  }
-  return def_all + min(tie_all, ties_allowed);
-}
-
-template <bool CACHED, int CL, class KeyFn, class ClassFn, class EmitFn, int ITEMS>
-__device__ int cluster_ordered_emit(int n, int ties_allowed, KeyFn key_of, const KeyCache<ITEMS>& kc, ClassFn classify,
-                                    EmitFn emit, SelectShared& sh) {
-  if constexpr (CACHED) return cached_ordered_emit<CL>(n, ties_allowed, kc, classify, emit, sh);
-  if (CL == 1) return block_ordered_emit<CACHED>(n, ties_allowed, key_of, kc, classify, emit, sh);
-  cg::cluster_group cluster = cg::this_cluster();
-  const int rank = (int)cluster.block_rank();
-  int dt = 0, tt = 0;
-  block_ordered_emit<CACHED>(n, 0, key_of, kc, classify, [](int, int) {}, sh, 0, 0, &dt, &tt);
-  if (threadIdx.x < CL) {
-    int* peer = cluster.map_shared_rank(&sh.totals[0][0], threadIdx.x);
-    peer[rank * 2 + 0] = dt;
-    peer[rank * 2 + 1] = tt;
-  }
-  cluster.sync();
-  int def_base = 0, tie_base = 0, def_all = 0, tie_all = 0;
-#pragma unroll
-  for (int r = 0; r < CL; ++r) {
-    if (r < rank) {
-      def_base += sh.totals[r][0];
-      tie_base += sh.totals[r][1];
-    }
-    def_all += sh.totals[r][0];
-    tie_all += sh.totals[r][1];
-  }
-  block_ordered_emit<CACHED>(n, ties_allowed, key_of, kc, classify, emit, sh, def_base, tie_base);
-  return def_all + min(tie_all, ties_allowed);
-}
-
-// Slice [lo, hi) of a unit of n elements owned by this CTA when the unit is split over CL CTAs (whole chunks of
-// kThreads elements per CTA so that the slices stay aligned).
-template <int CL>
-__device__ __forceinline__ void unit_slice(int n, int& lo, int& hi) {
-  if (CL == 1) {
-    lo = 0;
-    hi = n;
-    return;
-  }
-  const int rank = (int)cg::this_cluster().block_rank();
-  const int per = ((n + CL - 1) / CL + kThreads - 1) / kThreads * kThreads;
-  lo = min(n, rank * per);
-  hi = min(n, lo + per);
-}
-
-struct SeqInfo {
-  int start, n, K_eff, s_take, r_take, p;
-  bool bad;  // the sequence does not lie inside the token arrays (cu_seqlens is device data the host cannot check)
-};
-
-__device__ __forceinline__ SeqInfo seq_info(const ta_seq_desc& seq, int b, int K, int n_sink, int n_recent,
-                                            int k_protected) {
-  SeqInfo s;
-  s.start = ta_seq_begin(seq, b);
-  s.n = (seq.cu ? seq.cu[b + 1] : s.start + seq.n_uniform) - s.start;
-  s.bad = s.n < 0 || s.n > seq.max_n || s.start < 0 || (long long)s.start + s.n > seq.total;
-  if (s.bad) s.n = 0;
-  s.K_eff = min(K, s.n);
-  int p = k_protected < 0 ? s.K_eff - n_sink - n_recent : k_protected;
-  p = max(0, min(p, s.K_eff));
-  s.p = p;
-  const int K_main = s.K_eff - p;
-  // mandatory list: sinks 0.. then recents n-1, n-2, .. (no duplicates), truncated to K_main entries
-  const int sinks = min(n_sink, s.n);
-  const int recents = max(0, min(n_recent, s.n - sinks));
-  s.s_take = min(sinks, K_main);
-  s.r_take = min(recents, K_main - s.s_take);
-  return s;
-}
-
-template <bool CACHED, int CL, int ITEMS = kItems>
-__global__ void __launch_bounds__(kThreads) ta_forced_kernel(ta_seq_desc seq, int K, int n_sink, int n_recent,
-                                                             int k_protected, const float* __restrict__ voucher,
-                                                             uint8_t* __restrict__ forced,
-                                                             int32_t* __restrict__ r_main, ta_dev_status* status,
-                                                             const int32_t* __restrict__ class_K) {
-  __shared__ SelectShared sh;
-  // grid.x = classes * sequences * CL; without budget classes there is one class and K is the argument
-  const int b = (blockIdx.x / CL) % seq.batch;
-  if (class_K) {
-    const int cls = (blockIdx.x / CL) / seq.batch;
-    K = class_K[cls];
-    forced += (long long)cls * seq.total;
-    r_main += cls * seq.batch;
-  }
-  const SeqInfo s = seq_info(seq, b, K, n_sink, n_recent, k_protected);
-  if (s.bad) {
-    if (threadIdx.x == 0) {
-      if (atomicCAS(&status->code, 0, (int)TA_ERR_DEVICE_BOUNDS) == 0) {
-        status->where = 3;
-        status->detail0 = b;
-        status->detail1 = s.start;
-      }
-      r_main[b] = -2;  // poisoned: the select kernel writes an empty result
-    }
-    return;
-  }
-  if (s.K_eff == s.n) {
-    if (threadIdx.x == 0) r_main[b] = -1;  // keep everything
-    return;
-  }
-  int lo, hi;
-  unit_slice<CL>(s.n, lo, hi);
-  const float* V = voucher + s.start + lo;  // this CTA's slice; local index il <-> position lo + il
-  auto mandatory = [&](int i) { return i < s.s_take || i >= s.n - s.r_take; };
-  auto key_of = [&](int il, uint32_t& key) {
-    const float v = V[il];
-    key = sortable_key(v);
-    return v > 0.0f && !mandatory(lo + il);
-  };
-  KeyCache<ITEMS> kc;
-  if (CACHED) fill_cache(hi - lo, key_of, kc);
-  const SelectResult r = block_radix_select<CACHED, CL>(hi - lo, s.p, key_of, kc, sh);
-  uint8_t* f = forced + s.start + lo;
-  // ordered pass: mandatory tokens and vouchers above the threshold are forced for sure; vouchers equal to the
-  // threshold are forced while protected slots last, lowest position first
-  auto classify = [&](int il, bool cand, uint32_t key, bool& def, bool& tie) {
-    def = mandatory(lo + il) || (cand && !r.none && (r.all || key > r.thresh));
-    tie = !def && cand && !r.none && !r.all && key == r.thresh;
-    f[il] = 0;  // set by emit when taken (same thread, later)
-  };
-  auto emit = [&](int il, int rank) { f[il] = 1; };
-  const int taken = cluster_ordered_emit<CACHED, CL>(hi - lo, r.ties, key_of, kc, classify, emit, sh);
-  if (threadIdx.x == 0 && blockIdx.x % CL == 0) r_main[b] = s.K_eff - taken;
-}
-
-struct UnitSrc {  // where a unit's utility comes from
-  const float* u;         // fused: [L][Hkv][total]
-  const float* A;         // unfused
-  const float* P;
-  const float* u_static;  // per token
-  float alpha, delta;
-};
-
-__device__ __forceinline__ float unit_utility(const UnitSrc& src, long long unit_off, long long tok) {
-  const float u0 = src.u_static[tok];
-  if (src.u) return __fadd_rn(src.u[unit_off + tok], u0);
-  if (!src.A) return u0;
-  const float aA = __fmul_rn(src.alpha, src.A[unit_off + tok]);
-  const float dP = __fmul_rn(src.delta, src.P ? src.P[unit_off + tok] : 0.0f);
-  return __fadd_rn(__fadd_rn(aA, dP), u0);
-}
-
-// Small budgets and few units: the block that selected a unit also moves its retained K and V rows (Algorithm 1
-// step 9), which saves the launch of the gather kernel where that launch costs more than the copy. Same result as ta_compact_kernel:
-// rows at and beyond the retained count, and rows whose index lies outside the sequence, are zero.
-struct GatherDst {
-  ta_bf16_view k, v;
-  uint4* k_out;
-  uint4* v_out;
-};
-constexpr int kGatherMaxK = 16;  // one 16-byte piece per thread
-
-__device__ __forceinline__ void gather_unit(const GatherDst& gd, const ta_seq_desc& seq, int unit, int l, int b, int g,
-                                            int n, int K, const int32_t* out, int taken) {
-  constexpr int kLanesPerRow = TA_HEAD_DIM * 2 / 16;
-  __syncthreads();  // the unit's indices were written by other threads of this block
-  for (int t = threadIdx.x; t < K * 2 * kLanesPerRow; t += kThreads) {
-    const int r = t / (2 * kLanesPerRow), which = (t / kLanesPerRow) & 1, lane16 = t % kLanesPerRow;
-    const ta_bf16_view& src = which ? gd.v : gd.k;
-    uint4 val = make_uint4(0u, 0u, 0u, 0u);
-    if (r < taken) {
-      const int i = out[r];
-      if (i >= 0 && i < n) {
-        const long long base = (long long)l * src.stride_l + (long long)g * src.stride_h +
-                               (seq.cu ? (long long)seq.cu[b] * src.stride_n : (long long)b * src.stride_b);
-        val = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const uint16_t*>(src.ptr) + base +
-                                                   (long long)i * src.stride_n) + lane16);
-      }
-    }
-    (which ? gd.v_out : gd.k_out)[((long long)unit * K + r) * kLanesPerRow + lane16] = val;
-  }
-}
-
-// grid.x = units. scored: unit = (l*B + b)*Hkv + g; fast: unit = b.
-template <bool CACHED, int CL, int ITEMS = kItems, bool GATHER = false>
-__global__ void __launch_bounds__(kThreads) ta_select_kernel(ta_seq_desc seq, int n_layers, int Hkv, int K, int fast,
-                                                             UnitSrc src, const uint8_t* __restrict__ forced,
-                                                             const int32_t* __restrict__ r_main,
-                                                             int32_t* __restrict__ idx, int32_t* __restrict__ count,
-                                                             GatherDst gd, const int32_t* __restrict__ class_of) {
-  __shared__ SelectShared sh;
-  const int unit = blockIdx.x / CL;
-  const bool lead = blockIdx.x % CL == 0;
-  int b, l = 0, g = 0;
-  if (fast) {
-    b = unit;
-  } else {
-    g = unit % Hkv;
-    b = (unit / Hkv) % seq.batch;
-    l = unit / (Hkv * seq.batch);
-  }
-  if (class_of) {  // budgets per (layer, head): the forced set and the main-pool size of this pair's class
-    const int cls = class_of[l * Hkv + g];
-    forced += (long long)cls * seq.total;
-    r_main += cls * seq.batch;
-  }
-  const int start = ta_seq_begin(seq, b);
-  const int n = (seq.cu ? seq.cu[b + 1] : start + seq.n_uniform) - start;
-  int32_t* out = idx + (long long)unit * K;
-  const int want = r_main[b];
-  const int tid = threadIdx.x;
-  if (want == -2) {  // sequence rejected by ta_forced_kernel
-    if (lead) {
-      for (int r = tid; r < K; r += kThreads) out[r] = -1;
-      if (tid == 0) count[unit] = 0;
-    }
-    if constexpr (GATHER) gather_unit(gd, seq, unit, l, b, g, n, K, out, 0);
-    return;
-  }
-  if (want == -1) {  // K >= n: keep everything
-    if (lead) {
-      for (int r = tid; r < K; r += kThreads) out[r] = r < n ? r : -1;
-      if (tid == 0) count[unit] = n;
-    }
-    if constexpr (GATHER) gather_unit(gd, seq, unit, l, b, g, n, K, out, n);
-    return;
-  }
-  const long long unit_off = fast ? 0 : ((long long)l * Hkv + g) * seq.total;
-  int lo, hi;
-  unit_slice<CL>(n, lo, hi);
-  const uint8_t* f = forced + start + lo;
-  auto key_of = [&](int il, uint32_t& key) {
-    key = sortable_key(unit_utility(src, unit_off, (long long)start + lo + il));
-    return f[il] == 0;
-  };
-  KeyCache<ITEMS> kc;
-  if (CACHED) fill_cache(hi - lo, key_of, kc);
-  const SelectResult r = block_radix_select<CACHED, CL>(hi - lo, want, key_of, kc, sh);
-  auto classify = [&](int, bool elig, uint32_t key, bool& def, bool& tie) {
-    def = !elig || (!r.none && (r.all || key > r.thresh));
-    tie = !def && !r.none && !r.all && key == r.thresh;
-  };
-  auto emit = [&](int il, int rank) {
-    if (rank < K) out[rank] = lo + il;
-  };
-  const int taken = cluster_ordered_emit<CACHED, CL>(hi - lo, r.ties, key_of, kc, classify, emit, sh);
-  if (!lead) return;
-  for (int q = taken + tid; q < K; q += kThreads) out[q] = -1;
-  if (tid == 0) count[unit] = taken;
-  if constexpr (GATHER) gather_unit(gd, seq, unit, l, b, g, n, K, out, min(taken, K));
-}
+using namespace sel512;  // the launchers below name the 512-thread kernels unless they say otherwise
 
 __global__ void ta_broadcast_idx_kernel(int B, int Hkv, int K, int n_layers, const int32_t* __restrict__ idx_seq,
                                         const int32_t* __restrict__ count_seq, int32_t* __restrict__ idx,
@@ -650,10 +101,10 @@ int sm_count_of(const ta_select_args& a) {
 }
 
 template <class Kern, class... Args>
-cudaError_t launch_clustered(Kern kern, int units, int cl, cudaStream_t stream, Args... args) {
+cudaError_t launch_threads(int threads, Kern kern, int units, int cl, cudaStream_t stream, Args... args) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)(units * cl), 1, 1);
-  cfg.blockDim = dim3(kThreads, 1, 1);
+  cfg.blockDim = dim3((unsigned)threads, 1, 1);
   cfg.dynamicSmemBytes = 0;
   cfg.stream = stream;
   cudaLaunchAttribute attr[1];
@@ -664,6 +115,10 @@ cudaError_t launch_clustered(Kern kern, int units, int cl, cudaStream_t stream, 
   cfg.attrs = attr;
   cfg.numAttrs = cl > 1 ? 1 : 0;  // a plain launch when no cluster is needed
   return cudaLaunchKernelEx(&cfg, kern, args...);
+}
+template <class Kern, class... Args>
+cudaError_t launch_clustered(Kern kern, int units, int cl, cudaStream_t stream, Args... args) {
+  return launch_threads(kThreads, kern, units, cl, stream, args...);
 }
 
 cudaError_t ta_launch_forced(const ta_select_args& a, ta_dev_status* status, cudaStream_t stream) {
@@ -726,6 +181,20 @@ cudaError_t ta_launch_select_units(const ta_select_args& a, cudaStream_t stream)
   if (!split_units(units, a.seq.max_n, sms) && a.seq.max_n <= kItemsLong * kThreads)
     return launch_clustered(ta_select_kernel<true, 1, kItemsLong>, units, 1, stream, a.seq, a.n_layers, a.Hkv, a.K, a.fast,
                             src, a.forced, a.r_main, a.idx, a.count, gd, co);
+  if (!split_units(units, a.seq.max_n, sms) && a.seq.max_n <= sel1024::kItemsLong * sel1024::kThreads) {
+    // many long units: blocks of 1024 threads hold a unit of up to 32768 keys in registers (read once instead of
+    // once per radix pass and once more for the ordered write)
+    sel1024::UnitSrc src2;
+    src2.u = src.u;
+    src2.A = src.A;
+    src2.P = src.P;
+    src2.u_static = src.u_static;
+    src2.alpha = src.alpha;
+    src2.delta = src.delta;
+    sel1024::GatherDst gd2 = {};
+    return launch_threads(sel1024::kThreads, sel1024::ta_select_kernel<true, 1, sel1024::kItemsLong>, units, 1, stream,
+                          a.seq, a.n_layers, a.Hkv, a.K, a.fast, src2, a.forced, a.r_main, a.idx, a.count, gd2, co);
+  }
   if (!split_units(units, a.seq.max_n, sms))
     return launch_clustered(ta_select_kernel<false, 1>, units, 1, stream, a.seq, a.n_layers, a.Hkv, a.K, a.fast, src,
                             a.forced, a.r_main, a.idx, a.count, gd, co);

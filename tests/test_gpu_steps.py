@@ -359,6 +359,19 @@ def test_select_scored_given_scores_bit_exact(K):
     _select_case(w, oracle_policy(K, "THEOREM"), K, L, (A, P))
 
 
+@pytest.mark.parametrize("K", [64, 2048])
+def test_select_many_long_units_keys_in_registers_of_big_blocks(K):
+    # 48 units of up to 32768 tokens: too many to split each over a cluster, so a block of 1024 threads holds a
+    # unit's keys in registers; exact ties, a full-length unit, one just above the 512-thread limit and a short one
+    w = _workload([32768, 16385, 20011, 900], [[5, 6, 7], [9]], seed=100 + K, Hq=4, Hkv=2)
+    L = 6
+    gen = torch.Generator().manual_seed(K)
+    A = torch.rand((L, w.Hkv, w.total), generator=gen).cuda()
+    A = (A * 128).round() / 128
+    P = (torch.rand((L, w.Hkv, w.total), generator=gen) * 0.1).cuda()
+    _select_case(w, oracle_policy(K, "THEOREM"), K, L, (A, P))
+
+
 def test_select_sponsored_overflow_and_precedence():
     # far more sponsored tokens than protected slots: nearest-to-anchor first, earlier anchors win ties
     w = _workload([5000], [[1]], [12], alphabet=40, seed=4)
