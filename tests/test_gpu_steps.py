@@ -284,8 +284,9 @@ def test_score_scores_far_above_and_below_the_first_keys(W):
     g.close()
 
 
-def test_score_with_supplied_lse_matches_two_pass():
-    w, pol, Qh, Kh, Qd, Kd, A2, g = _score_case([1300, 70], 8, 2, 32, seed=5)
+@pytest.mark.parametrize("W", [32, 64])
+def test_score_with_supplied_lse_matches_two_pass(W):
+    w, pol, Qh, Kh, Qd, Kd, A2, g = _score_case([1300, 70], 8, 2, W, seed=5)
     try:
         # log-sum-exp of every window row, from a library softmax in fp64
         G = w.Hq // w.Hkv
