@@ -439,6 +439,22 @@ def measure_others(main_name, dev, steps, warmup):
     return out
 
 
+def window_lse(inp, w, L):
+    """Natural-log softmax normalisers [L][B][Hq][W] of the observation-window rows of a uniform batch, by torch on the
+    device (what a prefill attention kernel would have left behind; input preparation, never timed)."""
+    G, n, W = w.Hq // w.Hkv, int(w.lengths[0]), w.W
+    lse = torch.empty((L, w.B, w.Hq, W), dtype=torch.float32, device=inp.dev)
+    pos = torch.arange(n - W, n, device=inp.dev).view(1, -1, 1)
+    key = torch.arange(n, device=inp.dev).view(1, 1, -1)
+    for l in range(L):
+        for b in range(w.B):
+            k = inp.Kc[l, b].float().repeat_interleave(G, dim=0)           # [Hq, n, d]
+            s = torch.bmm(inp.Q[l, b].float(), k.transpose(1, 2)) / float(np.sqrt(w.d))  # [Hq, W, n]
+            s = s.masked_fill(key > pos, float("-inf"))
+            lse[l, b] = torch.logsumexp(s, dim=-1)
+    return lse
+
+
 def measure_variants(dev, steps=10, warmup=3):
     """Timings of the entry points beyond the one-shot ta_compress, on synthetic inputs of the main workload's shape:
     selection shared by the heads of a layer, a caller-supplied score, detector-confidence anchors, and the per-step
@@ -457,6 +473,16 @@ def measure_variants(dev, steps=10, warmup=3):
         ms = float(np.median(time_rounds(allheads, steps, warmup, 3)))
         out.append({"entry": "ta_compress_allheads", "workload": f"c2, {L} layers, K={K}", "ms_per_step": ms,
                     "value": w.total * L / (ms * 1e-3), "unit": UNIT})
+        # the same step when the caller's prefill kernel has left the softmax normalisers of the window rows: one pass
+        # over the keys. The normalisers are prepared here with torch (a stand-in for that kernel), outside the timing.
+        lse = window_lse(inp, w, L)
+
+        def with_lse():
+            ta.ta_compress_lse(r.ctx, r.pats, r.p, r.batch, w.Hq, w.Hkv, w.d, K, inp.ids, r.vq, inp.vk, inp.vv, lse, 0,
+                               r.ko, r.vo, r.idx, r.cnt, r.stream)
+        ms = float(np.median(time_rounds(with_lse, steps, warmup, 3)))
+        out.append({"entry": "ta_compress_lse", "workload": f"c2, {L} layers, K={K}, normalisers supplied",
+                    "ms_per_step": ms, "value": w.total * L / (ms * 1e-3), "unit": UNIT})
         score = torch.rand((L, w.Hkv, w.total), dtype=torch.float32, device=dev)
 
         def scores():

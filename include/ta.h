@@ -320,6 +320,14 @@ ta_status ta_compress(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* pol
                       ta_bf16_view v, uint64_t seq_epoch, void* k_out, void* v_out, int32_t* idx, int32_t* count,
                       void* stream);
 
+/* The same when the softmax normalisers of the observation-window rows are already known (a prefill attention kernel
+ * computes the log-sum-exp of every query row): lse_obs is DEVICE float [L][B][Hq][W], natural log, as for ta_score.
+ * The keys are then read once instead of twice and the scoring costs about half. Scored mode only. */
+ta_status ta_compress_lse(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* policy, const ta_batch* batch, int Hq,
+                          int Hkv, int d, int K, const int32_t* token_ids, ta_bf16_view q_obs, ta_bf16_view k,
+                          ta_bf16_view v, const float* lse_obs, uint64_t seq_epoch, void* k_out, void* v_out,
+                          int32_t* idx, int32_t* count, void* stream);
+
 /* ---- one selection per layer, shared by its KV heads (Eq. 1: A_i "across heads") -----------------------------
  * Eq. 1 and Appendix A Definition 1 define A_i as attention accumulated over ALL heads, which gives one retained
  * set per layer. ta_compress reads them per KV head (every head keeps its own K tokens); this entry point takes

@@ -91,6 +91,8 @@ def lib():
             "ta_compact_kv": (i32, [vp, PB, i32, i32, i32, ta_bf16_view, ta_bf16_view, vp, vp, vp, vp, vp]),
             "ta_compress": (i32, [vp, vp, PP, PB, i32, i32, i32, i32, vp, ta_bf16_view, ta_bf16_view, ta_bf16_view,
                                   u64, vp, vp, vp, vp, vp]),
+            "ta_compress_lse": (i32, [vp, vp, PP, PB, i32, i32, i32, i32, vp, ta_bf16_view, ta_bf16_view, ta_bf16_view, vp,
+                                      u64, vp, vp, vp, vp, vp]),
             "ta_compress_allheads": (i32, [vp, vp, PP, PB, i32, i32, i32, i32, vp, ta_bf16_view, ta_bf16_view,
                                            ta_bf16_view, u64, vp, vp, vp, vp, vp]),
             "ta_score_headsum": (i32, [vp, PP, PB, i32, i32, i32, ta_bf16_view, ta_bf16_view, vp, vp]),
@@ -241,6 +243,13 @@ def ta_score_weighted(ctx, policy, batch, Hq, Hkv, d, q_obs: ta_bf16_view, k: ta
 
 def ta_ctx_set_wait_limit(ctx, nanoseconds: int):
     _check(lib().ta_ctx_set_wait_limit(ctx, int(nanoseconds)), "ta_ctx_set_wait_limit")
+
+
+def ta_compress_lse(ctx, pats, policy, batch, Hq, Hkv, d, K, token_ids, q_obs: ta_bf16_view, k: ta_bf16_view,
+                    v: ta_bf16_view, lse_obs, seq_epoch, k_out, v_out, idx, count, stream=None):
+    _check(lib().ta_compress_lse(ctx, pats, C.byref(policy), C.byref(batch), Hq, Hkv, d, K, _ptr(token_ids), q_obs, k, v,
+                                 _ptr(lse_obs), seq_epoch, _ptr(k_out), _ptr(v_out), _ptr(idx), _ptr(count), stream),
+           "ta_compress_lse")
 
 
 def ta_score_headsum(ctx, policy, batch, Hq, Hkv, d, q_obs: ta_bf16_view, k: ta_bf16_view, u_heads, stream=None):

@@ -631,7 +631,8 @@ ta_status compress_impl(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* p
                         int Hkv, int d, int K, const int32_t* token_ids, ta_bf16_view q_obs, ta_bf16_view k,
                         ta_bf16_view v, uint64_t seq_epoch, void* k_out, void* v_out, int32_t* idx, int32_t* count,
                         void* stream_v, const float* ext_A, const float* ext_P, bool share_heads,
-                        const int32_t* budgets = nullptr, const float* ext_u_all = nullptr) {
+                        const int32_t* budgets = nullptr, const float* ext_u_all = nullptr,
+                        const float* lse_obs = nullptr) {
   Range range("ta_compress");
   if (!ctx || !pats || !token_ids || !k_out || !v_out || !idx || !count) return TA_ERR_INVALID_ARG;
   ta_status s = check_batch(batch);
@@ -759,7 +760,7 @@ ta_status compress_impl(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* p
   // ...but only while the score kernel is short. It is persistent, so kernels beside it need SMs of their own (4 are
   // left free); a long score kernel gains more from those SMs than the step gains from hiding the per-sequence work,
   // which then simply runs first.
-  const long long score_jobs = 2LL * batch->n_layers * batch->batch * Hkv * ((batch->max_n + 127) / 128) *
+  const long long score_jobs = (lse_obs ? 1LL : 2LL) * batch->n_layers * batch->batch * Hkv * ((batch->max_n + 127) / 128) *
                                (((Hq / Hkv) * policy->obs_window + 127) / 128);
   const bool fork = !reuse && !fast && !external && score_jobs <= 400LL * ctx->sm_count;
   if (fork) {
@@ -789,7 +790,7 @@ ta_status compress_impl(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* p
     a.W = policy->obs_window;
     a.q = q_obs;
     a.k = k;
-    a.lse_obs = nullptr;
+    a.lse_obs = lse_obs;  // the rows' normalisers from the caller's prefill kernel: one pass over the keys
     a.A = nullptr;
     a.P = nullptr;
     a.u = u;
@@ -850,6 +851,16 @@ ta_status ta_compress(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* pol
                       void* stream) {
   return compress_impl(ctx, pats, policy, batch, Hq, Hkv, d, K, token_ids, q_obs, k, v, seq_epoch, k_out, v_out, idx,
                        count, stream, nullptr, nullptr, false);
+}
+
+ta_status ta_compress_lse(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* policy, const ta_batch* batch, int Hq,
+                          int Hkv, int d, int K, const int32_t* token_ids, ta_bf16_view q_obs, ta_bf16_view k,
+                          ta_bf16_view v, const float* lse_obs, uint64_t seq_epoch, void* k_out, void* v_out,
+                          int32_t* idx, int32_t* count, void* stream) {
+  if (!policy || !lse_obs) return TA_ERR_INVALID_ARG;
+  if (policy->mode != TA_MODE_SCORED) return TA_ERR_INVALID_ARG;
+  return compress_impl(ctx, pats, policy, batch, Hq, Hkv, d, K, token_ids, q_obs, k, v, seq_epoch, k_out, v_out, idx,
+                       count, stream, nullptr, nullptr, false, nullptr, nullptr, lse_obs);
 }
 
 ta_status ta_compress_allheads(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* policy, const ta_batch* batch,

@@ -277,3 +277,58 @@ def test_weighted_odd_windows(W):
     # windows that are not a multiple of 8: G*W rows that end inside a 16-row group of the accumulator
     _weighted_case([700, 40, 3], 4, 1, W, seed=20 + W)
     _weighted_case([1400], 8, 2, W, seed=40 + W)
+
+
+def _lse_rows(w, Qh, Kh, L):
+    """Natural-log softmax normalisers of every window row (what a prefill attention kernel leaves behind), fp64."""
+    G = w.Hq // w.Hkv
+    lse = torch.zeros((L, w.B, w.Hq, w.W), dtype=torch.float64)
+    for l in range(L):
+        for b in range(w.B):
+            o, e = int(w.cu[b]), int(w.cu[b + 1])
+            n = e - o
+            if n == 0:
+                continue
+            for h in range(w.Hq):
+                k = Kh[l, h // G, o:e].double()
+                s = (Qh[l, b, h].double() @ k.T) / np.sqrt(128.0)
+                pos = torch.arange(n - w.W, n).view(-1, 1)
+                s = s.masked_fill(torch.arange(n).view(1, -1) > pos, float("-inf"))
+                lse[l, b, h] = torch.where(pos.view(-1) >= 0, torch.logsumexp(s, -1), torch.zeros(w.W).double())
+    return lse
+
+
+@pytest.mark.parametrize("W", [32, 64])
+def test_compress_with_supplied_normalisers_reads_the_keys_once(W):
+    from ta_testlib import assert_selection_matches, oracle_patterns, oracle_unit
+    w = _workload([1700, 90, 640], [[4, 5], [9]], seed=50 + W, Hq=8, Hkv=2, W=W)
+    K, L = 24, 2
+    pol = oracle_policy(K, "THEOREM", W=W)
+    Qh, Kh, Vh = tw.make_qkv(w, range(L))
+    lse = _lse_rows(w, Qh, Kh, L).float().cuda()
+    g = Gpu(w, pol, K, L)
+    try:
+        Qd, Kd, Vd = Qh.cuda(), Kh.cuda(), Vh.cuda()
+        idx = torch.full((L, w.B, w.Hkv, K), -7, dtype=torch.int32, device="cuda")
+        cnt = torch.full((L, w.B, w.Hkv), -7, dtype=torch.int32, device="cuda")
+        ko = torch.full((L, w.B, w.Hkv, K, w.d), 1.0, dtype=torch.bfloat16, device="cuda")
+        vo = torch.full_like(ko, 1.0)
+        ta.ta_compress_lse(g.ctx, g.pats, g.p, g.batch, w.Hq, w.Hkv, w.d, K, g.ids, ta.view(Qd), ta.view(Kd, True),
+                           ta.view(Vd, True), lse, 0, ko, vo, idx, cnt, g.stream)
+        torch.cuda.synchronize()
+        assert g.poll() == ta.TA_OK
+        idx, cnt = idx.cpu().numpy(), cnt.cpu().numpy()
+        f_o, V_o, u0_o = oracle.sponsor_mask(w.ids, w.cu, oracle_patterns(w), pol)
+        for l in range(L):
+            for b in range(w.B):
+                for h in range(w.Hkv):
+                    A, P, u, io, co = oracle_unit(w, pol, K, Qh, Kh, l, b, h, V_o, u0_o)
+                    assert_selection_matches(idx[l, b, h], cnt[l, b, h], io, co, u, f"l{l} b{b} h{h}")
+                    c = int(cnt[l, b, h])
+                    np.testing.assert_array_equal(bf16_bits(ko[l, b, h]),
+                                                  oracle.compact(unit_kv(w, Kh, l, b, h), idx[l, b, h], c, K))
+        with pytest.raises(ta.TAError):
+            ta.ta_compress_lse(g.ctx, g.pats, g.p, g.batch, w.Hq, w.Hkv, w.d, K, g.ids, ta.view(Qd), ta.view(Kd, True),
+                               ta.view(Vd, True), None, 0, ko, vo, idx, cnt, g.stream)
+    finally:
+        g.close()
