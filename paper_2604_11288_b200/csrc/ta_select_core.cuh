@@ -126,6 +126,13 @@ __device__ SelectResult block_radix_select(int n, int want, KeyFn key_of, const 
     const uint32_t prefix = sh.prefix, mask = sh.mask;
     sweep<CACHED>(n, key_of, kc, [&](int, bool, bool elig, uint32_t key) {
       const int bin = (elig && (key & mask) == prefix) ? (int)((key >> shift) & 255u) : -1;
+      // after the first pass most warps hold no candidate at all: a ballot is far cheaper than match.any
+      const unsigned have = __ballot_sync(0xffffffffu, bin >= 0);
+      if (have == 0u) return;
+      if ((have & (have - 1u)) == 0u) {  // a single candidate in the warp
+        if (bin >= 0) atomicAdd(&sh.hist[bin], 1u);
+        return;
+      }
       const unsigned peers = __match_any_sync(0xffffffffu, bin);
       if (bin >= 0 && lane == __ffs(peers) - 1) atomicAdd(&sh.hist[bin], (uint32_t)__popc(peers));
     });
