@@ -82,7 +82,8 @@ __global__ void ta_broadcast_heads_kernel(long long units_lb, int Hkv, int K, co
 // additionally idx_seq [B][K] and count_seq [B] (passed through a.idx / a.count by the caller when it wants the
 // per-sequence result only).
 // Sequences that fit kItems keys per thread run one CTA per unit with the keys in registers; longer ones are split
-// over a cluster of kSelectCluster CTAs (keys in registers up to kSelectCluster * kItemsLong * kThreads elements).
+// over a cluster of kSelectCluster CTAs (keys in registers up to kSelectCluster * 32 * 1024 elements; beyond 65536
+// elements the cluster's blocks have 1024 threads).
 // Splitting pays only while the clusters of all units fit on the device about at once; with many units one CTA per
 // unit (keys re-read in batches when they do not fit in registers) keeps every SM busy without cluster barriers.
 bool split_units(int units, int max_n, int sms) {
@@ -138,9 +139,16 @@ cudaError_t ta_launch_forced(const ta_select_args& a, ta_dev_status* status, cud
   if (a.seq.max_n <= kSelectCluster * kItems * kThreads)
     return launch_clustered(ta_forced_kernel<true, kSelectCluster>, B, kSelectCluster, stream, a.seq, a.K, a.n_sink,
                             a.n_recent, a.k_protected, a.voucher, a.forced, a.r_main, status, ck);
-  if (a.seq.max_n <= kSelectCluster * kItemsLong * kThreads)
-    return launch_clustered(ta_forced_kernel<true, kSelectCluster, kItemsLong>, B, kSelectCluster, stream, a.seq, a.K,
-                            a.n_sink, a.n_recent, a.k_protected, a.voucher, a.forced, a.r_main, status, ck);
+  // few very long sequences: the chain of per-thread sweeps and cluster barriers sets the time, so blocks of 1024
+  // threads (half the keys per thread) roughly halve it
+  if (a.seq.max_n <= kSelectCluster * sel1024::kItems * sel1024::kThreads)
+    return launch_threads(sel1024::kThreads, sel1024::ta_forced_kernel<true, kSelectCluster>, B, kSelectCluster,
+                          stream, a.seq, a.K, a.n_sink, a.n_recent, a.k_protected, a.voucher, a.forced, a.r_main,
+                          status, ck);
+  if (a.seq.max_n <= kSelectCluster * sel1024::kItemsLong * sel1024::kThreads)
+    return launch_threads(sel1024::kThreads, sel1024::ta_forced_kernel<true, kSelectCluster, sel1024::kItemsLong>, B,
+                          kSelectCluster, stream, a.seq, a.K, a.n_sink, a.n_recent, a.k_protected, a.voucher,
+                          a.forced, a.r_main, status, ck);
   return launch_clustered(ta_forced_kernel<false, kSelectCluster>, B, kSelectCluster, stream, a.seq, a.K, a.n_sink,
                           a.n_recent, a.k_protected, a.voucher, a.forced, a.r_main, status, ck);
 }
@@ -181,17 +189,17 @@ cudaError_t ta_launch_select_units(const ta_select_args& a, cudaStream_t stream)
   if (!split_units(units, a.seq.max_n, sms) && a.seq.max_n <= kItemsLong * kThreads)
     return launch_clustered(ta_select_kernel<true, 1, kItemsLong>, units, 1, stream, a.seq, a.n_layers, a.Hkv, a.K, a.fast,
                             src, a.forced, a.r_main, a.idx, a.count, gd, co);
+  sel1024::UnitSrc src2;  // the same fields for the kernels built for 1024 threads
+  src2.u = src.u;
+  src2.A = src.A;
+  src2.P = src.P;
+  src2.u_static = src.u_static;
+  src2.alpha = src.alpha;
+  src2.delta = src.delta;
+  sel1024::GatherDst gd2 = {};
   if (!split_units(units, a.seq.max_n, sms) && a.seq.max_n <= sel1024::kItemsLong * sel1024::kThreads) {
     // many long units: blocks of 1024 threads hold a unit of up to 32768 keys in registers (read once instead of
     // once per radix pass and once more for the ordered write)
-    sel1024::UnitSrc src2;
-    src2.u = src.u;
-    src2.A = src.A;
-    src2.P = src.P;
-    src2.u_static = src.u_static;
-    src2.alpha = src.alpha;
-    src2.delta = src.delta;
-    sel1024::GatherDst gd2 = {};
     return launch_threads(sel1024::kThreads, sel1024::ta_select_kernel<true, 1, sel1024::kItemsLong>, units, 1, stream,
                           a.seq, a.n_layers, a.Hkv, a.K, a.fast, src2, a.forced, a.r_main, a.idx, a.count, gd2, co);
   }
@@ -201,9 +209,14 @@ cudaError_t ta_launch_select_units(const ta_select_args& a, cudaStream_t stream)
   if (a.seq.max_n <= kSelectCluster * kItems * kThreads)
     return launch_clustered(ta_select_kernel<true, kSelectCluster>, units, kSelectCluster, stream, a.seq, a.n_layers,
                             a.Hkv, a.K, a.fast, src, a.forced, a.r_main, a.idx, a.count, gd, co);
-  if (a.seq.max_n <= kSelectCluster * kItemsLong * kThreads)
-    return launch_clustered(ta_select_kernel<true, kSelectCluster, kItemsLong>, units, kSelectCluster, stream, a.seq,
-                            a.n_layers, a.Hkv, a.K, a.fast, src, a.forced, a.r_main, a.idx, a.count, gd, co);
+  if (a.seq.max_n <= kSelectCluster * sel1024::kItems * sel1024::kThreads)  // as in ta_launch_forced
+    return launch_threads(sel1024::kThreads, sel1024::ta_select_kernel<true, kSelectCluster>, units, kSelectCluster,
+                          stream, a.seq, a.n_layers, a.Hkv, a.K, a.fast, src2, a.forced, a.r_main, a.idx, a.count, gd2,
+                          co);
+  if (a.seq.max_n <= kSelectCluster * sel1024::kItemsLong * sel1024::kThreads)
+    return launch_threads(sel1024::kThreads, sel1024::ta_select_kernel<true, kSelectCluster, sel1024::kItemsLong>,
+                          units, kSelectCluster, stream, a.seq, a.n_layers, a.Hkv, a.K, a.fast, src2, a.forced,
+                          a.r_main, a.idx, a.count, gd2, co);
   return launch_clustered(ta_select_kernel<false, kSelectCluster>, units, kSelectCluster, stream, a.seq, a.n_layers,
                           a.Hkv, a.K, a.fast, src, a.forced, a.r_main, a.idx, a.count, gd, co);
 }
