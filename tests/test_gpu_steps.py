@@ -373,6 +373,21 @@ def test_select_many_long_units_keys_in_registers_of_big_blocks(K):
     _select_case(w, oracle_policy(K, "THEOREM"), K, L, (A, P))
 
 
+@pytest.mark.parametrize("lengths", [[100000, 65537, 70], [200000, 131073], [262144]])
+def test_select_few_very_long_units_split_over_clusters_of_big_blocks(lengths):
+    # few units beyond 65536 tokens: each is split over a cluster of 8 blocks of 1024 threads (16 keys per thread up
+    # to 131072 tokens, 32 up to 262144); exact ties across the slices, slices that end inside the last block
+    K = 4096
+    w = _workload(lengths, [[5, 6, 7], [9]], seed=7 + len(lengths), Hq=2, Hkv=1)
+    gen = torch.Generator().manual_seed(len(lengths))
+    A = torch.rand((1, w.Hkv, w.total), generator=gen).cuda()
+    A = (A * 512).round() / 512
+    P = (torch.rand((1, w.Hkv, w.total), generator=gen) * 0.1).cuda()
+    P = (P * 256).round() / 256
+    _select_case(w, oracle_policy(K, "THEOREM"), K, 1, (A, P))
+    _select_case(w, oracle_policy(K, "THEOREM", fast=True), K)
+
+
 def test_select_sponsored_overflow_and_precedence():
     # far more sponsored tokens than protected slots: nearest-to-anchor first, earlier anchors win ties
     w = _workload([5000], [[1]], [12], alphabet=40, seed=4)
