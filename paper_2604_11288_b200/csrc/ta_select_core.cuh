@@ -27,14 +27,17 @@ struct SelectShared {
   uint32_t prefix, mask;
   int remaining;
   int done_all;
+  int ncand;  // elements in the digit bin the threshold fell into: the candidates of the next pass
   __align__(16) uint32_t warp_cnt[kWarps];  // per warp: definite count (low 16 bits) | tie count (high 16 bits)
+  // range of the eligible keys: per warp (smallest, largest, how many), and per CTA of a cluster
+  uint32_t wmin[kWarps], wmax[kWarps], wnum[kWarps];
+  uint32_t cl_range[8][4];
   // long sequences are split over the CTAs of a cluster: histogram of the whole unit (on rank 0, two buffers
   // alternating by pass) and every CTA's (definite, tie) totals
   uint32_t ghist[2][256];
   int totals[8][2];
-  // ordered write of a unit whose keys sit in registers: per (chunk of kThreads elements, warp) the counts of
-  // definite | tie elements (packed 16 | 16 bits, then their exclusive prefix) and the two ballots
-  uint32_t cnt[kItemsLong * kWarps];
+  // ordered write of a unit whose keys sit in registers: bitmaps of the definite and of the tie elements in position
+  // order (word e covers positions 32e .. 32e+31 of this CTA's slice)
   uint32_t bdef[kItemsLong * kWarps], btie[kItemsLong * kWarps];
   uint32_t wtot[kWarps];
   uint32_t total;
@@ -45,6 +48,7 @@ constexpr int kSelectCluster = 8;  // CTAs per unit when a sequence is longer th
 // re-read from L2 on every sweep in batches whose loads are all issued before the first use.
 constexpr int kItems = 16;
 constexpr int kBatch = 8;
+static_assert(kItems % 8 == 0 && kItemsLong % 8 == 0, "the cached load works in groups of 8 keys per thread");
 template <int ITEMS>
 struct KeyCache {
   uint32_t key[ITEMS];
@@ -196,6 +200,181 @@ __device__ SelectResult block_radix_select(int n, int want, KeyFn key_of, const 
   return r;
 }
 
+// Shared step of the radix passes: warp 0 walks the 256-bin histogram from the top bin down until `remaining`
+// elements are covered and publishes the bin it stops in (sh.prefix gets the digit at `shift`, sh.remaining what is
+// still to take inside that bin, sh.ncand the bin's population). Called by all threads of warp 0.
+__device__ __forceinline__ void radix_walk(const uint32_t* hist, int shift, uint32_t digit_mask, uint32_t prefix,
+                                           uint32_t mask, SelectShared& sh) {
+  const int lane = threadIdx.x & 31;
+  // lane l owns bins [8l, 8l+8)
+  uint32_t hl[8];
+#pragma unroll
+  for (int k = 0; k < 8; ++k) hl[k] = hist[8 * lane + k];
+  uint32_t tot = 0;
+#pragma unroll
+  for (int k = 0; k < 8; ++k) tot += hl[k];
+  uint32_t run = tot;  // inclusive sum over this lane and the lanes above it
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const uint32_t o = __shfl_down_sync(0xffffffffu, run, off);
+    if (lane + off < 32) run += o;
+  }
+  const uint32_t above = run - tot;
+  const uint32_t remaining = (uint32_t)sh.remaining;
+  if (above < remaining && remaining <= above + tot) {
+    uint32_t cum = above;
+    int k = 7;
+#pragma unroll
+    for (int kk = 7; kk > 0; --kk) {
+      if (k == kk && cum + hl[kk] < remaining) {
+        cum += hl[kk];
+        k = kk - 1;
+      }
+    }
+    uint32_t pop = hl[0];
+#pragma unroll
+    for (int kk = 1; kk < 8; ++kk)
+      if (k == kk) pop = hl[kk];
+    const int bin = 8 * lane + k;
+    sh.remaining = (int)(remaining - cum);
+    sh.ncand = (int)pop;
+    sh.prefix = prefix | ((uint32_t)bin << shift);
+    sh.mask = mask | (digit_mask << shift);
+  }
+}
+
+// Top-`want` of the eligible elements when the keys sit in registers. The eligible keys' range is taken first: the
+// bits above the highest bit in which two of them differ are common to all and need no pass, so the first 8-bit
+// digit already spreads the keys over the whole histogram (utilities of one unit span a few binades: the top byte of
+// a float alone would put most of them into two or three bins). The first pass counts every eligible element
+// (match.any merges equal digits of a warp into one shared-memory atomic); from then on each thread keeps a bit mask
+// of its elements that are still candidates, and the passes touch those only. The passes stop as soon as the
+// candidates left are exactly as many as are still to take. n_unit is the length of the whole unit (n is this CTA's
+// slice when CL > 1).
+template <int CL, int ITEMS>
+__device__ SelectResult cached_radix_select(int n, int n_unit, int want, const KeyCache<ITEMS>& kc, SelectShared& sh) {
+  SelectResult r;
+  r.thresh = 0;
+  r.ties = 0;
+  r.all = 0;
+  r.none = (want <= 0);
+  if (r.none) return r;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const unsigned lt = (1u << lane) - 1u;
+  uint32_t cand = kc.elig;
+  uint32_t kmin = 0xffffffffu, kmax = 0u;
+#pragma unroll
+  for (int it = 0; it < ITEMS; ++it) {
+    if ((cand >> it) & 1u) {
+      kmin = min(kmin, kc.key[it]);
+      kmax = max(kmax, kc.key[it]);
+    }
+  }
+  kmin = __reduce_min_sync(0xffffffffu, kmin);
+  kmax = __reduce_max_sync(0xffffffffu, kmax);
+  uint32_t num = __reduce_add_sync(0xffffffffu, (uint32_t)__popc(cand));
+  if (lane == 0) {
+    sh.wmin[warp] = kmin;
+    sh.wmax[warp] = kmax;
+    sh.wnum[warp] = num;
+  }
+  if (tid == 0) sh.remaining = want;
+  if (CL > 1) cg::this_cluster().sync();  // also: every CTA of the cluster runs before its shared memory is written
+  else __syncthreads();
+  static_assert(kWarps <= 32, "one lane per warp in the second reduction step");
+  kmin = __reduce_min_sync(0xffffffffu, lane < kWarps ? sh.wmin[lane] : 0xffffffffu);
+  kmax = __reduce_max_sync(0xffffffffu, lane < kWarps ? sh.wmax[lane] : 0u);
+  num = __reduce_add_sync(0xffffffffu, lane < kWarps ? sh.wnum[lane] : 0u);
+  uint32_t* ghist0 = nullptr;
+  if (CL > 1) {
+    cg::cluster_group cluster = cg::this_cluster();
+    const int rank = (int)cluster.block_rank();
+    ghist0 = cluster.map_shared_rank(&sh.ghist[0][0], 0);
+    if (tid < CL) {
+      uint32_t* peer = cluster.map_shared_rank(&sh.cl_range[0][0], tid);
+      peer[rank * 4 + 0] = kmin;
+      peer[rank * 4 + 1] = kmax;
+      peer[rank * 4 + 2] = num;
+    }
+    cluster.sync();
+    kmin = 0xffffffffu;
+    kmax = 0u;
+    num = 0u;
+#pragma unroll
+    for (int q = 0; q < CL; ++q) {
+      kmin = min(kmin, sh.cl_range[q][0]);
+      kmax = max(kmax, sh.cl_range[q][1]);
+      num += sh.cl_range[q][2];
+    }
+  }
+  if (num < (uint32_t)want) {  // fewer eligible elements than requested: all of them
+    r.all = 1;
+    return r;
+  }
+  const uint32_t diff = kmin ^ kmax;
+  if (diff == 0u) {  // all eligible keys are equal
+    r.thresh = kmin;
+    r.ties = want;
+    return r;
+  }
+  const int bits = 32 - __clz(diff);  // low bits still to resolve
+  uint32_t mask = bits == 32 ? 0u : (0xffffffffu << bits);
+  uint32_t prefix = kmax & mask;
+  int remaining = want;
+  int ncand = (int)num;
+  int done = 0, pass = 0;
+  while (done < bits) {
+    const int width = min(8, bits - done), shift = bits - done - width;
+    const uint32_t digit_mask = (1u << width) - 1u;
+    if (tid < 256) {
+      sh.hist[tid] = 0;
+      if (CL > 1) sh.ghist[pass & 1][tid] = 0;  // only rank 0's copy is used; its readers of two passes ago are done
+    }
+    if (CL > 1) cg::this_cluster().sync();
+    else __syncthreads();
+    if (pass == 0 || ncand * 4 > n_unit) {  // most elements are candidates (uniform over the unit's CTAs)
+#pragma unroll
+      for (int it = 0; it < ITEMS; ++it) {
+        if (it * kThreads < n) {
+          const bool c = ((cand >> it) & 1u) != 0 && (kc.key[it] & mask) == prefix;
+          if (!c) cand &= ~(1u << it);
+          const int bin = c ? (int)((kc.key[it] >> shift) & digit_mask) : -1;
+          const unsigned peers = __match_any_sync(0xffffffffu, bin);
+          if (c && (peers & lt) == 0u) atomicAdd(&sh.hist[bin], (uint32_t)__popc(peers));
+        }
+      }
+    } else if (cand != 0u) {
+#pragma unroll
+      for (int it = 0; it < ITEMS; ++it) {
+        if ((cand >> it) & 1u) {
+          if ((kc.key[it] & mask) != prefix) cand &= ~(1u << it);
+          else atomicAdd(&sh.hist[(kc.key[it] >> shift) & digit_mask], 1u);
+        }
+      }
+    }
+    __syncthreads();
+    const uint32_t* hist = sh.hist;
+    if (CL > 1) {  // merge the slices' histograms on rank 0, then every CTA takes the same decision from the sum
+      uint32_t* gh = ghist0 + (pass & 1) * 256;
+      if (tid < 256 && sh.hist[tid]) atomicAdd(&gh[tid], sh.hist[tid]);
+      cg::this_cluster().sync();
+      hist = gh;
+    }
+    if (tid < 32) radix_walk(hist, shift, digit_mask, prefix, mask, sh);
+    __syncthreads();
+    prefix = sh.prefix;
+    mask = sh.mask;
+    remaining = sh.remaining;
+    ncand = sh.ncand;
+    done += width;
+    ++pass;
+    if (ncand == remaining) break;  // every candidate left is taken: the low bits need no pass
+  }
+  r.thresh = prefix;  // with the unresolved low bits zero: candidates above it are definite, equal ones are ties
+  r.ties = remaining;
+  return r;
+}
+
 // Ordered pass over [0, n): classify(i, eligible, key, def, tie) marks element i `definite` (taken for sure) or a
 // `tie` (taken while ties last). Calls emit(i, rank) for every taken element with its rank in ascending position
 // order. Returns the number taken.
@@ -239,21 +418,19 @@ __device__ int block_ordered_emit(int n, int ties_allowed, KeyFn key_of, const K
   return def_base + min(tie_base, ties_allowed);
 }
 
-// The ordered pass for a unit split over CL CTAs (rank r owns a contiguous, ascending slice): a counting sweep
-// gives every CTA its (definite, tie) totals, the totals are exchanged through distributed shared memory, and the
-// emitting sweep starts from the sums of the lower ranks. Returns the number taken over the whole unit.
 // The ordered pass when the keys sit in registers (ITEMS chunks of kThreads elements, element tid + it*kThreads in
-// chunk it): one sweep classifies and records, per chunk and warp, the counts and ballots of definite and tie
-// elements; one block-wide exclusive scan over those (chunk-major = position order) gives every warp its base; a
-// second sweep emits. Three block barriers (and one cluster barrier for the totals of the lower ranks) instead of two
-// per chunk. classify is called exactly once per element.
+// chunk it). One sweep classifies every element and leaves two bitmaps in shared memory, definite and tie, in
+// position order: the ballot of warp w in chunk it is word it*kWarps + w and covers positions 32 * word .. + 31.
+// From there on thread j owns word j: a block-wide exclusive scan over the words' populations gives it the number
+// of definite and of tie elements before its 32 positions, and it writes its taken positions itself (two per word on
+// average) -- no key is needed for that. Three block barriers (and one cluster barrier for the totals of the lower
+// ranks). classify is called exactly once per element; emit may run on another thread than classify did.
 template <int CL, class ClassFn, class EmitFn, int ITEMS>
 __device__ int cached_ordered_emit(int n, int ties_allowed, const KeyCache<ITEMS>& kc, ClassFn classify, EmitFn emit,
                                    SelectShared& sh) {
   static_assert(ITEMS <= kItemsLong && ITEMS <= 32, "per-thread masks hold one bit per chunk");
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int chunks = (n + kThreads - 1) / kThreads;
-  uint32_t mdef = 0, mtie = 0;
 #pragma unroll
   for (int it = 0; it < ITEMS; ++it) {
     if (it < chunks) {
@@ -261,26 +438,26 @@ __device__ int cached_ordered_emit(int n, int ties_allowed, const KeyCache<ITEMS
       bool def = false, tie = false;
       if (i < n) classify(i, ((kc.elig >> it) & 1u) != 0, kc.key[it], def, tie);
       const unsigned bd = __ballot_sync(0xffffffffu, def), bt = __ballot_sync(0xffffffffu, tie);
-      if (def) mdef |= 1u << it;
-      if (tie) mtie |= 1u << it;
       if (lane == 0) {
-        sh.cnt[it * kWarps + warp] = (uint32_t)__popc(bd) | ((uint32_t)__popc(bt) << 16);
         sh.bdef[it * kWarps + warp] = bd;
         sh.btie[it * kWarps + warp] = bt;
       }
     }
   }
   __syncthreads();
-  // exclusive scan of the packed counts over the chunks * kWarps entries (entry tid belongs to thread tid)
-  static_assert(kItemsLong * kWarps <= kThreads, "one scan entry per thread");
-  const uint32_t mine = tid < chunks * kWarps ? sh.cnt[tid] : 0u;
+  // exclusive scan of the packed populations over the chunks * kWarps words (word tid belongs to thread tid)
+  static_assert(kItemsLong * kWarps <= kThreads, "one word per thread");
+  const bool owner = tid < chunks * kWarps;
+  const uint32_t wd = owner ? sh.bdef[tid] : 0u, wt = owner ? sh.btie[tid] : 0u;
+  const uint32_t mine = (uint32_t)__popc(wd) | ((uint32_t)__popc(wt) << 16);
   uint32_t run = mine;
 #pragma unroll
   for (int off = 1; off < 32; off <<= 1) {
     const uint32_t o = __shfl_up_sync(0xffffffffu, run, off);
     if (lane >= off) run += o;
   }
-  if (lane == 31) sh.wtot[warp] = run;
+  const uint32_t warp_total = __shfl_sync(0xffffffffu, run, 31);
+  if (lane == 0) sh.wtot[warp] = warp_total;
   __syncthreads();
   uint32_t before = 0, all = 0;
 #pragma unroll
@@ -289,7 +466,7 @@ __device__ int cached_ordered_emit(int n, int ties_allowed, const KeyCache<ITEMS
     if (w < warp) before += t;
     all += t;
   }
-  if (tid < chunks * kWarps) sh.cnt[tid] = before + run - mine;
+  const uint32_t ex = before + run - mine;
   int def_base = 0, tie_base = 0;
   int def_all = (int)(all & 0xffffu), tie_all = (int)(all >> 16);
   if (CL > 1) {
@@ -312,25 +489,28 @@ __device__ int cached_ordered_emit(int n, int ties_allowed, const KeyCache<ITEMS
       def_all += sh.totals[r][0];
       tie_all += sh.totals[r][1];
     }
-  } else {
-    __syncthreads();
   }
-  const unsigned lt = (1u << lane) - 1u;
-#pragma unroll
-  for (int it = 0; it < ITEMS; ++it) {
-    if (it < chunks) {
-      const int e = it * kWarps + warp;
-      const uint32_t ex = sh.cnt[e];
-      const int def_before = def_base + (int)(ex & 0xffffu) + __popc(sh.bdef[e] & lt);
-      const int ties_seen = tie_base + (int)(ex >> 16) + __popc(sh.btie[e] & lt);
-      const int i = tid + it * kThreads;
-      if ((mdef >> it) & 1u) emit(i, def_before + min(ties_seen, ties_allowed));
-      else if (((mtie >> it) & 1u) && ties_seen < ties_allowed) emit(i, def_before + ties_seen);
+  int def_before = def_base + (int)(ex & 0xffffu);
+  int ties_seen = tie_base + (int)(ex >> 16);
+  uint32_t m = wd | wt;
+  while (m) {
+    const int bit = __ffs((int)m) - 1;
+    m &= m - 1u;
+    const int i = 32 * tid + bit;
+    if ((wd >> bit) & 1u) {
+      emit(i, def_before + min(ties_seen, ties_allowed));
+      ++def_before;
+    } else {
+      if (ties_seen < ties_allowed) emit(i, def_before + ties_seen);
+      ++ties_seen;
     }
   }
   return def_all + min(tie_all, ties_allowed);
 }
 
+// The ordered pass for a unit split over CL CTAs (rank r owns a contiguous, ascending slice): a counting sweep
+// gives every CTA its (definite, tie) totals, the totals are exchanged through distributed shared memory, and the
+// emitting sweep starts from the sums of the lower ranks. Returns the number taken over the whole unit.
 template <bool CACHED, int CL, class KeyFn, class ClassFn, class EmitFn, int ITEMS>
 __device__ int cluster_ordered_emit(int n, int ties_allowed, KeyFn key_of, const KeyCache<ITEMS>& kc, ClassFn classify,
                                     EmitFn emit, SelectShared& sh) {
@@ -401,7 +581,7 @@ __device__ __forceinline__ SeqInfo seq_info(const ta_seq_desc& seq, int b, int K
 }
 
 template <bool CACHED, int CL, int ITEMS = kItems>
-__global__ void __launch_bounds__(kThreads) ta_forced_kernel(ta_seq_desc seq, int K, int n_sink, int n_recent,
+__global__ void __launch_bounds__(kThreads, 1024 / kThreads) ta_forced_kernel(ta_seq_desc seq, int K, int n_sink, int n_recent,
                                                              int k_protected, const float* __restrict__ voucher,
                                                              uint8_t* __restrict__ forced,
                                                              int32_t* __restrict__ r_main, ta_dev_status* status,
@@ -442,14 +622,16 @@ __global__ void __launch_bounds__(kThreads) ta_forced_kernel(ta_seq_desc seq, in
   };
   KeyCache<ITEMS> kc;
   if (CACHED) fill_cache(hi - lo, key_of, kc);
-  const SelectResult r = block_radix_select<CACHED, CL>(hi - lo, s.p, key_of, kc, sh);
+  SelectResult r;
+  if constexpr (CACHED) r = cached_radix_select<CL>(hi - lo, s.n, s.p, kc, sh);
+  else r = block_radix_select<CACHED, CL>(hi - lo, s.p, key_of, kc, sh);
   uint8_t* f = forced + s.start + lo;
   // ordered pass: mandatory tokens and vouchers above the threshold are forced for sure; vouchers equal to the
   // threshold are forced while protected slots last, lowest position first
   auto classify = [&](int il, bool cand, uint32_t key, bool& def, bool& tie) {
     def = mandatory(lo + il) || (cand && !r.none && (r.all || key > r.thresh));
     tie = !def && cand && !r.none && !r.all && key == r.thresh;
-    f[il] = 0;  // set by emit when taken (same thread, later)
+    f[il] = 0;  // set by emit when taken (later, after a block barrier; possibly by another thread)
   };
   auto emit = [&](int il, int rank) { f[il] = 1; };
   const int taken = cluster_ordered_emit<CACHED, CL>(hi - lo, r.ties, key_of, kc, classify, emit, sh);
@@ -506,7 +688,7 @@ __device__ __forceinline__ void gather_unit(const GatherDst& gd, const ta_seq_de
 
 // grid.x = units. scored: unit = (l*B + b)*Hkv + g; fast: unit = b.
 template <bool CACHED, int CL, int ITEMS = kItems, bool GATHER = false>
-__global__ void __launch_bounds__(kThreads) ta_select_kernel(ta_seq_desc seq, int n_layers, int Hkv, int K, int fast,
+__global__ void __launch_bounds__(kThreads, 1024 / kThreads) ta_select_kernel(ta_seq_desc seq, int n_layers, int Hkv, int K, int fast,
                                                              UnitSrc src, const uint8_t* __restrict__ forced,
                                                              const int32_t* __restrict__ r_main,
                                                              int32_t* __restrict__ idx, int32_t* __restrict__ count,
@@ -557,8 +739,48 @@ __global__ void __launch_bounds__(kThreads) ta_select_kernel(ta_seq_desc seq, in
     return f[il] == 0;
   };
   KeyCache<ITEMS> kc;
-  if (CACHED) fill_cache(hi - lo, key_of, kc);
-  const SelectResult r = block_radix_select<CACHED, CL>(hi - lo, want, key_of, kc, sh);
+  if constexpr (CACHED) {
+    if (src.u) {
+      // the attention part comes from HBM, the per-token arrays mostly from L2: issue all loads of the former first
+      // (they land in the registers that hold the keys afterwards), so one memory latency covers the whole unit
+      const int nl = hi - lo;
+      const float* up = src.u + unit_off + start + lo;
+      const float* sp = src.u_static + start + lo;
+      kc.elig = 0;
+      // loads as selects, never under a branch: nothing then keeps them from being in flight together
+      float uu[ITEMS];
+#pragma unroll
+      for (int it = 0; it < ITEMS; ++it) {
+        const int i = tid + it * kThreads;
+        uu[it] = i < nl ? up[i] : 0.0f;
+      }
+      // the per-token values in groups of 8 (registers: a group's loads are in flight together, no more)
+#pragma unroll
+      for (int g0 = 0; g0 < ITEMS; g0 += 8) {
+        float us[8];
+        uint8_t ff[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+          const int i = tid + (g0 + q) * kThreads;
+          us[q] = i < nl ? sp[i] : 0.0f;
+          ff[q] = i < nl ? f[i] : (uint8_t)1;
+        }
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+          const int it = g0 + q;
+          const bool in = tid + it * kThreads < nl;
+          kc.key[it] = in ? sortable_key(__fadd_rn(uu[it], us[q])) : 0u;
+          kc.elig |= (in && ff[q] == 0) ? (1u << it) : 0u;
+        }
+        asm volatile("" ::: "memory");  // keeps the next group's loads behind this group's use
+      }
+    } else {
+      fill_cache(hi - lo, key_of, kc);
+    }
+  }
+  SelectResult r;
+  if constexpr (CACHED) r = cached_radix_select<CL>(hi - lo, n, want, kc, sh);
+  else r = block_radix_select<CACHED, CL>(hi - lo, want, key_of, kc, sh);
   auto classify = [&](int, bool elig, uint32_t key, bool& def, bool& tie) {
     def = !elig || (!r.none && (r.all || key > r.thresh));
     tie = !def && !r.none && !r.all && key == r.thresh;
