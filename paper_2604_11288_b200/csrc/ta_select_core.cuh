@@ -22,6 +22,8 @@ struct SelectResult {
   int none;         // 1: nothing is taken
 };
 
+constexpr int kCandCap = 2048;  // candidates a split unit finishes locally
+
 struct SelectShared {
   uint32_t hist[256];
   uint32_t prefix, mask;
@@ -41,6 +43,10 @@ struct SelectShared {
   uint32_t bdef[kItemsLong * kWarps], btie[kItemsLong * kWarps];
   uint32_t wtot[kWarps];
   uint32_t total;
+  // a unit split over a cluster: once few candidates are left, their keys are collected (on rank 0, then copied by
+  // every CTA) and the remaining passes run on that list inside each CTA, without cluster barriers
+  uint32_t cand_n;
+  uint32_t cand_keys[kCandCap];
 };
 constexpr int kSelectCluster = 8;  // CTAs per unit when a sequence is longer than kItems * kThreads
 
@@ -200,6 +206,21 @@ __device__ SelectResult block_radix_select(int n, int want, KeyFn key_of, const 
   return r;
 }
 
+// A unit split over a cluster, keys in registers: clears the state that peers will add to and arrives at the
+// cluster barrier whose wait opens cached_radix_select(); the loads of the keys run in between.
+template <int CL>
+__device__ __forceinline__ void split_unit_begin(SelectShared& sh) {
+  if (CL > 1) {
+    const int tid = threadIdx.x;
+    if (tid < 256) {
+      sh.ghist[0][tid] = 0;
+      sh.ghist[1][tid] = 0;
+    }
+    if (tid == 0) sh.cand_n = 0;
+    cg::this_cluster().barrier_arrive();
+  }
+}
+
 // Shared step of the radix passes: warp 0 walks the 256-bin histogram from the top bin down until `remaining`
 // elements are covered and publishes the bin it stops in (sh.prefix gets the digit at `shift`, sh.remaining what is
 // still to take inside that bin, sh.ncand the bin's population). Called by all threads of warp 0.
@@ -243,6 +264,45 @@ __device__ __forceinline__ void radix_walk(const uint32_t* hist, int shift, uint
   }
 }
 
+// The remaining radix passes over the m candidate keys in sh.cand_keys (all of them match `prefix` under `mask`),
+// with block barriers only. On return prefix/remaining describe the threshold as at the end of the register passes.
+__device__ __forceinline__ void list_radix_finish(int m, int bits, int done, uint32_t& prefix, uint32_t& mask,
+                                                  int& remaining, SelectShared& sh) {
+  const int tid = threadIdx.x;
+  constexpr int kPer = (kCandCap + kThreads - 1) / kThreads;
+  uint32_t lk[kPer];
+  uint32_t live = 0;
+#pragma unroll
+  for (int q = 0; q < kPer; ++q) {
+    const int j = tid + q * kThreads;
+    lk[q] = j < m ? sh.cand_keys[j] : 0u;
+    if (j < m) live |= 1u << q;
+  }
+  if (tid == 0) sh.remaining = remaining;
+  while (done < bits) {
+    const int width = min(8, bits - done), shift = bits - done - width;
+    const uint32_t digit_mask = (1u << width) - 1u;
+    if (tid < 256) sh.hist[tid] = 0;
+    __syncthreads();
+#pragma unroll
+    for (int q = 0; q < kPer; ++q) {
+      if ((live >> q) & 1u) {
+        if ((lk[q] & mask) != prefix) live &= ~(1u << q);
+        else atomicAdd(&sh.hist[(lk[q] >> shift) & digit_mask], 1u);
+      }
+    }
+    __syncthreads();
+    if (tid < 32) radix_walk(sh.hist, shift, digit_mask, prefix, mask, sh);
+    __syncthreads();
+    prefix = sh.prefix;
+    mask = sh.mask;
+    remaining = sh.remaining;
+    const int ncand = sh.ncand;
+    done += width;
+    if (ncand == remaining) break;
+  }
+}
+
 // Top-`want` of the eligible elements when the keys sit in registers. The eligible keys' range is taken first: the
 // bits above the highest bit in which two of them differ are common to all and need no pass, so the first 8-bit
 // digit already spreads the keys over the whole histogram (utilities of one unit span a few binades: the top byte of
@@ -258,6 +318,9 @@ __device__ SelectResult cached_radix_select(int n, int n_unit, int want, const K
   r.ties = 0;
   r.all = 0;
   r.none = (want <= 0);
+  // the cluster barrier that split_unit_begin() arrived at before the keys were loaded: from here on every CTA of the
+  // cluster is known to run (its shared memory may be written) and to have zeroed its ghist and cand_n
+  if (CL > 1) cg::this_cluster().barrier_wait();
   if (r.none) return r;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const unsigned lt = (1u << lane) - 1u;
@@ -279,8 +342,7 @@ __device__ SelectResult cached_radix_select(int n, int n_unit, int want, const K
     sh.wnum[warp] = num;
   }
   if (tid == 0) sh.remaining = want;
-  if (CL > 1) cg::this_cluster().sync();  // also: every CTA of the cluster runs before its shared memory is written
-  else __syncthreads();
+  __syncthreads();
   static_assert(kWarps <= 32, "one lane per warp in the second reduction step");
   kmin = __reduce_min_sync(0xffffffffu, lane < kWarps ? sh.wmin[lane] : 0xffffffffu);
   kmax = __reduce_max_sync(0xffffffffu, lane < kWarps ? sh.wmax[lane] : 0u);
@@ -324,14 +386,60 @@ __device__ SelectResult cached_radix_select(int n, int n_unit, int want, const K
   int ncand = (int)num;
   int done = 0, pass = 0;
   while (done < bits) {
+    if (CL > 1 && ncand <= kCandCap) {
+      // Few candidates left (uniform over the cluster: ncand comes from the merged histogram, or is the number of
+      // eligible elements before the first pass). Every CTA appends its own to the list on rank 0; after one cluster
+      // barrier every CTA copies the list and finishes alone. The list's order does not matter: only the multiset of
+      // keys decides the threshold, so all CTAs arrive at the same one.
+      cg::cluster_group cluster = cg::this_cluster();
+      uint32_t* list0 = cluster.map_shared_rank(&sh.cand_keys[0], 0);
+      uint32_t* count0 = cluster.map_shared_rank(&sh.cand_n, 0);
+      uint32_t mine = 0;
+      if (cand != 0u) {
+#pragma unroll
+        for (int it = 0; it < ITEMS; ++it)
+          if (((cand >> it) & 1u) && (kc.key[it] & mask) == prefix) mine |= 1u << it;
+      }
+      // one remote atomic per warp reserves the warp's range of the list
+      const uint32_t cnt = (uint32_t)__popc(mine);
+      uint32_t incl = cnt;
+#pragma unroll
+      for (int off = 1; off < 32; off <<= 1) {
+        const uint32_t o = __shfl_up_sync(0xffffffffu, incl, off);
+        if (lane >= off) incl += o;
+      }
+      const uint32_t warp_n = __shfl_sync(0xffffffffu, incl, 31);
+      uint32_t base = 0;
+      if (lane == 0 && warp_n != 0u) base = atomicAdd(count0, warp_n);
+      base = __shfl_sync(0xffffffffu, base, 0);
+      uint32_t slot = base + incl - cnt;
+      if (mine != 0u) {
+#pragma unroll
+        for (int it = 0; it < ITEMS; ++it) {
+          if ((mine >> it) & 1u) {
+            if (slot < (uint32_t)kCandCap) list0[slot] = kc.key[it];
+            ++slot;
+          }
+        }
+      }
+      cluster.sync();
+      if (cluster.block_rank() != 0)
+        for (int j = tid; j < ncand; j += kThreads) sh.cand_keys[j] = list0[j];
+      __syncthreads();
+      list_radix_finish(ncand, bits, done, prefix, mask, remaining, sh);
+      break;
+    }
     const int width = min(8, bits - done), shift = bits - done - width;
     const uint32_t digit_mask = (1u << width) - 1u;
-    if (tid < 256) {
-      sh.hist[tid] = 0;
-      if (CL > 1) sh.ghist[pass & 1][tid] = 0;  // only rank 0's copy is used; its readers of two passes ago are done
+    if (tid < 256) sh.hist[tid] = 0;
+    if (CL > 1 && pass >= 2) {
+      // rank 0's merged histogram alternates between two buffers, both zero at the start; from the third pass on the
+      // buffer is cleared again (its readers of two passes ago are done) and the clearing made visible
+      if (tid < 256) sh.ghist[pass & 1][tid] = 0;
+      cg::this_cluster().sync();
+    } else {
+      __syncthreads();
     }
-    if (CL > 1) cg::this_cluster().sync();
-    else __syncthreads();
     if (pass == 0 || ncand * 4 > n_unit) {  // most elements are candidates (uniform over the unit's CTAs)
 #pragma unroll
       for (int it = 0; it < ITEMS; ++it) {
@@ -621,6 +729,7 @@ __global__ void __launch_bounds__(kThreads, 1024 / kThreads) ta_forced_kernel(ta
     return v > 0.0f && !mandatory(lo + il);
   };
   KeyCache<ITEMS> kc;
+  if constexpr (CACHED) split_unit_begin<CL>(sh);
   if (CACHED) fill_cache(hi - lo, key_of, kc);
   SelectResult r;
   if constexpr (CACHED) r = cached_radix_select<CL>(hi - lo, s.n, s.p, kc, sh);
@@ -740,6 +849,7 @@ __global__ void __launch_bounds__(kThreads, 1024 / kThreads) ta_select_kernel(ta
   };
   KeyCache<ITEMS> kc;
   if constexpr (CACHED) {
+    split_unit_begin<CL>(sh);
     if (src.u) {
       // the attention part comes from HBM, the per-token arrays mostly from L2: issue all loads of the former first
       // (they land in the registers that hold the keys afterwards), so one memory latency covers the whole unit
