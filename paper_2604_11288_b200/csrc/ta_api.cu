@@ -719,6 +719,14 @@ ta_status compress_impl(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* p
   sel.flags = flags;
   sel.voucher = voucher;
   sel.u_static = u_static;
+  // the forced-set kernel writes the static utilities of its sequence (one kernel less on the per-sequence chain)
+  sel.static_out = u_static;
+  sel.static_ids = token_ids;
+  sel.static_hist = hist;
+  sel.static_vocab = policy->vocab_size;
+  sel.beta = policy->beta;
+  sel.gamma = policy->gamma;
+  sel.lambda = policy->lambda;
   sel.u = external ? nullptr : u;
   sel.A = ext_A;
   sel.P = ext_P;
@@ -771,9 +779,9 @@ ta_status compress_impl(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* p
   if (!reuse) {
     if (timing && e == cudaSuccess) e = cudaEventRecord(ctx->ev[5], seq_stream);
     if (e == cudaSuccess)
-      e = ta_launch_mask(pats, *policy, seq, token_ids, flags, voucher, u_static, hist, ctx->d_status, seq_stream);
+      e = ta_launch_mask(pats, *policy, seq, token_ids, flags, voucher, nullptr, hist, ctx->d_status, seq_stream);
     if (e == cudaSuccess) e = ta_launch_forced(sel, ctx->d_status, seq_stream);
-    launches += 3;  // mask, static utility, forced set
+    launches += 2;  // mask, forced set (which also writes the static utilities)
     if (timing && e == cudaSuccess) {
       e = cudaEventRecord(ctx->ev[6], seq_stream);
       ctx->ev_ran[0] = 1;

@@ -76,7 +76,22 @@ __host__ __device__ inline int ta_seq_begin(const ta_seq_desc& s, int b, const i
   return s.cu ? s.cu[b] : b * s.n_uniform;
 }
 
+#ifdef __CUDACC__
+// Static part of a token's utility (Eq. 3): u_static = ((beta*R + gamma*S) - lambda*F) + V with R = (i0+1)/n,
+// S = 1 on anchor tokens, F = count(id)/n; one rounding per operation. i0 is the 0-based position in the sequence.
+__device__ __forceinline__ float ta_static_utility(int i0, int n, int count, bool anchor_token, float V, float beta,
+                                                   float gamma, float lambda) {
+  const float R = __fdiv_rn((float)(i0 + 1), (float)n);
+  const float S = anchor_token ? 1.0f : 0.0f;
+  const float F = __fdiv_rn((float)count, (float)n);
+  const float t0 = __fadd_rn(__fmul_rn(beta, R), __fmul_rn(gamma, S));
+  const float t1 = __fsub_rn(t0, __fmul_rn(lambda, F));
+  return __fadd_rn(t1, V);
+}
+#endif
+
 // ---- step 1 ------------------------------------------------------------------------------------------------
+// u_static may be null: the caller then has ta_launch_forced compute it (ta_select_args::static_out).
 cudaError_t ta_launch_mask(const ta_patterns* pats, const ta_policy& pol, const ta_seq_desc& seq, const int32_t* ids,
                            uint8_t* flags, float* voucher, float* u_static, int32_t* hist /*[B][vocab]*/,
                            ta_dev_status* status, cudaStream_t stream);
@@ -112,6 +127,15 @@ cudaError_t ta_launch_wait_selftest(ta_dev_status* status, unsigned long long li
                                     cudaStream_t stream);
 
 // ---- step 3 ------------------------------------------------------------------------------------------------
+struct ta_static_out {  // what ta_forced_kernel needs to write the static utilities of its sequence (out null: off)
+  float* out;
+  const int32_t* ids;
+  const uint8_t* flags;
+  const int32_t* hist;
+  int vocab;
+  float beta, gamma, lambda;
+};
+
 struct ta_select_args {
   ta_seq_desc seq;
   int n_layers, Hkv, K;
@@ -139,6 +163,13 @@ struct ta_select_args {
   ta_bf16_view gather_k, gather_v;
   void* gather_k_out;  // null: no gather
   void* gather_v_out;
+  // optional: ta_launch_forced also writes the static utilities (what ta_launch_mask does when it is given the
+  // array), saving a kernel on the per-sequence chain. static_out null: not asked for.
+  float* static_out;
+  const int32_t* static_ids;
+  const int32_t* static_hist;  // [B][vocab] token counts per sequence
+  int static_vocab;
+  float beta, gamma, lambda;
 };
 bool ta_select_gathers(const ta_select_args& a);  // whether ta_launch_select_units will do the gather itself
 cudaError_t ta_launch_select(const ta_select_args& a, ta_dev_status* status, cudaStream_t stream);  // both below

@@ -305,12 +305,8 @@ __global__ void __launch_bounds__(256) ta_ustatic_kernel(ta_seq_desc seq, const 
   const int n = (seq.cu ? seq.cu[b + 1] : start + seq.n_uniform) - start;
   const int id = ids[tok];
   const int c = (id >= 0 && id < vocab) ? hist[(long long)b * vocab + id] : 0;
-  const float R = __fdiv_rn((float)((int)(tok - start) + 1), (float)n);
-  const float S = (flags[tok] & TA_FLAG_ANCHOR_TOKEN) ? 1.0f : 0.0f;
-  const float F = __fdiv_rn((float)c, (float)n);
-  const float t0 = __fadd_rn(__fmul_rn(beta, R), __fmul_rn(gamma, S));
-  const float t1 = __fsub_rn(t0, __fmul_rn(lambda, F));
-  u_static[tok] = __fadd_rn(t1, voucher[tok]);
+  u_static[tok] = ta_static_utility((int)(tok - start), n, c, (flags[tok] & TA_FLAG_ANCHOR_TOKEN) != 0, voucher[tok],
+                                    beta, gamma, lambda);
 }
 
 }  // namespace
@@ -318,6 +314,7 @@ __global__ void __launch_bounds__(256) ta_ustatic_kernel(ta_seq_desc seq, const 
 namespace {
 cudaError_t finish_static_utility(const ta_policy& pol, const ta_seq_desc& seq, const int32_t* ids, const uint8_t* flags,
                                   const float* voucher, const int32_t* hist, float* u_static, cudaStream_t stream) {
+  if (!u_static) return cudaSuccess;  // left to the forced-set kernel
   const int blocks = (int)((seq.total + 255) / 256);
   ta_ustatic_kernel<<<blocks, 256, 0, stream>>>(seq, ids, flags, voucher, hist, pol.vocab_size, pol.beta, pol.gamma,
                                                 pol.lambda, u_static);

@@ -127,30 +127,39 @@ cudaError_t ta_launch_forced(const ta_select_args& a, ta_dev_status* status, cud
   const int B = a.seq.batch * (a.n_classes > 0 ? a.n_classes : 1);  // blocks: (class, sequence)
   const int32_t* ck = a.n_classes > 0 ? a.class_K : nullptr;
   const int sms = sm_count_of(a);
+  ta_static_out so = {};
+  so.out = a.static_out;
+  so.ids = a.static_ids;
+  so.flags = a.flags;
+  so.hist = a.static_hist;
+  so.vocab = a.static_vocab;
+  so.beta = a.beta;
+  so.gamma = a.gamma;
+  so.lambda = a.lambda;
   if (a.seq.max_n <= kItems * kThreads)
     return launch_clustered(ta_forced_kernel<true, 1>, B, 1, stream, a.seq, a.K, a.n_sink, a.n_recent, a.k_protected,
-                            a.voucher, a.forced, a.r_main, status, ck);
+                            a.voucher, a.forced, a.r_main, status, ck, so);
   if (!split_units(B, a.seq.max_n, sms) && a.seq.max_n <= kItemsLong * kThreads)
     return launch_clustered(ta_forced_kernel<true, 1, kItemsLong>, B, 1, stream, a.seq, a.K, a.n_sink, a.n_recent,
-                            a.k_protected, a.voucher, a.forced, a.r_main, status, ck);
+                            a.k_protected, a.voucher, a.forced, a.r_main, status, ck, so);
   if (!split_units(B, a.seq.max_n, sms))
     return launch_clustered(ta_forced_kernel<false, 1>, B, 1, stream, a.seq, a.K, a.n_sink, a.n_recent, a.k_protected,
-                            a.voucher, a.forced, a.r_main, status, ck);
+                            a.voucher, a.forced, a.r_main, status, ck, so);
   if (a.seq.max_n <= kSelectCluster * kItems * kThreads)
     return launch_clustered(ta_forced_kernel<true, kSelectCluster>, B, kSelectCluster, stream, a.seq, a.K, a.n_sink,
-                            a.n_recent, a.k_protected, a.voucher, a.forced, a.r_main, status, ck);
+                            a.n_recent, a.k_protected, a.voucher, a.forced, a.r_main, status, ck, so);
   // few very long sequences: the chain of per-thread sweeps and cluster barriers sets the time, so blocks of 1024
   // threads (half the keys per thread) roughly halve it
   if (a.seq.max_n <= kSelectCluster * sel1024::kItems * sel1024::kThreads)
     return launch_threads(sel1024::kThreads, sel1024::ta_forced_kernel<true, kSelectCluster>, B, kSelectCluster,
                           stream, a.seq, a.K, a.n_sink, a.n_recent, a.k_protected, a.voucher, a.forced, a.r_main,
-                          status, ck);
+                          status, ck, so);
   if (a.seq.max_n <= kSelectCluster * sel1024::kItemsLong * sel1024::kThreads)
     return launch_threads(sel1024::kThreads, sel1024::ta_forced_kernel<true, kSelectCluster, sel1024::kItemsLong>, B,
                           kSelectCluster, stream, a.seq, a.K, a.n_sink, a.n_recent, a.k_protected, a.voucher,
-                          a.forced, a.r_main, status, ck);
+                          a.forced, a.r_main, status, ck, so);
   return launch_clustered(ta_forced_kernel<false, kSelectCluster>, B, kSelectCluster, stream, a.seq, a.K, a.n_sink,
-                          a.n_recent, a.k_protected, a.voucher, a.forced, a.r_main, status, ck);
+                          a.n_recent, a.k_protected, a.voucher, a.forced, a.r_main, status, ck, so);
 }
 
 bool ta_select_gathers(const ta_select_args& a) {

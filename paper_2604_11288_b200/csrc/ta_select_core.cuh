@@ -693,17 +693,44 @@ __global__ void __launch_bounds__(kThreads, 1024 / kThreads) ta_forced_kernel(ta
                                                              int k_protected, const float* __restrict__ voucher,
                                                              uint8_t* __restrict__ forced,
                                                              int32_t* __restrict__ r_main, ta_dev_status* status,
-                                                             const int32_t* __restrict__ class_K) {
+                                                             const int32_t* __restrict__ class_K, ta_static_out so) {
   __shared__ SelectShared sh;
   // grid.x = classes * sequences * CL; without budget classes there is one class and K is the argument
   const int b = (blockIdx.x / CL) % seq.batch;
+  const int cls = (blockIdx.x / CL) / seq.batch;
   if (class_K) {
-    const int cls = (blockIdx.x / CL) / seq.batch;
     K = class_K[cls];
     forced += (long long)cls * seq.total;
     r_main += cls * seq.batch;
   }
   const SeqInfo s = seq_info(seq, b, K, n_sink, n_recent, k_protected);
+  if (so.out && cls == 0) {  // the static utilities of this CTA's slice (a rejected sequence has s.n == 0)
+    int slo, shi;
+    unit_slice<CL>(s.n, slo, shi);
+    // eight tokens per thread and step: their loads (id, then count of that id, flags, voucher) are in flight together
+    for (int i0 = slo + (int)threadIdx.x; i0 < shi; i0 += 8 * kThreads) {
+      int id[8], c[8];
+      uint8_t fl[8];
+      float V[8];
+#pragma unroll
+      for (int q = 0; q < 8; ++q) {
+        const int i = i0 + q * kThreads;
+        const long long tok = (long long)s.start + i;
+        id[q] = i < shi ? so.ids[tok] : -1;
+        fl[q] = i < shi ? so.flags[tok] : (uint8_t)0;
+        V[q] = i < shi ? voucher[tok] : 0.0f;
+      }
+#pragma unroll
+      for (int q = 0; q < 8; ++q) c[q] = (id[q] >= 0 && id[q] < so.vocab) ? so.hist[(long long)b * so.vocab + id[q]] : 0;
+#pragma unroll
+      for (int q = 0; q < 8; ++q) {
+        const int i = i0 + q * kThreads;
+        if (i < shi)
+          so.out[(long long)s.start + i] = ta_static_utility(i, s.n, c[q], (fl[q] & TA_FLAG_ANCHOR_TOKEN) != 0, V[q],
+                                                             so.beta, so.gamma, so.lambda);
+      }
+    }
+  }
   if (s.bad) {
     if (threadIdx.x == 0) {
       if (atomicCAS(&status->code, 0, (int)TA_ERR_DEVICE_BOUNDS) == 0) {
