@@ -1,12 +1,14 @@
 // Step 3 of the retention path: budget-K selection with the partition of Section 3.3 (Algorithm 1 step 8).
 //
-// The retained set is reported in ascending position order, so no sort of the winners is needed: a 4-pass 8-bit
-// radix select finds the threshold key (and how many tokens that tie with it still fit), and one ordered
+// The retained set is reported in ascending position order, so no sort of the winners is needed: a radix select
+// over the order-preserving integer image of the values (8-bit digits, starting below the bits that all keys of the
+// unit share) finds the threshold key and how many tokens that tie with it still fit, and one ordered
 // stream-compaction pass writes the indices. Order is total and deterministic: larger value first, lower
 // position first among equal values.
 //
 //   ta_forced_kernel   one block per sequence: mandatory sinks/recents and the protected pool (largest vouchers
-//                      among sponsored tokens). Independent of layer and head, so it runs once per sequence.
+//                      among sponsored tokens). Independent of layer and head, so it runs once per sequence; on
+//                      request it also writes the sequence's static utilities (Eq. 3).
 //   ta_select_kernel   one block per unit (layer, sequence, KV head) in scored mode, per sequence in fast mode:
 //                      main pool by utility among the tokens not forced, then the ordered write of
 //                      forced + chosen positions.
