@@ -388,6 +388,19 @@ def test_select_few_very_long_units_split_over_clusters_of_big_blocks(lengths):
     _select_case(w, oracle_policy(K, "THEOREM", fast=True), K)
 
 
+@pytest.mark.parametrize("lengths,L", [([200000], 1), ([32768, 20000, 9000, 700], 6)])
+def test_select_three_distinct_utilities_keep_every_pass_crowded(lengths, L):
+    # utilities that take three values only (no recency, anchor or frequency term): a third of the keys stays a
+    # candidate through every radix pass, so the passes over all keys, the passes of a split unit beyond the second
+    # and the tie rule (lowest position first) all run; one unit split over a cluster, and 48 units of one block each
+    K = 4096
+    w = _workload(lengths, [[5, 6, 7], [9]], seed=31 + L, Hq=4, Hkv=2)
+    gen = torch.Generator().manual_seed(L)
+    A = (torch.randint(1, 4, (L, w.Hkv, w.total), generator=gen).float() / 4).cuda()
+    P = torch.zeros((L, w.Hkv, w.total)).cuda()
+    _select_case(w, oracle_policy(K, "THEOREM", beta=0.0, gamma=0.0, lam=0.0), K, L, (A, P))
+
+
 def test_select_sponsored_overflow_and_precedence():
     # far more sponsored tokens than protected slots: nearest-to-anchor first, earlier anchors win ties
     w = _workload([5000], [[1]], [12], alphabet=40, seed=4)
