@@ -40,7 +40,8 @@ struct SelectShared {
   int totals[8][2];
   // ordered write of a unit whose keys sit in registers: bitmaps of the definite and of the tie elements in position
   // order (word e covers positions 32e .. 32e+31 of this CTA's slice)
-  uint32_t bdef[kItemsLong * kWarps], btie[kItemsLong * kWarps];
+  // (a row of kWarps words per chunk, padded by one word so that the 32 rows a warp writes fall into 32 banks)
+  uint32_t bdef[kItemsLong * (kWarps + 1)], btie[kItemsLong * (kWarps + 1)];
   uint32_t wtot[kWarps];
   uint32_t total;
   // a unit split over a cluster: once few candidates are left, their keys are collected (on rank 0, then copied by
@@ -526,37 +527,73 @@ __device__ int block_ordered_emit(int n, int ties_allowed, KeyFn key_of, const K
   return def_base + min(tie_base, ties_allowed);
 }
 
+// Bit `it` set for every chunk in which this thread's slot (tid + it * kThreads) lies inside [0, n).
+__device__ __forceinline__ uint32_t exist_mask(int n) {
+  const int tid = threadIdx.x;
+  const int cnt = n > tid ? (n - tid + kThreads - 1) / kThreads : 0;
+  return cnt >= 32 ? 0xffffffffu : ((1u << cnt) - 1u);
+}
+
+// Transpose of a 32 x 32 bit matrix held one row per lane: on return lane i holds, in bit l, what was bit i of lane l.
+// Five butterfly steps, each swapping the off-diagonal blocks of size s with the lane s away.
+__device__ __forceinline__ uint32_t warp_transpose32(uint32_t x, int lane) {
+#pragma unroll
+  for (int s = 16; s >= 1; s >>= 1) {
+    const uint32_t m = s == 16 ? 0x0000ffffu : s == 8 ? 0x00ff00ffu : s == 4 ? 0x0f0f0f0fu : s == 2 ? 0x33333333u : 0x55555555u;
+    const uint32_t y = __shfl_xor_sync(0xffffffffu, x, s);
+    x = (lane & s) ? ((x & ~m) | ((y >> s) & m)) : ((x & m) | ((y << s) & ~m));
+  }
+  return x;
+}
+
 // The ordered pass when the keys sit in registers (ITEMS chunks of kThreads elements, element tid + it*kThreads in
-// chunk it). One sweep classifies every element and leaves two bitmaps in shared memory, definite and tie, in
-// position order: the ballot of warp w in chunk it is word it*kWarps + w and covers positions 32 * word .. + 31.
+// chunk it). One sweep classifies every element (each thread collects its own 32 bits, one in-warp bit transpose turns
+// them into what 32 ballots would give) and leaves two bitmaps in shared memory, definite and tie, in position
+// order: the bits of warp w in chunk it are word it*kWarps + w and cover positions 32 * word .. + 31.
 // From there on thread j owns word j: a block-wide exclusive scan over the words' populations gives it the number
 // of definite and of tie elements before its 32 positions, and it writes its taken positions itself (two per word on
 // average) -- no key is needed for that. Three block barriers (and one cluster barrier for the totals of the lower
-// ranks). classify is called exactly once per element; emit may run on another thread than classify did.
-template <int CL, class ClassFn, class EmitFn, int ITEMS>
-__device__ int cached_ordered_emit(int n, int ties_allowed, const KeyCache<ITEMS>& kc, ClassFn classify, EmitFn emit,
-                                   SelectShared& sh) {
+// ranks). emit may run on another thread than the one that holds the element's key.
+template <int CL, class EmitFn, int ITEMS>
+__device__ int cached_ordered_emit(int n, const SelectResult& r, const KeyCache<ITEMS>& kc, uint32_t always,
+                                   EmitFn emit, SelectShared& sh) {
   static_assert(ITEMS <= kItemsLong && ITEMS <= 32, "per-thread masks hold one bit per chunk");
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int chunks = (n + kThreads - 1) / kThreads;
+  // per thread: bit `it` of mdef / mtie = its element of chunk `it` is definite / a tie. `always` marks the elements
+  // taken whatever their key (not eligible for the search); eligible ones are definite above the threshold and ties
+  // at it. The elig bits exist only for elements inside the unit.
+  const int ties_allowed = r.ties;
+  uint32_t mdef = always, mtie = 0;
+  if (!r.none) {
+    if (r.all) {
+      mdef |= kc.elig;
+    } else {
+      uint32_t above = 0, equal = 0;
 #pragma unroll
-  for (int it = 0; it < ITEMS; ++it) {
-    if (it < chunks) {
-      const int i = tid + it * kThreads;
-      bool def = false, tie = false;
-      if (i < n) classify(i, ((kc.elig >> it) & 1u) != 0, kc.key[it], def, tie);
-      const unsigned bd = __ballot_sync(0xffffffffu, def), bt = __ballot_sync(0xffffffffu, tie);
-      if (lane == 0) {
-        sh.bdef[it * kWarps + warp] = bd;
-        sh.btie[it * kWarps + warp] = bt;
+      for (int it = 0; it < ITEMS; ++it) {
+        if (it < chunks) {
+          above |= kc.key[it] > r.thresh ? (1u << it) : 0u;
+          equal |= kc.key[it] == r.thresh ? (1u << it) : 0u;
+        }
       }
+      mdef |= kc.elig & above;
+      mtie = kc.elig & equal;
     }
+  }
+  // the warp's 32 x 32 bits transposed: lane `it` then holds the ballot of chunk `it` (bit l = lane l's element)
+  mdef = warp_transpose32(mdef, lane);
+  mtie = warp_transpose32(mtie, lane);
+  if (lane < chunks) {
+    sh.bdef[lane * (kWarps + 1) + warp] = mdef;
+    sh.btie[lane * (kWarps + 1) + warp] = mtie;
   }
   __syncthreads();
   // exclusive scan of the packed populations over the chunks * kWarps words (word tid belongs to thread tid)
   static_assert(kItemsLong * kWarps <= kThreads, "one word per thread");
   const bool owner = tid < chunks * kWarps;
-  const uint32_t wd = owner ? sh.bdef[tid] : 0u, wt = owner ? sh.btie[tid] : 0u;
+  const int slot = tid + tid / kWarps;  // word tid = (chunk tid / kWarps, warp tid % kWarps) in the padded rows
+  const uint32_t wd = owner ? sh.bdef[slot] : 0u, wt = owner ? sh.btie[slot] : 0u;
   const uint32_t mine = (uint32_t)__popc(wd) | ((uint32_t)__popc(wt) << 16);
   uint32_t run = mine;
 #pragma unroll
@@ -622,7 +659,7 @@ __device__ int cached_ordered_emit(int n, int ties_allowed, const KeyCache<ITEMS
 template <bool CACHED, int CL, class KeyFn, class ClassFn, class EmitFn, int ITEMS>
 __device__ int cluster_ordered_emit(int n, int ties_allowed, KeyFn key_of, const KeyCache<ITEMS>& kc, ClassFn classify,
                                     EmitFn emit, SelectShared& sh) {
-  if constexpr (CACHED) return cached_ordered_emit<CL>(n, ties_allowed, kc, classify, emit, sh);
+  static_assert(!CACHED, "keys in registers: call cached_ordered_emit");
   if (CL == 1) return block_ordered_emit<CACHED>(n, ties_allowed, key_of, kc, classify, emit, sh);
   cg::cluster_group cluster = cg::this_cluster();
   const int rank = (int)cluster.block_rank();
@@ -770,7 +807,21 @@ __global__ void __launch_bounds__(kThreads, 1024 / kThreads) ta_forced_kernel(ta
     f[il] = 0;  // set by emit when taken (later, after a block barrier; possibly by another thread)
   };
   auto emit = [&](int il, int rank) { f[il] = 1; };
-  const int taken = cluster_ordered_emit<CACHED, CL>(hi - lo, r.ties, key_of, kc, classify, emit, sh);
+  int taken;
+  if constexpr (CACHED) {
+    uint32_t always = 0;  // the mandatory tokens; every flag is cleared here and set by emit after a block barrier
+#pragma unroll
+    for (int it = 0; it < ITEMS; ++it) {
+      const int il = (int)threadIdx.x + it * kThreads;
+      if (il < hi - lo) {
+        f[il] = 0;
+        if (mandatory(lo + il)) always |= 1u << it;
+      }
+    }
+    taken = cached_ordered_emit<CL>(hi - lo, r, kc, always, emit, sh);
+  } else {
+    taken = cluster_ordered_emit<CACHED, CL>(hi - lo, r.ties, key_of, kc, classify, emit, sh);
+  }
   if (threadIdx.x == 0 && blockIdx.x % CL == 0) r_main[b] = s.K_eff - taken;
 }
 
@@ -925,7 +976,11 @@ __global__ void __launch_bounds__(kThreads, 1024 / kThreads) ta_select_kernel(ta
   auto emit = [&](int il, int rank) {
     if (rank < K) out[rank] = lo + il;
   };
-  const int taken = cluster_ordered_emit<CACHED, CL>(hi - lo, r.ties, key_of, kc, classify, emit, sh);
+  int taken;
+  if constexpr (CACHED)  // forced tokens (not eligible, inside the unit) are taken whatever their key
+    taken = cached_ordered_emit<CL>(hi - lo, r, kc, exist_mask(hi - lo) & ~kc.elig, emit, sh);
+  else
+    taken = cluster_ordered_emit<CACHED, CL>(hi - lo, r.ties, key_of, kc, classify, emit, sh);
   if (!lead) return;
   for (int q = taken + tid; q < K; q += kThreads) out[q] = -1;
   if (tid == 0) count[unit] = taken;
