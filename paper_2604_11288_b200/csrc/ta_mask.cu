@@ -97,21 +97,33 @@ __global__ void __launch_bounds__(kTile) ta_mask_kernel(ta_seq_desc seq, const i
       s_pbud[0] = ca.budget;
     }
   } else {
-    for (int i = tid; i < n_pat * TA_MAX_PATTERN_LEN; i += kTile) s_pid[i] = p_ids[i];
-    for (int i = tid; i < n_pat; i += kTile) {
-      s_plen[i] = p_len[i];
-      s_pspan[i] = p_span[i];
-      s_pbud[i] = p_budget[i];
+    // the pattern tables: every load is requested before the first is stored (one memory latency for all of them)
+    static_assert(TA_MAX_PATTERNS <= kTile && TA_MAX_PATTERNS * TA_MAX_PATTERN_LEN <= 4 * kTile, "slots per thread");
+    int32_t r_pid[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const int i = tid + q * kTile;
+      r_pid[q] = i < n_pat * TA_MAX_PATTERN_LEN ? p_ids[i] : 0;
     }
-    if (tid < 32) s_bloom[tid] = n_pat ? p_bloom[tid] : 0u;
+    const int32_t r_len = tid < n_pat ? p_len[tid] : 0, r_span = tid < n_pat ? p_span[tid] : 0;
+    const float r_bud = tid < n_pat ? p_budget[tid] : 0.0f;
+    const uint32_t r_bloom = (tid < 32 && n_pat) ? p_bloom[tid] : 0u;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const int i = tid + q * kTile;
+      if (i < n_pat * TA_MAX_PATTERN_LEN) s_pid[i] = r_pid[q];
+    }
+    if (tid < n_pat) {
+      s_plen[tid] = r_len;
+      s_pspan[tid] = r_span;
+      s_pbud[tid] = r_bud;
+    }
+    if (tid < 32) s_bloom[tid] = r_bloom;
   }
-  if (tid == 0) {
-    float w = voucher_decay;
-    s_w[0] = 1.0f;
-    for (int k = 1; k <= TA_MAX_SPAN; ++k) {
-      s_w[k] = w;
-      w = __fmul_rn(w, voucher_decay);
-    }
+  if (tid <= TA_MAX_SPAN) {  // s_w[k] = decay^k by repeated multiplication (one rounding per step), thread k on its own
+    float w = 1.0f;
+    for (int k = 0; k < tid; ++k) w = __fmul_rn(w, voucher_decay);
+    s_w[tid] = w;
   }
 
   // phase a: ids + sequence starts for tile and halo; histogram for the tile proper
@@ -279,10 +291,21 @@ __global__ void __launch_bounds__(kTile) ta_mask_kernel(ta_seq_desc seq, const i
       const bool head = (tok == start);
       const int reach = (head || q == 0) ? -1 : s_reach[q - 1];
       if (reach >= i) {
+        // which of the kmax positions before this token hold an anchor whose span reaches it: independent loads,
+        // collected in a bit mask; the sum then runs over the few set bits, nearest anchor first
         const int kmax = (int)min((long long)max_span, tok - start);
+        static_assert(TA_MAX_SPAN <= 64, "one bit per distance");
+        unsigned long long reaching = 0;
+#pragma unroll 8
         for (int k = 1; k <= kmax; ++k) {
           const int p = s_apat[i - k];
-          if (p >= 0 && k <= s_pspan[p]) V = __fadd_rn(V, __fmul_rn(s_abud[i - k], s_w[k]));
+          const int span = p >= 0 ? s_pspan[p] : 0;
+          if (k <= span) reaching |= 1ull << (k - 1);
+        }
+        while (reaching) {
+          const int k = __ffsll((long long)reaching);
+          reaching &= reaching - 1ull;
+          V = __fadd_rn(V, __fmul_rn(s_abud[i - k], s_w[k]));
         }
       }
       flags[tok] = (uint8_t)((anchor_tok ? TA_FLAG_ANCHOR_TOKEN : 0) | (anchor_end ? TA_FLAG_ANCHOR_END : 0) |
