@@ -771,6 +771,12 @@ ta_status compress_impl(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* p
   const long long score_jobs = (lse_obs ? 1LL : 2LL) * batch->n_layers * batch->batch * Hkv * ((batch->max_n + 127) / 128) *
                                (((Hq / Hkv) * policy->obs_window + 127) / 128);
   const bool fork = !reuse && !fast && !external && score_jobs <= 400LL * ctx->sm_count;
+  // Kernels of the chain that directly follow another kernel of the chain on their stream are launched as its
+  // programmatic dependents: their launch overlaps its tail, and they wait for it before they touch memory. The
+  // forced-set kernel follows the mask kernel; the selection follows the score kernel, the forced-set kernel or the
+  // head sum (not across the join with the side stream); the broadcast and the gather follow the selection.
+  sel.pdl_forced = 1;
+  sel.pdl_units = fork ? 0 : 1;
   if (fork) {
     seq_stream = ctx->side;
     e = cudaEventRecord(ctx->ev_fork, stream);
@@ -821,7 +827,7 @@ ta_status compress_impl(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* p
   if (e == cudaSuccess && share_heads)
     e = ta_launch_broadcast_heads(batch->n_layers, batch->batch, Hkv, K, idx_lb, count_lb, idx, count, stream);
   if (e == cudaSuccess && fast)
-    e = ta_launch_broadcast_idx(batch->batch, Hkv, K, batch->n_layers, idx_seq, count_seq, idx, count, stream);
+    e = ta_launch_broadcast_idx(batch->batch, Hkv, K, batch->n_layers, idx_seq, count_seq, idx, count, stream, true);
   mark(3);
   if (e == cudaSuccess && !select_gathers) {
     ta_compact_args a = {};
@@ -835,6 +841,7 @@ ta_status compress_impl(ta_ctx* ctx, const ta_patterns* pats, const ta_policy* p
     a.count = count;
     a.k_out = k_out;
     a.v_out = v_out;
+    a.pdl = 1;
     e = ta_launch_compact(a, ctx->sm_count, stream);
   }
   mark(4);

@@ -31,6 +31,7 @@ __global__ void __launch_bounds__(kThreads) ta_compact_kernel(ta_seq_desc seq, i
                                                               ta_bf16_view kv1, const int32_t* __restrict__ idx,
                                                               const int32_t* __restrict__ count,
                                                               uint4* __restrict__ out0, uint4* __restrict__ out1) {
+  ta_wait_for_prior_grid();
   const int unit = blockIdx.x;
   const int g = unit % Hkv;
   const int b = (unit / Hkv) % seq.batch;
@@ -71,8 +72,14 @@ cudaError_t ta_launch_compact(const ta_compact_args& a, int sm_count, cudaStream
   const int units = a.n_layers * a.seq.batch * a.Hkv;
   if (units == 0 || a.K == 0) return cudaSuccess;
   dim3 grid(units, (a.K + kRowsPerBlock - 1) / kRowsPerBlock, 2);
-  ta_compact_kernel<<<grid, kThreads, 0, stream>>>(a.seq, a.Hkv, a.K, a.k, a.v, a.idx, a.count,
-                                                   reinterpret_cast<uint4*>(a.k_out),
-                                                   reinterpret_cast<uint4*>(a.v_out));
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = dim3(kThreads, 1, 1);
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  if (a.pdl) ta_pdl_attribute(&attr[0]);
+  cfg.attrs = attr;
+  cfg.numAttrs = a.pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, ta_compact_kernel, a.seq, a.Hkv, a.K, a.k, a.v, a.idx, a.count,
+                            reinterpret_cast<uint4*>(a.k_out), reinterpret_cast<uint4*>(a.v_out));
 }

@@ -76,7 +76,16 @@ __host__ __device__ inline int ta_seq_begin(const ta_seq_desc& s, int b, const i
   return s.cu ? s.cu[b] : b * s.n_uniform;
 }
 
+// Programmatic dependent launch: a kernel launched with ta_pdl_attribute() may be scheduled while the kernel before it
+// on the stream is still draining (its launch latency overlaps that kernel's tail); it must call
+// ta_wait_for_prior_grid() before its first access to memory. The call returns at once in a kernel launched normally.
+inline void ta_pdl_attribute(cudaLaunchAttribute* attr) {
+  attr->id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr->val.programmaticStreamSerializationAllowed = 1;
+}
 #ifdef __CUDACC__
+__device__ __forceinline__ void ta_wait_for_prior_grid() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // Static part of a token's utility (Eq. 3): u_static = ((beta*R + gamma*S) - lambda*F) + V with R = (i0+1)/n,
 // S = 1 on anchor tokens, F = count(id)/n; one rounding per operation. i0 is the 0-based position in the sequence.
 __device__ __forceinline__ float ta_static_utility(int i0, int n, int count, bool anchor_token, float V, float beta,
@@ -165,6 +174,7 @@ struct ta_select_args {
   void* gather_v_out;
   // optional: ta_launch_forced also writes the static utilities (what ta_launch_mask does when it is given the
   // array), saving a kernel on the per-sequence chain. static_out null: not asked for.
+  int pdl_forced, pdl_units;  // launch the forced-set / the selection kernel as a programmatic dependent of the kernel before it
   float* static_out;
   const int32_t* static_ids;
   const int32_t* static_hist;  // [B][vocab] token counts per sequence
@@ -176,7 +186,8 @@ cudaError_t ta_launch_select(const ta_select_args& a, ta_dev_status* status, cud
 cudaError_t ta_launch_forced(const ta_select_args& a, ta_dev_status* status, cudaStream_t stream);
 cudaError_t ta_launch_select_units(const ta_select_args& a, cudaStream_t stream);
 cudaError_t ta_launch_broadcast_idx(int B, int Hkv, int K, int n_layers, const int32_t* idx_seq,
-                                    const int32_t* count_seq, int32_t* idx, int32_t* count, cudaStream_t stream);
+                                    const int32_t* count_seq, int32_t* idx, int32_t* count, cudaStream_t stream,
+                                    bool pdl = false);
 
 // selection shared by the KV heads of a layer: head sum of the utilities, copy of the result to every head
 cudaError_t ta_launch_headsum(int n_layers, int Hkv, long long total, const float* u, float* u_all,
@@ -216,5 +227,6 @@ struct ta_compact_args {
   const int32_t* count;
   void* k_out;
   void* v_out;
+  int pdl;  // launch as a programmatic dependent of the kernel before it on the stream
 };
 cudaError_t ta_launch_compact(const ta_compact_args& a, int sm_count, cudaStream_t stream);

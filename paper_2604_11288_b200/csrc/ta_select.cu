@@ -40,6 +40,7 @@ using namespace sel512;  // the launchers below name the 512-thread kernels unle
 __global__ void ta_broadcast_idx_kernel(int B, int Hkv, int K, int n_layers, const int32_t* __restrict__ idx_seq,
                                         const int32_t* __restrict__ count_seq, int32_t* __restrict__ idx,
                                         int32_t* __restrict__ count) {
+  ta_wait_for_prior_grid();
   const long long total = (long long)n_layers * B * Hkv * K;
   for (long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x; t < total;
        t += (long long)gridDim.x * blockDim.x) {
@@ -103,29 +104,40 @@ int sm_count_of(const ta_select_args& a) {
   return sms;
 }
 
+// stream_pdl: the stream, and whether the kernel is launched as a programmatic dependent of the kernel before it
+struct StreamPdl {
+  cudaStream_t stream;
+  bool pdl;
+};
 template <class Kern, class... Args>
-cudaError_t launch_threads(int threads, Kern kern, int units, int cl, cudaStream_t stream, Args... args) {
+cudaError_t launch_threads(int threads, Kern kern, int units, int cl, StreamPdl sp, Args... args) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)(units * cl), 1, 1);
   cfg.blockDim = dim3((unsigned)threads, 1, 1);
   cfg.dynamicSmemBytes = 0;
-  cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = (unsigned)cl;
-  attr[0].val.clusterDim.y = 1;
-  attr[0].val.clusterDim.z = 1;
+  cfg.stream = sp.stream;
+  cudaLaunchAttribute attr[2];
+  int n = 0;
+  if (cl > 1) {  // no cluster attribute when no cluster is needed
+    attr[n].id = cudaLaunchAttributeClusterDimension;
+    attr[n].val.clusterDim.x = (unsigned)cl;
+    attr[n].val.clusterDim.y = 1;
+    attr[n].val.clusterDim.z = 1;
+    ++n;
+  }
+  if (sp.pdl) ta_pdl_attribute(&attr[n++]);
   cfg.attrs = attr;
-  cfg.numAttrs = cl > 1 ? 1 : 0;  // a plain launch when no cluster is needed
+  cfg.numAttrs = n;
   return cudaLaunchKernelEx(&cfg, kern, args...);
 }
 template <class Kern, class... Args>
-cudaError_t launch_clustered(Kern kern, int units, int cl, cudaStream_t stream, Args... args) {
-  return launch_threads(kThreads, kern, units, cl, stream, args...);
+cudaError_t launch_clustered(Kern kern, int units, int cl, StreamPdl sp, Args... args) {
+  return launch_threads(kThreads, kern, units, cl, sp, args...);
 }
 
-cudaError_t ta_launch_forced(const ta_select_args& a, ta_dev_status* status, cudaStream_t stream) {
+cudaError_t ta_launch_forced(const ta_select_args& a, ta_dev_status* status, cudaStream_t stream_) {
   if (a.seq.batch == 0 || a.n_layers == 0) return cudaSuccess;
+  const StreamPdl stream = {stream_, a.pdl_forced != 0};
   const int B = a.seq.batch * (a.n_classes > 0 ? a.n_classes : 1);  // blocks: (class, sequence)
   const int32_t* ck = a.n_classes > 0 ? a.class_K : nullptr;
   const int sms = sm_count_of(a);
@@ -173,8 +185,9 @@ bool ta_select_gathers(const ta_select_args& a) {
   return a.seq.max_n <= kItems * kThreads && units <= 4 * sm_count_of(a);
 }
 
-cudaError_t ta_launch_select_units(const ta_select_args& a, cudaStream_t stream) {
+cudaError_t ta_launch_select_units(const ta_select_args& a, cudaStream_t stream_) {
   if (a.seq.batch == 0 || a.n_layers == 0) return cudaSuccess;
+  const StreamPdl stream = {stream_, a.pdl_units != 0};
   UnitSrc src;
   src.u = a.fast ? nullptr : a.u;
   src.A = a.fast ? nullptr : a.A;
@@ -239,12 +252,20 @@ cudaError_t ta_launch_select(const ta_select_args& a, ta_dev_status* status, cud
 }
 
 cudaError_t ta_launch_broadcast_idx(int B, int Hkv, int K, int n_layers, const int32_t* idx_seq,
-                                    const int32_t* count_seq, int32_t* idx, int32_t* count, cudaStream_t stream) {
+                                    const int32_t* count_seq, int32_t* idx, int32_t* count, cudaStream_t stream,
+                                    bool pdl) {
   const long long total = (long long)n_layers * B * Hkv * K;
   if (total == 0) return cudaSuccess;
   const int blocks = (int)((total + 255) / 256 < 4096 ? (total + 255) / 256 : 4096);
-  ta_broadcast_idx_kernel<<<blocks, 256, 0, stream>>>(B, Hkv, K, n_layers, idx_seq, count_seq, idx, count);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)blocks, 1, 1);
+  cfg.blockDim = dim3(256, 1, 1);
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  if (pdl) ta_pdl_attribute(&attr[0]);
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, ta_broadcast_idx_kernel, B, Hkv, K, n_layers, idx_seq, count_seq, idx, count);
 }
 
 cudaError_t ta_launch_headsum(int n_layers, int Hkv, long long total, const float* u, float* u_all,

@@ -732,6 +732,7 @@ __global__ void __launch_bounds__(kThreads, 1024 / kThreads) ta_forced_kernel(ta
                                                              int32_t* __restrict__ r_main, ta_dev_status* status,
                                                              const int32_t* __restrict__ class_K, ta_static_out so) {
   __shared__ SelectShared sh;
+  ta_wait_for_prior_grid();
   // grid.x = classes * sequences * CL; without budget classes there is one class and K is the argument
   const int b = (blockIdx.x / CL) % seq.batch;
   const int cls = (blockIdx.x / CL) / seq.batch;
@@ -881,6 +882,7 @@ __global__ void __launch_bounds__(kThreads, 1024 / kThreads) ta_select_kernel(ta
                                                              int32_t* __restrict__ idx, int32_t* __restrict__ count,
                                                              GatherDst gd, const int32_t* __restrict__ class_of) {
   __shared__ SelectShared sh;
+  ta_wait_for_prior_grid();
   const int unit = blockIdx.x / CL;
   const bool lead = blockIdx.x % CL == 0;
   int b, l = 0, g = 0;
