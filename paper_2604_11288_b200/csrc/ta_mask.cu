@@ -321,6 +321,7 @@ __global__ void __launch_bounds__(256) ta_ustatic_kernel(ta_seq_desc seq, const 
                                                          const float* __restrict__ voucher,
                                                          const int32_t* __restrict__ hist, int vocab, float beta,
                                                          float gamma, float lambda, float* __restrict__ u_static) {
+  ta_wait_for_prior_grid();  // launched as a programmatic dependent of the mask kernel
   const long long tok = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (tok >= seq.total) return;
   const int b = seq_of(seq, tok);
@@ -339,9 +340,16 @@ cudaError_t finish_static_utility(const ta_policy& pol, const ta_seq_desc& seq, 
                                   const float* voucher, const int32_t* hist, float* u_static, cudaStream_t stream) {
   if (!u_static) return cudaSuccess;  // left to the forced-set kernel
   const int blocks = (int)((seq.total + 255) / 256);
-  ta_ustatic_kernel<<<blocks, 256, 0, stream>>>(seq, ids, flags, voucher, hist, pol.vocab_size, pol.beta, pol.gamma,
-                                                pol.lambda, u_static);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)blocks, 1, 1);
+  cfg.blockDim = dim3(256, 1, 1);
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  ta_pdl_attribute(&attr[0]);  // always directly behind the mask kernel
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, ta_ustatic_kernel, seq, ids, flags, voucher, hist, pol.vocab_size, pol.beta,
+                            pol.gamma, pol.lambda, u_static);
 }
 }  // namespace
 

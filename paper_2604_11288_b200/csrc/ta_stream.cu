@@ -111,6 +111,7 @@ __global__ void ta_stream_step_kernel(ta_stream_dev st, const ta_stream_seq_info
                                       int n_recent, int k_protected, int32_t* __restrict__ evicted_pos,
                                       ta_dev_status* status) {
   extern __shared__ __align__(16) unsigned char smem[];
+  ta_wait_for_prior_grid();  // launched as a programmatic dependent of the per-sequence kernel
   const int u = blockIdx.x, tid = threadIdx.x, nt = blockDim.x;
   const int b = (u / st.Hkv) % st.B;
   const int K = st.K, C = K + 1, len = st.len, n = len + 1;
@@ -332,8 +333,17 @@ cudaError_t ta_launch_stream_step(const ta_stream_dev& st, const ta_policy& pol,
     if (e != cudaSuccess) return e;
     attr_set[dev & 63].store(true, std::memory_order_release);
   }
-  ta_stream_step_kernel<<<U, threads, smem, stream>>>(st, info, attn, pol.vocab_size, pol.alpha, pol.beta, pol.gamma,
-                                                      pol.delta, pol.lambda, pol.pension_rho, pol.budget_decay,
-                                                      pol.n_sink, pol.n_recent, pol.k_protected, evicted_pos, status);
-  return cudaGetLastError();
+  // the launch overlaps the tail of the kernel before it on the stream (ta_stream_seq_kernel in ta_stream_step)
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)U, 1, 1);
+  cfg.blockDim = dim3((unsigned)threads, 1, 1);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  ta_pdl_attribute(&attr[0]);
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, ta_stream_step_kernel, st, info, attn, pol.vocab_size, pol.alpha, pol.beta, pol.gamma,
+                            pol.delta, pol.lambda, pol.pension_rho, pol.budget_decay, pol.n_sink, pol.n_recent,
+                            pol.k_protected, evicted_pos, status);
 }
