@@ -31,7 +31,8 @@
 // pass), so a fixed share of the exponentials (2 of every 16 with 256 score rows) is evaluated on the FMA pipe instead: the argument is
 // clamped to [-126, 126] with a saturating multiply-add, split into integer and fraction with the 1.5*2^23 rounding
 // trick, 2^fraction comes from a cubic polynomial (relative error 7.5e-5) and the integer part goes into the exponent
-// field with an integer add.
+// field with an integer add. The other exponentials take their scale-and-shift and their running sums two at a time
+// (fma.rn.f32x2, add.rn.f32x2: the same roundings as the scalar forms, a third fewer issue slots per element).
 //
 // Every wait on an mbarrier is bounded by wall time; when one runs out the CTA records TA_ERR_TIMEOUT, its producer
 // and MMA warps stop issuing work, the copies and MMAs in flight are drained, and the softmax warps finish their loops
@@ -162,6 +163,19 @@ __device__ __forceinline__ float exp2_poly(float s, float c252, float bias) {
   p = fmaf(p, f, kC1);
   p = fmaf(p, f, kC0);
   return __int_as_float((__float_as_int(y) << 23) + __float_as_int(p));
+}
+// two multiply-adds / two adds in one instruction (same roundings as the scalar forms)
+__device__ __forceinline__ void fma2(float& d0, float& d1, float a0, float a1, float b, float c0, float c1) {
+  asm("{\n\t.reg .b64 ra, rb, rc, rd;\n\tmov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %4};\n\tmov.b64 rc, {%5, %6};\n\t"
+      "fma.rn.f32x2 rd, ra, rb, rc;\n\tmov.b64 {%0, %1}, rd;\n\t}"
+      : "=f"(d0), "=f"(d1)
+      : "f"(a0), "f"(a1), "f"(b), "f"(c0), "f"(c1));
+}
+__device__ __forceinline__ void add2(float& d0, float& d1, float a0, float a1) {
+  asm("{\n\t.reg .b64 ra, rd;\n\tmov.b64 ra, {%2, %3};\n\tmov.b64 rd, {%0, %1};\n\tadd.rn.f32x2 rd, rd, ra;\n\t"
+      "mov.b64 {%0, %1}, rd;\n\t}"
+      : "+f"(d0), "+f"(d1)
+      : "f"(a0), "f"(a1));
 }
 __device__ __forceinline__ float poly_bias(float beta) { return (126.0f - beta) * (1.0f / kPolyRange); }
 
@@ -461,9 +475,18 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
               if (kbase + q > lim) v[q] = -INFINITY;
           }
 #pragma unroll
-          for (int q = 0; q < 16; ++q) {
-            const float e = (mix && poly_slot<MB>(q)) ? exp2_poly(v[q], c252, pbias) : ex2(fmaf(v[q], c, -rc));
-            s4[q & 3] += e;
+          for (int q = 0; q < 16; q += 2) {
+            if (mix && (poly_slot<MB>(q) || poly_slot<MB>(q + 1))) {
+#pragma unroll
+              for (int e2 = 0; e2 < 2; ++e2) {
+                const float e = poly_slot<MB>(q + e2) ? exp2_poly(v[q + e2], c252, pbias) : ex2(fmaf(v[q + e2], c, -rc));
+                s4[(q + e2) & 3] += e;
+              }
+            } else {
+              float a0, a1;
+              fma2(a0, a1, v[q], v[q + 1], c, -rc, -rc);
+              add2(s4[q & 3], s4[(q & 3) + 1], ex2(a0), ex2(a1));
+            }
           }
           if (track) {
             float t4[4];
@@ -665,9 +688,18 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             const float tbv[4] = {tb.x, tb.y, tb.z, tb.w};
             float a[4];
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              a[e] = (!masked && poly_slot<MB>(4 * q4 + e)) ? exp2_poly(cur[4 * q4 + e], c252, tbv[e])
-                                                        : ex2(fmaf(cur[4 * q4 + e], c, tbv[e]));
+            for (int e = 0; e < 4; e += 2) {
+              if (!masked && (poly_slot<MB>(4 * q4 + e) || poly_slot<MB>(4 * q4 + e + 1))) {
+#pragma unroll
+                for (int e2 = e; e2 < e + 2; ++e2)
+                  a[e2] = poly_slot<MB>(4 * q4 + e2) ? exp2_poly(cur[4 * q4 + e2], c252, tbv[e2])
+                                                     : ex2(fmaf(cur[4 * q4 + e2], c, tbv[e2]));
+              } else {
+                float x0, x1;
+                fma2(x0, x1, cur[4 * q4 + e], cur[4 * q4 + e + 1], c, tbv[e], tbv[e + 1]);
+                a[e] = ex2(x0);
+                a[e + 1] = ex2(x1);
+              }
             }
             if (masked) {  // row r sees key i only if i <= the row's own position
 #pragma unroll
@@ -678,8 +710,8 @@ ta_score_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 if (key > lim) a[e] = 0.0f;
               }
             }
-#pragma unroll
-            for (int e = 0; e < 4; ++e) sA4[e] += a[e];
+            add2(sA4[0], sA4[1], a[0], a[1]);
+            add2(sA4[2], sA4[3], a[2], a[3]);
             if (PM == kOutAP) {
               const float4 ws = w4[cc * 8 + hi * 4 + q4];
               sP = fmaf(ws.x, a[0], sP);
